@@ -1,0 +1,156 @@
+/*
+ * libomc -- Online Model Compression (arXiv 2205.03494) parameter store for one NVIDIA B200.
+ *
+ * Model parameters live in a reduced-bit-width floating-point format (Sec. 2.2) with a
+ * per-variable linear transformation (Sec. 2.3); they are decompressed on the fly into a transient
+ * FP32 copy for the forward pass and, in the backward pass, decompressed, updated with the gradient
+ * and compressed again without the FP32 value ever being stored (Sec. 2.1, Fig. 1).  Only weight
+ * matrices are quantised (Sec. 2.4), and only a chosen subset of them (Sec. 2.5, Sec. 3.1).
+ *
+ * Conventions
+ *   - Every function returns OMC_OK (0) or a negative omc_status.  Nothing throws, aborts or traps.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA device memory owned by
+ *     the caller, 16-byte aligned, valid until the work queued on `stream` has finished.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device calls only
+ *     enqueue work; they do not synchronise.  Apart from omc_plan_prepare they allocate nothing.
+ *   - Non-finite values are data, never errors: they propagate as IEEE-754 prescribes.
+ *   - A plan is not thread-safe; distinct plans are independent.
+ *
+ * Memory layouts (all fixed by the plan; query them with omc_plan_sizes / omc_plan_var)
+ *   full   : FP32 arena holding every variable, variable i at element offset full_off[i]; every
+ *            offset is a multiple of 4 elements, the gap after a variable is padding that the
+ *            library may read but never interprets.  Gradients and decompressed output use it.
+ *   resid  : FP32 arena with only the variables that stay in FP32, same alignment rule.
+ *   packed : byte arena with the codes of the quantised variables.  Variable i occupies
+ *            packed_bytes[i] = roundup16(ceil(numel*B/8)) bytes at packed_off[i]; inside it code k
+ *            occupies bits [k*B, (k+1)*B) of a little-endian bit stream (bit j of the stream is
+ *            bit j%8 of byte j/8); the bits after the last code are zero.  A code is
+ *            sign<<(E+M) | exponent_field<<M | mantissa_field.
+ *   sb     : float[2 * n_quantised]; sb[2*slot] = s and sb[2*slot+1] = b of Sec. 2.3.
+ */
+#ifndef OMC_H_
+#define OMC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* SxEyMz of Sec. 3.1: x sign, y exponent, z mantissa bits.  Accepted: sign_bits == 1,
+ * 2 <= exp_bits <= 8, 0 <= man_bits <= 23 (so 3 <= B <= 32).  S1E8M23 is FP32, S1E5M10 is FP16
+ * (Sec. 2.2, Sec. 3.4); the family is the IEEE-754 interchange parametrisation (bias
+ * 2^(E-1)-1, gradual underflow, top exponent field = Inf/NaN), rounding to nearest, ties to even.
+ * `flags` must be 0. */
+typedef struct {
+    uint8_t sign_bits, exp_bits, man_bits, flags;
+} omc_format_t;
+
+/* What a variable is (Sec. 2.4): only weight matrices are ever quantised. */
+enum { OMC_KIND_WEIGHT_MATRIX = 0, OMC_KIND_BIAS = 1, OMC_KIND_NORM = 2, OMC_KIND_OTHER = 3 };
+
+typedef struct {
+    uint64_t numel;    /* number of FP32 elements, > 0 */
+    uint32_t kind;     /* OMC_KIND_* */
+    uint32_t reserved; /* 0 */
+} omc_var_desc_t;
+
+typedef struct omc_plan omc_plan_t; /* opaque, owned by the library */
+
+/* Plan flags: the switches of the paper's ablation (Table 4). */
+#define OMC_PLAN_PVT 1u          /* fit and apply the per-variable transformation (Sec. 2.3)   */
+#define OMC_PLAN_WEIGHTS_ONLY 2u /* only OMC_KIND_WEIGHT_MATRIX is eligible (Sec. 2.4)         */
+#define OMC_PLAN_DEFAULT (OMC_PLAN_PVT | OMC_PLAN_WEIGHTS_ONLY)
+
+typedef enum {
+    OMC_OK = 0,
+    OMC_ERR_INVALID_ARG = -1,   /* a size, index, fraction or flag is out of range             */
+    OMC_ERR_BAD_FORMAT = -2,    /* omc_format_t outside the accepted family                    */
+    OMC_ERR_NULL_PTR = -3,      /* a required pointer is NULL                                  */
+    OMC_ERR_MISALIGNED = -4,    /* a device pointer is not 16-byte aligned                     */
+    OMC_ERR_PLAN_MISMATCH = -5, /* the plan was not prepared, or not for this call             */
+    OMC_ERR_CUDA = -6,          /* a CUDA runtime call failed (see omc_last_cuda_error)        */
+    OMC_ERR_NO_MEMORY = -7      /* host allocation failed                                      */
+} omc_status;
+
+const char *omc_strerror(int status);
+/* cudaError_t of the most recent failing runtime call on the calling thread (0 if none). */
+int omc_last_cuda_error(void);
+
+/*
+ * omc_plan -- decide which variables are compressed and lay out the arenas (host only; touches no
+ * device memory and needs no GPU).
+ *   Sec. 2.4: with OMC_PLAN_WEIGHTS_ONLY only weight matrices are eligible; biases and
+ *   normalisation parameters stay FP32.  Sec. 2.5 / Sec. 3.1: a fraction of the eligible
+ *   variables is quantised, chosen at random (the paper's default is 0.9 and a new draw per round
+ *   and per client: make one plan per draw).
+ *   vars[nvars]  host; the model's variables in the order the arenas will hold them.
+ *   fraction     in (0, 1]: k = floor(fraction * W + 1/2) of the W eligible variables.
+ *   seed         used iff mask == NULL: the eligible indices, ascending, are shuffled by
+ *                Fisher-Yates (i = W-1 .. 1, j = next() mod (i+1)) driven by SplitMix64(seed); the
+ *                first k are quantised.
+ *   mask         optional host array of nvars bytes; non-zero = quantise variable i.  Overrides
+ *                fraction and seed; a marked variable that is not eligible is an error.
+ *   flags        OMC_PLAN_* bits.
+ *   out          receives the plan; release it with omc_plan_destroy.
+ */
+int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t fmt, double fraction,
+             uint64_t seed, const uint8_t *mask, uint32_t flags, omc_plan_t **out);
+int omc_plan_destroy(omc_plan_t *plan); /* also frees the plan's device tables, if any */
+
+/*
+ * Sizes the caller must allocate (any output pointer may be NULL).
+ *   closed_form_bytes: the stored size of the model as the paper counts it (Tables 1 and 2):
+ *   sum over quantised variables of ceil(numel*B/8) + 8, plus 4*numel for the others.
+ */
+int omc_plan_sizes(const omc_plan_t *plan, uint64_t *full_elems, uint64_t *resid_elems,
+                   uint64_t *packed_bytes, uint32_t *n_quantised, uint64_t *workspace_bytes,
+                   uint64_t *closed_form_bytes);
+/* Where variable i lives.  resid_off_elems is meaningful iff !quantised; packed_* and sb_slot iff
+ * quantised. */
+int omc_plan_var(const omc_plan_t *plan, uint32_t i, int *quantised, uint64_t *full_off_elems,
+                 uint64_t *resid_off_elems, uint64_t *packed_off_bytes, uint64_t *packed_bytes,
+                 uint32_t *sb_slot);
+
+/*
+ * omc_plan_prepare -- copy the plan's tables to the current device (the one allocation the
+ * library makes; synchronous) and clear `workspace` (device, workspace_bytes) on `stream`.
+ * Must precede the first device call with this plan; the workspace then stays valid from call
+ * to call (each kernel leaves it cleared) as long as calls using it do not overlap on the GPU.
+ */
+int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream);
+
+/*
+ * omc_compress -- initial compression of a full-precision model (Sec. 2.2, 2.3).
+ * For each quantised variable V: codes = Q(V); Vt = Q^-1(codes); (s, b) = argmin ||s*Vt+b-V||_2
+ * from fp64 sums, stored FP32 (s = 1 when all Vt are equal or the denominator is 0 / not finite;
+ * s = 1, b = 0 without OMC_PLAN_PVT).  Other variables are copied to the resid arena.
+ *   params  device, full layout, read only.     packed, resid, sb  device, written.
+ */
+int omc_compress(const omc_plan_t *plan, const float *params, uint8_t *packed, float *resid,
+                 float *sb, void *workspace, void *stream);
+
+/*
+ * omc_decompress -- forward path of Fig. 1: the transient FP32 copy of variables
+ * [first_var, first_var + n_vars), written at their offsets in `out` (device, full layout):
+ * Vbar_k = fma(s, Vt_k, b) for quantised variables (one rounding), a copy for the others.
+ */
+int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, const float *resid,
+                   const float *sb, uint32_t first_var, uint32_t n_vars, float *out, void *stream);
+
+/*
+ * omc_update_recompress -- backward path of Fig. 1 in one launch: per element
+ * W = fma(-lr, g, fma(s, Vt, b)), re-quantised at once; (s, b) refitted per variable from fp64
+ * sums over (W, Q^-1 Q(W)); FP32 variables take W = fma(-lr, g, V) in place.  W itself is never
+ * stored, unless debug_w_out (device, full layout, may be NULL) asks for it.
+ *   packed, resid, sb  device, updated in place.    grads  device, full layout, read only.
+ * A NaN produced by the arithmetic is encoded as the positive NaN with all mantissa bits set.
+ */
+int omc_update_recompress(const omc_plan_t *plan, uint8_t *packed, float *resid, float *sb,
+                          const float *grads, float lr, float *debug_w_out, void *workspace,
+                          void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OMC_H_ */

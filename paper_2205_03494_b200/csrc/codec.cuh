@@ -1,0 +1,188 @@
+// SxEyMz codec arithmetic for the device side (Sec. 2.2 of the OMC paper; notation of Sec. 3.1).
+//
+// A code is sign<<(E+M) | exponent_field<<M | mantissa_field with the IEEE-754 interchange
+// parametrisation: bias 2^(E-1)-1, exponent field 0 = zero/subnormal, all ones = Inf/NaN.
+// Encoding rounds to nearest, ties to even, with gradual underflow and overflow to infinity.
+//
+// Each operation has a "fast" form that is exact for every finite in-range input and an "exact"
+// form that also handles Inf/NaN/overflow; callers test once per group of elements whether the
+// exact form is needed (it almost never is) instead of paying for it per element.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace omc {
+
+template <int E_, int M_>
+struct Fmt {
+    static_assert(E_ >= 2 && E_ <= 8 && M_ >= 0 && M_ <= 23, "format outside the accepted family");
+    static constexpr int E = E_, M = M_, B = 1 + E_ + M_;
+    static constexpr int BIAS = (1 << (E_ - 1)) - 1;
+    static constexpr int EMIN = 1 - BIAS, EMAX = BIAS;
+    static constexpr int SH = 23 - M_;                                   // fp32 mantissa bits dropped
+    static constexpr uint32_t CODE_MASK = (B == 32) ? 0xFFFFFFFFu : ((1u << (B % 32)) - 1u);
+    static constexpr uint32_t MAG_MASK = (1u << (E_ + M_)) - 1u;         // exponent + mantissa fields
+    static constexpr uint32_t INF_MAG = ((1u << E_) - 1u) << M_;         // magnitude code of infinity
+    static constexpr uint32_t SIGN_BIT = 1u << (E_ + M_);
+    // fp32 bit pattern of 2^k
+    __host__ __device__ static constexpr uint32_t pow2_bits(int k) { return (uint32_t)(k + 127) << 23; }
+    // Smallest FP32 magnitude that rounds to infinity: 2^EMAX * (2 - 2^-(M+1)) (a tie, which goes
+    // to the even side = infinity); with M == 23 that is not an FP32 value and 2^(EMAX+1) is.
+    __host__ __device__ static constexpr uint32_t ovf_bits()
+    {
+        if (E_ == 8) return 0x7F800000u;
+        if (M_ == 23) return pow2_bits(EMAX + 1);
+        return pow2_bits(EMAX) | (((1u << (M_ + 1)) - 1u) << (M_ == 23 ? 0 : 22 - M_));
+    }
+    static constexpr uint32_t OVF_BITS = ovf_bits();
+};
+
+__device__ __forceinline__ uint32_t f2u(float x) { return __float_as_uint(x); }
+__device__ __forceinline__ float u2f(uint32_t u) { return __uint_as_float(u); }
+
+// ---------------------------------------------------------------------------------------------
+// decode
+
+// Exact for every code whose exponent field is not all ones.
+template <class F>
+__device__ __forceinline__ float decode_fast(uint32_t c)
+{
+    if constexpr (F::E == 8) {
+        return u2f(c << F::SH);      // S1E8Mz is FP32 with the low mantissa bits dropped
+    } else {
+        // Put the fields where FP32 keeps them: the result has the code's exponent field as its
+        // own (subnormal codes become FP32 subnormals), so one exact multiplication by
+        // 2^(127-BIAS) rebiases normal and subnormal codes alike.
+        const uint32_t mag = (c & F::MAG_MASK) << F::SH;
+        const float v = __fmul_rn(u2f(mag), u2f(F::pow2_bits(127 - F::BIAS)));
+        return u2f(f2u(v) | ((c >> (F::E + F::M)) << 31));
+    }
+}
+
+template <class F>
+__device__ __forceinline__ bool code_is_special(uint32_t c)
+{
+    if constexpr (F::E == 8) return false;   // decode_fast is already exact
+    return (c & F::MAG_MASK) >= F::INF_MAG;
+}
+
+// Every code, Inf and NaN included (NaN: mantissa field kept in the top bits of the payload).
+template <class F>
+__device__ __forceinline__ float decode_exact(uint32_t c)
+{
+    if constexpr (F::E < 8) {
+        if ((c & F::MAG_MASK) >= F::INF_MAG) {
+            const uint32_t m = c & ((1u << F::M) - 1u);
+            return u2f(((c >> (F::E + F::M)) << 31) | 0x7F800000u | (m << F::SH));
+        }
+    }
+    return decode_fast<F>(c);
+}
+
+// ---------------------------------------------------------------------------------------------
+// encode: returns the code and the decoded value Q^-1(Q(w)) (needed by the Sec. 2.3 fit).
+
+// Exact iff !needs_exact_encode(w).
+template <class F>
+__device__ __forceinline__ uint32_t encode_fast(float w, float &vt)
+{
+    const uint32_t u = f2u(w);
+    if constexpr (F::M == 23 && F::E == 8) {
+        vt = w;
+        return u;
+    } else if constexpr (F::E == 8) {
+        // Only mantissa bits are dropped: round the FP32 pattern as an integer (a carry out of
+        // the mantissa moves into the exponent, up to infinity, exactly as it should).
+        const uint32_t a = u & 0x7FFFFFFFu;
+        const uint32_t lsb = (a >> F::SH) & 1u;
+        const uint32_t mag = (a + ((1u << (F::SH - 1)) - 1u) + lsb) >> F::SH;
+        const uint32_t c = mag | ((u >> 31) << (F::E + F::M));
+        vt = u2f(c << F::SH);
+        return c;
+    } else {
+        // Let the FP32 adder do the rounding: adding 2^(e_q+23-M), e_q = max(exponent, EMIN),
+        // leaves exactly the bits above the target spacing 2^(e_q-M), rounded to nearest even.
+        const float a = fabsf(w);
+        float r;
+        if constexpr (F::M <= 22) {
+            const float x2 = __fmul_rn(a, u2f(F::pow2_bits(F::SH)));
+            const uint32_t eb = max(f2u(x2) & 0x7F800000u, F::pow2_bits(F::EMIN + F::SH));
+            const float magic = u2f(eb);
+            r = __fsub_rn(__fadd_rn(a, magic), magic);
+        } else {
+            // M == 23: normal-range values are kept as they are, only the subnormal range rounds
+            const float magic = u2f(F::pow2_bits(F::EMIN));
+            const float rs = __fsub_rn(__fadd_rn(a, magic), magic);
+            r = (f2u(a) >= F::pow2_bits(F::EMIN)) ? a : rs;
+        }
+        // r is a value of the format: rebias exactly and read the fields off the FP32 pattern.
+        const float t = __fmul_rn(r, u2f(F::pow2_bits(F::BIAS - 127)));
+        const uint32_t c = (f2u(t) >> F::SH) | ((u >> 31) << (F::E + F::M));
+        vt = u2f(f2u(r) | (u & 0x80000000u));
+        return c;
+    }
+}
+
+// True for NaN, infinity (E < 8) and finite values that round to infinity (E < 8).
+template <class F>
+__device__ __forceinline__ bool needs_exact_encode(float w)
+{
+    const uint32_t a = f2u(w) & 0x7FFFFFFFu;
+    if constexpr (F::E == 8) return a > 0x7F800000u;
+    return a >= F::OVF_BITS;
+}
+
+// NaN -> sign, all-ones exponent, top M payload bits (a quiet bit is forced if those are zero;
+// with M == 0 there is no NaN code and infinity is written).
+template <class F>
+__device__ __forceinline__ uint32_t encode_exact(float w, float &vt)
+{
+    const uint32_t u = f2u(w);
+    const uint32_t a = u & 0x7FFFFFFFu;
+    const uint32_t sign = (u >> 31) << (F::E + F::M);
+    if (a > 0x7F800000u) {
+        uint32_t c;
+        if constexpr (F::M == 0) {
+            c = sign | F::INF_MAG;
+        } else {
+            uint32_t m = (u & 0x7FFFFFu) >> F::SH;
+            if (m == 0) m = 1u << (F::M - 1);
+            c = sign | F::INF_MAG | m;
+        }
+        vt = decode_exact<F>(c);
+        return c;
+    }
+    if constexpr (F::E < 8) {
+        if (a >= F::OVF_BITS) {
+            vt = u2f(0x7F800000u | (u & 0x80000000u));
+            return sign | F::INF_MAG;
+        }
+    }
+    return encode_fast<F>(w, vt);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Codes inside a run of 32-bit words (little-endian bit stream, code i at bits [i*B, (i+1)*B)).
+// With i a compile-time constant after unrolling, every shift below is an immediate.
+
+template <class F, int NW>
+__device__ __forceinline__ uint32_t get_code(const uint32_t (&w)[NW], int i)
+{
+    const int pos = i * F::B, wi = pos >> 5, sh = pos & 31;
+    uint32_t c;
+    if (sh + F::B <= 32)
+        c = w[wi] >> sh;
+    else
+        c = __funnelshift_r(w[wi], w[(wi + 1 < NW) ? wi + 1 : wi], sh);
+    return c & F::CODE_MASK;
+}
+
+template <class F, int NW>
+__device__ __forceinline__ void put_code(uint32_t (&w)[NW], int i, uint32_t c)
+{
+    const int pos = i * F::B, wi = pos >> 5, sh = pos & 31;
+    w[wi] |= c << sh;
+    if (sh + F::B > 32) w[(wi + 1 < NW) ? wi + 1 : wi] |= c >> (32 - sh);
+}
+
+}  // namespace omc

@@ -1,0 +1,6 @@
+// Kernel instantiations for one group of formats (split so the groups compile in parallel).
+#include "kernels.cuh"
+namespace omc {
+OMC_DEFINE_FORMAT(5, 2)
+OMC_DEFINE_FORMAT(4, 3)
+}  // namespace omc

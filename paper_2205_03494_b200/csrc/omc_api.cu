@@ -1,0 +1,144 @@
+// Device-side C-ABI entry points: argument checks, launch geometry, dispatch on the format.
+#include <cuda_runtime.h>
+
+#include "omc_internal.h"
+
+namespace omc {
+int note_cuda(cudaError_t e);
+
+#define OMC_DECLARE_FORMAT(E_, M_) extern const FmtOps ops_E##E_##M##M_;
+#define OMC_FORMAT_LIST(X)                                                                      \
+    X(5, 2) X(4, 3) X(5, 6) X(5, 10) /* benchmark configurations                              */ \
+    X(4, 14) X(3, 7) X(2, 3)         /* Tables 1 and 2 of the paper                           */ \
+    X(3, 9) X(4, 8) X(5, 7)          /* the 13-bit formats of Sec. 3.5.3                      */ \
+    X(8, 7) X(8, 23)                 /* bfloat16 and FP32 itself                              */
+OMC_FORMAT_LIST(OMC_DECLARE_FORMAT)
+
+const FmtOps *find_ops(int E, int M)
+{
+#define OMC_ADDR(E_, M_) &ops_E##E_##M##M_,
+    static const FmtOps *const table[] = {OMC_FORMAT_LIST(OMC_ADDR)};
+    for (const FmtOps *o : table)
+        if (o->E == E && o->M == M) return o;
+    return nullptr;
+}
+}  // namespace omc
+
+using omc::KParams;
+
+static bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
+{
+    if (!plan || !workspace) return OMC_ERR_NULL_PTR;
+    if (misaligned(workspace)) return OMC_ERR_MISALIGNED;
+    int dev = 0;
+    int rc = omc::note_cuda(cudaGetDevice(&dev));
+    if (rc) return rc;
+    if (plan->d_vars && plan->device != dev) return OMC_ERR_PLAN_MISMATCH;
+    if (!plan->d_vars) {
+        const size_t bytes = sizeof(omc::VarDev) * (size_t)plan->nvars;
+        rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), bytes));
+        if (rc) { plan->d_vars = nullptr; return rc; }
+        rc = omc::note_cuda(cudaMemcpy(plan->d_vars, plan->vars.data(), bytes, cudaMemcpyHostToDevice));
+        if (rc) { (void)cudaFree(plan->d_vars); plan->d_vars = nullptr; return rc; }
+        plan->device = dev;
+    }
+    return omc::note_cuda(cudaMemsetAsync(workspace, 0, plan->ws_bytes, static_cast<cudaStream_t>(stream)));
+}
+
+static int check_ready(const omc_plan_t *plan)
+{
+    if (!plan) return OMC_ERR_NULL_PTR;
+    if (!plan->d_vars) return OMC_ERR_PLAN_MISMATCH;
+    int dev = 0;
+    int rc = omc::note_cuda(cudaGetDevice(&dev));
+    if (rc) return rc;
+    return dev == plan->device ? OMC_OK : OMC_ERR_PLAN_MISMATCH;
+}
+
+static KParams whole_model(const omc_plan_t *plan, void *workspace)
+{
+    KParams p{};
+    p.vars = plan->d_vars;
+    p.var_begin = 0;
+    p.var_end = plan->nvars;
+    p.tile_begin = 0;
+    p.tile_count = plan->ntiles;
+    p.nwarps = plan->nwarps;
+    p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
+    p.tickets = reinterpret_cast<uint32_t *>(static_cast<char *>(workspace) + plan->ws_tickets_off);
+    p.slots = reinterpret_cast<omc::Partial *>(static_cast<char *>(workspace) + plan->ws_slots_off);
+    return p;
+}
+
+static int grid_for(uint32_t nwarps) { return (int)((nwarps + omc::WARPS_PER_CTA - 1) / omc::WARPS_PER_CTA); }
+
+extern "C" int omc_compress(const omc_plan_t *plan, const float *params, uint8_t *packed, float *resid,
+                            float *sb, void *workspace, void *stream)
+{
+    int rc = check_ready(plan);
+    if (rc) return rc;
+    if (!params || !workspace) return OMC_ERR_NULL_PTR;
+    if (plan->nq && (!packed || !sb)) return OMC_ERR_NULL_PTR;
+    if (plan->resid_elems && !resid) return OMC_ERR_NULL_PTR;
+    if (misaligned(params) || misaligned(packed) || misaligned(resid) || misaligned(sb) || misaligned(workspace))
+        return OMC_ERR_MISALIGNED;
+    KParams p = whole_model(plan, workspace);
+    p.packed = packed; p.resid = resid; p.sb = sb; p.fin = params;
+    plan->ops->compress(p, grid_for(p.nwarps), stream);
+    return omc::note_cuda(cudaGetLastError());
+}
+
+extern "C" int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, const float *resid,
+                              const float *sb, uint32_t first_var, uint32_t n_vars, float *out, void *stream)
+{
+    int rc = check_ready(plan);
+    if (rc) return rc;
+    if (n_vars == 0 || first_var >= plan->nvars || n_vars > plan->nvars - first_var) return OMC_ERR_INVALID_ARG;
+    if (!out) return OMC_ERR_NULL_PTR;
+    bool any_q = false, any_r = false;
+    for (uint32_t i = first_var; i < first_var + n_vars; ++i)
+        (plan->vars[i].quantised ? any_q : any_r) = true;
+    if (any_q && (!packed || !sb)) return OMC_ERR_NULL_PTR;
+    if (any_r && !resid) return OMC_ERR_NULL_PTR;
+    if (misaligned(packed) || misaligned(resid) || misaligned(sb) || misaligned(out)) return OMC_ERR_MISALIGNED;
+    KParams p{};
+    p.vars = plan->d_vars;
+    p.var_begin = first_var;
+    p.var_end = first_var + n_vars;
+    p.tile_begin = plan->vars[first_var].tile_start;
+    const omc::VarDev &lastv = plan->vars[first_var + n_vars - 1];
+    p.tile_count = lastv.tile_start + lastv.ntiles - p.tile_begin;
+    const uint64_t max_warps = (uint64_t)plan->n_cta * omc::WARPS_PER_CTA;
+    p.nwarps = (uint32_t)(p.tile_count < max_warps ? p.tile_count : max_warps);
+    p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
+    p.packed = const_cast<uint8_t *>(packed);
+    p.resid = const_cast<float *>(resid);
+    p.sb = const_cast<float *>(sb);
+    p.fout = out;
+    plan->ops->decompress(p, grid_for(p.nwarps), stream);
+    return omc::note_cuda(cudaGetLastError());
+}
+
+extern "C" int omc_update_recompress(const omc_plan_t *plan, uint8_t *packed, float *resid, float *sb,
+                                     const float *grads, float lr, float *debug_w_out, void *workspace,
+                                     void *stream)
+{
+    int rc = check_ready(plan);
+    if (rc) return rc;
+    if (!grads || !workspace) return OMC_ERR_NULL_PTR;
+    if (plan->nq && (!packed || !sb)) return OMC_ERR_NULL_PTR;
+    if (plan->resid_elems && !resid) return OMC_ERR_NULL_PTR;
+    if (misaligned(grads) || misaligned(packed) || misaligned(resid) || misaligned(sb) ||
+        misaligned(workspace) || misaligned(debug_w_out))
+        return OMC_ERR_MISALIGNED;
+    KParams p = whole_model(plan, workspace);
+    p.packed = packed; p.resid = resid; p.sb = sb; p.fin = grads; p.fout = debug_w_out;
+    p.neg_lr = -lr;
+    if (debug_w_out)
+        plan->ops->update_w(p, grid_for(p.nwarps), stream);
+    else
+        plan->ops->update(p, grid_for(p.nwarps), stream);
+    return omc::note_cuda(cudaGetLastError());
+}

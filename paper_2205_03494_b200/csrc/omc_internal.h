@@ -1,0 +1,87 @@
+// Internal declarations shared by the host-side plan code and the kernel launchers.
+#pragma once
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/omc.h"
+
+namespace omc {
+
+constexpr int TILE = 1024;         // elements per tile: the unit of work a warp takes
+constexpr int WARPS_PER_CTA = 8;
+constexpr int THREADS = 32 * WARPS_PER_CTA;
+constexpr int CTAS_PER_SM = 2;
+constexpr int DEFAULT_SMS = 148;   // B200; used when no device can be queried at plan time
+
+// One per variable, in the caller's order; lives in device memory after omc_plan_prepare.
+struct VarDev {
+    uint64_t n;             // elements
+    uint64_t full_off;      // element offset in the full FP32 layout
+    uint64_t store_off;     // quantised: byte offset in the packed arena; else element offset in resid
+    uint64_t packed_bytes;  // quantised: padded byte size of the code stream; else 0
+    uint64_t tile_start;    // index of the variable's first tile among all tiles of the plan
+    uint32_t ntiles;
+    uint32_t quantised;
+    uint32_t sb_slot;       // index into sb[] and the ticket array
+    uint32_t slot_base;     // first partial-sum slot of this variable in the workspace
+    uint32_t first_warp;    // the warp (of the plan-wide partition) that owns the first tile
+    uint32_t nslots;        // number of warps that own at least one tile of this variable
+};
+static_assert(sizeof(VarDev) == 64, "VarDev is laid out for 16-byte loads");
+
+// Per-warp partial sums of the Sec. 2.3 fit, one slot per (variable, warp that touched it).
+struct Partial {
+    double sx, sy, sxy, syy;   // Sum W, Sum Vt, Sum W*Vt, Sum Vt^2
+    float mn, mx;              // min / max of Vt (equal <=> degenerate case)
+    float pad[2];
+};
+static_assert(sizeof(Partial) == 48, "");
+
+constexpr uint64_t WS_HEADER_BYTES = 256;
+
+// Arguments of one kernel launch.
+struct KParams {
+    const VarDev *vars;
+    uint32_t var_begin, var_end;   // variables covered by this launch
+    uint64_t tile_begin;           // first tile covered
+    uint64_t tile_count;           // number of tiles covered
+    uint32_t nwarps;               // warps the tiles are divided among (<= tile_count)
+    uint32_t pvt;
+    uint8_t *packed;
+    float *resid;
+    float *sb;
+    const float *fin;              // compress: params; update: grads (full layout)
+    float *fout;                   // decompress: out; update: optional W (full layout)
+    float neg_lr;
+    Partial *slots;
+    uint32_t *tickets;
+};
+
+struct FmtOps {
+    int E, M;
+    void (*compress)(const KParams &, int grid, void *stream);
+    void (*decompress)(const KParams &, int grid, void *stream);
+    void (*update)(const KParams &, int grid, void *stream);     // W not stored
+    void (*update_w)(const KParams &, int grid, void *stream);   // W stored to fout
+};
+const FmtOps *find_ops(int E, int M);
+
+}  // namespace omc
+
+struct omc_plan {
+    omc_format_t fmt;
+    uint32_t flags;
+    uint32_t nvars, nq;
+    std::vector<omc::VarDev> vars;
+    std::vector<uint64_t> resid_off;   // per variable (valid iff !quantised)
+    uint64_t full_elems, resid_elems, packed_bytes, closed_form_bytes;
+    uint64_t ntiles;                   // all tiles
+    uint32_t n_sm, n_cta, nwarps;      // launch geometry the partition was made for
+    uint32_t nslots;
+    uint64_t ws_tickets_off, ws_slots_off, ws_bytes;
+    const omc::FmtOps *ops;
+    // device side
+    omc::VarDev *d_vars;
+    int device;                        // device the tables live on, -1 before prepare
+};

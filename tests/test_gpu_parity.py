@@ -1,0 +1,277 @@
+"""GPU parity: the CUDA library (through its C-ABI) against the CPU oracle on the same seeded
+inputs.  Packed codes (whole arena, zero padding included), decompressed values, the updated FP32
+values W and the FP32 variables must be bit-exact.  (s, b) come from fp64 sums whose order the
+paper does not fix: the oracle sums exactly, the GPU in a fixed order in fp64, so the two may
+differ by one FP32 unit in the last place in rare near-midpoint cases; the tests allow that, count
+it, and then continue from the oracle's (s, b) so that a difference cannot compound.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2205_03494_b200 as omc
+from paper_2205_03494_b200 import workloads
+from oracle import omc_oracle as orc
+from harness import DeviceModel, from_full, same_f32, to_full, ulp_diff
+
+pytestmark = pytest.mark.gpu
+
+ALL_FORMATS = [(5, 2), (4, 3), (5, 6), (5, 10), (4, 14), (3, 7), (2, 3), (3, 9), (4, 8), (5, 7), (8, 7),
+               (8, 23)]
+
+
+class Lockstep:
+    """Runs the oracle and the GPU side by side on a (sub)set of variables and compares."""
+
+    def __init__(self, numel, kinds, fmt, params, *, fraction=1.0, seed=0, mask=None,
+                 flags=omc.PLAN_DEFAULT, sample=None, threads=4):
+        self.E, self.M = fmt
+        self.B = 1 + self.E + self.M
+        self.plan = omc.Plan(numel, kinds, fmt, fraction=fraction, seed=seed, mask=mask, flags=flags)
+        self.pvt = bool(flags & omc.PLAN_PVT)
+        self.dm = DeviceModel(self.plan)
+        self.idx = list(range(len(numel))) if sample is None else list(sample)
+        self.threads = threads
+        self.sb_ulp_cases = 0
+        self.sb_checked = 0
+        # initial compression on both sides
+        full = self.dm.upload_full(params)
+        self.dm.compress(full)
+        del full
+        sel = [self.plan.quantised[i] for i in self.idx]
+        self.st = orc.compress([params[i] for i in self.idx], sel, self.E, self.M, self.pvt, threads)
+        self.check_state("compress")
+
+    def check_state(self, what, resync=True):
+        packed, resid, sb = self.dm.host_state()
+        fix = []
+        for k, i in enumerate(self.idx):
+            if self.plan.quantised[i]:
+                got = self.dm.var_packed(packed, i)
+                assert np.array_equal(got, self.st["packed"][k]), \
+                    "%s: codes of variable %d differ at byte %s" % (
+                        what, i, np.flatnonzero(got != self.st["packed"][k])[:5])
+                s, b = self.dm.var_sb(sb, i)
+                for name, g, w in (("s", s, self.st["s"][k]), ("b", b, self.st["b"][k])):
+                    d = ulp_diff(g, w)
+                    self.sb_checked += 1
+                    assert d <= 1, "%s: %s of variable %d: gpu %r oracle %r" % (what, name, i, g, w)
+                    if d:
+                        self.sb_ulp_cases += 1
+                        fix.append((i, k))
+            else:
+                assert same_f32(self.dm.var_resid(resid, i), self.st["fp32"][k]), (what, i)
+        if fix and resync:
+            for i, k in fix:
+                slot = self.plan.sb_slot[i]
+                self.dm.sb[2 * slot] = float(self.st["s"][k])
+                self.dm.sb[2 * slot + 1] = float(self.st["b"][k])
+        return packed
+
+    def check_padding(self, packed):
+        """The bits after a variable's last code, up to its 16-byte boundary, are zero."""
+        for i in range(self.plan.nvars):
+            if self.plan.quantised[i]:
+                arr = self.dm.var_packed(packed, i)
+                nbits = self.plan.numel[i] * self.B
+                assert arr.size % 16 == 0 and not arr[(nbits + 7) // 8:].any(), i
+                if nbits % 8:
+                    assert int(arr[nbits // 8]) >> (nbits % 8) == 0, i
+
+    def check_decompress(self, first=0, count=None):
+        out = self.dm.decompress(first, count)
+        torch.cuda.synchronize()
+        out = out.cpu().numpy()
+        want = orc.decompress(self.st, self.threads)
+        hi = self.plan.nvars if count is None else first + count
+        for k, i in enumerate(self.idx):
+            if first <= i < hi:
+                assert same_f32(from_full(self.plan, out, i), want[k]), ("decompress", i)
+        return out
+
+    def round(self, grads, lr, want_w=True):
+        """grads: list over all variables (GPU) -- the oracle takes the sampled ones."""
+        gfull = self.dm.upload_full(grads)
+        w_out = torch.zeros(self.plan.full_elems, dtype=torch.float32, device=self.dm.dev) if want_w else None
+        self.dm.update(gfull, lr, w_out)
+        ws = orc.update_recompress(self.st, [grads[i] for i in self.idx], lr, self.threads, want_w=True)
+        packed = self.check_state("update")
+        if want_w:
+            w_host = w_out.cpu().numpy()
+            for k, i in enumerate(self.idx):
+                assert same_f32(from_full(self.plan, w_host, i), ws[k]), ("W", i)
+        return packed
+
+
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("lr", [0.01, 10.0])
+def test_tiny_set_one_round(lr):
+    """Tiny set, 1/5/2, all four matrices: compress, decompress, one update round.  lr = 10 makes
+    the step larger than the code spacing so that the re-encode path really changes codes."""
+    wl = workloads.tiny()
+    params = wl.all_params()
+    ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params)
+    before = ls.dm.packed.cpu().numpy().copy()
+    ls.check_decompress()
+    packed = ls.round(wl.all_grads(0), lr)
+    ls.check_padding(packed)
+    ls.check_decompress()
+    changed = np.count_nonzero(before != packed[:before.size])
+    if lr == 10.0:
+        assert changed > before.size // 10
+    assert ls.sb_ulp_cases <= 2
+
+
+@pytest.mark.parametrize("wl", list(workloads.sweep()), ids=lambda w: "p%g-E%dM%d" % (w.fraction, *w.fmt))
+def test_partial_quantisation_sweep(wl):
+    """Quantised fraction x format sweep on the tiny set: parity, stored bytes against the closed
+    form, and the quantisation error against the half-spacing bound."""
+    params = wl.all_params()
+    ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params, fraction=wl.fraction, seed=wl.sel_seed)
+    E, M = wl.fmt
+    B = 1 + E + M
+    sel = orc.select(wl.kinds, wl.fraction, wl.sel_seed)
+    assert ls.plan.quantised == list(sel)
+    assert ls.plan.closed_form_bytes == orc.model_bytes(wl.numel, sel, B)
+    out = ls.check_decompress()
+    # error of the plain code against the bound 2^(max(e, emin) - M - 1)
+    emin = 2 - (1 << (E - 1))
+    for i in range(len(params)):
+        if not sel[i]:
+            continue
+        v = params[i].astype(np.float64)
+        vt = orc.decode(orc.unpack(ls.dm.var_packed(ls.dm.packed.cpu().numpy(), i), v.size, B), E, M)
+        nz = v != 0
+        bound = np.exp2(np.maximum(np.floor(np.log2(np.abs(v[nz]))), emin) - M - 1)
+        assert np.all(np.abs(vt[nz] - v[nz]) <= bound)
+        rec = from_full(ls.plan, out, i).astype(np.float64)
+        assert np.linalg.norm(rec - v) <= np.linalg.norm(vt - v) * (1 + 1e-6)
+    for r in range(2):
+        ls.round(wl.all_grads(r), 0.01 if r == 0 else 5.0)
+    ls.check_decompress()
+
+
+@pytest.mark.parametrize("fmt", ALL_FORMATS, ids=lambda f: "E%dM%d" % f)
+def test_ragged_small_all_formats(fmt):
+    """Ragged list (sizes 1 .. a few tiles, not multiples of anything), mixed kinds, three rounds
+    with a step large enough to move codes across binades and into the subnormal range."""
+    rng = np.random.default_rng(fmt[0] * 100 + fmt[1])
+    numel = [1, 2, 3, 5, 31, 32, 33, 127, 128, 129, 1023, 1024, 1025, 2047, 4096, 5000, 3 * 1024 + 7,
+             777, 8, 16, 12289]
+    kinds = [0] * len(numel)
+    for j in (3, 9, 14):
+        kinds[j] = 1
+    E, M = fmt
+    span = min(2.0 ** ((1 << (E - 1)) - 2), 4.0)
+    params = []
+    for j, n in enumerate(numel):
+        scale = span * 10.0 ** (-(j % 6))
+        params.append((rng.standard_normal(n) * scale).astype(np.float32))
+    ls = Lockstep(numel, kinds, fmt, params)
+    packed = ls.check_state("compress-again", resync=False)
+    ls.check_padding(packed)
+    ls.check_decompress()
+    ls.check_decompress(first=4, count=9)
+    for r in range(3):
+        grads = [(rng.standard_normal(n) * 0.3 * span * 10.0 ** (-(j % 6))).astype(np.float32)
+                 for j, n in enumerate(numel)]
+        packed = ls.round(grads, [0.01, 1.0, 0.5][r])
+        ls.check_padding(packed)
+    ls.check_decompress()
+    assert ls.sb_ulp_cases <= 3, ls.sb_ulp_cases
+
+
+@pytest.mark.parametrize("fmt", [(5, 2), (5, 6), (5, 10), (4, 3), (3, 7), (8, 7), (2, 3)],
+                         ids=lambda f: "E%dM%d" % f)
+def test_special_values(fmt):
+    """Zeros of both signs, FP32 subnormals, ties, the overflow threshold, infinities and NaNs with
+    payloads, a constant variable, a one-element variable."""
+    E, M = fmt
+    bias = (1 << (E - 1)) - 1
+    emin, emax = 1 - bias, bias
+    tiny = 2.0 ** (emin - M)
+    top = 2.0 ** emax * (2 - 2.0 ** -M)
+    thr = 2.0 ** emax * (2 - 2.0 ** -(M + 1))
+    f32 = np.float32
+    specials = np.array([0.0, -0.0, 1e-45, -1e-45, 1e-40, tiny, tiny / 2, -tiny / 2, 1.5 * tiny, 2.5 * tiny,
+                         np.nextafter(f32(tiny / 2), f32(1)), 2.0 ** emin, np.nextafter(f32(2.0 ** emin), f32(0)),
+                         1.0, 1 + 2.0 ** -(M + 1), 1 + 3 * 2.0 ** -(M + 1), np.nextafter(f32(2.0), f32(0)),
+                         min(top, 3.4e38), min(thr, 3.4e38), np.nextafter(f32(min(thr, 3.4e38)), f32(0)),
+                         -min(thr, 3.4e38), 3.4028235e38, -3.4028235e38, np.inf, -np.inf], np.float32)
+    nans = np.array([0x7FC00000, 0xFFC00000, 0x7F800001, 0xFF800001, 0x7FFFFFFF, 0x7FA00000, 0x7F801000],
+                    np.uint32).view(np.float32)
+    rng = np.random.default_rng(5)
+    body = (rng.standard_normal(3000) * 0.05).astype(np.float32)
+    v_finite = np.concatenate([specials[:-4], body])           # no Inf/NaN: the fit stays finite
+    v_inf = np.concatenate([specials, body[:100]])
+    v_nan = np.concatenate([nans, body[:200]])
+    v_const = np.full(1500, 0.3, np.float32)
+    v_cell = np.linspace(0.26, 0.2600001, 700).astype(np.float32)       # one quantisation cell
+    v_one = np.array([0.7], np.float32)
+    v_zero = np.zeros(130, np.float32)
+    v_pm0 = np.array([0.0, -0.0] * 40, np.float32)
+    params = [v_finite, v_inf, v_nan, v_const, v_cell, v_one, v_zero, v_pm0, body]
+    numel = [p.size for p in params]
+    ls = Lockstep(numel, [0] * len(numel), fmt, params)
+    ls.check_decompress()
+    grads = [(rng.standard_normal(n) * 0.05).astype(np.float32) for n in numel]
+    grads[0][:8] = [np.inf, -np.inf, np.nan, 1e38, -1e38, 0.0, -0.0, 1e-45]
+    ls.round(grads, 1.0)
+    ls.check_decompress()
+    grads = [(rng.standard_normal(n) * 0.05).astype(np.float32) for n in numel]
+    ls.round(grads, 0.5)
+    ls.check_decompress()
+
+
+def test_plan_switches():
+    """Per-variable transformation off (s = 1, b = 0 stay put), weights-only off, explicit mask."""
+    wl = workloads.tiny()
+    params = wl.all_params()
+    ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params, flags=omc.PLAN_WEIGHTS_ONLY)
+    _, _, sb = ls.dm.host_state()
+    assert np.array_equal(sb[:8], np.array([1, 0] * 4, np.float32))
+    ls.round(wl.all_grads(0), 10.0)
+    ls.check_decompress()
+    ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params, flags=omc.PLAN_PVT)
+    assert all(ls.plan.quantised)
+    ls.round(wl.all_grads(0), 10.0)
+    ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params, mask=[1, 0, 0, 0, 0, 0, 1, 0])
+    assert sum(ls.plan.quantised) == 2
+    ls.round(wl.all_grads(0), 10.0)
+    ls.check_decompress()
+
+
+def test_repeatable_and_workspace_reuse():
+    """Two runs from the same state give identical bytes; the workspace needs no clearing between
+    calls; a second plan with its own workspace is independent."""
+    wl = workloads.ragged(nvars=300, hi=30000)
+    params = wl.all_params()
+    plan = omc.Plan(wl.numel, wl.kinds, wl.fmt)
+    outs = []
+    for rep in range(2):
+        dm = DeviceModel(plan)
+        dm.compress(dm.upload_full(params))
+        for r in range(3):
+            dm.update(dm.upload_full(wl.all_grads(r)), 0.5)
+        outs.append(dm.host_state())
+    for a, b in zip(*outs):
+        assert np.array_equal(a.view(np.uint8), b.view(np.uint8))
+
+
+def test_device_call_argument_errors():
+    wl = workloads.tiny()
+    plan = omc.Plan(wl.numel, wl.kinds, wl.fmt)
+    dm = DeviceModel(plan)
+    L = omc.lib()
+    h, ws, pk, rs, sb = plan._h, dm.ws.data_ptr(), dm.packed.data_ptr(), dm.resid.data_ptr(), dm.sb.data_ptr()
+    full = torch.zeros(plan.full_elems, device="cuda")
+    assert L.omc_compress(h, None, pk, rs, sb, ws, None) == -3
+    assert L.omc_compress(h, full.data_ptr() + 4, pk, rs, sb, ws, None) == -4
+    assert L.omc_decompress(h, pk, rs, sb, 0, 0, full.data_ptr(), None) == -1
+    assert L.omc_decompress(h, pk, rs, sb, 7, 2, full.data_ptr(), None) == -1
+    assert L.omc_decompress(h, pk, rs, sb, 0, 8, None, None) == -3
+    assert L.omc_update_recompress(h, pk, rs, sb, None, 0.1, None, ws, None) == -3
+    assert L.omc_update_recompress(h, pk + 8, rs, sb, full.data_ptr(), 0.1, None, ws, None) == -4
+    assert L.omc_plan_prepare(h, None, None) == -3
+    torch.cuda.synchronize()
