@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Throughput of the OMC hot path on B200: one step = one round of the fused
+decode -> SGD update -> re-encode over a whole synthetic parameter set (one kernel launch).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload conformer|large|large20|ragged|tiny]
+    python bench.py --impl reference ...      # times the CPU oracle instead (rank 0 only)
+
+Prints one JSON line.  Multi-GPU runs are independent replicas (the path has no exchange step):
+every rank runs the same workload on its own GPU; the value is all ranks' parameters over the
+slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "params/s, fused decode->update->re-encode"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per launch of the fused kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by workload name; None until a capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def make_workload(name):
+    from paper_2205_03494_b200 import workloads
+    if name == "conformer":
+        return workloads.conformer_like()
+    if name == "large":
+        return workloads.large_transformer()
+    if name == "large20":
+        return workloads.large_transformer(layers=20)
+    if name == "ragged":
+        return workloads.ragged()
+    if name == "tiny":
+        return workloads.tiny()
+    raise SystemExit("unknown workload " + name)
+
+
+def algorithmic_bytes(plan) -> int:
+    """Bytes one fused round must move: code in + gradient in + code out per quantised parameter
+    (4 + B/4), 12 per FP32 parameter, 16 for each variable's (s, b) read and written."""
+    total = 0
+    for i, n in enumerate(plan.numel):
+        if plan.quantised[i]:
+            total += n * 4 + 2 * ((n * plan.B + 7) // 8) + 16
+        else:
+            total += 12 * n
+    return total
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            c = [x.strip() for x in r.split(",")]
+            if len(c) < 7:
+                continue
+            try:
+                sm.append(float(c[0])); mx.append(float(c[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+
+def cpu_oracle_rate(wl, threads, which, rounds=1):
+    """Parameters per second of the CPU oracle's update-recompress on variables `which`."""
+    from oracle import omc_oracle as orc
+    from paper_2205_03494_b200 import workloads  # noqa: F401
+    params = wl.all_params(which=which)
+    grads = wl.all_grads(0, which=which)
+    sel = orc.select(wl.kinds, wl.fraction, wl.sel_seed)
+    st = orc.compress(params, [bool(sel[i]) for i in which], wl.fmt[0], wl.fmt[1], True, threads)
+    n = sum(wl.numel[i] for i in which)
+    t0 = time.perf_counter()
+    for _ in range(rounds):
+        orc.update_recompress(st, grads, wl.lr, threads)
+    dt = time.perf_counter() - t0
+    return n * rounds / dt, n, dt
+
+
+def sample_vars(wl, budget_params):
+    """Leading variables of the workload up to a parameter budget (at least one)."""
+    which, tot = [], 0
+    for i, n in enumerate(wl.numel):
+        if which and tot + n > budget_params:
+            break
+        which.append(i)
+        tot += n
+    return which
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle as it stands, on the host cores, on a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2205_03494_b200.workloads import default_threads
+    wl = make_workload(args.workload)
+    threads = default_threads()
+    which = sample_vars(wl, 12_500_000)
+    from oracle import omc_oracle as orc
+    params = wl.all_params(which=which)
+    grads = wl.all_grads(0, which=which)
+    sel = orc.select(wl.kinds, wl.fraction, wl.sel_seed)
+    st = orc.compress(params, [bool(sel[i]) for i in which], wl.fmt[0], wl.fmt[1], True, threads)
+    n = sum(wl.numel[i] for i in which)
+    for _ in range(args.warmup):
+        orc.update_recompress(st, grads, wl.lr, threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.update_recompress(st, grads, wl.lr, threads)
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = "first %d variables (%d params) of %s per step" % (len(which), n, wl.name)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "params/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": "%s S1E%dM%d p=%g" % (wl.name, wl.fmt[0], wl.fmt[1], wl.fraction),
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "params/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "params/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import paper_2205_03494_b200 as omc
+    from paper_2205_03494_b200.workloads import default_threads
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl = make_workload(args.workload)
+    plan = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=wl.fraction, seed=wl.sel_seed)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def full_array(arrays, pinned=False):
+        t = torch.zeros(plan.full_elems, dtype=torch.float32, pin_memory=pinned)
+        a = t.numpy()
+        for i, x in enumerate(arrays):
+            a[plan.full_off[i]:plan.full_off[i] + plan.numel[i]] = x
+        return t
+
+    z = lambda n, dt: torch.zeros(max(int(n), 16), dtype=dt, device=dev)
+    packed, resid = z(plan.packed_bytes, torch.uint8), z(plan.resid_elems, torch.float32)
+    sb, ws = z(2 * plan.n_quantised, torch.float32), z(plan.workspace_bytes, torch.uint8)
+    plan.prepare(ws.data_ptr(), stream)
+    params = full_array(wl.all_params()).to(dev)
+    plan.compress(params.data_ptr(), packed.data_ptr(), resid.data_ptr(), sb.data_ptr(), ws.data_ptr(), stream)
+    torch.cuda.synchronize()
+    del params
+    host_grads = full_array(wl.all_grads(0), pinned=True)
+    grads = host_grads.to(dev)
+    nparams = wl.total
+    step_bytes = algorithmic_bytes(plan)
+
+    def step():
+        plan.update_recompress(packed.data_ptr(), resid.data_ptr(), sb.data_ptr(), grads.data_ptr(), wl.lr,
+                               ws.data_ptr(), None, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+
+    # ---- end to end: gradients start in pinned host memory, (s, b) is read back, every step
+    host_sb = torch.zeros(max(2 * plan.n_quantised, 1), dtype=torch.float32, pin_memory=True)
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        plan.update_recompress_host(packed.data_ptr(), resid.data_ptr(), sb.data_ptr(), host_grads.data_ptr(),
+                                    wl.lr, grads.data_ptr(), host_sb.data_ptr(), ws.data_ptr(), stream)
+
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+
+    # ---- the two other kernels, for context (not part of the step)
+    extra = {}
+    if rank == 0 and not args.no_extra:
+        out = torch.empty(plan.full_elems, dtype=torch.float32, device=dev)
+        for name, fn, nbytes in (
+            ("decompress", lambda: plan.decompress(packed.data_ptr(), resid.data_ptr(), sb.data_ptr(),
+                                                   out.data_ptr(), 0, None, stream),
+             sum((n * plan.B + 7) // 8 + 4 * n if q else 8 * n for n, q in zip(plan.numel, plan.quantised))),
+            ("compress", lambda: plan.compress(out.data_ptr(), packed.data_ptr(), resid.data_ptr(), sb.data_ptr(),
+                                               ws.data_ptr(), stream),
+             sum((n * plan.B + 7) // 8 + 4 * n if q else 8 * n for n, q in zip(plan.numel, plan.quantised))),
+        ):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            reps = 20
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            t_ms = e0.elapsed_time(e1) / reps
+            extra[name] = {"ms": t_ms, "params_per_s": nparams / (t_ms * 1e-3), "gbs": nbytes / (t_ms * 1e6)}
+
+    if dist is not None:
+        dist.barrier()
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    achieved = step_bytes / (ms_per_step * 1e6)       # GB/s
+    threads = default_threads()
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        which = list(range(len(wl.numel))) if wl.total <= 120_000_000 else sample_vars(wl, 100_000_000)
+        rate, n_s, dt = cpu_oracle_rate(wl, threads, which)
+        cpu = {"value": rate, "unit": "params/s", "cores": threads, "kind": "oracle",
+               "sample": "1 round over %d variables (%d params) of %s, %.1f s wall" % (len(which), n_s, wl.name, dt)}
+    line = {
+        "metric": METRIC, "value": world * nparams / (ms_per_step * 1e-3), "unit": "params/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "%s S1E%dM%d p=%g" % (wl.name, wl.fmt[0], wl.fmt[1], wl.fraction),
+                   "params": nparams, "variables": plan.nvars, "quantised_variables": plan.n_quantised,
+                   "bytes_per_step": step_bytes, "lr": wl.lr, "gradients": "one seeded buffer reused every step",
+                   "l2": "inputs per step (%.0f MB) exceed the 126 MB L2; no flush" % (step_bytes / 1e6),
+                   "multi_gpu": "replicas only"},
+        "hbm_gbs": achieved, "pct_of_8tbs": 100 * achieved / NOMINAL_HBM_GBS,
+        "clocks": clocks,
+        "e2e": {"value": world * nparams / (e2e_ms / e2e_steps * 1e-3), "unit": "params/s",
+                "h2d_bytes_per_step": 4 * plan.full_elems, "d2h_bytes_per_step": 8 * plan.n_quantised,
+                "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_source": peak_kind + " copy bandwidth", "kernel": "omc_kernel<UPDATE>",
+                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name)},
+        "cpu_baseline": cpu,
+        "other_kernels": extra,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="conformer")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-extra", action="store_true", help="skip timing the decompress / compress kernels")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

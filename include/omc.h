@@ -19,7 +19,7 @@
  * Memory layouts (all fixed by the plan; query them with omc_plan_sizes / omc_plan_var)
  *   full   : FP32 arena holding every variable, variable i at element offset full_off[i]; every
  *            offset is a multiple of 4 elements, the gap after a variable is padding that the
- *            library may read but never interprets.  Gradients and decompressed output use it.
+ *            library may read and overwrite but never interprets.  Gradients and decompressed output use it.
  *   resid  : FP32 arena with only the variables that stay in FP32, same alignment rule.
  *   packed : byte arena with the codes of the quantised variables.  Variable i occupies
  *            packed_bytes[i] = roundup16(ceil(numel*B/8)) bytes at packed_off[i]; inside it code k
@@ -121,6 +121,15 @@ int omc_plan_var(const omc_plan_t *plan, uint32_t i, int *quantised, uint64_t *f
 int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream);
 
 /*
+ * omc_plan_status -- waits for `stream`, then reports the plan's device status word in
+ * *host_status (host): 0 = every kernel launched with this plan so far ran to completion;
+ * non-zero = a kernel gave up waiting for one of its own asynchronous copies (its outputs are
+ * then incomplete; the context stays usable).  The kernels never wait for each other, so this
+ * is not expected to happen; the bounded wait exists so that a fault cannot hang the GPU.
+ */
+int omc_plan_status(const omc_plan_t *plan, void *stream, uint32_t *host_status);
+
+/*
  * omc_compress -- initial compression of a full-precision model (Sec. 2.2, 2.3).
  * For each quantised variable V: codes = Q(V); Vt = Q^-1(codes); (s, b) = argmin ||s*Vt+b-V||_2
  * from fp64 sums, stored FP32 (s = 1 when all Vt are equal or the denominator is 0 / not finite;
@@ -149,6 +158,16 @@ int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, const float *r
 int omc_update_recompress(const omc_plan_t *plan, uint8_t *packed, float *resid, float *sb,
                           const float *grads, float lr, float *debug_w_out, void *workspace,
                           void *stream);
+
+/*
+ * omc_update_recompress_host -- the same round (Sec. 2.1) for a caller whose gradients arrive in
+ * host memory: copies host_grads (host, full layout, pinned for full speed) into grads_staging
+ * (device, full layout), runs omc_update_recompress, copies the refitted (s, b) array back into
+ * host_sb_out (host, 2*n_quantised floats, may be NULL) and waits for `stream` before returning.
+ */
+int omc_update_recompress_host(const omc_plan_t *plan, uint8_t *packed, float *resid, float *sb,
+                               const float *host_grads, float lr, float *grads_staging,
+                               float *host_sb_out, void *workspace, void *stream);
 
 #ifdef __cplusplus
 }

@@ -19,8 +19,8 @@ PLAN_PVT, PLAN_WEIGHTS_ONLY = 1, 2
 PLAN_DEFAULT = PLAN_PVT | PLAN_WEIGHTS_ONLY
 
 EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_sizes",
-           "omc_plan_var", "omc_plan_prepare", "omc_compress", "omc_decompress",
-           "omc_update_recompress"]
+           "omc_plan_var", "omc_plan_prepare", "omc_plan_status", "omc_compress", "omc_decompress",
+           "omc_update_recompress", "omc_update_recompress_host"]
 
 
 class OmcError(RuntimeError):
@@ -62,9 +62,11 @@ def lib():
         L.omc_plan_sizes.argtypes = [vp, u64p, u64p, u64p, u32p, u64p, u64p]
         L.omc_plan_var.argtypes = [vp, C.c_uint32, C.POINTER(C.c_int), u64p, u64p, u64p, u64p, u32p]
         L.omc_plan_prepare.argtypes = [vp, vp, vp]
+        L.omc_plan_status.argtypes = [vp, vp, u32p]
         L.omc_compress.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.omc_decompress.argtypes = [vp, vp, vp, vp, C.c_uint32, C.c_uint32, vp, vp]
         L.omc_update_recompress.argtypes = [vp, vp, vp, vp, vp, C.c_float, vp, vp, vp]
+        L.omc_update_recompress_host.argtypes = [vp, vp, vp, vp, vp, C.c_float, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -131,6 +133,11 @@ class Plan:
     def prepare(self, workspace, stream=0):
         _check(lib().omc_plan_prepare(self._h, workspace, stream), "omc_plan_prepare")
 
+    def status(self, stream=0) -> int:
+        st = C.c_uint32(0)
+        _check(lib().omc_plan_status(self._h, stream, C.byref(st)), "omc_plan_status")
+        return st.value
+
     def compress(self, params, packed, resid, sb, workspace, stream=0):
         _check(lib().omc_compress(self._h, params, packed, resid, sb, workspace, stream),
                "omc_compress")
@@ -144,3 +151,9 @@ class Plan:
                           stream=0):
         _check(lib().omc_update_recompress(self._h, packed, resid, sb, grads, float(lr),
                                            debug_w_out, workspace, stream), "omc_update_recompress")
+
+    def update_recompress_host(self, packed, resid, sb, host_grads, lr, grads_staging, host_sb_out,
+                               workspace, stream=0):
+        _check(lib().omc_update_recompress_host(self._h, packed, resid, sb, host_grads, float(lr),
+                                                grads_staging, host_sb_out, workspace, stream),
+               "omc_update_recompress_host")

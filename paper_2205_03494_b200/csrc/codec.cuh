@@ -8,6 +8,7 @@
 // form that also handles Inf/NaN/overflow; callers test once per group of elements whether the
 // exact form is needed (it almost never is) instead of paying for it per element.
 #pragma once
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -37,6 +38,13 @@ struct Fmt {
     static constexpr uint32_t OVF_BITS = ovf_bits();
 };
 
+// Formats with E = 5 and M <= 10 are FP16 with the low mantissa bits dropped: code << (10-M) is
+// an IEEE half, so the hardware half conversions do the exponent work (specials included).
+template <class F>
+struct HalfPath {
+    static constexpr bool value = (F::E == 5 && F::M <= 10);
+};
+
 __device__ __forceinline__ uint32_t f2u(float x) { return __float_as_uint(x); }
 __device__ __forceinline__ float u2f(uint32_t u) { return __uint_as_float(u); }
 
@@ -49,6 +57,8 @@ __device__ __forceinline__ float decode_fast(uint32_t c)
 {
     if constexpr (F::E == 8) {
         return u2f(c << F::SH);      // S1E8Mz is FP32 with the low mantissa bits dropped
+    } else if constexpr (HalfPath<F>::value) {
+        return __half2float(__ushort_as_half((unsigned short)(c << (10 - F::M))));   // exact, all codes
     } else {
         // Put the fields where FP32 keeps them: the result has the code's exponent field as its
         // own (subnormal codes become FP32 subnormals), so one exact multiplication by
@@ -62,7 +72,7 @@ __device__ __forceinline__ float decode_fast(uint32_t c)
 template <class F>
 __device__ __forceinline__ bool code_is_special(uint32_t c)
 {
-    if constexpr (F::E == 8) return false;   // decode_fast is already exact
+    if constexpr (F::E == 8 || HalfPath<F>::value) return false;   // decode_fast is already exact
     return (c & F::MAG_MASK) >= F::INF_MAG;
 }
 
@@ -70,7 +80,7 @@ __device__ __forceinline__ bool code_is_special(uint32_t c)
 template <class F>
 __device__ __forceinline__ float decode_exact(uint32_t c)
 {
-    if constexpr (F::E < 8) {
+    if constexpr (F::E < 8 && !HalfPath<F>::value) {
         if ((c & F::MAG_MASK) >= F::INF_MAG) {
             const uint32_t m = c & ((1u << F::M) - 1u);
             return u2f(((c >> (F::E + F::M)) << 31) | 0x7F800000u | (m << F::SH));
@@ -90,6 +100,12 @@ __device__ __forceinline__ uint32_t encode_fast(float w, float &vt)
     if constexpr (F::M == 23 && F::E == 8) {
         vt = w;
         return u;
+    } else if constexpr (HalfPath<F>::value && F::M == 10) {
+        // FP16 itself: the hardware conversion rounds to nearest even, underflows gradually,
+        // overflows to infinity and turns any NaN into 0x7FFF.
+        const __half h = __float2half_rn(w);
+        vt = __half2float(h);
+        return (uint32_t)__half_as_ushort(h);
     } else if constexpr (F::E == 8) {
         // Only mantissa bits are dropped: round the FP32 pattern as an integer (a carry out of
         // the mantissa moves into the exponent, up to infinity, exactly as it should).
@@ -115,19 +131,26 @@ __device__ __forceinline__ uint32_t encode_fast(float w, float &vt)
             const float rs = __fsub_rn(__fadd_rn(a, magic), magic);
             r = (f2u(a) >= F::pow2_bits(F::EMIN)) ? a : rs;
         }
-        // r is a value of the format: rebias exactly and read the fields off the FP32 pattern.
-        const float t = __fmul_rn(r, u2f(F::pow2_bits(F::BIAS - 127)));
-        const uint32_t c = (f2u(t) >> F::SH) | ((u >> 31) << (F::E + F::M));
         vt = u2f(f2u(r) | (u & 0x80000000u));
-        return c;
+        if constexpr (HalfPath<F>::value) {
+            // r is an FP16 value with zero low mantissa bits: the half conversion is exact
+            return (uint32_t)__half_as_ushort(__float2half_rn(vt)) >> (10 - F::M);
+        } else {
+            // r is a value of the format: rebias exactly and read the fields off the FP32 pattern.
+            const float t = __fmul_rn(r, u2f(F::pow2_bits(F::BIAS - 127)));
+            return (f2u(t) >> F::SH) | ((u >> 31) << (F::E + F::M));
+        }
     }
 }
 
-// True for NaN, infinity (E < 8) and finite values that round to infinity (E < 8).
-template <class F>
+// True when encode_fast would be wrong: NaN, and for E < 8 infinity and finite values that round
+// to infinity.  KEEP_PAYLOAD = false means the caller accepts the positive all-ones NaN code for
+// any NaN input, which is what the FP16 hardware conversion produces by itself.
+template <class F, bool KEEP_PAYLOAD>
 __device__ __forceinline__ bool needs_exact_encode(float w)
 {
     const uint32_t a = f2u(w) & 0x7FFFFFFFu;
+    if constexpr (HalfPath<F>::value && F::M == 10) return KEEP_PAYLOAD ? (a > 0x7F800000u) : false;
     if constexpr (F::E == 8) return a > 0x7F800000u;
     return a >= F::OVF_BITS;
 }

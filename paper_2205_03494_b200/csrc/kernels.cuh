@@ -1,10 +1,20 @@
 // The three OMC kernels (compress, decompress, fused update-recompress) as one warp-tiled
-// template.  Work is a flat list of 1024-element tiles over all variables; the tiles are divided
-// into contiguous runs, one per warp, so that ragged variable lists load-balance and a warp keeps
-// the fit's running sums in registers across the tiles of a variable.  Per (variable, warp) one
-// partial-sum record goes to the workspace; the warp that completes a variable's last tile adds the
-// records in a fixed order and finalises (s, b) -- deterministic, no floating-point atomics, and
-// nothing ever waits on another warp.
+// template.
+//
+// Work is a flat list of 1024-element tiles over all variables; the tiles are divided into
+// contiguous runs, one per warp, so that ragged variable lists load-balance and a warp keeps the
+// fit's running sums in registers across the tiles of a variable.  Every warp is its own
+// producer/consumer pipeline: lane 0 streams the next full tile (packed codes and FP32 operand)
+// into the warp's shared-memory stage with 1-D TMA bulk copies that complete on an mbarrier while
+// the warp computes on the current stage; results leave through a bulk store from shared memory.
+// There is no block-wide barrier anywhere.  Ragged last tiles and FP32-only variables take a
+// plain path with predicated vector loads and stores.
+//
+// Per (variable, warp) one partial-sum record goes to the workspace; the warp that completes a
+// variable's last tile adds the records in a fixed order and finalises (s, b): deterministic, no
+// floating-point atomics, and no warp ever waits for another.  The only waits are on the warp's
+// own copies; they are bounded, and a wait that runs out sets the plan's status word and ends
+// the warp.
 #pragma once
 #include "codec.cuh"
 #include "omc_internal.h"
@@ -12,6 +22,9 @@
 namespace omc {
 
 enum Mode { COMPRESS = 0, DECOMPRESS = 1, UPDATE = 2 };
+
+constexpr int STAGES = 2;
+constexpr uint32_t WAIT_LIMIT = 1u << 24;   // polls of one mbarrier before giving up
 
 // How many consecutive elements one lane takes per step: the smallest run whose codes fill
 // whole 32-bit words.
@@ -21,17 +34,81 @@ struct Unit {
     static constexpr int NWORDS = LU * F::B / 32;
     static constexpr int STEP = 32 * LU;          // elements per warp step
     static constexpr int STEPS = TILE / STEP;     // steps per tile
-    static constexpr int K = STEPS < 4 ? STEPS : 4;   // steps whose loads are issued together
 };
 
+// Shared-memory budget of one warp.
+template <class F, int MODE, bool WOUT>
+struct Smem {
+    static constexpr int CB = TILE * F::B / 8;    // bytes of one tile's codes
+    static constexpr int FB = TILE * 4;           // bytes of one tile's FP32 operand
+    static constexpr int IN_C = (MODE != COMPRESS) ? CB : 0;
+    static constexpr int IN_F = (MODE != DECOMPRESS) ? FB : 0;
+    static constexpr int STAGE = IN_C + IN_F;
+    static constexpr int OUT_C = (MODE == COMPRESS) ? CB : 0;      // UPDATE rewrites the codes in place
+    static constexpr int OUT_F = (MODE == DECOMPRESS || WOUT) ? FB : 0;
+    static constexpr int PER_WARP = STAGES * STAGE + OUT_C + OUT_F;
+    static constexpr int BAR_BYTES = 128;         // WARPS_PER_CTA * STAGES mbarriers
+    static constexpr int TOTAL = BAR_BYTES + WARPS_PER_CTA * PER_WARP;
+    static_assert(WARPS_PER_CTA * STAGES * 8 <= BAR_BYTES, "");
+    static_assert(STAGE % 16 == 0 && CB % 16 == 0, "bulk copies move multiples of 16 bytes");
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers: mbarrier and 1-D bulk copies (TMA without a tensor map)
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// ---------------------------------------------------------------------------------------------
+// Running sums of the Sec. 2.3 fit.
+
 struct Acc {
-    double sx, sy, sxy, syy;
-    float mn, mx;
+    double sx, sy, sxy, syy;   // Sum W, Sum Vt, Sum W*Vt, Sum Vt^2
+    uint32_t band, bor;        // AND / OR of the bit patterns of Vt: all Vt equal <=> band == bor
     __device__ __forceinline__ void reset()
     {
         sx = sy = sxy = syy = 0.0;
-        mn = __int_as_float(0x7F800000);
-        mx = __int_as_float(0xFF800000);
+        band = 0xFFFFFFFFu;
+        bor = 0u;
     }
     // Sec. 2.3: the sums are taken in fp64; the two products are exact there (24-bit factors).
     __device__ __forceinline__ void add(float w, float vt)
@@ -41,13 +118,11 @@ struct Acc {
         sy += dv;
         sxy = fma(dw, dv, sxy);
         syy = fma(dv, dv, syy);
-        mn = fminf(mn, vt);
-        mx = fmaxf(mx, vt);
     }
     __device__ __forceinline__ void merge(const Acc &o)
     {
         sx += o.sx; sy += o.sy; sxy += o.sxy; syy += o.syy;
-        mn = fminf(mn, o.mn); mx = fmaxf(mx, o.mx);
+        band &= o.band; bor |= o.bor;
     }
     __device__ __forceinline__ void warp_reduce()
     {
@@ -58,21 +133,23 @@ struct Acc {
             o.sy = __shfl_xor_sync(0xFFFFFFFFu, sy, d);
             o.sxy = __shfl_xor_sync(0xFFFFFFFFu, sxy, d);
             o.syy = __shfl_xor_sync(0xFFFFFFFFu, syy, d);
-            o.mn = __shfl_xor_sync(0xFFFFFFFFu, mn, d);
-            o.mx = __shfl_xor_sync(0xFFFFFFFFu, mx, d);
+            o.band = __shfl_xor_sync(0xFFFFFFFFu, band, d);
+            o.bor = __shfl_xor_sync(0xFFFFFFFFu, bor, d);
             merge(o);
         }
     }
 };
 
 // Sec. 2.3 closed form from the four sums (normal equations of min ||s*Vt + b - V||), fp64 with
-// every operation rounded separately, stored as FP32.  Degenerate case: s = 1.
+// every operation rounded separately, stored as FP32.  Degenerate case (all Vt equal, which
+// includes zeros of mixed sign; or a zero / non-finite denominator): s = 1.
 __device__ __forceinline__ void fit_from_sums(const Acc &a, uint64_t n, float &s, float &b)
 {
     const double nn = (double)n;
     const double num = __dsub_rn(__dmul_rn(nn, a.sxy), __dmul_rn(a.sx, a.sy));
     const double den = __dsub_rn(__dmul_rn(nn, a.syy), __dmul_rn(a.sy, a.sy));
-    const bool degenerate = (a.mn == a.mx) || den == 0.0 || !isfinite(den);
+    const bool all_equal = (a.band == a.bor) || ((a.bor & 0x7FFFFFFFu) == 0u);
+    const bool degenerate = all_equal || den == 0.0 || !isfinite(den);
     const double s64 = degenerate ? 1.0 : __ddiv_rn(num, den);
     s = __double2float_rn(s64);
     b = __double2float_rn(__ddiv_rn(__dsub_rn(a.sx, __dmul_rn(s64, a.sy)), nn));
@@ -91,7 +168,7 @@ static __device__ __noinline__ void flush_and_maybe_finalise(Partial *slots, uin
     if (lane == 0) {
         Partial q;
         q.sx = acc.sx; q.sy = acc.sy; q.sxy = acc.sxy; q.syy = acc.syy;
-        q.mn = acc.mn; q.mx = acc.mx; q.pad[0] = q.pad[1] = 0.f;
+        q.band = acc.band; q.bor = acc.bor; q.pad[0] = q.pad[1] = 0u;
         slots[my_slot] = q;
         __threadfence();
         const uint32_t old = atomicAdd(ticket, cnt);
@@ -105,9 +182,9 @@ static __device__ __noinline__ void flush_and_maybe_finalise(Partial *slots, uin
     for (uint32_t i = lane; i < nslots; i += 32) {
         const double2 a = __ldcg(reinterpret_cast<const double2 *>(slots + i));
         const double2 c = __ldcg(reinterpret_cast<const double2 *>(slots + i) + 1);
-        const float2 m = __ldcg(reinterpret_cast<const float2 *>(slots + i) + 4);
+        const uint2 m = __ldcg(reinterpret_cast<const uint2 *>(slots + i) + 4);
         Acc o;
-        o.sx = a.x; o.sy = a.y; o.sxy = c.x; o.syy = c.y; o.mn = m.x; o.mx = m.y;
+        o.sx = a.x; o.sy = a.y; o.sxy = c.x; o.syy = c.y; o.band = m.x; o.bor = m.y;
         tot.merge(o);
     }
     tot.warp_reduce();
@@ -119,6 +196,82 @@ static __device__ __noinline__ void flush_and_maybe_finalise(Partial *slots, uin
         *ticket = 0;      // leave the workspace clean for the next launch
     }
 }
+
+// ---------------------------------------------------------------------------------------------
+// Arithmetic of one lane's unit: LU consecutive elements held in registers.
+//   win  : the unit's codes (read unless COMPRESS)       fv : the unit's FP32 operand (params / grads)
+//   wout : the unit's new codes (written unless DECOMPRESS)  fo : FP32 result (decompressed value / W)
+//   valid: number of leading elements that exist (LU except in a ragged tile)
+
+template <class F, int MODE, bool TAIL>
+__device__ __forceinline__ void compute_unit(const uint32_t (&win)[Unit<F>::NWORDS], const float4 (&fv)[Unit<F>::LU / 4],
+                                             uint32_t (&wout)[Unit<F>::NWORDS], float4 (&fo)[Unit<F>::LU / 4],
+                                             float s, float b, float neg_lr, Acc &acc, int valid)
+{
+    constexpr int LU = Unit<F>::LU, NW = Unit<F>::NWORDS;
+    constexpr bool HAS_CIN = (MODE != COMPRESS);
+    constexpr bool KEEP_PAYLOAD = (MODE == COMPRESS);    // UPDATE gives arithmetic NaNs one pattern
+#pragma unroll
+    for (int j = 0; j < NW; ++j) wout[j] = 0u;
+    uint32_t ref = 0u, diff = 0u;
+#pragma unroll
+    for (int g = 0; g < LU / 4; ++g) {
+        const float fin4[4] = {fv[g].x, fv[g].y, fv[g].z, fv[g].w};
+        uint32_t cin[4], cout[4];
+        float w[4], vt[4];
+        bool bad = false;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if constexpr (HAS_CIN) {
+                cin[j] = get_code<F, NW>(win, 4 * g + j);
+                bad |= code_is_special<F>(cin[j]);
+                const float vbar = __fmaf_rn(s, decode_fast<F>(cin[j]), b);
+                w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
+            } else {
+                w[j] = fin4[j];
+            }
+            if constexpr (MODE != DECOMPRESS) {
+                bad |= needs_exact_encode<F, KEEP_PAYLOAD>(w[j]);
+                cout[j] = encode_fast<F>(w[j], vt[j]);
+            }
+        }
+        if (bad) {   // Inf / NaN / overflow somewhere in these four: redo them carefully
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if constexpr (HAS_CIN) {
+                    const float vbar = __fmaf_rn(s, decode_exact<F>(cin[j]), b);
+                    w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
+                    // a NaN made by the arithmetic gets one fixed pattern
+                    if (MODE == UPDATE && w[j] != w[j]) w[j] = u2f(0x7FFFFFFFu);
+                }
+                if constexpr (MODE != DECOMPRESS) cout[j] = encode_exact<F>(w[j], vt[j]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const bool ok = !TAIL || (4 * g + j < valid);
+            if constexpr (MODE != DECOMPRESS) {
+                if (ok) {
+                    acc.add(w[j], vt[j]);
+                    put_code<F, NW>(wout, 4 * g + j, cout[j]);
+                    if (g == 0 && j == 0) ref = f2u(vt[0]);      // element 0 exists whenever the unit does
+                    else diff |= f2u(vt[j]) ^ ref;
+                }
+            }
+            if (TAIL && !ok) w[j] = 0.f;
+        }
+        fo[g] = make_float4(w[0], w[1], w[2], w[3]);
+    }
+    if constexpr (MODE != DECOMPRESS) {
+        if (!TAIL || valid > 0) {
+            acc.band &= ref & ~diff;
+            acc.bor |= ref | diff;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Register <-> memory moves of a unit (global or shared: the address space is inferred).
 
 template <int N>
 __device__ __forceinline__ void load_words(uint32_t (&w)[N], const uint32_t *p)
@@ -157,129 +310,85 @@ __device__ __forceinline__ void store_words(const uint32_t (&w)[N], uint32_t *p)
     }
 }
 
-// One tile of a quantised variable.  `n_rem` = elements of the variable from the tile's start on
-// (>= TILE for a full tile); `w_rem` = 32-bit words of its code stream from the tile's start on.
-template <class F, int MODE, bool WOUT, bool TAIL>
-__device__ __forceinline__ void tile_quantised(uint32_t *__restrict__ cw, const float *__restrict__ fin,
-                                               float *__restrict__ fout, uint64_t n_rem,
-                                               uint64_t w_rem, float s, float b, float neg_lr,
-                                               Acc &acc, int lane)
+// A full tile whose inputs sit in the warp's shared-memory stage.
+template <class F, int MODE, bool WOUT>
+__device__ __forceinline__ void tile_from_smem(uint32_t *s_cin, const float *s_fin, uint32_t *s_cout,
+                                               float *s_fout, float s, float b, float neg_lr, Acc &acc,
+                                               int lane)
 {
     using U = Unit<F>;
-    constexpr int LU = U::LU, NW = U::NWORDS, K = U::K;
-    constexpr bool HAS_FIN = (MODE != DECOMPRESS);
-    constexpr bool HAS_CIN = (MODE != COMPRESS);
-    constexpr bool HAS_FOUT = (MODE == DECOMPRESS) || WOUT;
-    const uint64_t n_pad = (n_rem + 3) & ~3ull;       // floats that exist in the full layout
-
+    constexpr int LU = U::LU, NW = U::NWORDS;
+    constexpr int G = U::STEPS >= 2 ? 2 : 1;      // steps whose operands are fetched together
 #pragma unroll 1
-    for (int s0 = 0; s0 < U::STEPS; s0 += K) {
-        if (TAIL && (uint64_t)s0 * U::STEP >= n_rem) break;
-        uint32_t win[K][NW];
-        float4 fv[K][LU / 4];
-        // ---- all loads of K steps first: the codes are updated in place, so the compiler could
-        //      not move a later step's loads above an earlier step's stores by itself
+    for (int k0 = 0; k0 < U::STEPS; k0 += G) {
+        uint32_t win[G][NW];
+        float4 fv[G][LU / 4];
+        // fetch first: the codes are rewritten in place, so the compiler may not move a later
+        // step's loads above an earlier step's stores by itself
 #pragma unroll
-        for (int k = 0; k < K; ++k) {
-            const uint32_t unit = (uint32_t)(s0 + k) * 32u + (uint32_t)lane;
-            const uint64_t e0 = (uint64_t)unit * LU;
-            if constexpr (HAS_CIN) {
-                if (!TAIL) {
-                    load_words<NW>(win[k], cw + (size_t)unit * NW);
-                } else {
+        for (int g = 0; g < G; ++g) {
+            const int unit = (k0 + g) * 32 + lane;
+            if constexpr (MODE != COMPRESS) load_words<NW>(win[g], s_cin + unit * NW);
+            if constexpr (MODE != DECOMPRESS) {
 #pragma unroll
-                    for (int j = 0; j < NW; ++j)
-                        win[k][j] = ((uint64_t)unit * NW + j < w_rem) ? cw[(size_t)unit * NW + j] : 0u;
-                }
-            }
-            if constexpr (HAS_FIN) {
-#pragma unroll
-                for (int j = 0; j < LU / 4; ++j) {
-                    if (!TAIL || e0 + 4 * j < n_pad)
-                        fv[k][j] = __ldcs(reinterpret_cast<const float4 *>(fin + e0) + j);
-                    else
-                        fv[k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
+                for (int j = 0; j < LU / 4; ++j) fv[g][j] = reinterpret_cast<const float4 *>(s_fin + unit * LU)[j];
             }
         }
-        // ---- compute and store
 #pragma unroll
-        for (int k = 0; k < K; ++k) {
-            const uint32_t unit = (uint32_t)(s0 + k) * 32u + (uint32_t)lane;
-            const uint64_t e0 = (uint64_t)unit * LU;
+        for (int g = 0; g < G; ++g) {
+            const int unit = (k0 + g) * 32 + lane;
             uint32_t wout[NW];
+            float4 fo[LU / 4];
+            compute_unit<F, MODE, false>(win[g], fv[g], wout, fo, s, b, neg_lr, acc, LU);
+            if constexpr (MODE != DECOMPRESS) store_words<NW>(wout, s_cout + unit * NW);
+            if constexpr (MODE == DECOMPRESS || WOUT) {
 #pragma unroll
-            for (int j = 0; j < NW; ++j) wout[j] = 0u;
-#pragma unroll
-            for (int g = 0; g < LU / 4; ++g) {
-                const float fin4[4] = {fv[k][g].x, fv[k][g].y, fv[k][g].z, fv[k][g].w};
-                uint32_t cin[4], cout[4];
-                float w[4], vt[4];
-                bool bad = false;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if constexpr (HAS_CIN) {
-                        cin[j] = get_code<F, NW>(win[k], 4 * g + j);
-                        bad |= code_is_special<F>(cin[j]);
-                        const float vbar = __fmaf_rn(s, decode_fast<F>(cin[j]), b);
-                        w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
-                    } else {
-                        w[j] = fin4[j];
-                    }
-                    if constexpr (MODE != DECOMPRESS) {
-                        bad |= needs_exact_encode<F>(w[j]);
-                        cout[j] = encode_fast<F>(w[j], vt[j]);
-                    }
-                }
-                if (bad) {   // Inf / NaN / overflow somewhere in these four: redo them carefully
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if constexpr (HAS_CIN) {
-                            const float vbar = __fmaf_rn(s, decode_exact<F>(cin[j]), b);
-                            w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
-                            // a NaN made by the arithmetic gets one fixed pattern
-                            if (MODE == UPDATE && w[j] != w[j]) w[j] = u2f(0x7FFFFFFFu);
-                        }
-                        if constexpr (MODE != DECOMPRESS) cout[j] = encode_exact<F>(w[j], vt[j]);
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const bool valid = !TAIL || (e0 + 4 * g + j < n_rem);
-                    if constexpr (MODE != DECOMPRESS) {
-                        if (valid) {
-                            acc.add(w[j], vt[j]);
-                            put_code<F, NW>(wout, 4 * g + j, cout[j]);
-                        }
-                    }
-                    if (TAIL && !valid) w[j] = 0.f;
-                }
-                if constexpr (HAS_FOUT) {
-                    if (!TAIL || e0 + 4 * g < n_pad)
-                        reinterpret_cast<float4 *>(fout + e0)[g] = make_float4(w[0], w[1], w[2], w[3]);
-                }
-            }
-            if constexpr (MODE != DECOMPRESS) {
-                if (!TAIL) {
-                    store_words<NW>(wout, cw + (size_t)unit * NW);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < NW; ++j)
-                        if ((uint64_t)unit * NW + j < w_rem) cw[(size_t)unit * NW + j] = wout[j];
-                }
+                for (int j = 0; j < LU / 4; ++j) reinterpret_cast<float4 *>(s_fout + unit * LU)[j] = fo[j];
             }
         }
     }
 }
 
-// The ragged last tile of a variable: rare, kept out of line so that it costs the main loop no
-// registers.
+// The ragged last tile of a variable, straight from and to global memory with predicated
+// accesses.  `n_rem` = elements left in the variable (< TILE); `w_rem` = 32-bit words left in
+// its padded code stream.  Rare: kept out of line so that it costs the main loop no registers.
 template <class F, int MODE, bool WOUT>
-__device__ __noinline__ Acc tile_quantised_tail(uint32_t *cw, const float *fin, float *fout, uint64_t n_rem,
-                                                uint64_t w_rem, float s, float b, float neg_lr, Acc acc,
-                                                int lane)
+__device__ __noinline__ Acc tile_ragged(uint32_t *cw, const float *fin, float *fout, uint32_t n_rem,
+                                        uint32_t w_rem, float s, float b, float neg_lr, Acc acc, int lane)
 {
-    tile_quantised<F, MODE, WOUT, true>(cw, fin, fout, n_rem, w_rem, s, b, neg_lr, acc, lane);
+    using U = Unit<F>;
+    constexpr int LU = U::LU, NW = U::NWORDS;
+    const uint32_t n_pad = (n_rem + 3u) & ~3u;       // floats that exist in the full layout
+#pragma unroll 1
+    for (int k = 0; k < U::STEPS; ++k) {
+        if ((uint32_t)k * U::STEP >= n_rem) break;
+        const uint32_t unit = (uint32_t)k * 32u + (uint32_t)lane;
+        const uint32_t e0 = unit * LU;
+        uint32_t win[NW], wout[NW];
+        float4 fv[LU / 4], fo[LU / 4];
+        if constexpr (MODE != COMPRESS) {
+#pragma unroll
+            for (int j = 0; j < NW; ++j) win[j] = (unit * NW + j < w_rem) ? cw[unit * NW + j] : 0u;
+        }
+        if constexpr (MODE != DECOMPRESS) {
+#pragma unroll
+            for (int j = 0; j < LU / 4; ++j)
+                fv[j] = (e0 + 4 * j < n_pad) ? reinterpret_cast<const float4 *>(fin + e0)[j]
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        const int valid = e0 >= n_rem ? 0 : (n_rem - e0 < (uint32_t)LU ? (int)(n_rem - e0) : LU);
+        compute_unit<F, MODE, true>(win, fv, wout, fo, s, b, neg_lr, acc, valid);
+        if constexpr (MODE != DECOMPRESS) {
+#pragma unroll
+            for (int j = 0; j < NW; ++j)
+                if (unit * NW + j < w_rem) cw[unit * NW + j] = wout[j];
+        }
+        if constexpr (MODE == DECOMPRESS || WOUT) {
+#pragma unroll
+            for (int j = 0; j < LU / 4; ++j)
+                if (e0 + 4 * j < n_pad) reinterpret_cast<float4 *>(fout + e0)[j] = fo[j];
+        }
+    }
     return acc;
 }
 
@@ -289,7 +398,7 @@ __device__ __forceinline__ void tile_resid(float *__restrict__ r, const float *_
                                            float *__restrict__ fout, uint64_t n_rem, float neg_lr,
                                            int lane)
 {
-    const uint64_t n4 = ((n_rem < (uint64_t)TILE ? n_rem : (uint64_t)TILE) + 3) / 4;   // float4s
+    const uint32_t n4 = (uint32_t)(((n_rem < (uint64_t)TILE ? n_rem : (uint64_t)TILE) + 3) / 4);   // float4s
     float4 a[TILE / 128], g[TILE / 128];
 #pragma unroll
     for (int j = 0; j < TILE / 128; ++j) {
@@ -320,12 +429,32 @@ __device__ __forceinline__ void tile_resid(float *__restrict__ r, const float *_
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+
 template <class F, int MODE, bool WOUT>
 __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams p)
 {
+    using SM = Smem<F, MODE, WOUT>;
+    extern __shared__ __align__(128) uint8_t smem_raw[];
     const int lane = threadIdx.x & 31;
-    const uint32_t warp = blockIdx.x * WARPS_PER_CTA + (threadIdx.x >> 5);
+    const int wid = threadIdx.x >> 5;
+    const uint32_t warp = blockIdx.x * WARPS_PER_CTA + wid;
     if (warp >= p.nwarps) return;
+
+    // this warp's slice of shared memory: STAGES input stages, then the output buffers
+    uint8_t *const wbase = smem_raw + SM::BAR_BYTES + wid * SM::PER_WARP;
+    uint8_t *const out_c = wbase + STAGES * SM::STAGE;
+    uint8_t *const out_f = out_c + SM::OUT_C;
+    const uint32_t bar0 = smem_addr(smem_raw) + (uint32_t)wid * STAGES * 8u;
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < STAGES; ++i) mbar_init(bar0 + 8u * i, 1u);
+        fence_mbar_init();
+        fence_proxy_async();
+    }
+    __syncwarp();
+    uint32_t k = 0;   // bulk-loaded tiles so far: tile k uses stage k % STAGES, barrier phase (k / STAGES) & 1
+
     uint64_t t = p.tile_begin + (uint64_t)warp * p.tile_count / p.nwarps;
     const uint64_t tend = p.tile_begin + (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
     // variable that holds tile t
@@ -335,7 +464,8 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
         if (__ldg(&p.vars[mid].tile_start) <= t) lo = mid; else hi = mid;
     }
     uint32_t v = lo;
-    while (t < tend) {
+    bool failed = false;
+    while (t < tend && !failed) {
         VarDev var;
         {
             const VarDev *src = p.vars + v;
@@ -359,19 +489,66 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
             }
             Acc acc;
             acc.reset();
-            uint32_t *cw_var = reinterpret_cast<uint32_t *>(p.packed + var.store_off);
-            for (uint32_t i = 0; i < cnt; ++i) {
-                const uint64_t e0 = (uint64_t)(local + i) * TILE;
-                const uint64_t w0 = e0 / 32 * F::B;              // first word of the tile's codes
-                uint32_t *cw = cw_var + w0;
-                const float *fin = (MODE != DECOMPRESS) ? p.fin + var.full_off + e0 : nullptr;
-                float *fout = ((MODE == DECOMPRESS) || WOUT) ? p.fout + var.full_off + e0 : nullptr;
-                const uint64_t n_rem = var.n - e0;
-                if (n_rem >= (uint64_t)TILE)
-                    tile_quantised<F, MODE, WOUT, false>(cw, fin, fout, n_rem, 0, s, b, p.neg_lr, acc, lane);
-                else
-                    acc = tile_quantised_tail<F, MODE, WOUT>(cw, fin, fout, n_rem, var.packed_bytes / 4 - w0,
-                                                             s, b, p.neg_lr, acc, lane);
+            uint8_t *const codes = p.packed + var.store_off;
+            const float *const fin = (MODE != DECOMPRESS) ? p.fin + var.full_off : nullptr;
+            float *const fout = (MODE == DECOMPRESS || WOUT) ? p.fout + var.full_off : nullptr;
+            // full tiles of this run: all but a ragged last tile of the variable
+            const uint32_t full_in_var = (uint32_t)(var.n / TILE);
+            const uint32_t nfull = local + cnt <= full_in_var ? cnt : full_in_var - local;
+
+            auto issue = [&](uint32_t tile, uint32_t kk) {      // lane 0 only
+                const uint32_t st = kk % STAGES;
+                const uint32_t bar = bar0 + 8u * st;
+                uint8_t *dst = wbase + st * SM::STAGE;
+                mbar_expect_tx(bar, (uint32_t)SM::STAGE);
+                if constexpr (SM::IN_C > 0)
+                    bulk_load(smem_addr(dst), codes + (size_t)tile * SM::CB, SM::CB, bar);
+                if constexpr (SM::IN_F > 0)
+                    bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)tile * TILE, SM::FB, bar);
+            };
+
+            if (nfull > 0 && lane == 0) {
+                bulk_wait_read0();             // the stage may still feed an earlier store
+                issue(local, k);
+            }
+            for (uint32_t i = 0; i < nfull; ++i, ++k) {
+                const uint32_t tile = local + i;
+                if (lane == 0) {
+                    bulk_wait_read0();         // earlier stores have left shared memory
+                    if (i + 1 < nfull) issue(tile + 1, k + 1);
+                }
+                __syncwarp();
+                // wait for this tile's bytes (bounded)
+                const uint32_t st = k % STAGES, bar = bar0 + 8u * st, parity = (k / STAGES) & 1u;
+                uint32_t polls = 0;
+                while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) {
+                    if (++polls > WAIT_LIMIT) { failed = true; break; }
+                }
+                if (failed) break;
+                uint8_t *stage = wbase + st * SM::STAGE;
+                tile_from_smem<F, MODE, WOUT>(reinterpret_cast<uint32_t *>(stage),
+                                              reinterpret_cast<const float *>(stage + SM::IN_C),
+                                              reinterpret_cast<uint32_t *>(MODE == UPDATE ? stage : out_c),
+                                              reinterpret_cast<float *>(out_f), s, b, p.neg_lr, acc, lane);
+                fence_proxy_async();           // make the results visible to the bulk store
+                __syncwarp();
+                if (lane == 0) {
+                    if constexpr (MODE != DECOMPRESS)
+                        bulk_store(codes + (size_t)tile * SM::CB, smem_addr(MODE == UPDATE ? stage : out_c), SM::CB);
+                    if constexpr (MODE == DECOMPRESS || WOUT)
+                        bulk_store(fout + (size_t)tile * TILE, smem_addr(out_f), SM::FB);
+                    bulk_commit();
+                }
+            }
+            if (failed) break;
+            if (nfull < cnt) {     // the variable's ragged last tile
+                const uint32_t tile = local + nfull;
+                const uint64_t e0 = (uint64_t)tile * TILE;
+                const uint64_t w0 = e0 / 32 * F::B;
+                acc = tile_ragged<F, MODE, WOUT>(reinterpret_cast<uint32_t *>(codes) + w0,
+                                                 fin ? fin + e0 : nullptr, fout ? fout + e0 : nullptr,
+                                                 (uint32_t)(var.n - e0), (uint32_t)(var.packed_bytes / 4 - w0),
+                                                 s, b, p.neg_lr, acc, lane);
             }
             if constexpr (MODE != DECOMPRESS) {
                 if (p.pvt) {
@@ -395,12 +572,22 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
         t += cnt;
         ++v;
     }
+    if (failed && lane == 0) atomicExch(p.status, 1u);   // a bulk load never arrived
+    if (lane == 0) bulk_wait_all();                      // stores must finish before the CTA's memory goes
 }
 
 template <class F, int MODE, bool WOUT>
 void launch(const KParams &p, int grid, void *stream)
 {
-    omc_kernel<F, MODE, WOUT><<<grid, THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    using SM = Smem<F, MODE, WOUT>;
+    static bool configured[64] = {};    // once per device and instantiation
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        cudaFuncSetAttribute(omc_kernel<F, MODE, WOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL);
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    omc_kernel<F, MODE, WOUT><<<grid, THREADS, SM::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
 }
 
 #define OMC_DEFINE_FORMAT(E_, M_)                                                               \

@@ -38,10 +38,12 @@ extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
     if (plan->d_vars && plan->device != dev) return OMC_ERR_PLAN_MISMATCH;
     if (!plan->d_vars) {
         const size_t bytes = sizeof(omc::VarDev) * (size_t)plan->nvars;
-        rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), bytes));
+        rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), bytes + 16));
         if (rc) { plan->d_vars = nullptr; return rc; }
         rc = omc::note_cuda(cudaMemcpy(plan->d_vars, plan->vars.data(), bytes, cudaMemcpyHostToDevice));
+        if (!rc) rc = omc::note_cuda(cudaMemset(plan->d_vars + plan->nvars, 0, 16));
         if (rc) { (void)cudaFree(plan->d_vars); plan->d_vars = nullptr; return rc; }
+        plan->d_status = reinterpret_cast<uint32_t *>(plan->d_vars + plan->nvars);
         plan->device = dev;
     }
     return omc::note_cuda(cudaMemsetAsync(workspace, 0, plan->ws_bytes, static_cast<cudaStream_t>(stream)));
@@ -67,6 +69,7 @@ static KParams whole_model(const omc_plan_t *plan, void *workspace)
     p.tile_count = plan->ntiles;
     p.nwarps = plan->nwarps;
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
+    p.status = plan->d_status;
     p.tickets = reinterpret_cast<uint32_t *>(static_cast<char *>(workspace) + plan->ws_tickets_off);
     p.slots = reinterpret_cast<omc::Partial *>(static_cast<char *>(workspace) + plan->ws_slots_off);
     return p;
@@ -113,6 +116,7 @@ extern "C" int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, con
     const uint64_t max_warps = (uint64_t)plan->n_cta * omc::WARPS_PER_CTA;
     p.nwarps = (uint32_t)(p.tile_count < max_warps ? p.tile_count : max_warps);
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
+    p.status = plan->d_status;
     p.packed = const_cast<uint8_t *>(packed);
     p.resid = const_cast<float *>(resid);
     p.sb = const_cast<float *>(sb);
@@ -141,4 +145,37 @@ extern "C" int omc_update_recompress(const omc_plan_t *plan, uint8_t *packed, fl
     else
         plan->ops->update(p, grid_for(p.nwarps), stream);
     return omc::note_cuda(cudaGetLastError());
+}
+
+extern "C" int omc_update_recompress_host(const omc_plan_t *plan, uint8_t *packed, float *resid, float *sb,
+                                          const float *host_grads, float lr, float *grads_staging,
+                                          float *host_sb_out, void *workspace, void *stream)
+{
+    int rc = check_ready(plan);
+    if (rc) return rc;
+    if (!host_grads || !grads_staging) return OMC_ERR_NULL_PTR;
+    if (misaligned(grads_staging)) return OMC_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = omc::note_cuda(cudaMemcpyAsync(grads_staging, host_grads, sizeof(float) * plan->full_elems,
+                                        cudaMemcpyHostToDevice, st));
+    if (rc) return rc;
+    rc = omc_update_recompress(plan, packed, resid, sb, grads_staging, lr, nullptr, workspace, stream);
+    if (rc) return rc;
+    if (host_sb_out && plan->nq) {
+        rc = omc::note_cuda(cudaMemcpyAsync(host_sb_out, sb, sizeof(float) * 2 * plan->nq,
+                                            cudaMemcpyDeviceToHost, st));
+        if (rc) return rc;
+    }
+    return omc::note_cuda(cudaStreamSynchronize(st));
+}
+
+extern "C" int omc_plan_status(const omc_plan_t *plan, void *stream, uint32_t *host_status)
+{
+    int rc = check_ready(plan);
+    if (rc) return rc;
+    if (!host_status) return OMC_ERR_NULL_PTR;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = omc::note_cuda(cudaMemcpyAsync(host_status, plan->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    if (rc) return rc;
+    return omc::note_cuda(cudaStreamSynchronize(st));
 }

@@ -33,8 +33,8 @@ static_assert(sizeof(VarDev) == 64, "VarDev is laid out for 16-byte loads");
 // Per-warp partial sums of the Sec. 2.3 fit, one slot per (variable, warp that touched it).
 struct Partial {
     double sx, sy, sxy, syy;   // Sum W, Sum Vt, Sum W*Vt, Sum Vt^2
-    float mn, mx;              // min / max of Vt (equal <=> degenerate case)
-    float pad[2];
+    uint32_t band, bor;        // AND / OR of the bit patterns of Vt (equal <=> all Vt equal)
+    uint32_t pad[2];
 };
 static_assert(sizeof(Partial) == 48, "");
 
@@ -56,6 +56,7 @@ struct KParams {
     float neg_lr;
     Partial *slots;
     uint32_t *tickets;
+    uint32_t *status;              // the plan's device status word: set non-zero if a copy never arrived
 };
 
 struct FmtOps {
@@ -82,6 +83,7 @@ struct omc_plan {
     uint64_t ws_tickets_off, ws_slots_off, ws_bytes;
     const omc::FmtOps *ops;
     // device side
-    omc::VarDev *d_vars;
+    omc::VarDev *d_vars;               // one allocation: the tables, then the status word
+    uint32_t *d_status;
     int device;                        // device the tables live on, -1 before prepare
 };

@@ -86,6 +86,7 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         pl->nvars = nvars;
         pl->ops = ops;
         pl->d_vars = nullptr;
+        pl->d_status = nullptr;
         pl->device = -1;
         const uint32_t B = 1u + fmt.exp_bits + fmt.man_bits;
 

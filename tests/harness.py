@@ -59,6 +59,7 @@ class DeviceModel:
     # ---- per-variable views on the host
     def host_state(self):
         torch.cuda.synchronize()
+        assert self.plan.status(self._s()) == 0, "a kernel gave up waiting for one of its copies"
         return (self.packed.cpu().numpy(), self.resid.cpu().numpy(), self.sb.cpu().numpy())
 
     def var_packed(self, packed_host, i):
