@@ -2,7 +2,7 @@
 """Throughput of the OMC hot path on B200: one step = one round of the fused
 decode -> SGD update -> re-encode over a whole synthetic parameter set (one kernel launch).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload conformer|large|large20|ragged|tiny]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload conformer|large|large:<layers>|ragged|tiny]
     python bench.py --impl reference ...      # times the CPU oracle instead (rank 0 only)
 
 Prints one JSON line.  Multi-GPU runs are independent replicas (the path has no exchange step):
@@ -38,8 +38,8 @@ def make_workload(name):
         return workloads.conformer_like()
     if name == "large":
         return workloads.large_transformer()
-    if name == "large20":
-        return workloads.large_transformer(layers=20)
+    if name.startswith("large:"):            # e.g. large:20 = the 20-layer cut (1,006,632,960 params)
+        return workloads.large_transformer(layers=int(name.split(":")[1]))
     if name == "ragged":
         return workloads.ragged()
     if name == "tiny":

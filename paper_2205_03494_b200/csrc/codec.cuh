@@ -143,6 +143,38 @@ __device__ __forceinline__ uint32_t encode_fast(float w, float &vt)
     }
 }
 
+// Two elements at once.  On the half path the two conversions to FP16 share one packed
+// instruction (the single-value conversion runs on a unit with a quarter of the throughput).
+template <class F>
+__device__ __forceinline__ void encode_fast2(float w0, float w1, uint32_t &c0, uint32_t &c1, float &vt0,
+                                             float &vt1)
+{
+    if constexpr (HalfPath<F>::value && F::M == 10) {
+        const __half2 h = __floats2half2_rn(w0, w1);     // low half = w0
+        const uint32_t x = *reinterpret_cast<const uint32_t *>(&h);
+        c0 = x & 0xFFFFu;
+        c1 = x >> 16;
+        vt0 = __low2float(h);
+        vt1 = __high2float(h);
+    } else if constexpr (HalfPath<F>::value && F::M <= 9) {
+        const uint32_t u0 = f2u(w0), u1 = f2u(w1);
+        const float a0 = fabsf(w0), a1 = fabsf(w1);
+        const float x0 = __fmul_rn(a0, u2f(F::pow2_bits(F::SH))), x1 = __fmul_rn(a1, u2f(F::pow2_bits(F::SH)));
+        const float m0 = u2f(max(f2u(x0) & 0x7F800000u, F::pow2_bits(F::EMIN + F::SH)));
+        const float m1 = u2f(max(f2u(x1) & 0x7F800000u, F::pow2_bits(F::EMIN + F::SH)));
+        const float r0 = __fsub_rn(__fadd_rn(a0, m0), m0), r1 = __fsub_rn(__fadd_rn(a1, m1), m1);
+        vt0 = u2f(f2u(r0) | (u0 & 0x80000000u));
+        vt1 = u2f(f2u(r1) | (u1 & 0x80000000u));
+        const __half2 h = __floats2half2_rn(vt0, vt1);   // exact: both are FP16 values
+        const uint32_t x = *reinterpret_cast<const uint32_t *>(&h);
+        c0 = (x & 0xFFFFu) >> (10 - F::M);
+        c1 = x >> (26 - F::M);
+    } else {
+        c0 = encode_fast<F>(w0, vt0);
+        c1 = encode_fast<F>(w1, vt1);
+    }
+}
+
 // True when encode_fast would be wrong: NaN, and for E < 8 infinity and finite values that round
 // to infinity.  KEEP_PAYLOAD = false means the caller accepts the positive all-ones NaN code for
 // any NaN input, which is what the FP16 hardware conversion produces by itself.

@@ -4,11 +4,11 @@
 // Work is a flat list of 1024-element tiles over all variables; the tiles are divided into
 // contiguous runs, one per warp, so that ragged variable lists load-balance and a warp keeps the
 // fit's running sums in registers across the tiles of a variable.  Every warp is its own
-// producer/consumer pipeline: lane 0 streams the next full tile (packed codes and FP32 operand)
-// into the warp's shared-memory stage with 1-D TMA bulk copies that complete on an mbarrier while
-// the warp computes on the current stage; results leave through a bulk store from shared memory.
-// There is no block-wide barrier anywhere.  Ragged last tiles and FP32-only variables take a
-// plain path with predicated vector loads and stores.
+// producer/consumer pipeline: lane 0 streams the next granule (a tile or half a tile: packed codes
+// and FP32 operand) into one of the warp's shared-memory stages with 1-D TMA bulk copies that
+// complete on an mbarrier while the warp computes on the current stage; results go to an output
+// buffer and leave through a bulk store.  There is no block-wide barrier anywhere.  Ragged ends of
+// variables and FP32-only variables take a plain path with predicated vector loads and stores.
 //
 // Per (variable, warp) one partial-sum record goes to the workspace; the warp that completes a
 // variable's last tile adds the records in a fixed order and finalises (s, b): deterministic, no
@@ -23,8 +23,16 @@ namespace omc {
 
 enum Mode { COMPRESS = 0, DECOMPRESS = 1, UPDATE = 2 };
 
-constexpr int STAGES = 2;
+constexpr int STAGES = 2;                   // input stages per warp
 constexpr uint32_t WAIT_LIMIT = 1u << 24;   // polls of one mbarrier before giving up
+
+// Build-time overrides for tuning runs: granule size and number of output buffers for all formats.
+#ifndef OMC_SUB
+#define OMC_SUB 0
+#endif
+#ifndef OMC_OUTBUFS
+#define OMC_OUTBUFS 0
+#endif
 
 // How many consecutive elements one lane takes per step: the smallest run whose codes fill
 // whole 32-bit words.
@@ -33,23 +41,33 @@ struct Unit {
     static constexpr int LU = (F::B % 8 == 0) ? 4 : (F::B % 4 == 0) ? 8 : (F::B % 2 == 0) ? 16 : 32;
     static constexpr int NWORDS = LU * F::B / 32;
     static constexpr int STEP = 32 * LU;          // elements per warp step
-    static constexpr int STEPS = TILE / STEP;     // steps per tile
+    // Pipeline granule: the elements one pair of bulk copies brings in and one bulk store takes out.
+    // 16-bit codes run best with half-tile granules and two output buffers (measured); the narrower
+    // codes, which spend more instructions per byte, with whole tiles and one buffer.
+    static constexpr int SUB_DEFAULT = (F::B == 16) ? 512 : TILE;
+    static constexpr int SUB = (OMC_SUB ? OMC_SUB : SUB_DEFAULT) > STEP ? (OMC_SUB ? OMC_SUB : SUB_DEFAULT) : STEP;
+    static constexpr int SUB_STEPS = SUB / STEP;
+    static constexpr int OUTBUFS = OMC_OUTBUFS ? OMC_OUTBUFS : (SUB < TILE ? 2 : 1);
+    static_assert(TILE % SUB == 0 && (OUTBUFS == 1 || OUTBUFS == 2), "");
 };
 
-// Shared-memory budget of one warp.
+// Shared-memory budget of one warp: STAGES input stages and OUTBUFS output buffers of one granule.
 template <class F, int MODE, bool WOUT>
 struct Smem {
-    static constexpr int CB = TILE * F::B / 8;    // bytes of one tile's codes
-    static constexpr int FB = TILE * 4;           // bytes of one tile's FP32 operand
+    static constexpr int SUB = Unit<F>::SUB;
+    static constexpr int OUTBUFS = Unit<F>::OUTBUFS;
+    static constexpr int CB = SUB * F::B / 8;     // bytes of one granule's codes
+    static constexpr int FB = SUB * 4;            // bytes of one granule's FP32 operand
     static constexpr int IN_C = (MODE != COMPRESS) ? CB : 0;
     static constexpr int IN_F = (MODE != DECOMPRESS) ? FB : 0;
     static constexpr int STAGE = IN_C + IN_F;
-    static constexpr int OUT_C = (MODE == COMPRESS) ? CB : 0;      // UPDATE rewrites the codes in place
+    static constexpr int DIST = STAGES - 1;       // granules fetched ahead
+    static constexpr int OUT_C = (MODE != DECOMPRESS) ? CB : 0;
     static constexpr int OUT_F = (MODE == DECOMPRESS || WOUT) ? FB : 0;
-    static constexpr int PER_WARP = STAGES * STAGE + OUT_C + OUT_F;
-    static constexpr int BAR_BYTES = 128;         // WARPS_PER_CTA * STAGES mbarriers
-    static constexpr int TOTAL = BAR_BYTES + WARPS_PER_CTA * PER_WARP;
-    static_assert(WARPS_PER_CTA * STAGES * 8 <= BAR_BYTES, "");
+    static constexpr int OUT = OUT_C + OUT_F;
+    static constexpr int PER_WARP = STAGES * STAGE + OUTBUFS * OUT;
+    static constexpr int BAR_PAD = (8 * STAGES * WARPS_PER_CTA + 127) / 128 * 128;   // the mbarriers
+    static constexpr int TOTAL = BAR_PAD + WARPS_PER_CTA * PER_WARP;
     static_assert(STAGE % 16 == 0 && CB % 16 == 0, "bulk copies move multiples of 16 bytes");
 };
 
@@ -96,6 +114,7 @@ __device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------------------------
@@ -230,10 +249,11 @@ __device__ __forceinline__ void compute_unit(const uint32_t (&win)[Unit<F>::NWOR
             } else {
                 w[j] = fin4[j];
             }
-            if constexpr (MODE != DECOMPRESS) {
-                bad |= needs_exact_encode<F, KEEP_PAYLOAD>(w[j]);
-                cout[j] = encode_fast<F>(w[j], vt[j]);
-            }
+            if constexpr (MODE != DECOMPRESS) bad |= needs_exact_encode<F, KEEP_PAYLOAD>(w[j]);
+        }
+        if constexpr (MODE != DECOMPRESS) {
+            encode_fast2<F>(w[0], w[1], cout[0], cout[1], vt[0], vt[1]);
+            encode_fast2<F>(w[2], w[3], cout[2], cout[3], vt[2], vt[3]);
         }
         if (bad) {   // Inf / NaN / overflow somewhere in these four: redo them carefully
 #pragma unroll
@@ -310,21 +330,20 @@ __device__ __forceinline__ void store_words(const uint32_t (&w)[N], uint32_t *p)
     }
 }
 
-// A full tile whose inputs sit in the warp's shared-memory stage.
+// A full granule (SUB elements) whose inputs sit in the warp's shared-memory stage.
 template <class F, int MODE, bool WOUT>
-__device__ __forceinline__ void tile_from_smem(uint32_t *s_cin, const float *s_fin, uint32_t *s_cout,
-                                               float *s_fout, float s, float b, float neg_lr, Acc &acc,
-                                               int lane)
+__device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const float *s_fin, uint32_t *s_cout,
+                                                  float *s_fout, float s, float b, float neg_lr, Acc &acc,
+                                                  int lane)
 {
     using U = Unit<F>;
     constexpr int LU = U::LU, NW = U::NWORDS;
-    constexpr int G = U::STEPS >= 2 ? 2 : 1;      // steps whose operands are fetched together
+    constexpr int G = (U::SUB_STEPS >= 2 && LU == 4) ? 2 : 1;   // steps whose operands are fetched together
 #pragma unroll 1
-    for (int k0 = 0; k0 < U::STEPS; k0 += G) {
+    for (int k0 = 0; k0 < U::SUB_STEPS; k0 += G) {
         uint32_t win[G][NW];
         float4 fv[G][LU / 4];
-        // fetch first: the codes are rewritten in place, so the compiler may not move a later
-        // step's loads above an earlier step's stores by itself
+        // fetch first, so that the loads of both steps are in flight before the arithmetic starts
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             const int unit = (k0 + g) * 32 + lane;
@@ -349,9 +368,9 @@ __device__ __forceinline__ void tile_from_smem(uint32_t *s_cin, const float *s_f
     }
 }
 
-// The ragged last tile of a variable, straight from and to global memory with predicated
-// accesses.  `n_rem` = elements left in the variable (< TILE); `w_rem` = 32-bit words left in
-// its padded code stream.  Rare: kept out of line so that it costs the main loop no registers.
+// The ragged end of a variable (fewer than SUB elements), straight from and to global memory
+// with predicated accesses.  `n_rem` = elements left in the variable; `w_rem` = 32-bit words left
+// in its padded code stream.  Rare: kept out of line so that it costs the main loop no registers.
 template <class F, int MODE, bool WOUT>
 __device__ __noinline__ Acc tile_ragged(uint32_t *cw, const float *fin, float *fout, uint32_t n_rem,
                                         uint32_t w_rem, float s, float b, float neg_lr, Acc acc, int lane)
@@ -360,7 +379,7 @@ __device__ __noinline__ Acc tile_ragged(uint32_t *cw, const float *fin, float *f
     constexpr int LU = U::LU, NW = U::NWORDS;
     const uint32_t n_pad = (n_rem + 3u) & ~3u;       // floats that exist in the full layout
 #pragma unroll 1
-    for (int k = 0; k < U::STEPS; ++k) {
+    for (int k = 0; k < U::SUB_STEPS; ++k) {
         if ((uint32_t)k * U::STEP >= n_rem) break;
         const uint32_t unit = (uint32_t)k * 32u + (uint32_t)lane;
         const uint32_t e0 = unit * LU;
@@ -442,9 +461,8 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
     if (warp >= p.nwarps) return;
 
     // this warp's slice of shared memory: STAGES input stages, then the output buffers
-    uint8_t *const wbase = smem_raw + SM::BAR_BYTES + wid * SM::PER_WARP;
-    uint8_t *const out_c = wbase + STAGES * SM::STAGE;
-    uint8_t *const out_f = out_c + SM::OUT_C;
+    uint8_t *const wbase = smem_raw + SM::BAR_PAD + wid * SM::PER_WARP;
+    uint8_t *const outs = wbase + STAGES * SM::STAGE;
     const uint32_t bar0 = smem_addr(smem_raw) + (uint32_t)wid * STAGES * 8u;
     if (lane == 0) {
 #pragma unroll
@@ -453,7 +471,8 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
         fence_proxy_async();
     }
     __syncwarp();
-    uint32_t k = 0;   // bulk-loaded tiles so far: tile k uses stage k % STAGES, barrier phase (k / STAGES) & 1
+    uint32_t k = 0;   // granules so far: granule k uses stage k % STAGES (barrier phase (k / STAGES) & 1)
+                      // and output buffer k % OUTBUFS
 
     uint64_t t = p.tile_begin + (uint64_t)warp * p.tile_count / p.nwarps;
     const uint64_t tend = p.tile_begin + (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
@@ -492,33 +511,37 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
             uint8_t *const codes = p.packed + var.store_off;
             const float *const fin = (MODE != DECOMPRESS) ? p.fin + var.full_off : nullptr;
             float *const fout = (MODE == DECOMPRESS || WOUT) ? p.fout + var.full_off : nullptr;
-            // full tiles of this run: all but a ragged last tile of the variable
-            const uint32_t full_in_var = (uint32_t)(var.n / TILE);
-            const uint32_t nfull = local + cnt <= full_in_var ? cnt : full_in_var - local;
+            // this run's elements of the variable: whole granules through the pipeline, the rest
+            // (only at the variable's end) through the predicated path
+            constexpr uint32_t SUB = Unit<F>::SUB;
+            const uint64_t e_begin = (uint64_t)local * TILE;
+            const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
+            const uint32_t g0 = (uint32_t)(e_begin / SUB);                  // first granule
+            const uint32_t ng = (uint32_t)((e_end - e_begin) / SUB);        // whole granules
 
-            auto issue = [&](uint32_t tile, uint32_t kk) {      // lane 0 only
+            auto issue = [&](uint32_t g, uint32_t kk) {          // lane 0 only
                 const uint32_t st = kk % STAGES;
                 const uint32_t bar = bar0 + 8u * st;
                 uint8_t *dst = wbase + st * SM::STAGE;
                 mbar_expect_tx(bar, (uint32_t)SM::STAGE);
                 if constexpr (SM::IN_C > 0)
-                    bulk_load(smem_addr(dst), codes + (size_t)tile * SM::CB, SM::CB, bar);
+                    bulk_load(smem_addr(dst), codes + (size_t)g * SM::CB, SM::CB, bar);
                 if constexpr (SM::IN_F > 0)
-                    bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)tile * TILE, SM::FB, bar);
+                    bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)g * SUB, SM::FB, bar);
             };
 
-            if (nfull > 0 && lane == 0) {
-                bulk_wait_read0();             // the stage may still feed an earlier store
-                issue(local, k);
+            if (lane == 0) {
+                for (uint32_t i = 0; i < (uint32_t)SM::DIST && i < ng; ++i) issue(g0 + i, k + i);
             }
-            for (uint32_t i = 0; i < nfull; ++i, ++k) {
-                const uint32_t tile = local + i;
+            for (uint32_t i = 0; i < ng; ++i, ++k) {
+                const uint32_t g = g0 + i;
                 if (lane == 0) {
-                    bulk_wait_read0();         // earlier stores have left shared memory
-                    if (i + 1 < nfull) issue(tile + 1, k + 1);
+                    if (i + SM::DIST < ng) issue(g + SM::DIST, k + SM::DIST);   // its stage was consumed last round
+                    // the output buffer written next must have left with its last store
+                    if constexpr (SM::OUTBUFS == 2) bulk_wait_read1(); else bulk_wait_read0();
                 }
                 __syncwarp();
-                // wait for this tile's bytes (bounded)
+                // wait for this granule's bytes (bounded)
                 const uint32_t st = k % STAGES, bar = bar0 + 8u * st, parity = (k / STAGES) & 1u;
                 uint32_t polls = 0;
                 while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) {
@@ -526,28 +549,28 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
                 }
                 if (failed) break;
                 uint8_t *stage = wbase + st * SM::STAGE;
-                tile_from_smem<F, MODE, WOUT>(reinterpret_cast<uint32_t *>(stage),
-                                              reinterpret_cast<const float *>(stage + SM::IN_C),
-                                              reinterpret_cast<uint32_t *>(MODE == UPDATE ? stage : out_c),
-                                              reinterpret_cast<float *>(out_f), s, b, p.neg_lr, acc, lane);
+                uint8_t *ob = outs + (k % SM::OUTBUFS) * SM::OUT;
+                granule_from_smem<F, MODE, WOUT>(reinterpret_cast<const uint32_t *>(stage),
+                                                 reinterpret_cast<const float *>(stage + SM::IN_C),
+                                                 reinterpret_cast<uint32_t *>(ob),
+                                                 reinterpret_cast<float *>(ob + SM::OUT_C), s, b, p.neg_lr, acc, lane);
                 fence_proxy_async();           // make the results visible to the bulk store
                 __syncwarp();
                 if (lane == 0) {
                     if constexpr (MODE != DECOMPRESS)
-                        bulk_store(codes + (size_t)tile * SM::CB, smem_addr(MODE == UPDATE ? stage : out_c), SM::CB);
+                        bulk_store(codes + (size_t)g * SM::CB, smem_addr(ob), SM::CB);
                     if constexpr (MODE == DECOMPRESS || WOUT)
-                        bulk_store(fout + (size_t)tile * TILE, smem_addr(out_f), SM::FB);
+                        bulk_store(fout + (size_t)g * SUB, smem_addr(ob + SM::OUT_C), SM::FB);
                     bulk_commit();
                 }
             }
             if (failed) break;
-            if (nfull < cnt) {     // the variable's ragged last tile
-                const uint32_t tile = local + nfull;
-                const uint64_t e0 = (uint64_t)tile * TILE;
-                const uint64_t w0 = e0 / 32 * F::B;
+            const uint64_t e_rag = e_begin + (uint64_t)ng * SUB;
+            if (e_rag < e_end) {     // the variable's ragged end
+                const uint64_t w0 = e_rag / 32 * F::B;
                 acc = tile_ragged<F, MODE, WOUT>(reinterpret_cast<uint32_t *>(codes) + w0,
-                                                 fin ? fin + e0 : nullptr, fout ? fout + e0 : nullptr,
-                                                 (uint32_t)(var.n - e0), (uint32_t)(var.packed_bytes / 4 - w0),
+                                                 fin ? fin + e_rag : nullptr, fout ? fout + e_rag : nullptr,
+                                                 (uint32_t)(var.n - e_rag), (uint32_t)(var.packed_bytes / 4 - w0),
                                                  s, b, p.neg_lr, acc, lane);
             }
             if constexpr (MODE != DECOMPRESS) {

@@ -8,10 +8,18 @@
 
 namespace omc {
 
+// Launch shape (overridable at build time for tuning runs).
+#ifndef OMC_WARPS_PER_CTA
+#define OMC_WARPS_PER_CTA 8
+#endif
+#ifndef OMC_CTAS_PER_SM
+#define OMC_CTAS_PER_SM 2
+#endif
+
 constexpr int TILE = 1024;         // elements per tile: the unit of work a warp takes
-constexpr int WARPS_PER_CTA = 8;
+constexpr int WARPS_PER_CTA = OMC_WARPS_PER_CTA;
 constexpr int THREADS = 32 * WARPS_PER_CTA;
-constexpr int CTAS_PER_SM = 2;
+constexpr int CTAS_PER_SM = OMC_CTAS_PER_SM;
 constexpr int DEFAULT_SMS = 148;   // B200; used when no device can be queried at plan time
 
 // One per variable, in the caller's order; lives in device memory after omc_plan_prepare.
