@@ -70,7 +70,8 @@ typedef enum {
     OMC_ERR_MISALIGNED = -4,    /* a device pointer is not 16-byte aligned                     */
     OMC_ERR_PLAN_MISMATCH = -5, /* the plan was not prepared, or not for this call             */
     OMC_ERR_CUDA = -6,          /* a CUDA runtime call failed (see omc_last_cuda_error)        */
-    OMC_ERR_NO_MEMORY = -7      /* host allocation failed                                      */
+    OMC_ERR_NO_MEMORY = -7,     /* host allocation failed                                      */
+    OMC_ERR_TOO_LARGE = -8      /* beyond the fixed capacity of omc_compress_var_static        */
 } omc_status;
 
 const char *omc_strerror(int status);
@@ -168,6 +169,38 @@ int omc_update_recompress(const omc_plan_t *plan, uint8_t *packed, float *resid,
 int omc_update_recompress_host(const omc_plan_t *plan, uint8_t *packed, float *resid, float *sb,
                                const float *host_grads, float lr, float *grads_staging,
                                float *host_sb_out, void *workspace, void *stream);
+
+/*
+ * omc_compress_var_static -- compress ONE variable without a plan, a workspace or any allocation.
+ * (The paper has no counterpart: this is a convenience of this library, not part of the method.)
+ *
+ * For code that must not allocate device memory when it needs a variable compressed: a callback
+ * running while another framework owns the device's memory pool, a real-time or
+ * fragmentation-sensitive service whose buffers are all reserved at start-up, or a plug-in that is
+ * handed its input and output buffers and nothing else.  Such a caller cannot use omc_compress,
+ * because omc_plan_prepare allocates the plan's device table and the caller would have to provide a
+ * workspace.  Here the table entry, the ticket, the status word and the per-warp partial sums of
+ * the Sec. 2.3 fit live in a fixed 196,864-byte array inside the library's device image (every GPU
+ * that loads the library carries it until the process ends).  The function calls no cudaMalloc,
+ * cudaFree or other allocating routine; the result is bit-identical to omc_compress on a
+ * one-variable plan.
+ *
+ *   values  device, numel floats (readable up to the next multiple of 4), 16-byte aligned.
+ *   numel   1 .. OMC_STATIC_MAX_NUMEL; anything larger returns OMC_ERR_TOO_LARGE and does nothing.
+ *   fmt     as for omc_plan.      flags   0 or OMC_PLAN_PVT (without it s = 1, b = 0 are written).
+ *   packed  device, roundup16(ceil(numel*B/8)) bytes, 16-byte aligned; written, padding zeroed.
+ *   sb      device, 2 floats (s, b), 8-byte aligned; written.
+ *
+ * The first call on a device looks up the array's address on that device (with that device
+ * current); make that first call outside any stream capture.  All calls share the one array, which
+ * keeps the previous call's contents: each call rewrites the table entry and clears the counters it
+ * needs on `stream` before its kernel runs, so back-to-back calls on one stream are fine, but two
+ * calls whose work overlaps on the same GPU (different streams or host threads) race on the array
+ * and give wrong results.  Asynchronous like the other device calls.
+ */
+#define OMC_STATIC_MAX_NUMEL (1ull << 28)
+int omc_compress_var_static(const float *values, uint64_t numel, omc_format_t fmt, uint32_t flags,
+                            uint8_t *packed, float *sb, void *stream);
 
 #ifdef __cplusplus
 }

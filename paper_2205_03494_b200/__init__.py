@@ -20,7 +20,8 @@ PLAN_DEFAULT = PLAN_PVT | PLAN_WEIGHTS_ONLY
 
 EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_sizes",
            "omc_plan_var", "omc_plan_prepare", "omc_plan_status", "omc_compress", "omc_decompress",
-           "omc_update_recompress", "omc_update_recompress_host"]
+           "omc_update_recompress", "omc_update_recompress_host", "omc_compress_var_static"]
+STATIC_MAX_NUMEL = 1 << 28
 
 
 class OmcError(RuntimeError):
@@ -67,6 +68,7 @@ def lib():
         L.omc_decompress.argtypes = [vp, vp, vp, vp, C.c_uint32, C.c_uint32, vp, vp]
         L.omc_update_recompress.argtypes = [vp, vp, vp, vp, vp, C.c_float, vp, vp, vp]
         L.omc_update_recompress_host.argtypes = [vp, vp, vp, vp, vp, C.c_float, vp, vp, vp, vp]
+        L.omc_compress_var_static.argtypes = [vp, C.c_uint64, Format, C.c_uint32, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -157,3 +159,11 @@ class Plan:
         _check(lib().omc_update_recompress_host(self._h, packed, resid, sb, host_grads, float(lr),
                                                 grads_staging, host_sb_out, workspace, stream),
                "omc_update_recompress_host")
+
+
+def compress_var_static(values, numel, fmt, packed, sb, flags=PLAN_PVT, stream=0):
+    """omc_compress_var_static: one variable, no plan, no workspace, no allocation (addresses are
+    ints).  Raises OmcError like the other calls (status -8 = numel beyond STATIC_MAX_NUMEL)."""
+    S, E, M = (1, fmt[0], fmt[1]) if len(fmt) == 2 else fmt
+    _check(lib().omc_compress_var_static(values, int(numel), Format(S, E, M, 0), int(flags), packed, sb,
+                                         stream), "omc_compress_var_static")

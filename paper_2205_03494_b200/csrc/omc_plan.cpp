@@ -33,6 +33,7 @@ extern "C" const char *omc_strerror(int status)
         case OMC_ERR_PLAN_MISMATCH: return "plan not prepared, or not usable for this call";
         case OMC_ERR_CUDA: return "CUDA runtime error (see omc_last_cuda_error)";
         case OMC_ERR_NO_MEMORY: return "out of host memory";
+        case OMC_ERR_TOO_LARGE: return "size beyond the fixed capacity of the allocation-free entry point";
         default: return "unknown status";
     }
 }
