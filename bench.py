@@ -181,6 +181,21 @@ def run_reference(args):
     }))
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The slowest rank's time: what a multi-rank (replica) run reports."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_value(nparams: int, world: int, ms_per_step: float) -> float:
+    """Whole-job parameters per second of `world` independent replicas."""
+    return world * nparams / (ms_per_step * 1e-3)
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -247,10 +262,7 @@ def run_ours(args):
     barrier()
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, dev)
     ms_per_step = ms / args.steps
 
     # ---- end to end: gradients start in pinned host memory, (s, b) is read back, every step
@@ -269,10 +281,7 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
 
     # ---- the two other kernels, for context (not part of the step)
     extra = {}
@@ -315,7 +324,7 @@ def run_ours(args):
         cpu = {"value": rate, "unit": "params/s", "cores": threads, "kind": "oracle",
                "sample": "1 round over %d variables (%d params) of %s, %.1f s wall" % (len(which), n_s, wl.name, dt)}
     line = {
-        "metric": METRIC, "value": world * nparams / (ms_per_step * 1e-3), "unit": "params/s",
+        "metric": METRIC, "value": replica_value(nparams, world, ms_per_step), "unit": "params/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "%s S1E%dM%d p=%g" % (wl.name, wl.fmt[0], wl.fmt[1], wl.fraction),
@@ -325,7 +334,7 @@ def run_ours(args):
                    "multi_gpu": "replicas only"},
         "hbm_gbs": achieved, "pct_of_8tbs": 100 * achieved / NOMINAL_HBM_GBS,
         "clocks": clocks,
-        "e2e": {"value": world * nparams / (e2e_ms / e2e_steps * 1e-3), "unit": "params/s",
+        "e2e": {"value": replica_value(nparams, world, e2e_ms / e2e_steps), "unit": "params/s",
                 "h2d_bytes_per_step": 4 * plan.full_elems, "d2h_bytes_per_step": 8 * plan.n_quantised,
                 "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
         "gpu_launches": args.steps,
