@@ -13,6 +13,7 @@ int note_cuda(cudaError_t e);
     X(3, 9) X(4, 8) X(5, 7)          /* the 13-bit formats of Sec. 3.5.3                      */ \
     X(8, 7) X(8, 23)                 /* bfloat16 and FP32 itself                              */
 OMC_FORMAT_LIST(OMC_DECLARE_FORMAT)
+extern const FmtOps ops_dynamic;   // any other format of the family, at run time
 
 const FmtOps *find_ops(int E, int M)
 {
@@ -20,6 +21,7 @@ const FmtOps *find_ops(int E, int M)
     static const FmtOps *const table[] = {OMC_FORMAT_LIST(OMC_ADDR)};
     for (const FmtOps *o : table)
         if (o->E == E && o->M == M) return o;
+    if (E >= 2 && E <= 8 && M >= 0 && M <= 23) return &ops_dynamic;
     return nullptr;
 }
 }  // namespace omc
@@ -69,6 +71,8 @@ static KParams whole_model(const omc_plan_t *plan, void *workspace)
     p.tile_count = plan->ntiles;
     p.nwarps = plan->nwarps;
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
+    p.dyn_e = plan->fmt.exp_bits;
+    p.dyn_m = plan->fmt.man_bits;
     p.status = plan->d_status;
     p.tickets = reinterpret_cast<uint32_t *>(static_cast<char *>(workspace) + plan->ws_tickets_off);
     p.slots = reinterpret_cast<omc::Partial *>(static_cast<char *>(workspace) + plan->ws_slots_off);
@@ -116,6 +120,8 @@ extern "C" int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, con
     const uint64_t max_warps = (uint64_t)plan->n_cta * omc::WARPS_PER_CTA;
     p.nwarps = (uint32_t)(p.tile_count < max_warps ? p.tile_count : max_warps);
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
+    p.dyn_e = plan->fmt.exp_bits;
+    p.dyn_m = plan->fmt.man_bits;
     p.status = plan->d_status;
     p.packed = const_cast<uint8_t *>(packed);
     p.resid = const_cast<float *>(resid);

@@ -56,6 +56,7 @@ struct KParams {
     uint64_t tile_count;           // number of tiles covered
     uint32_t nwarps;               // warps the tiles are divided among (<= tile_count)
     uint32_t pvt;
+    uint32_t dyn_e, dyn_m;         // the format, for the kernels that take it at run time
     uint8_t *packed;
     float *resid;
     float *sb;

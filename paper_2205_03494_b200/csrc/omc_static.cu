@@ -107,6 +107,8 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     p.tile_count = tiles;
     p.nwarps = nwarps;
     p.pvt = (flags & OMC_PLAN_PVT) ? 1u : 0u;
+    p.dyn_e = fmt.exp_bits;
+    p.dyn_m = fmt.man_bits;
     p.packed = packed;
     p.resid = nullptr;
     p.sb = sb;

@@ -3,7 +3,9 @@ inputs.  Packed codes (whole arena, zero padding included), decompressed values,
 values W and the FP32 variables must be bit-exact.  (s, b) come from fp64 sums whose order the
 paper does not fix: the oracle sums exactly, the GPU in a fixed order in fp64, so the two may
 differ by one FP32 unit in the last place in rare near-midpoint cases; the tests allow that, count
-it, and then continue from the oracle's (s, b) so that a difference cannot compound.
+it, and then continue from the oracle's (s, b) so that a difference cannot compound.  For nearly
+lossless formats b is a difference of almost equal sums; there the bound is the summation error
+itself, 4 n 2^-53 mean|V|, far below anything a stored value can show.
 """
 import numpy as np
 import pytest
@@ -17,7 +19,9 @@ from harness import DeviceModel, from_full, same_f32, to_full, ulp_diff
 pytestmark = pytest.mark.gpu
 
 ALL_FORMATS = [(5, 2), (4, 3), (5, 6), (5, 10), (4, 14), (3, 7), (2, 3), (3, 9), (4, 8), (5, 7), (8, 7),
-               (8, 23)]
+               (8, 23),
+               # no compiled specialisation: these take the run-time-format kernels
+               (2, 0), (3, 2), (6, 5), (7, 22), (4, 23), (8, 10), (5, 3), (2, 23)]
 
 
 class Lockstep:
@@ -33,6 +37,7 @@ class Lockstep:
         self.idx = list(range(len(numel))) if sample is None else list(sample)
         self.threads = threads
         self.sb_ulp_cases = 0
+        self.b_cancellation_cases = 0
         self.sb_checked = 0
         # initial compression on both sides
         full = self.dm.upload_full(params)
@@ -55,6 +60,17 @@ class Lockstep:
                 for name, g, w in (("s", s, self.st["s"][k]), ("b", b, self.st["b"][k])):
                     d = ulp_diff(g, w)
                     self.sb_checked += 1
+                    if d > 1 and name == "b" and np.isfinite(g) and np.isfinite(w):
+                        # b = (Sum V - s Sum Vt)/n cancels almost completely when the code is nearly
+                        # lossless; what the fixed-order fp64 sums can differ by is then larger than
+                        # an ulp of the tiny b: 4 n 2^-53 mean|V| bounds it (worst-case summation).
+                        n = self.plan.numel[i]
+                        scale = float(np.mean(np.abs(orc.decompress_var(
+                            self.st["packed"][k], n, self.E, self.M, self.st["s"][k], self.st["b"][k]))))
+                        assert abs(float(g) - float(w)) <= 4 * n * 2.0 ** -53 * scale, (what, i, g, w, scale)
+                        self.b_cancellation_cases += 1
+                        fix.append((i, k))
+                        continue
                     assert d <= 1, "%s: %s of variable %d: gpu %r oracle %r" % (what, name, i, g, w)
                     if d:
                         self.sb_ulp_cases += 1
@@ -182,7 +198,7 @@ def test_ragged_small_all_formats(fmt):
     assert ls.sb_ulp_cases <= 3, ls.sb_ulp_cases
 
 
-@pytest.mark.parametrize("fmt", [(5, 2), (5, 6), (5, 10), (4, 3), (3, 7), (8, 7), (2, 3)],
+@pytest.mark.parametrize("fmt", [(5, 2), (5, 6), (5, 10), (4, 3), (3, 7), (8, 7), (2, 3), (6, 5), (8, 10), (3, 0)],
                          ids=lambda f: "E%dM%d" % f)
 def test_special_values(fmt):
     """Zeros of both signs, FP32 subnormals, ties, the overflow threshold, infinities and NaNs with
