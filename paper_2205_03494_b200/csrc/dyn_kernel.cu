@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(THREADS) omc_dyn_kernel(const KParams p, const
             if (MODE != DECOMPRESS) {
                 if (p.pvt) {
                     flush_and_maybe_finalise(p.slots + var.slot_base, warp - var.first_warp, var.nslots,
-                                             p.tickets + var.sb_slot, cnt, var.ntiles, var.n,
+                                             p.tickets + var.sb_slot, cnt, var.ntiles, var.n, 0x7FFFFFFFu,
                                              p.sb + 2 * var.sb_slot, acc, lane);
                 } else if (MODE == COMPRESS && local == 0 && lane == 0) {
                     p.sb[2 * var.sb_slot] = 1.f;

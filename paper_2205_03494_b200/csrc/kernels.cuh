@@ -122,7 +122,7 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 
 struct Acc {
     double sx, sy, sxy, syy;   // Sum W, Sum Vt, Sum W*Vt, Sum Vt^2
-    uint32_t band, bor;        // AND / OR of the bit patterns of Vt: all Vt equal <=> band == bor
+    uint32_t band, bor;        // AND / OR of ValuePattern(Vt): all Vt equal <=> band == bor
     __device__ __forceinline__ void reset()
     {
         sx = sy = sxy = syy = 0.0;
@@ -162,12 +162,13 @@ struct Acc {
 // Sec. 2.3 closed form from the four sums (normal equations of min ||s*Vt + b - V||), fp64 with
 // every operation rounded separately, stored as FP32.  Degenerate case (all Vt equal, which
 // includes zeros of mixed sign; or a zero / non-finite denominator): s = 1.
-__device__ __forceinline__ void fit_from_sums(const Acc &a, uint64_t n, float &s, float &b)
+__device__ __forceinline__ void fit_from_sums(const Acc &a, uint64_t n, uint32_t magnitude_mask, float &s,
+                                              float &b)
 {
     const double nn = (double)n;
     const double num = __dsub_rn(__dmul_rn(nn, a.sxy), __dmul_rn(a.sx, a.sy));
     const double den = __dsub_rn(__dmul_rn(nn, a.syy), __dmul_rn(a.sy, a.sy));
-    const bool all_equal = (a.band == a.bor) || ((a.bor & 0x7FFFFFFFu) == 0u);
+    const bool all_equal = (a.band == a.bor) || ((a.bor & magnitude_mask) == 0u);
     const bool degenerate = all_equal || den == 0.0 || !isfinite(den);
     const double s64 = degenerate ? 1.0 : __ddiv_rn(num, den);
     s = __double2float_rn(s64);
@@ -180,7 +181,8 @@ __device__ __forceinline__ void fit_from_sums(const Acc &a, uint64_t n, float &s
 static __device__ __noinline__ void flush_and_maybe_finalise(Partial *slots, uint32_t my_slot,
                                                              uint32_t nslots, uint32_t *ticket,
                                                              uint32_t cnt, uint32_t ntiles, uint64_t n,
-                                                             float *sb, Acc acc, int lane)
+                                                             uint32_t magnitude_mask, float *sb, Acc acc,
+                                                             int lane)
 {
     acc.warp_reduce();
     uint32_t last = 0;
@@ -209,12 +211,37 @@ static __device__ __noinline__ void flush_and_maybe_finalise(Partial *slots, uin
     tot.warp_reduce();
     if (lane == 0) {
         float s, b;
-        fit_from_sums(tot, n, s, b);
+        fit_from_sums(tot, n, magnitude_mask, s, b);
         sb[0] = s;
         sb[1] = b;
         *ticket = 0;      // leave the workspace clean for the next launch
     }
 }
+
+// Formats whose full units take compute_unit_pairs (two elements per register) instead of
+// compute_unit.  Measured on B200: a gain for 8-bit codes only (the 12- and 16-bit kernels are
+// no faster with it), so only S1E5M2 uses it; the switch lets a tuning build change that.
+#ifndef OMC_PAIR_PATH_BITS
+#define OMC_PAIR_PATH_BITS 8
+#endif
+template <class F>
+struct PairPath {
+    static constexpr bool value = HalfPath<F>::value && (F::B == 8 || F::B == 12 || F::B == 16) &&
+                                  (F::B <= OMC_PAIR_PATH_BITS);
+};
+
+// A 32-bit pattern that identifies the value Q^-1(code) up to the sign of zero; the fit only needs
+// to know whether all of a variable's values are equal.  Pair-path formats use the FP16 pattern in
+// both halves (so that two codes can be compared per operation), the others the FP32 pattern.
+template <class F>
+struct ValuePattern {
+    static constexpr uint32_t MAGNITUDE_MASK = PairPath<F>::value ? 0x7FFF7FFFu : 0x7FFFFFFFu;
+    __device__ static __forceinline__ uint32_t of(uint32_t code, float vt)
+    {
+        if constexpr (PairPath<F>::value) return ((code << (10 - F::M)) & 0xFFFFu) * 0x00010001u;
+        return f2u(vt);
+    }
+};
 
 // ---------------------------------------------------------------------------------------------
 // Arithmetic of one lane's unit: LU consecutive elements held in registers.
@@ -274,8 +301,9 @@ __device__ __forceinline__ void compute_unit(const uint32_t (&win)[Unit<F>::NWOR
                 if (ok) {
                     acc.add(w[j], vt[j]);
                     put_code<F, NW>(wout, 4 * g + j, cout[j]);
-                    if (g == 0 && j == 0) ref = f2u(vt[0]);      // element 0 exists whenever the unit does
-                    else diff |= f2u(vt[j]) ^ ref;
+                    const uint32_t pat = ValuePattern<F>::of(cout[j], vt[j]);
+                    if (g == 0 && j == 0) ref = pat;             // element 0 exists whenever the unit does
+                    else diff |= pat ^ ref;
                 }
             }
             if (TAIL && !ok) w[j] = 0.f;
@@ -288,6 +316,142 @@ __device__ __forceinline__ void compute_unit(const uint32_t (&win)[Unit<F>::NWOR
             acc.bor |= ref | diff;
         }
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same arithmetic for full units of the half-path formats with 8-, 12- and 16-bit codes, two
+// elements at a time: a pair lives in one register as two FP16 patterns (code << (10-M), element
+// 2p in the low half).  Byte permutes unpack and pack, and Inf/NaN/overflow are detected on the
+// packed result (exponent field 31) once per unit, which then goes to compute_unit out of line.
+// Results are identical to compute_unit.
+
+// Out-of-line entry to compute_unit for the rare unit that holds a special value, so that the
+// careful path costs the main loop neither registers nor instruction-cache space.
+template <class F, int MODE>
+__device__ __noinline__ void compute_unit_careful(const uint32_t *win_p, const float4 *fv_p, uint32_t *wout_p,
+                                                  float4 *fo_p, float s, float b, float neg_lr, Acc *acc_p)
+{
+    constexpr int LU = Unit<F>::LU, NW = Unit<F>::NWORDS;
+    uint32_t win[NW], wout[NW];
+    float4 fv[LU / 4], fo[LU / 4];
+#pragma unroll
+    for (int j = 0; j < NW; ++j) win[j] = win_p[j];
+#pragma unroll
+    for (int j = 0; j < LU / 4; ++j) fv[j] = fv_p[j];
+    Acc acc = *acc_p;
+    compute_unit<F, MODE, false>(win, fv, wout, fo, s, b, neg_lr, acc, LU);
+    *acc_p = acc;
+#pragma unroll
+    for (int j = 0; j < NW; ++j) wout_p[j] = wout[j];
+#pragma unroll
+    for (int j = 0; j < LU / 4; ++j) fo_p[j] = fo[j];
+}
+
+template <class F>
+__device__ __forceinline__ void unpack_pairs(const uint32_t (&w)[Unit<F>::NWORDS], uint32_t (&X)[Unit<F>::LU / 2])
+{
+    if constexpr (F::B == 16) {
+        X[0] = w[0]; X[1] = w[1];
+    } else if constexpr (F::B == 8) {            // a code is the top byte of its FP16 pattern
+        X[0] = __byte_perm(w[0], 0u, 0x1404);
+        X[1] = __byte_perm(w[0], 0u, 0x3424);
+    } else {                                     // B == 12: pair p is bytes 3p .. 3p+2 of the unit
+        const uint32_t t[4] = {__byte_perm(w[0], 0u, 0x2110), __byte_perm(w[0], w[1], 0x5443),
+                               __byte_perm(w[1], w[2], 0x4332), __byte_perm(w[2], 0u, 0x3221)};
+#pragma unroll
+        for (int p = 0; p < 4; ++p)              // low half: code << 4; high half: already in place
+            X[p] = ((t[p] << 4) & 0x0000FFF0u) | (t[p] & 0xFFF00000u);
+    }
+}
+
+template <class F>
+__device__ __forceinline__ void pack_pairs(const uint32_t (&Y)[Unit<F>::LU / 2], uint32_t (&w)[Unit<F>::NWORDS])
+{
+    if constexpr (F::B == 16) {
+        w[0] = Y[0]; w[1] = Y[1];
+    } else if constexpr (F::B == 8) {
+        w[0] = __byte_perm(Y[0], Y[1], 0x7531);
+    } else {                                     // B == 12: 24 bits per pair, four pairs in three words
+        uint32_t q[4];
+#pragma unroll
+        for (int p = 0; p < 4; ++p) q[p] = ((Y[p] >> 4) & 0x00000FFFu) | ((Y[p] >> 8) & 0x00FFF000u);
+        w[0] = __byte_perm(q[0], q[1], 0x4210);
+        w[1] = __byte_perm(q[1], q[2], 0x5421);
+        w[2] = __byte_perm(q[2], q[3], 0x6542);
+    }
+}
+
+template <class F, int MODE>
+__device__ __forceinline__ void compute_unit_pairs(const uint32_t (&win)[Unit<F>::NWORDS],
+                                                   const float4 (&fv)[Unit<F>::LU / 4],
+                                                   uint32_t (&wout)[Unit<F>::NWORDS], float4 (&fo)[Unit<F>::LU / 4],
+                                                   float s, float b, float neg_lr, Acc &acc)
+{
+    constexpr int LU = Unit<F>::LU, NP = LU / 2;
+    uint32_t X[NP], Y[NP];
+    float w[LU], vt[LU];
+    if constexpr (MODE != COMPRESS) unpack_pairs<F>(win, X);
+    uint32_t special = 0u;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        const float g0 = (p & 1) ? fv[p / 2].z : fv[p / 2].x, g1 = (p & 1) ? fv[p / 2].w : fv[p / 2].y;
+        if constexpr (MODE != COMPRESS) {
+            const __half2 hx = *reinterpret_cast<const __half2 *>(&X[p]);
+            const float v0 = __low2float(hx), v1 = __high2float(hx);     // exact, all codes
+            const float vb0 = __fmaf_rn(s, v0, b), vb1 = __fmaf_rn(s, v1, b);
+            w[2 * p] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, g0, vb0) : vb0;
+            w[2 * p + 1] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, g1, vb1) : vb1;
+        } else {
+            w[2 * p] = g0;
+            w[2 * p + 1] = g1;
+        }
+        if constexpr (MODE != DECOMPRESS) {
+            __half2 h;
+            if constexpr (F::M == 10) {
+                h = __floats2half2_rn(w[2 * p], w[2 * p + 1]);
+                vt[2 * p] = __low2float(h);
+                vt[2 * p + 1] = __high2float(h);
+            } else {
+                uint32_t c0, c1;                              // unused: the codes are read off Y
+                encode_fast2<F>(w[2 * p], w[2 * p + 1], c0, c1, vt[2 * p], vt[2 * p + 1]);
+                h = __floats2half2_rn(vt[2 * p], vt[2 * p + 1]);   // exact unless out of range
+            }
+            Y[p] = *reinterpret_cast<const uint32_t *>(&h);
+            special |= (Y[p] & 0x7FFF7FFFu) + 0x04000400u;    // bit 15 of a half set <=> exponent field 31
+        }
+    }
+    if constexpr (MODE != DECOMPRESS) {
+        if (special & 0x80008000u) {      // Inf, NaN or overflow in this unit: take the careful path,
+            // on copies, so that only they (and not the registers of the main path) have addresses
+            uint32_t win_c[Unit<F>::NWORDS], wout_c[Unit<F>::NWORDS];
+            float4 fv_c[LU / 4], fo_c[LU / 4];
+            Acc acc_c = acc;
+#pragma unroll
+            for (int j = 0; j < Unit<F>::NWORDS; ++j) win_c[j] = (MODE != COMPRESS) ? win[j] : 0u;
+#pragma unroll
+            for (int j = 0; j < LU / 4; ++j) fv_c[j] = fv[j];
+            compute_unit_careful<F, MODE>(win_c, fv_c, wout_c, fo_c, s, b, neg_lr, &acc_c);
+            acc = acc_c;
+#pragma unroll
+            for (int j = 0; j < Unit<F>::NWORDS; ++j) wout[j] = wout_c[j];
+#pragma unroll
+            for (int j = 0; j < LU / 4; ++j) fo[j] = fo_c[j];
+            return;
+        }
+        const uint32_t ref = __byte_perm(Y[0], 0u, 0x1010);   // element 0's pattern in both halves
+        uint32_t diff = 0u;
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            acc.add(w[2 * p], vt[2 * p]);
+            acc.add(w[2 * p + 1], vt[2 * p + 1]);
+            diff |= Y[p] ^ ref;
+        }
+        acc.band &= ref & ~diff;
+        acc.bor |= ref | diff;
+        pack_pairs<F>(Y, wout);
+    }
+#pragma unroll
+    for (int g = 0; g < LU / 4; ++g) fo[g] = make_float4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -358,7 +522,10 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
             const int unit = (k0 + g) * 32 + lane;
             uint32_t wout[NW];
             float4 fo[LU / 4];
-            compute_unit<F, MODE, false>(win[g], fv[g], wout, fo, s, b, neg_lr, acc, LU);
+            if constexpr (PairPath<F>::value)
+                compute_unit_pairs<F, MODE>(win[g], fv[g], wout, fo, s, b, neg_lr, acc);
+            else
+                compute_unit<F, MODE, false>(win[g], fv[g], wout, fo, s, b, neg_lr, acc, LU);
             if constexpr (MODE != DECOMPRESS) store_words<NW>(wout, s_cout + unit * NW);
             if constexpr (MODE == DECOMPRESS || WOUT) {
 #pragma unroll
@@ -577,7 +744,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
                 if (p.pvt) {
                     flush_and_maybe_finalise(p.slots + var.slot_base, warp - var.first_warp, var.nslots,
                                              p.tickets + var.sb_slot, cnt, var.ntiles, var.n,
-                                             p.sb + 2 * var.sb_slot, acc, lane);
+                                             ValuePattern<F>::MAGNITUDE_MASK, p.sb + 2 * var.sb_slot, acc, lane);
                 } else if (MODE == COMPRESS && local == 0 && lane == 0) {
                     p.sb[2 * var.sb_slot] = 1.f;
                     p.sb[2 * var.sb_slot + 1] = 0.f;
