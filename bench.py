@@ -307,6 +307,36 @@ def run_ours(args):
             t_ms = e0.elapsed_time(e1) / reps
             extra[name] = {"ms": t_ms, "params_per_s": nparams / (t_ms * 1e-3), "gbs": nbytes / (t_ms * 1e6)}
 
+        # re-selection between two random 90% subsets (Sec. 3.1), state A -> state B
+        pa = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=1)
+        pb = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=2)
+        if pa.n_quantised and pa.quantised != pb.quantised:
+            bufs = {}
+            for nm, pl in (("a", pa), ("b", pb)):
+                bufs[nm] = (z(pl.packed_bytes, torch.uint8), z(pl.resid_elems, torch.float32),
+                            z(2 * pl.n_quantised, torch.float32), z(pl.workspace_bytes, torch.uint8))
+                pl.prepare(bufs[nm][3].data_ptr(), stream)
+            A, Bf = bufs["a"], bufs["b"]
+            pa.compress(out.data_ptr(), A[0].data_ptr(), A[1].data_ptr(), A[2].data_ptr(), A[3].data_ptr(), stream)
+            fn = lambda: omc.transition(pa, pb, A[0].data_ptr(), A[1].data_ptr(), A[2].data_ptr(), Bf[0].data_ptr(),
+                                        Bf[1].data_ptr(), Bf[2].data_ptr(), Bf[3].data_ptr(), stream)
+            nbytes = 0
+            for n, qa, qb in zip(pa.numel, pa.quantised, pb.quantised):
+                cb = (n * pa.B + 7) // 8
+                nbytes += 2 * cb if (qa and qb) else 8 * n if not (qa or qb) else cb + 4 * n
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(20):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            t_ms = e0.elapsed_time(e1) / 20
+            extra["transition_90pct_to_90pct"] = {"ms": t_ms, "params_per_s": nparams / (t_ms * 1e-3),
+                                                  "gbs": nbytes / (t_ms * 1e6),
+                                                  "variables_changing": sum(a != b for a, b in zip(pa.quantised, pb.quantised))}
+
     if dist is not None:
         dist.barrier()
     if rank != 0:

@@ -171,6 +171,22 @@ int omc_update_recompress_host(const omc_plan_t *plan, uint8_t *packed, float *r
                                float *host_sb_out, void *workspace, void *stream);
 
 /*
+ * omc_transition -- re-selection (Sec. 2.5, Sec. 3.1: the quantised subset of weight matrices
+ * changes from round to round and from client to client).  Takes a model's state under plan `from`
+ * to its state under plan `to` in one launch.  Both plans must be prepared on the current device
+ * and describe the same variables (count, sizes) in the same format, else OMC_ERR_PLAN_MISMATCH.
+ * Per variable: quantised in both -> codes and (s, b) copied; FP32 in both -> copied; quantised only
+ * in `from` -> decompressed into resid_to (fma(s, Vt, b)); quantised only in `to` -> quantised from
+ * its FP32 values with a fresh (s, b) fit, exactly as omc_compress would.
+ *   *_from  device, state under `from`, read only.     *_to  device, state under `to`, written.
+ *   workspace_to  device, `to`'s workspace (prepared).  The two states must not overlap.
+ * Formats without a compiled specialisation return OMC_ERR_BAD_FORMAT.
+ */
+int omc_transition(const omc_plan_t *from, const omc_plan_t *to, const uint8_t *packed_from,
+                   const float *resid_from, const float *sb_from, uint8_t *packed_to, float *resid_to,
+                   float *sb_to, void *workspace_to, void *stream);
+
+/*
  * omc_compress_var_static -- compress ONE variable without a plan, a workspace or any allocation.
  * (The paper has no counterpart: this is a convenience of this library, not part of the method.)
  *

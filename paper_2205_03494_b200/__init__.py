@@ -20,7 +20,8 @@ PLAN_DEFAULT = PLAN_PVT | PLAN_WEIGHTS_ONLY
 
 EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_sizes",
            "omc_plan_var", "omc_plan_prepare", "omc_plan_status", "omc_compress", "omc_decompress",
-           "omc_update_recompress", "omc_update_recompress_host", "omc_compress_var_static"]
+           "omc_update_recompress", "omc_update_recompress_host", "omc_transition",
+           "omc_compress_var_static"]
 STATIC_MAX_NUMEL = 1 << 28
 
 
@@ -68,6 +69,7 @@ def lib():
         L.omc_decompress.argtypes = [vp, vp, vp, vp, C.c_uint32, C.c_uint32, vp, vp]
         L.omc_update_recompress.argtypes = [vp, vp, vp, vp, vp, C.c_float, vp, vp, vp]
         L.omc_update_recompress_host.argtypes = [vp, vp, vp, vp, vp, C.c_float, vp, vp, vp, vp]
+        L.omc_transition.argtypes = [vp] * 10
         L.omc_compress_var_static.argtypes = [vp, C.c_uint64, Format, C.c_uint32, vp, vp, vp]
         _lib = L
     return _lib
@@ -159,6 +161,13 @@ class Plan:
         _check(lib().omc_update_recompress_host(self._h, packed, resid, sb, host_grads, float(lr),
                                                 grads_staging, host_sb_out, workspace, stream),
                "omc_update_recompress_host")
+
+
+def transition(plan_from: Plan, plan_to: Plan, packed_from, resid_from, sb_from, packed_to, resid_to, sb_to,
+               workspace_to, stream=0):
+    """omc_transition: state under plan_from -> state under plan_to (addresses are ints)."""
+    _check(lib().omc_transition(plan_from._h, plan_to._h, packed_from, resid_from, sb_from, packed_to, resid_to,
+                                sb_to, workspace_to, stream), "omc_transition")
 
 
 def compress_var_static(values, numel, fmt, packed, sb, flags=PLAN_PVT, stream=0):

@@ -617,6 +617,107 @@ __device__ __forceinline__ void tile_resid(float *__restrict__ r, const float *_
 
 // ---------------------------------------------------------------------------------------------
 
+// The state of a warp's pipeline: its slice of shared memory, its mbarriers, how many granules it
+// has moved so far (which fixes the stage, the barrier phase and the output buffer of the next
+// one) and whether a wait ran out.
+struct WarpPipe {
+    uint8_t *wbase;
+    uint32_t bar0;
+    uint32_t k;
+    bool failed;
+};
+
+// Elements [e_begin, e_end) of one quantised variable (e_begin on a tile boundary, e_end on a tile
+// boundary or at the variable's end): whole granules through the warp's pipeline, the rest (only
+// at the variable's end) through the predicated path.  `codes`, `fin`, `fout` point at the
+// variable's first element in their arenas.
+template <class F, int MODE, bool WOUT>
+__device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, const float *fin, float *fout,
+                                             uint64_t e_begin, uint64_t e_end, uint64_t n, uint64_t packed_bytes,
+                                             float s, float b, float neg_lr, Acc &acc, int lane)
+{
+    using SM = Smem<F, MODE, WOUT>;
+    uint8_t *const wbase = pipe.wbase;
+    uint8_t *const outs = wbase + STAGES * SM::STAGE;
+    const uint32_t bar0 = pipe.bar0;
+    uint32_t k = pipe.k;
+    bool failed = false;
+    constexpr uint32_t SUB = Unit<F>::SUB;
+    const uint32_t g0 = (uint32_t)(e_begin / SUB);                  // first granule
+    const uint32_t ng = (uint32_t)((e_end - e_begin) / SUB);        // whole granules
+
+    auto issue = [&](uint32_t g, uint32_t kk) {          // lane 0 only
+        const uint32_t st = kk % STAGES;
+        const uint32_t bar = bar0 + 8u * st;
+        uint8_t *dst = wbase + st * SM::STAGE;
+        mbar_expect_tx(bar, (uint32_t)SM::STAGE);
+        if constexpr (SM::IN_C > 0)
+            bulk_load(smem_addr(dst), codes + (size_t)g * SM::CB, SM::CB, bar);
+        if constexpr (SM::IN_F > 0)
+            bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)g * SUB, SM::FB, bar);
+    };
+
+    if (lane == 0) {
+        for (uint32_t i = 0; i < (uint32_t)SM::DIST && i < ng; ++i) issue(g0 + i, k + i);
+    }
+    for (uint32_t i = 0; i < ng; ++i, ++k) {
+        const uint32_t g = g0 + i;
+        if (lane == 0) {
+            if (i + SM::DIST < ng) issue(g + SM::DIST, k + SM::DIST);   // its stage was consumed last round
+            // the output buffer written next must have left with its last store
+            if constexpr (SM::OUTBUFS == 2) bulk_wait_read1(); else bulk_wait_read0();
+        }
+        __syncwarp();
+        // wait for this granule's bytes (bounded)
+        const uint32_t st = k % STAGES, bar = bar0 + 8u * st, parity = (k / STAGES) & 1u;
+        uint32_t polls = 0;
+        while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) {
+            if (++polls > WAIT_LIMIT) { failed = true; break; }
+        }
+        if (failed) break;
+        uint8_t *stage = wbase + st * SM::STAGE;
+        uint8_t *ob = outs + (k % SM::OUTBUFS) * SM::OUT;
+        granule_from_smem<F, MODE, WOUT>(reinterpret_cast<const uint32_t *>(stage),
+                                         reinterpret_cast<const float *>(stage + SM::IN_C),
+                                         reinterpret_cast<uint32_t *>(ob),
+                                         reinterpret_cast<float *>(ob + SM::OUT_C), s, b, neg_lr, acc, lane);
+        fence_proxy_async();           // make the results visible to the bulk store
+        __syncwarp();
+        if (lane == 0) {
+            if constexpr (MODE != DECOMPRESS)
+                bulk_store(codes + (size_t)g * SM::CB, smem_addr(ob), SM::CB);
+            if constexpr (MODE == DECOMPRESS || WOUT)
+                bulk_store(fout + (size_t)g * SUB, smem_addr(ob + SM::OUT_C), SM::FB);
+            bulk_commit();
+        }
+    }
+    if (failed) { pipe.k = k; pipe.failed = true; return; }
+    const uint64_t e_rag = e_begin + (uint64_t)ng * SUB;
+    if (e_rag < e_end) {     // the variable's ragged end
+        const uint64_t w0 = e_rag / 32 * F::B;
+        acc = tile_ragged<F, MODE, WOUT>(reinterpret_cast<uint32_t *>(codes) + w0,
+                                         fin ? fin + e_rag : nullptr, fout ? fout + e_rag : nullptr,
+                                         (uint32_t)(n - e_rag), (uint32_t)(packed_bytes / 4 - w0),
+                                         s, b, neg_lr, acc, lane);
+    }
+    pipe.k = k;
+}
+
+// One table entry, through the read-only path with 16-byte loads (all lanes read the same entry).
+__device__ __forceinline__ VarDev load_var(const VarDev *src)
+{
+    VarDev var;
+    const ulonglong2 a = __ldg(reinterpret_cast<const ulonglong2 *>(src));
+    const ulonglong2 c = __ldg(reinterpret_cast<const ulonglong2 *>(src) + 1);
+    const uint4 d = __ldg(reinterpret_cast<const uint4 *>(src) + 2);
+    const uint4 e = __ldg(reinterpret_cast<const uint4 *>(src) + 3);
+    var.n = a.x; var.full_off = a.y; var.store_off = c.x; var.packed_bytes = c.y;
+    var.tile_start = ((uint64_t)d.y << 32) | d.x;
+    var.ntiles = d.z; var.quantised = d.w;
+    var.sb_slot = e.x; var.slot_base = e.y; var.first_warp = e.z; var.nslots = e.w;
+    return var;
+}
+
 template <class F, int MODE, bool WOUT>
 __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams p)
 {
@@ -628,9 +729,12 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
     if (warp >= p.nwarps) return;
 
     // this warp's slice of shared memory: STAGES input stages, then the output buffers
-    uint8_t *const wbase = smem_raw + SM::BAR_PAD + wid * SM::PER_WARP;
-    uint8_t *const outs = wbase + STAGES * SM::STAGE;
-    const uint32_t bar0 = smem_addr(smem_raw) + (uint32_t)wid * STAGES * 8u;
+    WarpPipe pipe;
+    pipe.wbase = smem_raw + SM::BAR_PAD + wid * SM::PER_WARP;
+    pipe.bar0 = smem_addr(smem_raw) + (uint32_t)wid * STAGES * 8u;
+    pipe.k = 0;
+    pipe.failed = false;
+    const uint32_t bar0 = pipe.bar0;
     if (lane == 0) {
 #pragma unroll
         for (int i = 0; i < STAGES; ++i) mbar_init(bar0 + 8u * i, 1u);
@@ -638,8 +742,6 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
         fence_proxy_async();
     }
     __syncwarp();
-    uint32_t k = 0;   // granules so far: granule k uses stage k % STAGES (barrier phase (k / STAGES) & 1)
-                      // and output buffer k % OUTBUFS
 
     uint64_t t = p.tile_begin + (uint64_t)warp * p.tile_count / p.nwarps;
     const uint64_t tend = p.tile_begin + (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
@@ -650,20 +752,8 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
         if (__ldg(&p.vars[mid].tile_start) <= t) lo = mid; else hi = mid;
     }
     uint32_t v = lo;
-    bool failed = false;
-    while (t < tend && !failed) {
-        VarDev var;
-        {
-            const VarDev *src = p.vars + v;
-            const ulonglong2 a = __ldg(reinterpret_cast<const ulonglong2 *>(src));
-            const ulonglong2 c = __ldg(reinterpret_cast<const ulonglong2 *>(src) + 1);
-            const uint4 d = __ldg(reinterpret_cast<const uint4 *>(src) + 2);
-            const uint4 e = __ldg(reinterpret_cast<const uint4 *>(src) + 3);
-            var.n = a.x; var.full_off = a.y; var.store_off = c.x; var.packed_bytes = c.y;
-            var.tile_start = ((uint64_t)d.y << 32) | d.x;
-            var.ntiles = d.z; var.quantised = d.w;
-            var.sb_slot = e.x; var.slot_base = e.y; var.first_warp = e.z; var.nslots = e.w;
-        }
+    while (t < tend && !pipe.failed) {
+        const VarDev var = load_var(p.vars + v);
         const uint32_t local = (uint32_t)(t - var.tile_start);
         const uint64_t left = tend - t;
         const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
@@ -678,68 +768,11 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
             uint8_t *const codes = p.packed + var.store_off;
             const float *const fin = (MODE != DECOMPRESS) ? p.fin + var.full_off : nullptr;
             float *const fout = (MODE == DECOMPRESS || WOUT) ? p.fout + var.full_off : nullptr;
-            // this run's elements of the variable: whole granules through the pipeline, the rest
-            // (only at the variable's end) through the predicated path
-            constexpr uint32_t SUB = Unit<F>::SUB;
             const uint64_t e_begin = (uint64_t)local * TILE;
             const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
-            const uint32_t g0 = (uint32_t)(e_begin / SUB);                  // first granule
-            const uint32_t ng = (uint32_t)((e_end - e_begin) / SUB);        // whole granules
-
-            auto issue = [&](uint32_t g, uint32_t kk) {          // lane 0 only
-                const uint32_t st = kk % STAGES;
-                const uint32_t bar = bar0 + 8u * st;
-                uint8_t *dst = wbase + st * SM::STAGE;
-                mbar_expect_tx(bar, (uint32_t)SM::STAGE);
-                if constexpr (SM::IN_C > 0)
-                    bulk_load(smem_addr(dst), codes + (size_t)g * SM::CB, SM::CB, bar);
-                if constexpr (SM::IN_F > 0)
-                    bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)g * SUB, SM::FB, bar);
-            };
-
-            if (lane == 0) {
-                for (uint32_t i = 0; i < (uint32_t)SM::DIST && i < ng; ++i) issue(g0 + i, k + i);
-            }
-            for (uint32_t i = 0; i < ng; ++i, ++k) {
-                const uint32_t g = g0 + i;
-                if (lane == 0) {
-                    if (i + SM::DIST < ng) issue(g + SM::DIST, k + SM::DIST);   // its stage was consumed last round
-                    // the output buffer written next must have left with its last store
-                    if constexpr (SM::OUTBUFS == 2) bulk_wait_read1(); else bulk_wait_read0();
-                }
-                __syncwarp();
-                // wait for this granule's bytes (bounded)
-                const uint32_t st = k % STAGES, bar = bar0 + 8u * st, parity = (k / STAGES) & 1u;
-                uint32_t polls = 0;
-                while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) {
-                    if (++polls > WAIT_LIMIT) { failed = true; break; }
-                }
-                if (failed) break;
-                uint8_t *stage = wbase + st * SM::STAGE;
-                uint8_t *ob = outs + (k % SM::OUTBUFS) * SM::OUT;
-                granule_from_smem<F, MODE, WOUT>(reinterpret_cast<const uint32_t *>(stage),
-                                                 reinterpret_cast<const float *>(stage + SM::IN_C),
-                                                 reinterpret_cast<uint32_t *>(ob),
-                                                 reinterpret_cast<float *>(ob + SM::OUT_C), s, b, p.neg_lr, acc, lane);
-                fence_proxy_async();           // make the results visible to the bulk store
-                __syncwarp();
-                if (lane == 0) {
-                    if constexpr (MODE != DECOMPRESS)
-                        bulk_store(codes + (size_t)g * SM::CB, smem_addr(ob), SM::CB);
-                    if constexpr (MODE == DECOMPRESS || WOUT)
-                        bulk_store(fout + (size_t)g * SUB, smem_addr(ob + SM::OUT_C), SM::FB);
-                    bulk_commit();
-                }
-            }
-            if (failed) break;
-            const uint64_t e_rag = e_begin + (uint64_t)ng * SUB;
-            if (e_rag < e_end) {     // the variable's ragged end
-                const uint64_t w0 = e_rag / 32 * F::B;
-                acc = tile_ragged<F, MODE, WOUT>(reinterpret_cast<uint32_t *>(codes) + w0,
-                                                 fin ? fin + e_rag : nullptr, fout ? fout + e_rag : nullptr,
-                                                 (uint32_t)(var.n - e_rag), (uint32_t)(var.packed_bytes / 4 - w0),
-                                                 s, b, p.neg_lr, acc, lane);
-            }
+            run_elements<F, MODE, WOUT>(pipe, codes, fin, fout, e_begin, e_end, var.n, var.packed_bytes, s, b,
+                                        p.neg_lr, acc, lane);
+            if (pipe.failed) break;
             if constexpr (MODE != DECOMPRESS) {
                 if (p.pvt) {
                     flush_and_maybe_finalise(p.slots + var.slot_base, warp - var.first_warp, var.nslots,
@@ -762,7 +795,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
         t += cnt;
         ++v;
     }
-    if (failed && lane == 0) atomicExch(p.status, 1u);   // a bulk load never arrived
+    if (pipe.failed && lane == 0) atomicExch(p.status, 1u);   // a bulk load never arrived
     if (lane == 0) bulk_wait_all();                      // stores must finish before the CTA's memory goes
 }
 
@@ -780,10 +813,140 @@ void launch(const KParams &p, int grid, void *stream)
     omc_kernel<F, MODE, WOUT><<<grid, THREADS, SM::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Re-selection (Sec. 3.1: the quantised subset changes from round to round): the state of a model
+// under one plan becomes its state under another plan of the same variables and format, in one
+// launch over the destination plan's tile list.  Per variable: still quantised -> its codes and
+// (s, b) are copied; still FP32 -> copied; released -> decompressed into the FP32 arena
+// (fma(s, Vt, b)); newly selected -> quantised from its FP32 values with a fresh fit.  Most bytes
+// are plain copies; the two converting cases use the predicated global-memory path.
+
+// Shared memory of the transition kernel: a warp's slice must hold either converting pipeline.
+template <class F>
+struct TransitionSmem {
+    using C = Smem<F, COMPRESS, false>;
+    using D = Smem<F, DECOMPRESS, false>;
+    static constexpr int PER_WARP = C::PER_WARP > D::PER_WARP ? C::PER_WARP : D::PER_WARP;
+    static constexpr int TOTAL = C::BAR_PAD + WARPS_PER_CTA * PER_WARP;
+};
+
+// 16-byte copy of `count` units by one warp, eight loads in flight per lane.
+__device__ __forceinline__ void warp_copy16(uint4 *__restrict__ to, const uint4 *__restrict__ from, uint64_t count,
+                                            int lane)
+{
+    uint64_t i = lane;
+    for (; i + 7 * 32 < count; i += 8 * 32) {
+        uint4 r[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r[j] = __ldcs(from + i + j * 32);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) to[i + j * 32] = r[j];
+    }
+    for (; i < count; i += 32) to[i] = __ldcs(from + i);
+}
+
+template <class F>
+__global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_transition_kernel(const KParams p)
+{
+    using TS = TransitionSmem<F>;
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    const int lane = threadIdx.x & 31;
+    const int wid = threadIdx.x >> 5;
+    const uint32_t warp = blockIdx.x * WARPS_PER_CTA + wid;
+    if (warp >= p.nwarps) return;
+    WarpPipe pipe;
+    pipe.wbase = smem_raw + TS::C::BAR_PAD + wid * TS::PER_WARP;
+    pipe.bar0 = smem_addr(smem_raw) + (uint32_t)wid * STAGES * 8u;
+    pipe.k = 0;
+    pipe.failed = false;
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < STAGES; ++i) mbar_init(pipe.bar0 + 8u * i, 1u);
+        fence_mbar_init();
+        fence_proxy_async();
+    }
+    __syncwarp();
+
+    uint64_t t = p.tile_begin + (uint64_t)warp * p.tile_count / p.nwarps;
+    const uint64_t tend = p.tile_begin + (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
+    uint32_t lo = p.var_begin, hi = p.var_end;
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (__ldg(&p.vars[mid].tile_start) <= t) lo = mid; else hi = mid;
+    }
+    uint32_t v = lo;
+    while (t < tend && !pipe.failed) {
+        const VarDev var = load_var(p.vars + v);            // where the variable goes
+        const VarDev src = load_var(p.vars_from + v);       // where it is now
+        const uint32_t local = (uint32_t)(t - var.tile_start);
+        const uint64_t left = tend - t;
+        const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
+        const uint64_t e_begin = (uint64_t)local * TILE;
+        const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
+        if (var.quantised && src.quantised) {
+            // same codes, other place: this run's share of the padded stream
+            const uint64_t b0 = e_begin / 8 * F::B;
+            const uint64_t b1 = (uint64_t)(local + cnt) == var.ntiles ? var.packed_bytes : e_end / 8 * F::B;
+            warp_copy16(reinterpret_cast<uint4 *>(p.packed + var.store_off + b0),
+                        reinterpret_cast<const uint4 *>(p.packed_from + src.store_off + b0), (b1 - b0) / 16, lane);
+            if (local == 0 && lane == 0) {
+                p.sb[2 * var.sb_slot] = p.sb_from[2 * src.sb_slot];
+                p.sb[2 * var.sb_slot + 1] = p.sb_from[2 * src.sb_slot + 1];
+            }
+        } else if (!var.quantised && !src.quantised) {
+            warp_copy16(reinterpret_cast<uint4 *>(p.resid + var.store_off + e_begin),
+                        reinterpret_cast<const uint4 *>(p.resid_from + src.store_off + e_begin),
+                        (e_end - e_begin + 3) / 4, lane);
+        } else if (src.quantised) {
+            // released: decompress into the FP32 arena
+            const float s = __ldcg(p.sb_from + 2 * src.sb_slot), b = __ldcg(p.sb_from + 2 * src.sb_slot + 1);
+            Acc none;
+            none.reset();
+            run_elements<F, DECOMPRESS, false>(pipe, const_cast<uint8_t *>(p.packed_from) + src.store_off, nullptr,
+                                               p.resid + var.store_off, e_begin, e_end, var.n, src.packed_bytes,
+                                               s, b, 0.f, none, lane);
+        } else {
+            // newly selected: quantise the FP32 values, fit (s, b)
+            Acc acc;
+            acc.reset();
+            run_elements<F, COMPRESS, false>(pipe, p.packed + var.store_off, p.resid_from + src.store_off, nullptr,
+                                             e_begin, e_end, var.n, var.packed_bytes, 1.f, 0.f, 0.f, acc, lane);
+            if (pipe.failed) break;
+            if (p.pvt) {
+                flush_and_maybe_finalise(p.slots + var.slot_base, warp - var.first_warp, var.nslots,
+                                         p.tickets + var.sb_slot, cnt, var.ntiles, var.n,
+                                         ValuePattern<F>::MAGNITUDE_MASK, p.sb + 2 * var.sb_slot, acc, lane);
+            } else if (local == 0 && lane == 0) {
+                p.sb[2 * var.sb_slot] = 1.f;
+                p.sb[2 * var.sb_slot + 1] = 0.f;
+            }
+        }
+        t += cnt;
+        ++v;
+    }
+    if (pipe.failed && lane == 0) atomicExch(p.status, 1u);
+    if (lane == 0) bulk_wait_all();
+}
+
+template <class F>
+void launch_transition(const KParams &p, int grid, void *stream)
+{
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        cudaFuncSetAttribute(omc_transition_kernel<F>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             TransitionSmem<F>::TOTAL);
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    omc_transition_kernel<F><<<grid, THREADS, TransitionSmem<F>::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
+}
+
 #define OMC_DEFINE_FORMAT(E_, M_)                                                               \
     extern const FmtOps ops_E##E_##M##M_ = {E_, M_, launch<Fmt<E_, M_>, COMPRESS, false>,       \
                                             launch<Fmt<E_, M_>, DECOMPRESS, false>,             \
                                             launch<Fmt<E_, M_>, UPDATE, false>,                 \
-                                            launch<Fmt<E_, M_>, UPDATE, true>};
+                                            launch<Fmt<E_, M_>, UPDATE, true>,                  \
+                                            launch_transition<Fmt<E_, M_>>};
 
 }  // namespace omc

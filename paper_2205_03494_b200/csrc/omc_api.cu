@@ -185,3 +185,32 @@ extern "C" int omc_plan_status(const omc_plan_t *plan, void *stream, uint32_t *h
     if (rc) return rc;
     return omc::note_cuda(cudaStreamSynchronize(st));
 }
+
+extern "C" int omc_transition(const omc_plan_t *from, const omc_plan_t *to, const uint8_t *packed_from,
+                              const float *resid_from, const float *sb_from, uint8_t *packed_to,
+                              float *resid_to, float *sb_to, void *workspace_to, void *stream)
+{
+    int rc = check_ready(from);
+    if (rc) return rc;
+    rc = check_ready(to);
+    if (rc) return rc;
+    if (from->nvars != to->nvars || from->fmt.exp_bits != to->fmt.exp_bits || from->fmt.man_bits != to->fmt.man_bits)
+        return OMC_ERR_PLAN_MISMATCH;
+    for (uint32_t i = 0; i < to->nvars; ++i)
+        if (from->vars[i].n != to->vars[i].n) return OMC_ERR_PLAN_MISMATCH;
+    if (!to->ops->transition) return OMC_ERR_BAD_FORMAT;
+    if (!workspace_to) return OMC_ERR_NULL_PTR;
+    if (from->nq && (!packed_from || !sb_from)) return OMC_ERR_NULL_PTR;
+    if (from->resid_elems && !resid_from) return OMC_ERR_NULL_PTR;
+    if (to->nq && (!packed_to || !sb_to)) return OMC_ERR_NULL_PTR;
+    if (to->resid_elems && !resid_to) return OMC_ERR_NULL_PTR;
+    if (misaligned(packed_from) || misaligned(resid_from) || misaligned(sb_from) || misaligned(packed_to) ||
+        misaligned(resid_to) || misaligned(sb_to) || misaligned(workspace_to))
+        return OMC_ERR_MISALIGNED;
+    KParams p = whole_model(to, workspace_to);
+    p.packed = packed_to; p.resid = resid_to; p.sb = sb_to;
+    p.vars_from = from->d_vars;
+    p.packed_from = packed_from; p.resid_from = resid_from; p.sb_from = sb_from;
+    to->ops->transition(p, grid_for(p.nwarps), stream);
+    return omc::note_cuda(cudaGetLastError());
+}

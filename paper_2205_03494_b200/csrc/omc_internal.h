@@ -65,6 +65,11 @@ struct KParams {
     float neg_lr;
     Partial *slots;
     uint32_t *tickets;
+    // plan-to-plan transition only: the source plan's table and state
+    const VarDev *vars_from;
+    const uint8_t *packed_from;
+    const float *resid_from;
+    const float *sb_from;
     uint32_t *status;              // the plan's device status word: set non-zero if a copy never arrived
 };
 
@@ -74,6 +79,7 @@ struct FmtOps {
     void (*decompress)(const KParams &, int grid, void *stream);
     void (*update)(const KParams &, int grid, void *stream);     // W not stored
     void (*update_w)(const KParams &, int grid, void *stream);   // W stored to fout
+    void (*transition)(const KParams &, int grid, void *stream); // plan-to-plan; NULL if unsupported
 };
 const FmtOps *find_ops(int E, int M);
 

@@ -291,3 +291,64 @@ def test_device_call_argument_errors():
     assert L.omc_update_recompress(h, pk + 8, rs, sb, full.data_ptr(), 0.1, None, ws, None) == -4
     assert L.omc_plan_prepare(h, None, None) == -3
     torch.cuda.synchronize()
+
+
+def oracle_transition(st, sel_to):
+    """The oracle's state under another selection, composed from its own operations: released
+    variables are decompressed, newly selected ones compressed, the others kept."""
+    E, M, pvt = st["E"], st["M"], st["pvt"]
+    new = {"E": E, "M": M, "pvt": pvt, "n": list(st["n"]), "sel": [bool(x) for x in sel_to],
+           "packed": {}, "s": {}, "b": {}, "fp32": {}}
+    for i, n in enumerate(st["n"]):
+        was, now = st["sel"][i], bool(sel_to[i])
+        if was and now:
+            new["packed"][i], new["s"][i], new["b"][i] = st["packed"][i], st["s"][i], st["b"][i]
+        elif not was and not now:
+            new["fp32"][i] = st["fp32"][i]
+        elif was:
+            new["fp32"][i] = orc.decompress_var(st["packed"][i], n, E, M, st["s"][i], st["b"][i])
+        else:
+            new["packed"][i], new["s"][i], new["b"][i] = orc.compress_var(st["fp32"][i], E, M, pvt)
+    return new
+
+
+@pytest.mark.parametrize("fmt", [(5, 2), (5, 6), (5, 10), (4, 14), (3, 7)], ids=lambda f: "E%dM%d" % f)
+def test_transition_between_selections(fmt):
+    """Re-selection: a round under one random subset, then the state is carried to another subset
+    (other seed, other fraction) and training continues there; every step against the oracle."""
+    rng = np.random.default_rng(99)
+    numel = [5000, 1, 1024, 70000, 333, 2048, 12289, 4096, 100, 9000, 513, 65536]
+    kinds = [0, 0, 0, 0, 1, 0, 0, 0, 2, 0, 0, 0]
+    params = [(rng.standard_normal(n) * 0.1).astype(np.float32) for n in numel]
+    ls = Lockstep(numel, kinds, fmt, params, fraction=0.5, seed=1)
+    ls.round([(rng.standard_normal(n) * 0.05).astype(np.float32) for n in numel], 1.0)
+    for frac, seed in [(0.6, 2), (1.0, 3), (0.3, 4)]:
+        plan_to = omc.Plan(numel, kinds, fmt, fraction=frac, seed=seed)
+        assert plan_to.quantised != ls.plan.quantised
+        dm_to = DeviceModel(plan_to)
+        a, b = ls.dm, dm_to
+        omc.transition(ls.plan, plan_to, a.packed.data_ptr(), a.resid.data_ptr(), a.sb.data_ptr(),
+                       b.packed.data_ptr(), b.resid.data_ptr(), b.sb.data_ptr(), b.ws.data_ptr(),
+                       torch.cuda.current_stream().cuda_stream)
+        ls.st = oracle_transition(ls.st, plan_to.quantised)
+        ls.plan, ls.dm = plan_to, dm_to
+        packed = ls.check_state("transition")
+        ls.check_padding(packed)
+        ls.check_decompress()
+        ls.round([(rng.standard_normal(n) * 0.05).astype(np.float32) for n in numel], 0.5)
+    assert ls.sb_ulp_cases <= 2
+
+
+def test_transition_refuses_mismatched_plans():
+    a = omc.Plan([100, 200], [0, 0], (5, 2))
+    b = omc.Plan([100, 201], [0, 0], (5, 2))
+    c = omc.Plan([100, 200], [0, 0], (5, 6))
+    da, db, dc = DeviceModel(a), DeviceModel(b), DeviceModel(c)
+    args = lambda x, y: (x.packed.data_ptr(), x.resid.data_ptr(), x.sb.data_ptr(), y.packed.data_ptr(),
+                         y.resid.data_ptr(), y.sb.data_ptr(), y.ws.data_ptr(), None)
+    L = omc.lib()
+    assert L.omc_transition(a._h, b._h, *args(da, db)) == -5
+    assert L.omc_transition(a._h, c._h, *args(da, dc)) == -5
+    never = omc.Plan([100, 200], [0, 0], (5, 2))
+    assert L.omc_transition(a._h, never._h, *args(da, da)) == -5
+    torch.cuda.synchronize()
