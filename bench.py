@@ -215,6 +215,10 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     wl = make_workload(args.workload)
+    if args.format:
+        wl.fmt = tuple(int(x) for x in args.format.split(","))
+    if args.fraction:
+        wl.fraction = args.fraction
     plan = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=wl.fraction, seed=wl.sel_seed)
     stream = torch.cuda.current_stream().cuda_stream
 
@@ -386,6 +390,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="conformer")
+    ap.add_argument("--format", default="", help="override the workload's format: E,M (e.g. 3,7 = S1E3M7)")
+    ap.add_argument("--fraction", type=float, default=0.0, help="override the quantised fraction of weight matrices")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-extra", action="store_true", help="skip timing the decompress / compress kernels")
     args = ap.parse_args()

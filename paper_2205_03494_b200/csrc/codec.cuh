@@ -220,10 +220,11 @@ __device__ __forceinline__ uint32_t encode_exact(float w, float &vt)
 // Codes inside a run of 32-bit words (little-endian bit stream, code i at bits [i*B, (i+1)*B)).
 // With i a compile-time constant after unrolling, every shift below is an immediate.
 
+// The code at bit position `pos` of the words (pos = i*B for code i of an array that starts at code 0).
 template <class F, int NW>
-__device__ __forceinline__ uint32_t get_code(const uint32_t (&w)[NW], int i)
+__device__ __forceinline__ uint32_t get_code_at(const uint32_t (&w)[NW], int pos)
 {
-    const int pos = i * F::B, wi = pos >> 5, sh = pos & 31;
+    const int wi = pos >> 5, sh = pos & 31;
     uint32_t c;
     if (sh + F::B <= 32)
         c = w[wi] >> sh;
@@ -233,9 +234,9 @@ __device__ __forceinline__ uint32_t get_code(const uint32_t (&w)[NW], int i)
 }
 
 template <class F, int NW>
-__device__ __forceinline__ void put_code(uint32_t (&w)[NW], int i, uint32_t c)
+__device__ __forceinline__ void put_code_at(uint32_t (&w)[NW], int pos, uint32_t c)
 {
-    const int pos = i * F::B, wi = pos >> 5, sh = pos & 31;
+    const int wi = pos >> 5, sh = pos & 31;
     w[wi] |= c << sh;
     if (sh + F::B > 32) w[(wi + 1 < NW) ? wi + 1 : wi] |= c >> (32 - sh);
 }

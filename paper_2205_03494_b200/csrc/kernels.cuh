@@ -49,6 +49,7 @@ struct Unit {
     static constexpr int SUB_STEPS = SUB / STEP;
     static constexpr int OUTBUFS = OMC_OUTBUFS ? OMC_OUTBUFS : (SUB < TILE ? 2 : 1);
     static_assert(TILE % SUB == 0 && (OUTBUFS == 1 || OUTBUFS == 2), "");
+    static_assert(LU != 32 || SUB == STEP, "row layout: one 32-element row per lane and granule");
 };
 
 // Shared-memory budget of one warp: STAGES input stages and OUTBUFS output buffers of one granule.
@@ -56,11 +57,14 @@ template <class F, int MODE, bool WOUT>
 struct Smem {
     static constexpr int SUB = Unit<F>::SUB;
     static constexpr int OUTBUFS = Unit<F>::OUTBUFS;
+    static constexpr bool ROWS = (Unit<F>::LU == 32);   // FP32 data in padded rows, one per lane
     static constexpr int CB = SUB * F::B / 8;     // bytes of one granule's codes
-    static constexpr int FB = SUB * 4;            // bytes of one granule's FP32 operand
+    static constexpr int FB = ROWS ? 32 * 144 : SUB * 4;   // shared-memory bytes of one granule's FP32 data
+    static constexpr int FB_GLOBAL = SUB * 4;     // ... and its bytes in global memory
     static constexpr int IN_C = (MODE != COMPRESS) ? CB : 0;
     static constexpr int IN_F = (MODE != DECOMPRESS) ? FB : 0;
     static constexpr int STAGE = IN_C + IN_F;
+    static constexpr int TX_BYTES = IN_C + (IN_F ? FB_GLOBAL : 0);   // what the stage's copies bring in
     static constexpr int DIST = STAGES - 1;       // granules fetched ahead
     static constexpr int OUT_C = (MODE != DECOMPRESS) ? CB : 0;
     static constexpr int OUT_F = (MODE == DECOMPRESS || WOUT) ? FB : 0;
@@ -249,65 +253,79 @@ struct ValuePattern {
 //   wout : the unit's new codes (written unless DECOMPRESS)  fo : FP32 result (decompressed value / W)
 //   valid: number of leading elements that exist (LU except in a ragged tile)
 
+// Four consecutive elements (group g of the unit): codes from `win`, FP32 operand `fin4`; results
+// into `wout` (codes), `w` (FP32 values), the running sums and the equality trackers ref / diff.
+// `win` / `wout` hold the bits from position `bitbase` of the unit's code stream on (bitbase = 0
+// when they hold the whole unit).
+template <class F, int MODE, bool TAIL, int NWI, int NWO>
+__device__ __forceinline__ void compute_group(const uint32_t (&win)[NWI], int g, const float (&fin4)[4],
+                                              uint32_t (&wout)[NWO], float (&w)[4], float s, float b,
+                                              float neg_lr, Acc &acc, uint32_t &ref, uint32_t &diff, int valid,
+                                              int bitbase = 0)
+{
+    constexpr bool HAS_CIN = (MODE != COMPRESS);
+    constexpr bool KEEP_PAYLOAD = (MODE == COMPRESS);    // UPDATE gives arithmetic NaNs one pattern
+    uint32_t cin[4], cout[4];
+    float vt[4];
+    bool bad = false;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if constexpr (HAS_CIN) {
+            cin[j] = get_code_at<F, NWI>(win, (4 * g + j) * F::B - bitbase);
+            bad |= code_is_special<F>(cin[j]);
+            const float vbar = __fmaf_rn(s, decode_fast<F>(cin[j]), b);
+            w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
+        } else {
+            w[j] = fin4[j];
+        }
+        if constexpr (MODE != DECOMPRESS) bad |= needs_exact_encode<F, KEEP_PAYLOAD>(w[j]);
+    }
+    if constexpr (MODE != DECOMPRESS) {
+        encode_fast2<F>(w[0], w[1], cout[0], cout[1], vt[0], vt[1]);
+        encode_fast2<F>(w[2], w[3], cout[2], cout[3], vt[2], vt[3]);
+    }
+    if (bad) {   // Inf / NaN / overflow somewhere in these four: redo them carefully
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if constexpr (HAS_CIN) {
+                const float vbar = __fmaf_rn(s, decode_exact<F>(cin[j]), b);
+                w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
+                // a NaN made by the arithmetic gets one fixed pattern
+                if (MODE == UPDATE && w[j] != w[j]) w[j] = u2f(0x7FFFFFFFu);
+            }
+            if constexpr (MODE != DECOMPRESS) cout[j] = encode_exact<F>(w[j], vt[j]);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const bool ok = !TAIL || (4 * g + j < valid);
+        if constexpr (MODE != DECOMPRESS) {
+            if (ok) {
+                acc.add(w[j], vt[j]);
+                put_code_at<F, NWO>(wout, (4 * g + j) * F::B - bitbase, cout[j]);
+                const uint32_t pat = ValuePattern<F>::of(cout[j], vt[j]);
+                if (g == 0 && j == 0) ref = pat;             // element 0 exists whenever the unit does
+                else diff |= pat ^ ref;
+            }
+        }
+        if (TAIL && !ok) w[j] = 0.f;
+    }
+}
+
 template <class F, int MODE, bool TAIL>
 __device__ __forceinline__ void compute_unit(const uint32_t (&win)[Unit<F>::NWORDS], const float4 (&fv)[Unit<F>::LU / 4],
                                              uint32_t (&wout)[Unit<F>::NWORDS], float4 (&fo)[Unit<F>::LU / 4],
                                              float s, float b, float neg_lr, Acc &acc, int valid)
 {
     constexpr int LU = Unit<F>::LU, NW = Unit<F>::NWORDS;
-    constexpr bool HAS_CIN = (MODE != COMPRESS);
-    constexpr bool KEEP_PAYLOAD = (MODE == COMPRESS);    // UPDATE gives arithmetic NaNs one pattern
 #pragma unroll
     for (int j = 0; j < NW; ++j) wout[j] = 0u;
     uint32_t ref = 0u, diff = 0u;
 #pragma unroll
     for (int g = 0; g < LU / 4; ++g) {
         const float fin4[4] = {fv[g].x, fv[g].y, fv[g].z, fv[g].w};
-        uint32_t cin[4], cout[4];
-        float w[4], vt[4];
-        bool bad = false;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if constexpr (HAS_CIN) {
-                cin[j] = get_code<F, NW>(win, 4 * g + j);
-                bad |= code_is_special<F>(cin[j]);
-                const float vbar = __fmaf_rn(s, decode_fast<F>(cin[j]), b);
-                w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
-            } else {
-                w[j] = fin4[j];
-            }
-            if constexpr (MODE != DECOMPRESS) bad |= needs_exact_encode<F, KEEP_PAYLOAD>(w[j]);
-        }
-        if constexpr (MODE != DECOMPRESS) {
-            encode_fast2<F>(w[0], w[1], cout[0], cout[1], vt[0], vt[1]);
-            encode_fast2<F>(w[2], w[3], cout[2], cout[3], vt[2], vt[3]);
-        }
-        if (bad) {   // Inf / NaN / overflow somewhere in these four: redo them carefully
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if constexpr (HAS_CIN) {
-                    const float vbar = __fmaf_rn(s, decode_exact<F>(cin[j]), b);
-                    w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
-                    // a NaN made by the arithmetic gets one fixed pattern
-                    if (MODE == UPDATE && w[j] != w[j]) w[j] = u2f(0x7FFFFFFFu);
-                }
-                if constexpr (MODE != DECOMPRESS) cout[j] = encode_exact<F>(w[j], vt[j]);
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const bool ok = !TAIL || (4 * g + j < valid);
-            if constexpr (MODE != DECOMPRESS) {
-                if (ok) {
-                    acc.add(w[j], vt[j]);
-                    put_code<F, NW>(wout, 4 * g + j, cout[j]);
-                    const uint32_t pat = ValuePattern<F>::of(cout[j], vt[j]);
-                    if (g == 0 && j == 0) ref = pat;             // element 0 exists whenever the unit does
-                    else diff |= pat ^ ref;
-                }
-            }
-            if (TAIL && !ok) w[j] = 0.f;
-        }
+        float w[4];
+        compute_group<F, MODE, TAIL, NW, NW>(win, g, fin4, wout, w, s, b, neg_lr, acc, ref, diff, valid);
         fo[g] = make_float4(w[0], w[1], w[2], w[3]);
     }
     if constexpr (MODE != DECOMPRESS) {
@@ -315,6 +333,64 @@ __device__ __forceinline__ void compute_unit(const uint32_t (&win)[Unit<F>::NWOR
             acc.band &= ref & ~diff;
             acc.bor |= ref | diff;
         }
+    }
+}
+
+// A full unit of 32 elements per lane (odd code widths) whose FP32 operand and FP32 result live in
+// shared-memory rows: the operand is fetched four elements at a time right where it is used and
+// the result is stored at once, so that a lane never holds 32 values in registers.
+constexpr int ROW_FLOATS = 36;     // 32 values + 16 bytes: lanes 144 bytes apart hit different banks
+
+__device__ __forceinline__ uint32_t lds_volatile(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_addr(p)));
+    return v;
+}
+
+// Everything is streamed, four elements at a time: the code words and the operand are fetched
+// right where they are used (volatile loads, so that the compiler does not hoist them all to the
+// top), finished output words are stored at once, and a word shared by two groups is carried in
+// one register.  `cin` / `cout` / `fin_row` / `fout_row` are this lane's slices in shared memory.
+template <class F, int MODE, bool WOUT>
+__device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const float *fin_row, uint32_t *cout,
+                                                  float *fout_row, float s, float b, float neg_lr, Acc &acc)
+{
+    constexpr int LU = Unit<F>::LU, B = F::B;
+    constexpr int GW = (4 * B + 31) / 32 + 1;      // words a group of four codes can touch
+    uint32_t ref = 0u, diff = 0u, carry = 0u;
+#pragma unroll
+    for (int g = 0; g < LU / 4; ++g) {
+        const int bit0 = 4 * g * B, f0 = bit0 >> 5, cnt = ((bit0 + 4 * B - 1) >> 5) - f0 + 1;
+        const bool ends_on_word = ((bit0 + 4 * B) & 31) == 0;
+        uint32_t gw[GW], ow[GW];
+#pragma unroll
+        for (int q = 0; q < GW; ++q) {
+            gw[q] = (MODE != COMPRESS && q < cnt) ? lds_volatile(cin + f0 + q) : 0u;
+            ow[q] = 0u;
+        }
+        ow[0] = carry;
+        float fin4[4] = {0.f, 0.f, 0.f, 0.f};
+        if constexpr (MODE != DECOMPRESS) {
+            float4 v;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(smem_addr(fin_row + 4 * g)));
+            fin4[0] = v.x; fin4[1] = v.y; fin4[2] = v.z; fin4[3] = v.w;
+        }
+        float w[4];
+        compute_group<F, MODE, false, GW, GW>(gw, g, fin4, ow, w, s, b, neg_lr, acc, ref, diff, LU, 32 * f0);
+        if constexpr (MODE != DECOMPRESS) {
+#pragma unroll
+            for (int q = 0; q < GW; ++q)
+                if (q < cnt - 1 || (q == cnt - 1 && ends_on_word)) cout[f0 + q] = ow[q];
+            carry = ends_on_word ? 0u : ow[cnt - 1];
+        }
+        if constexpr (MODE == DECOMPRESS || WOUT)
+            reinterpret_cast<float4 *>(fout_row)[g] = make_float4(w[0], w[1], w[2], w[3]);
+    }
+    if constexpr (MODE != DECOMPRESS) {
+        acc.band &= ref & ~diff;
+        acc.bor |= ref | diff;
     }
 }
 
@@ -502,6 +578,11 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
 {
     using U = Unit<F>;
     constexpr int LU = U::LU, NW = U::NWORDS;
+    if constexpr (LU == 32) {       // one unit per lane; FP32 data in rows of ROW_FLOATS
+        compute_unit_rows<F, MODE, WOUT>(s_cin + lane * NW, s_fin + lane * ROW_FLOATS, s_cout + lane * NW,
+                                         s_fout + lane * ROW_FLOATS, s, b, neg_lr, acc);
+        return;
+    }
     constexpr int G = (U::SUB_STEPS >= 2 && LU == 4) ? 2 : 1;   // steps whose operands are fetched together
 #pragma unroll 1
     for (int k0 = 0; k0 < U::SUB_STEPS; k0 += G) {
@@ -646,24 +727,30 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
     const uint32_t g0 = (uint32_t)(e_begin / SUB);                  // first granule
     const uint32_t ng = (uint32_t)((e_end - e_begin) / SUB);        // whole granules
 
-    auto issue = [&](uint32_t g, uint32_t kk) {          // lane 0 only
+    constexpr bool ROWS_IN = SM::ROWS && SM::IN_F > 0;      // every lane copies its own row in
+    constexpr bool ROWS_OUT = SM::ROWS && SM::OUT_F > 0;    // ... and stores its own row
+    auto issue = [&](uint32_t g, uint32_t kk) {           // called by the whole warp
         const uint32_t st = kk % STAGES;
         const uint32_t bar = bar0 + 8u * st;
         uint8_t *dst = wbase + st * SM::STAGE;
-        mbar_expect_tx(bar, (uint32_t)SM::STAGE);
-        if constexpr (SM::IN_C > 0)
-            bulk_load(smem_addr(dst), codes + (size_t)g * SM::CB, SM::CB, bar);
-        if constexpr (SM::IN_F > 0)
-            bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)g * SUB, SM::FB, bar);
+        if (lane == 0) {
+            mbar_expect_tx(bar, (uint32_t)SM::TX_BYTES);
+            if constexpr (SM::IN_C > 0)
+                bulk_load(smem_addr(dst), codes + (size_t)g * SM::CB, SM::CB, bar);
+            if constexpr (SM::IN_F > 0 && !ROWS_IN)
+                bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)g * SUB, SM::FB, bar);
+        }
+        if constexpr (ROWS_IN) {
+            __syncwarp();      // the expectation is posted before any of the row copies can complete
+            bulk_load(smem_addr(dst + SM::IN_C + lane * (ROW_FLOATS * 4)), fin + (size_t)g * SUB + lane * 32, 128u, bar);
+        }
     };
 
-    if (lane == 0) {
-        for (uint32_t i = 0; i < (uint32_t)SM::DIST && i < ng; ++i) issue(g0 + i, k + i);
-    }
+    for (uint32_t i = 0; i < (uint32_t)SM::DIST && i < ng; ++i) issue(g0 + i, k + i);
     for (uint32_t i = 0; i < ng; ++i, ++k) {
         const uint32_t g = g0 + i;
-        if (lane == 0) {
-            if (i + SM::DIST < ng) issue(g + SM::DIST, k + SM::DIST);   // its stage was consumed last round
+        if (i + SM::DIST < ng) issue(g + SM::DIST, k + SM::DIST);   // its stage was consumed last round
+        if (lane == 0 || ROWS_OUT) {
             // the output buffer written next must have left with its last store
             if constexpr (SM::OUTBUFS == 2) bulk_wait_read1(); else bulk_wait_read0();
         }
@@ -686,10 +773,12 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
         if (lane == 0) {
             if constexpr (MODE != DECOMPRESS)
                 bulk_store(codes + (size_t)g * SM::CB, smem_addr(ob), SM::CB);
-            if constexpr (MODE == DECOMPRESS || WOUT)
+            if constexpr (SM::OUT_F > 0 && !ROWS_OUT)
                 bulk_store(fout + (size_t)g * SUB, smem_addr(ob + SM::OUT_C), SM::FB);
-            bulk_commit();
         }
+        if constexpr (ROWS_OUT)
+            bulk_store(fout + (size_t)g * SUB + lane * 32, smem_addr(ob + SM::OUT_C + lane * (ROW_FLOATS * 4)), 128u);
+        if (lane == 0 || ROWS_OUT) bulk_commit();
     }
     if (failed) { pipe.k = k; pipe.failed = true; return; }
     const uint64_t e_rag = e_begin + (uint64_t)ng * SUB;
@@ -796,7 +885,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams
         ++v;
     }
     if (pipe.failed && lane == 0) atomicExch(p.status, 1u);   // a bulk load never arrived
-    if (lane == 0) bulk_wait_all();                      // stores must finish before the CTA's memory goes
+    bulk_wait_all();                                     // stores must finish before the CTA's memory goes
 }
 
 template <class F, int MODE, bool WOUT>
@@ -925,7 +1014,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_transition_kernel(co
         ++v;
     }
     if (pipe.failed && lane == 0) atomicExch(p.status, 1u);
-    if (lane == 0) bulk_wait_all();
+    bulk_wait_all();
 }
 
 template <class F>
