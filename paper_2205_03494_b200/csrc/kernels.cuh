@@ -16,6 +16,8 @@
 // own copies; they are bounded, and a wait that runs out sets the plan's status word and ends
 // the warp.
 #pragma once
+#include <type_traits>
+
 #include "codec.cuh"
 #include "omc_internal.h"
 
@@ -253,6 +255,23 @@ struct ValuePattern {
 //   wout : the unit's new codes (written unless DECOMPRESS)  fo : FP32 result (decompressed value / W)
 //   valid: number of leading elements that exist (LU except in a ragged tile)
 
+// A loop whose index is a compile-time constant in every iteration (what "#pragma unroll" only
+// asks for): bit positions inside the code stream must fold to immediates.
+template <int I, int N>
+struct StaticFor {
+    template <class Fn>
+    __device__ __forceinline__ static void run(Fn &&fn)
+    {
+        fn(std::integral_constant<int, I>{});
+        StaticFor<I + 1, N>::run(fn);
+    }
+};
+template <int N>
+struct StaticFor<N, N> {
+    template <class Fn>
+    __device__ __forceinline__ static void run(Fn &&) {}
+};
+
 // Four consecutive elements (group g of the unit): codes from `win`, FP32 operand `fin4`; results
 // into `wout` (codes), `w` (FP32 values), the running sums and the equality trackers ref / diff.
 // `win` / `wout` hold the bits from position `bitbase` of the unit's code stream on (bitbase = 0
@@ -341,10 +360,10 @@ __device__ __forceinline__ void compute_unit(const uint32_t (&win)[Unit<F>::NWOR
 // the result is stored at once, so that a lane never holds 32 values in registers.
 constexpr int ROW_FLOATS = 36;     // 32 values + 16 bytes: lanes 144 bytes apart hit different banks
 
-__device__ __forceinline__ uint32_t lds_volatile(const uint32_t *p)
+__device__ __forceinline__ uint32_t lds_volatile(uint32_t shared_addr)
 {
     uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_addr(p)));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(shared_addr));
     return v;
 }
 
@@ -359,14 +378,15 @@ __device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const flo
     constexpr int LU = Unit<F>::LU, B = F::B;
     constexpr int GW = (4 * B + 31) / 32 + 1;      // words a group of four codes can touch
     uint32_t ref = 0u, diff = 0u, carry = 0u;
-#pragma unroll
-    for (int g = 0; g < LU / 4; ++g) {
-        const int bit0 = 4 * g * B, f0 = bit0 >> 5, cnt = ((bit0 + 4 * B - 1) >> 5) - f0 + 1;
-        const bool ends_on_word = ((bit0 + 4 * B) & 31) == 0;
+    const uint32_t cin_a = smem_addr(cin), fin_a = smem_addr(fin_row);     // shared-window addresses, once
+    StaticFor<0, LU / 4>::run([&](auto gi) {
+        constexpr int g = decltype(gi)::value;
+        constexpr int bit0 = 4 * g * B, f0 = bit0 >> 5, cnt = ((bit0 + 4 * B - 1) >> 5) - f0 + 1;
+        constexpr bool ends_on_word = ((bit0 + 4 * B) & 31) == 0;
         uint32_t gw[GW], ow[GW];
 #pragma unroll
         for (int q = 0; q < GW; ++q) {
-            gw[q] = (MODE != COMPRESS && q < cnt) ? lds_volatile(cin + f0 + q) : 0u;
+            gw[q] = (MODE != COMPRESS && q < cnt) ? lds_volatile(cin_a + 4u * (f0 + q)) : 0u;
             ow[q] = 0u;
         }
         ow[0] = carry;
@@ -374,7 +394,7 @@ __device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const flo
         if constexpr (MODE != DECOMPRESS) {
             float4 v;
             asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(smem_addr(fin_row + 4 * g)));
+                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(fin_a + 16u * g));
             fin4[0] = v.x; fin4[1] = v.y; fin4[2] = v.z; fin4[3] = v.w;
         }
         float w[4];
@@ -387,7 +407,7 @@ __device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const flo
         }
         if constexpr (MODE == DECOMPRESS || WOUT)
             reinterpret_cast<float4 *>(fout_row)[g] = make_float4(w[0], w[1], w[2], w[3]);
-    }
+    });
     if constexpr (MODE != DECOMPRESS) {
         acc.band &= ref & ~diff;
         acc.bor |= ref | diff;
@@ -808,7 +828,8 @@ __device__ __forceinline__ VarDev load_var(const VarDev *src)
 }
 
 template <class F, int MODE, bool WOUT>
-__global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_kernel(const KParams p)
+__global__ void __launch_bounds__(THREADS, MODE == DECOMPRESS ? DECOMPRESS_CTAS_PER_SM : CTAS_PER_SM)
+omc_kernel(const KParams p)
 {
     using SM = Smem<F, MODE, WOUT>;
     extern __shared__ __align__(128) uint8_t smem_raw[];

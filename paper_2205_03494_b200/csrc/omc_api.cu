@@ -117,7 +117,7 @@ extern "C" int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, con
     p.tile_begin = plan->vars[first_var].tile_start;
     const omc::VarDev &lastv = plan->vars[first_var + n_vars - 1];
     p.tile_count = lastv.tile_start + lastv.ntiles - p.tile_begin;
-    const uint64_t max_warps = (uint64_t)plan->n_cta * omc::WARPS_PER_CTA;
+    const uint64_t max_warps = (uint64_t)plan->n_sm * omc::DECOMPRESS_CTAS_PER_SM * omc::WARPS_PER_CTA;
     p.nwarps = (uint32_t)(p.tile_count < max_warps ? p.tile_count : max_warps);
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
     p.dyn_e = plan->fmt.exp_bits;

@@ -20,6 +20,12 @@ constexpr int TILE = 1024;         // elements per tile: the unit of work a warp
 constexpr int WARPS_PER_CTA = OMC_WARPS_PER_CTA;
 constexpr int THREADS = 32 * WARPS_PER_CTA;
 constexpr int CTAS_PER_SM = OMC_CTAS_PER_SM;
+#ifndef OMC_DECOMPRESS_CTAS_PER_SM
+#define OMC_DECOMPRESS_CTAS_PER_SM 2
+#endif
+// The decompress kernel keeps no running sums and needs fewer registers: it may run more CTAs per SM
+// (it divides its tiles at launch, so its grid is independent of the plan's partition).
+constexpr int DECOMPRESS_CTAS_PER_SM = OMC_DECOMPRESS_CTAS_PER_SM;
 constexpr int DEFAULT_SMS = 148;   // B200; used when no device can be queried at plan time
 
 // One per variable, in the caller's order; lives in device memory after omc_plan_prepare.
