@@ -341,6 +341,37 @@ def run_ours(args):
                                                   "gbs": nbytes / (t_ms * 1e6),
                                                   "variables_changing": sum(a != b for a, b in zip(pa.quantised, pb.quantised))}
 
+        # server-side mean of 8 client replicas, each with its own random 90% subset (Sec. 2.5)
+        K = 8
+        cl = []
+        for k in range(K):
+            pl = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=100 + k)
+            b4 = (z(pl.packed_bytes, torch.uint8), z(pl.resid_elems, torch.float32),
+                  z(2 * pl.n_quantised, torch.float32), z(pl.workspace_bytes, torch.uint8))
+            pl.prepare(b4[3].data_ptr(), stream)
+            pl.compress(out.data_ptr(), b4[0].data_ptr(), b4[1].data_ptr(), b4[2].data_ptr(), b4[3].data_ptr(), stream)
+            cl.append((pl, b4))
+        mean = torch.empty(plan.full_elems, dtype=torch.float32, device=dev)
+        try:
+            fn = lambda: omc.aggregate([c[0] for c in cl], [c[1][0].data_ptr() for c in cl],
+                                       [c[1][1].data_ptr() for c in cl], [c[1][2].data_ptr() for c in cl],
+                                       mean.data_ptr(), stream)
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(20):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            t_ms = e0.elapsed_time(e1) / 20
+            nbytes = 4 * nparams + sum(((n * pl.B + 7) // 8) if q else 4 * n
+                                       for pl, _ in cl for n, q in zip(pl.numel, pl.quantised))
+            extra["aggregate_8_clients"] = {"ms": t_ms, "params_per_s": nparams / (t_ms * 1e-3),
+                                            "gbs": nbytes / (t_ms * 1e6)}
+        except omc.OmcError as err:
+            extra["aggregate_8_clients"] = {"unavailable": str(err)}
+
     if dist is not None:
         dist.barrier()
     if rank != 0:

@@ -187,6 +187,21 @@ int omc_transition(const omc_plan_t *from, const omc_plan_t *to, const uint8_t *
                    float *sb_to, void *workspace_to, void *stream);
 
 /*
+ * omc_aggregate -- server-side aggregation of client replicas (Sec. 1: the trained client models
+ * are transported back, in compressed form, and aggregated; Sec. 2.5: each client quantises its
+ * own subset, so for every parameter some clients deliver full-precision values).
+ * out[e] = (x_0[e] + x_1[e] + ... + x_{K-1}[e]) / K in FP32, the clients added in index order and
+ * one correctly rounded division at the end, where x_k[e] is client k's decompressed value
+ * fma(s_k, Vt_k, b_k) if k quantised the variable and its FP32 value otherwise.
+ *   plans[K]   host array: each client's prepared plan (same variables and format, own selection).
+ *   packed[K], resid[K], sb[K]   host arrays of device pointers: each client's state, read only.
+ *   out        device, full layout, written.       1 <= K <= 16 (else OMC_ERR_INVALID_ARG).
+ * Formats without a compiled specialisation return OMC_ERR_BAD_FORMAT.
+ */
+int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
+                  const float *const *resid, const float *const *sb, float *out, void *stream);
+
+/*
  * omc_compress_var_static -- compress ONE variable without a plan, a workspace or any allocation.
  * (The paper has no counterpart: this is a convenience of this library, not part of the method.)
  *

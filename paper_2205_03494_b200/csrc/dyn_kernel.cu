@@ -180,6 +180,6 @@ static void launch_dyn(const KParams &p, int grid, void *stream)
 }
 
 extern const FmtOps ops_dynamic = {-1, -1, launch_dyn<COMPRESS, false>, launch_dyn<DECOMPRESS, false>,
-                                   launch_dyn<UPDATE, false>, launch_dyn<UPDATE, true>, nullptr};
+                                   launch_dyn<UPDATE, false>, launch_dyn<UPDATE, true>, nullptr, nullptr};
 
 }  // namespace omc

@@ -1052,11 +1052,109 @@ void launch_transition(const KParams &p, int grid, void *stream)
     omc_transition_kernel<F><<<grid, THREADS, TransitionSmem<F>::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Server-side aggregation (Sec. 1: the clients' models are transported back and aggregated;
+// Sec. 2.5: each client quantises its own subset, so the server receives precise values of a
+// parameter from the clients that kept it in FP32).  out = (x_0 + x_1 + ... + x_{K-1}) / K per
+// element, FP32, clients added in index order, one rounded division at the end, where x_k is
+// client k's decompressed value fma(s_k, Vt_k, b_k) or its FP32 value.  Plain predicated
+// 128-bit global accesses; every element is read once per client and written once.
+
+template <class F>
+__global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_aggregate_kernel(const AggParams p)
+{
+    using U = Unit<F>;
+    constexpr int LU = U::LU, NW = U::NWORDS;
+    const int lane = threadIdx.x & 31;
+    const uint32_t warp = blockIdx.x * WARPS_PER_CTA + (threadIdx.x >> 5);
+    if (warp >= p.nwarps) return;
+    uint64_t t = (uint64_t)warp * p.tile_count / p.nwarps;
+    const uint64_t tend = (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
+    uint32_t lo = 0, hi = p.nvars;
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (__ldg(&p.vars[0][mid].tile_start) <= t) lo = mid; else hi = mid;
+    }
+    uint32_t v = lo;
+    const float kf = (float)p.nclients;
+    // per warp: what the unit loop needs to know about each client's copy of the current variable
+    struct ClientVar { uint64_t base; uint32_t nwords; uint32_t quantised; float s, b; uint32_t pad[2]; };
+    __shared__ ClientVar cv_all[WARPS_PER_CTA][MAX_CLIENTS];
+    ClientVar *cv = cv_all[threadIdx.x >> 5];
+    while (t < tend) {
+        const VarDev var = load_var(p.vars[0] + v);
+        __syncwarp();
+        if ((uint32_t)lane < p.nclients) {
+            const VarDev vk = load_var(p.vars[lane] + v);
+            ClientVar c;
+            c.quantised = vk.quantised;
+            c.nwords = (uint32_t)(vk.packed_bytes / 4);
+            c.base = vk.quantised ? reinterpret_cast<uint64_t>(p.packed[lane] + vk.store_off)
+                                  : reinterpret_cast<uint64_t>(p.resid[lane] + vk.store_off);
+            c.s = vk.quantised ? __ldg(p.sb[lane] + 2 * vk.sb_slot) : 1.f;
+            c.b = vk.quantised ? __ldg(p.sb[lane] + 2 * vk.sb_slot + 1) : 0.f;
+            c.pad[0] = c.pad[1] = 0u;
+            cv[lane] = c;
+        }
+        __syncwarp();
+        const uint32_t local = (uint32_t)(t - var.tile_start);
+        const uint64_t left = tend - t;
+        const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
+        const uint64_t e_begin = (uint64_t)local * TILE;
+        const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
+        const uint64_t n_pad = (var.n + 3) & ~3ull;
+        for (uint64_t e0 = e_begin + (uint64_t)lane * LU; e0 < e_end; e0 += U::STEP) {
+            float acc[LU];
+#pragma unroll
+            for (int j = 0; j < LU; ++j) acc[j] = 0.f;
+            for (uint32_t k = 0; k < p.nclients; ++k) {
+                const ClientVar c = cv[k];
+                float x[LU];
+                if (c.quantised) {
+                    const uint32_t *cw = reinterpret_cast<const uint32_t *>(c.base);
+                    const uint64_t w0 = e0 / LU * NW;
+                    uint32_t win[NW];
+#pragma unroll
+                    for (int j = 0; j < NW; ++j) win[j] = (w0 + j < c.nwords) ? __ldcs(cw + w0 + j) : 0u;
+#pragma unroll
+                    for (int j = 0; j < LU; ++j)
+                        x[j] = __fmaf_rn(c.s, decode_exact<F>(get_code_at<F, NW>(win, j * F::B)), c.b);
+                } else {
+                    const float *r = reinterpret_cast<const float *>(c.base) + e0;
+#pragma unroll
+                    for (int j = 0; j < LU / 4; ++j) {
+                        const float4 q = (e0 + 4 * j < n_pad) ? __ldcs(reinterpret_cast<const float4 *>(r) + j)
+                                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                        x[4 * j] = q.x; x[4 * j + 1] = q.y; x[4 * j + 2] = q.z; x[4 * j + 3] = q.w;
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < LU; ++j) acc[j] = (k == 0) ? x[j] : __fadd_rn(acc[j], x[j]);
+            }
+            float *o = p.out + var.full_off + e0;
+#pragma unroll
+            for (int j = 0; j < LU / 4; ++j)
+                if (e0 + 4 * j < n_pad)
+                    reinterpret_cast<float4 *>(o)[j] = make_float4(__fdiv_rn(acc[4 * j], kf), __fdiv_rn(acc[4 * j + 1], kf),
+                                                                   __fdiv_rn(acc[4 * j + 2], kf), __fdiv_rn(acc[4 * j + 3], kf));
+        }
+        t += cnt;
+        ++v;
+    }
+}
+
+template <class F>
+void launch_aggregate(const AggParams &p, int grid, void *stream)
+{
+    omc_aggregate_kernel<F><<<grid, THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p);
+}
+
 #define OMC_DEFINE_FORMAT(E_, M_)                                                               \
     extern const FmtOps ops_E##E_##M##M_ = {E_, M_, launch<Fmt<E_, M_>, COMPRESS, false>,       \
                                             launch<Fmt<E_, M_>, DECOMPRESS, false>,             \
                                             launch<Fmt<E_, M_>, UPDATE, false>,                 \
                                             launch<Fmt<E_, M_>, UPDATE, true>,                  \
-                                            launch_transition<Fmt<E_, M_>>};
+                                            launch_transition<Fmt<E_, M_>>,                     \
+                                            launch_aggregate<Fmt<E_, M_>>};
 
 }  // namespace omc

@@ -214,3 +214,39 @@ extern "C" int omc_transition(const omc_plan_t *from, const omc_plan_t *to, cons
     to->ops->transition(p, grid_for(p.nwarps), stream);
     return omc::note_cuda(cudaGetLastError());
 }
+
+extern "C" int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
+                             const float *const *resid, const float *const *sb, float *out, void *stream)
+{
+    if (!plans || !packed || !resid || !sb || !out) return OMC_ERR_NULL_PTR;
+    if (n_clients == 0 || n_clients > (uint32_t)omc::MAX_CLIENTS) return OMC_ERR_INVALID_ARG;
+    if (misaligned(out)) return OMC_ERR_MISALIGNED;
+    omc::AggParams p{};
+    const omc_plan_t *first = plans[0];
+    for (uint32_t k = 0; k < n_clients; ++k) {
+        const omc_plan_t *pl = plans[k];
+        int rc = check_ready(pl);
+        if (rc) return rc;
+        if (pl->nvars != first->nvars || pl->fmt.exp_bits != first->fmt.exp_bits ||
+            pl->fmt.man_bits != first->fmt.man_bits)
+            return OMC_ERR_PLAN_MISMATCH;
+        for (uint32_t i = 0; i < pl->nvars; ++i)
+            if (pl->vars[i].n != first->vars[i].n) return OMC_ERR_PLAN_MISMATCH;
+        if (pl->nq && (!packed[k] || !sb[k])) return OMC_ERR_NULL_PTR;
+        if (pl->resid_elems && !resid[k]) return OMC_ERR_NULL_PTR;
+        if (misaligned(packed[k]) || misaligned(resid[k]) || misaligned(sb[k])) return OMC_ERR_MISALIGNED;
+        p.vars[k] = pl->d_vars;
+        p.packed[k] = packed[k];
+        p.resid[k] = resid[k];
+        p.sb[k] = sb[k];
+    }
+    if (!first->ops->aggregate) return OMC_ERR_BAD_FORMAT;
+    p.nclients = n_clients;
+    p.nvars = first->nvars;
+    p.tile_count = first->ntiles;
+    const uint64_t max_warps = (uint64_t)first->n_cta * omc::WARPS_PER_CTA * 2;    // light kernel: 4 CTAs per SM fit
+    p.nwarps = (uint32_t)(p.tile_count < max_warps ? p.tile_count : max_warps);
+    p.out = out;
+    first->ops->aggregate(p, grid_for(p.nwarps), stream);
+    return omc::note_cuda(cudaGetLastError());
+}

@@ -79,6 +79,20 @@ struct KParams {
     uint32_t *status;              // the plan's device status word: set non-zero if a copy never arrived
 };
 
+// Arguments of the aggregation kernel: the states of up to MAX_CLIENTS replicas of one model.
+constexpr int MAX_CLIENTS = 16;
+struct AggParams {
+    const VarDev *vars[MAX_CLIENTS];     // each replica's plan table (same variables, own selection)
+    const uint8_t *packed[MAX_CLIENTS];
+    const float *resid[MAX_CLIENTS];
+    const float *sb[MAX_CLIENTS];
+    uint32_t nclients;
+    uint32_t nvars;
+    uint64_t tile_count;
+    uint32_t nwarps;
+    float *out;                          // full layout
+};
+
 struct FmtOps {
     int E, M;
     void (*compress)(const KParams &, int grid, void *stream);
@@ -86,6 +100,7 @@ struct FmtOps {
     void (*update)(const KParams &, int grid, void *stream);     // W not stored
     void (*update_w)(const KParams &, int grid, void *stream);   // W stored to fout
     void (*transition)(const KParams &, int grid, void *stream); // plan-to-plan; NULL if unsupported
+    void (*aggregate)(const AggParams &, int grid, void *stream); // mean of replicas; NULL if unsupported
 };
 const FmtOps *find_ops(int E, int M);
 

@@ -352,3 +352,45 @@ def test_transition_refuses_mismatched_plans():
     never = omc.Plan([100, 200], [0, 0], (5, 2))
     assert L.omc_transition(a._h, never._h, *args(da, da)) == -5
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("fmt", [(5, 2), (5, 6), (5, 10), (3, 7), (4, 14)], ids=lambda f: "E%dM%d" % f)
+def test_aggregate_client_replicas(fmt):
+    """Server-side mean of K clients that each quantised their own random subset (Sec. 2.5): the
+    oracle decompresses every client and averages in FP32, clients in index order, one division."""
+    rng = np.random.default_rng(7)
+    numel = [3000, 1, 1024, 5121, 333, 40000, 12289, 77]
+    kinds = [0, 0, 0, 0, 1, 0, 0, 2]
+    K = 5
+    base = [(rng.standard_normal(n) * 0.1).astype(np.float32) for n in numel]
+    clients = []
+    for k in range(K):
+        params = [(p + rng.standard_normal(p.size).astype(np.float32) * np.float32(0.01)) for p in base]
+        if k == 2:
+            params[0][:6] = [np.inf, -np.inf, np.nan, 1e30, -0.0, 1e-45]
+        ls = Lockstep(numel, kinds, fmt, params, fraction=0.6, seed=10 + k)
+        clients.append(ls)
+    assert len({tuple(c.plan.quantised) for c in clients}) > 1
+    out = torch.zeros(clients[0].plan.full_elems, dtype=torch.float32, device="cuda")
+    omc.aggregate([c.plan for c in clients], [c.dm.packed.data_ptr() for c in clients],
+                  [c.dm.resid.data_ptr() for c in clients], [c.dm.sb.data_ptr() for c in clients],
+                  out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    dec = [orc.decompress(c.st) for c in clients]
+    with np.errstate(all="ignore"):
+        for i, n in enumerate(numel):
+            acc = dec[0][i].copy()
+            for k in range(1, K):
+                acc = acc + dec[k][i]                     # FP32 adds, client order
+            want = acc / np.float32(K)
+            assert same_f32(from_full(clients[0].plan, got, i), want), i
+    # one client alone: the mean is its decompressed model
+    omc.aggregate([clients[1].plan], [clients[1].dm.packed.data_ptr()], [clients[1].dm.resid.data_ptr()],
+                  [clients[1].dm.sb.data_ptr()], out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    for i in range(len(numel)):
+        assert same_f32(from_full(clients[1].plan, got, i), dec[1][i]), i
+    L = omc.lib()
+    assert L.omc_aggregate(None, 1, None, None, None, out.data_ptr(), None) == -3
