@@ -219,7 +219,8 @@ def run_ours(args):
         wl.fmt = tuple(int(x) for x in args.format.split(","))
     if args.fraction:
         wl.fraction = args.fraction
-    plan = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=wl.fraction, seed=wl.sel_seed)
+    flags = (0 if args.no_pvt else omc.PLAN_PVT) | (0 if args.all_variables else omc.PLAN_WEIGHTS_ONLY)
+    plan = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=wl.fraction, seed=wl.sel_seed, flags=flags)
     stream = torch.cuda.current_stream().cuda_stream
 
     def full_array(arrays, pinned=False):
@@ -394,7 +395,7 @@ def run_ours(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "%s S1E%dM%d p=%g" % (wl.name, wl.fmt[0], wl.fmt[1], wl.fraction),
                    "params": nparams, "variables": plan.nvars, "quantised_variables": plan.n_quantised,
-                   "bytes_per_step": step_bytes, "lr": wl.lr, "gradients": "one seeded buffer reused every step",
+                   "bytes_per_step": step_bytes, "lr": wl.lr, "pvt": not args.no_pvt, "weights_only": not args.all_variables, "gradients": "one seeded buffer reused every step",
                    "l2": "inputs per step (%.0f MB) exceed the 126 MB L2; no flush" % (step_bytes / 1e6),
                    "multi_gpu": "replicas only"},
         "hbm_gbs": achieved, "pct_of_8tbs": 100 * achieved / NOMINAL_HBM_GBS,
@@ -423,6 +424,8 @@ def main():
     ap.add_argument("--workload", default="conformer")
     ap.add_argument("--format", default="", help="override the workload's format: E,M (e.g. 3,7 = S1E3M7)")
     ap.add_argument("--fraction", type=float, default=0.0, help="override the quantised fraction of weight matrices")
+    ap.add_argument("--no-pvt", action="store_true", help="ablation: without the per-variable transformation")
+    ap.add_argument("--all-variables", action="store_true", help="ablation: biases and norms are eligible too")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-extra", action="store_true", help="skip timing the decompress / compress kernels")
     args = ap.parse_args()
