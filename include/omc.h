@@ -202,6 +202,22 @@ int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint
                   const float *const *resid, const float *const *sb, float *out, void *stream);
 
 /*
+ * omc_matmul -- forward path of Fig. 1 with the decompression fused into the consumer (Sec. 2.1:
+ * a layer's parameters are decompressed only when the layer needs them; here they never exist in
+ * FP32 at all).  For variable `var` of the plan, read as an N x K matrix W (K contiguous):
+ *     Y = X * Wbar^T,  Wbar = s*Wt + b (Sec. 2.3),  computed as  s * (X * Wt^T) + b * rowsum(X)
+ * with X and the codes as FP16 operands of the tensor cores and FP32 accumulation (the paper
+ * computes "in full precision or other hardware-supported formats").
+ *   Only S1E5M10 plans (whose codes are IEEE half patterns), else OMC_ERR_BAD_FORMAT.
+ *   var must be quantised and N*K == its numel; N % 128 == 0, K % 64 == 0 (else OMC_ERR_INVALID_ARG).
+ *   packed, sb      device, the model state (read only).
+ *   x_half          device, M x K IEEE halves, K contiguous, 16-byte aligned.
+ *   y               device, M x N floats, written.       rowsum_scratch  device, M floats, written.
+ */
+int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *packed, const float *sb, const void *x_half,
+               uint32_t M, uint32_t N, uint32_t K, float *y, float *rowsum_scratch, void *stream);
+
+/*
  * omc_compress_var_static -- compress ONE variable without a plan, a workspace or any allocation.
  * (The paper has no counterpart: this is a convenience of this library, not part of the method.)
  *

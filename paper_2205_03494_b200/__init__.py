@@ -20,7 +20,7 @@ PLAN_DEFAULT = PLAN_PVT | PLAN_WEIGHTS_ONLY
 
 EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_sizes",
            "omc_plan_var", "omc_plan_prepare", "omc_plan_status", "omc_compress", "omc_decompress",
-           "omc_update_recompress", "omc_update_recompress_host", "omc_transition", "omc_aggregate",
+           "omc_update_recompress", "omc_update_recompress_host", "omc_transition", "omc_aggregate", "omc_matmul",
            "omc_compress_var_static"]
 STATIC_MAX_NUMEL = 1 << 28
 
@@ -70,6 +70,7 @@ def lib():
         L.omc_update_recompress.argtypes = [vp, vp, vp, vp, vp, C.c_float, vp, vp, vp]
         L.omc_update_recompress_host.argtypes = [vp, vp, vp, vp, vp, C.c_float, vp, vp, vp, vp]
         L.omc_transition.argtypes = [vp] * 10
+        L.omc_matmul.argtypes = [vp, C.c_uint32, vp, vp, vp, C.c_uint32, C.c_uint32, C.c_uint32, vp, vp, vp]
         L.omc_aggregate.argtypes = [C.POINTER(vp), C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp, vp]
         L.omc_compress_var_static.argtypes = [vp, C.c_uint64, Format, C.c_uint32, vp, vp, vp]
         _lib = L
@@ -169,6 +170,11 @@ def transition(plan_from: Plan, plan_to: Plan, packed_from, resid_from, sb_from,
     """omc_transition: state under plan_from -> state under plan_to (addresses are ints)."""
     _check(lib().omc_transition(plan_from._h, plan_to._h, packed_from, resid_from, sb_from, packed_to, resid_to,
                                 sb_to, workspace_to, stream), "omc_transition")
+
+
+def matmul(plan: Plan, var, packed, sb, x_half, M, N, K, y, rowsum_scratch, stream=0):
+    """omc_matmul: Y = X * Wbar^T straight from the codes of variable `var` (addresses are ints)."""
+    _check(lib().omc_matmul(plan._h, var, packed, sb, x_half, M, N, K, y, rowsum_scratch, stream), "omc_matmul")
 
 
 def aggregate(plans, packed, resid, sb, out, stream=0):

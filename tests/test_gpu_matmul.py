@@ -1,0 +1,61 @@
+"""omc_matmul: the forward-path product computed straight from the codes (tensor cores) against
+the definition: decompress the variable with the oracle, then Y = X Wbar^T in fp64 (numpy matmul).
+Tolerance: X and the codes are exact FP16 inputs and their products are exact in FP32, so the only
+errors are the FP32 accumulation over K (<= K 2^-23 of sum |x||w|) and the epilogue's two roundings;
+the test allows 1e-3 of sum_k |x||w| (+ the same for the b*rowsum term), four orders of magnitude
+below what a wrong tile, swizzle or index would produce."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2205_03494_b200 as omc
+from oracle import omc_oracle as orc
+from harness import DeviceModel
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 256, 192), (1000, 384, 512), (64, 128, 1024)])
+def test_matmul_from_codes_matches_definition(M, N, K):
+    rng = np.random.default_rng(M + N + K)
+    numel = [777, N * K, 64, 128 * 64]
+    kinds = [0, 0, 1, 0]
+    params = [(rng.standard_normal(n) * 0.05 + 0.01).astype(np.float32) for n in numel]
+    plan = omc.Plan(numel, kinds, (5, 10))
+    dm = DeviceModel(plan)
+    dm.compress(dm.upload_full(params))
+    st = orc.compress(params, plan.quantised, 5, 10)
+    x = (rng.standard_normal((M, K)) * 0.5).astype(np.float16)
+    xd = torch.from_numpy(x).cuda()
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    scratch = torch.zeros(M, dtype=torch.float32, device="cuda")
+    omc.matmul(plan, 1, dm.packed.data_ptr(), dm.sb.data_ptr(), xd.data_ptr(), M, N, K, y.data_ptr(),
+               scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    wbar = orc.decompress_var(st["packed"][1], N * K, 5, 10, st["s"][1], st["b"][1]).reshape(N, K).astype(np.float64)
+    x64 = x.astype(np.float64)
+    want = x64 @ wbar.T
+    bound = 1e-3 * (np.abs(x64) @ np.abs(wbar).T + abs(float(st["b"][1])) * np.abs(x64).sum(1, keepdims=True)) + 1e-7
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.all(np.abs(got - want) <= bound), float(np.max(np.abs(got - want) / bound))
+
+
+def test_matmul_argument_checks():
+    plan = omc.Plan([128 * 64, 100], [0, 1], (5, 10))
+    dm = DeviceModel(plan)
+    p8 = omc.Plan([128 * 64], [0], (5, 2))
+    d8 = DeviceModel(p8)
+    x = torch.zeros(128 * 64, dtype=torch.float16, device="cuda")
+    y = torch.zeros(128 * 128, dtype=torch.float32, device="cuda")
+    L = omc.lib()
+    a = (dm.packed.data_ptr(), dm.sb.data_ptr(), x.data_ptr())
+    assert L.omc_matmul(plan._h, 1, *a, 128, 128, 64, y.data_ptr(), y.data_ptr(), None) == -1     # FP32 variable
+    assert L.omc_matmul(plan._h, 0, *a, 128, 128, 32, y.data_ptr(), y.data_ptr(), None) == -1     # K % 64
+    assert L.omc_matmul(plan._h, 0, *a, 128, 64, 128, y.data_ptr(), y.data_ptr(), None) == -1     # N % 128
+    assert L.omc_matmul(plan._h, 0, *a, 128, 128, 128, y.data_ptr(), y.data_ptr(), None) == -1    # N*K != numel
+    assert L.omc_matmul(p8._h, 0, d8.packed.data_ptr(), d8.sb.data_ptr(), x.data_ptr(), 128, 128, 64, y.data_ptr(),
+                        y.data_ptr(), None) == -2
+    assert L.omc_matmul(plan._h, 0, *a, 128, 128, 64, None, y.data_ptr(), None) == -3
+    torch.cuda.synchronize()
