@@ -7,7 +7,7 @@
 // and from there into the 5th-generation tensor cores as the B operand: the transient FP32 copy of
 // the weights that omc_decompress would write, and a GEMM would read back, never exists.
 //
-// One CTA computes a 128 x 128 tile of Y: thread 0 runs a four-stage TMA pipeline over K (64
+// One CTA computes a 128 x 128 tile of Y: thread 0 runs a three-stage TMA pipeline over K (64
 // columns per stage), thread 32 issues tcgen05.mma (128x128x16, FP16 inputs, FP32 accumulator in
 // tensor memory) and commits each stage back to the producer, then all four warps read the
 // accumulator with tcgen05.ld and apply the epilogue above.  Every wait is bounded; a wait that
@@ -25,7 +25,7 @@ int note_cuda(cudaError_t e);
 namespace {
 
 constexpr int BM = 128, BN = 128, BK = 64;       // CTA tile; BK halves = one 128-byte swizzle row
-constexpr int STAGES = 4;
+constexpr int STAGES = 3;                      // 3 x 32 KB per CTA: two CTAs fit one SM, so one computes while the other stores
 constexpr int UMMA_K = 16;                       // K of one tcgen05.mma with 16-bit inputs
 constexpr int TILE_A_BYTES = BM * BK * 2, TILE_B_BYTES = BN * BK * 2;
 constexpr int STAGE_BYTES = TILE_A_BYTES + TILE_B_BYTES;
@@ -99,7 +99,7 @@ __global__ void rowsum_kernel(const __half *__restrict__ x, uint32_t M, uint32_t
     if (lane == 0) out[row] = acc;
 }
 
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(128, 2)
 matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
               const float *__restrict__ sb, const float *__restrict__ rowsum, float *__restrict__ y,
               uint32_t M, uint32_t N, uint32_t K, uint32_t *status)
