@@ -374,32 +374,34 @@ def run_ours(args):
             extra["aggregate_8_clients"] = {"unavailable": str(err)}
 
         # forward path fused into a GEMM (tensor cores): a 2048 x 8192 feed-forward matrix, 8192 tokens
-        try:
-            Mm, Nm, Km = 8192, 8192, 2048
-            pm = omc.Plan([Nm * Km], [0], (5, 10))
-            bm = (z(pm.packed_bytes, torch.uint8), z(16, torch.float32), z(2, torch.float32), z(pm.workspace_bytes, torch.uint8))
-            pm.prepare(bm[3].data_ptr(), stream)
-            wsrc = torch.randn(Nm * Km, device=dev) * 0.02
-            pm.compress(wsrc.data_ptr(), bm[0].data_ptr(), bm[1].data_ptr(), bm[2].data_ptr(), bm[3].data_ptr(), stream)
-            xh = (torch.randn(Mm, Km, device=dev) * 0.5).half()
-            yo = torch.empty(Mm, Nm, dtype=torch.float32, device=dev)
-            rs = torch.empty(Mm, dtype=torch.float32, device=dev)
-            fn = lambda: omc.matmul(pm, 0, bm[0].data_ptr(), bm[2].data_ptr(), xh.data_ptr(), Mm, Nm, Km, yo.data_ptr(),
-                                    rs.data_ptr(), stream)
-            for _ in range(3):
-                fn()
-            torch.cuda.synchronize()
-            e0.record()
-            for _ in range(10):
-                fn()
-            e1.record()
-            torch.cuda.synchronize()
-            t_ms = e0.elapsed_time(e1) / 10
-            extra["matmul_from_codes_8192x8192x2048"] = {"ms": t_ms, "tflops": 2.0 * Mm * Nm * Km / (t_ms * 1e9),
-                                                         "status": pm.status(stream)}
-            del wsrc, xh, yo
-        except omc.OmcError as err:
-            extra["matmul_from_codes_8192x8192x2048"] = {"unavailable": str(err)}
+        Mm, Nm, Km = 8192, 8192, 2048
+        wsrc = torch.randn(Nm * Km, device=dev) * 0.02
+        xh = (torch.randn(Mm, Km, device=dev) * 0.5).half()
+        yo = torch.empty(Mm, Nm, dtype=torch.float32, device=dev)
+        rs = torch.empty(Mm, dtype=torch.float32, device=dev)
+        for mfmt in ((5, 10), (5, 6), (5, 2)):
+            key = "matmul_from_codes_8192x8192x2048_S1E%dM%d" % mfmt
+            try:
+                pm = omc.Plan([Nm * Km], [0], mfmt)
+                bm = (z(pm.packed_bytes, torch.uint8), z(16, torch.float32), z(2, torch.float32),
+                      z(pm.workspace_bytes, torch.uint8))
+                pm.prepare(bm[3].data_ptr(), stream)
+                pm.compress(wsrc.data_ptr(), bm[0].data_ptr(), bm[1].data_ptr(), bm[2].data_ptr(), bm[3].data_ptr(), stream)
+                fn = lambda: omc.matmul(pm, 0, bm[0].data_ptr(), bm[2].data_ptr(), xh.data_ptr(), Mm, Nm, Km,
+                                        yo.data_ptr(), rs.data_ptr(), stream)
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(10):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                t_ms = e0.elapsed_time(e1) / 10
+                extra[key] = {"ms": t_ms, "tflops": 2.0 * Mm * Nm * Km / (t_ms * 1e9), "status": pm.status(stream)}
+            except omc.OmcError as err:
+                extra[key] = {"unavailable": str(err)}
+        del wsrc, xh, yo
 
     if dist is not None:
         dist.barrier()

@@ -15,16 +15,17 @@ from harness import DeviceModel
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("fmt", [(5, 10), (5, 6), (5, 2)], ids=lambda f: "E%dM%d" % f)
 @pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 256, 192), (1000, 384, 512), (64, 128, 1024)])
-def test_matmul_from_codes_matches_definition(M, N, K):
+def test_matmul_from_codes_matches_definition(M, N, K, fmt):
     rng = np.random.default_rng(M + N + K)
     numel = [777, N * K, 64, 128 * 64]
     kinds = [0, 0, 1, 0]
     params = [(rng.standard_normal(n) * 0.05 + 0.01).astype(np.float32) for n in numel]
-    plan = omc.Plan(numel, kinds, (5, 10))
+    plan = omc.Plan(numel, kinds, fmt)
     dm = DeviceModel(plan)
     dm.compress(dm.upload_full(params))
-    st = orc.compress(params, plan.quantised, 5, 10)
+    st = orc.compress(params, plan.quantised, *fmt)
     x = (rng.standard_normal((M, K)) * 0.5).astype(np.float16)
     xd = torch.from_numpy(x).cuda()
     y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
@@ -33,7 +34,7 @@ def test_matmul_from_codes_matches_definition(M, N, K):
                scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     assert plan.status() == 0
-    wbar = orc.decompress_var(st["packed"][1], N * K, 5, 10, st["s"][1], st["b"][1]).reshape(N, K).astype(np.float64)
+    wbar = orc.decompress_var(st["packed"][1], N * K, fmt[0], fmt[1], st["s"][1], st["b"][1]).reshape(N, K).astype(np.float64)
     x64 = x.astype(np.float64)
     want = x64 @ wbar.T
     bound = 1e-3 * (np.abs(x64) @ np.abs(wbar).T + abs(float(st["b"][1])) * np.abs(x64).sum(1, keepdims=True)) + 1e-7
@@ -45,7 +46,7 @@ def test_matmul_from_codes_matches_definition(M, N, K):
 def test_matmul_argument_checks():
     plan = omc.Plan([128 * 64, 100], [0, 1], (5, 10))
     dm = DeviceModel(plan)
-    p8 = omc.Plan([128 * 64], [0], (5, 2))
+    p8 = omc.Plan([128 * 64], [0], (4, 3))
     d8 = DeviceModel(p8)
     x = torch.zeros(128 * 64, dtype=torch.float16, device="cuda")
     y = torch.zeros(128 * 128, dtype=torch.float32, device="cuda")
