@@ -29,7 +29,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per launch of the fused kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by workload name; None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"conformer_like_17b_d512": 794_979_328}   # profiles/fused_update_conformer_100m_e5m10.md
+# The capture is of the default configuration (format, fraction and plan switches as the workload sets them).
+NCU_TRAFFIC_BYTES = {"conformer_like_17b_d512": 794_499_072}   # profiles/fused_update_conformer_100m_e5m10.md
 
 
 def make_workload(name):
@@ -436,7 +437,8 @@ def run_ours(args):
         "gpu_launches": args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": peak_kind + " copy bandwidth", "kernel": "omc_kernel<UPDATE>",
-                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name)},
+                     "traffic": None if (args.format or args.fraction or args.no_pvt or args.all_variables)
+                     else NCU_TRAFFIC_BYTES.get(wl.name)},
         "cpu_baseline": cpu,
         "other_kernels": extra,
     }
