@@ -1077,6 +1077,11 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_aggregate_kernel(con
     }
     uint32_t v = lo;
     const float kf = (float)p.nclients;
+    // Dividing by a power of two is a multiplication by its exact reciprocal: both are the correctly
+    // rounded value of the same real number.
+    const bool pow2 = (p.nclients & (p.nclients - 1)) == 0;
+    const float kinv = 1.f / kf;
+    auto mean_of = [&](float a) { return pow2 ? __fmul_rn(a, kinv) : __fdiv_rn(a, kf); };
     // per warp: what the unit loop needs to know about each client's copy of the current variable
     struct ClientVar { uint64_t base; uint32_t nwords; uint32_t quantised; float s, b; uint32_t pad[2]; };
     __shared__ ClientVar cv_all[WARPS_PER_CTA][MAX_CLIENTS];
@@ -1103,40 +1108,72 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_aggregate_kernel(con
         const uint64_t e_begin = (uint64_t)local * TILE;
         const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
         const uint64_t n_pad = (var.n + 3) & ~3ull;
-        for (uint64_t e0 = e_begin + (uint64_t)lane * LU; e0 < e_end; e0 += U::STEP) {
-            float acc[LU];
+        // A lane takes AL consecutive elements per step: at least 8, so that its codes are 8 to 16
+        // contiguous bytes per client (one vector load where the width allows it).
+        constexpr int UF = LU < 8 ? 8 / LU : 1, AL = LU * UF, ANW = NW * UF;
+        for (uint64_t e0 = e_begin + (uint64_t)lane * AL; e0 < e_end; e0 += 32 * AL) {
+            float acc[AL];
 #pragma unroll
-            for (int j = 0; j < LU; ++j) acc[j] = 0.f;
-            for (uint32_t k = 0; k < p.nclients; ++k) {
-                const ClientVar c = cv[k];
-                float x[LU];
-                if (c.quantised) {
-                    const uint32_t *cw = reinterpret_cast<const uint32_t *>(c.base);
-                    const uint64_t w0 = e0 / LU * NW;
-                    uint32_t win[NW];
+            for (int j = 0; j < AL; ++j) acc[j] = 0.f;
+            const uint64_t w0 = e0 / AL * ANW;
+            // clients in batches: first every load of the batch, then the arithmetic, in index order
+            constexpr int KB = AL >= 32 ? 1 : 4, WMAX = ANW > AL ? ANW : AL;
+            for (uint32_t k0 = 0; k0 < p.nclients; k0 += KB) {
+                uint32_t w[KB][WMAX];
 #pragma unroll
-                    for (int j = 0; j < NW; ++j) win[j] = (w0 + j < c.nwords) ? __ldcs(cw + w0 + j) : 0u;
+                for (int kk = 0; kk < KB; ++kk) {
+                    if (k0 + kk >= p.nclients) break;
+                    const ClientVar c = cv[k0 + kk];
+                    if (c.quantised) {
+                        // packed sizes are multiples of 16 bytes: an aligned 8- or 16-byte group is inside or outside as a whole
+                        const uint32_t *cw = reinterpret_cast<const uint32_t *>(c.base) + w0;
+                        if constexpr (ANW == 4) {
+                            const uint4 q = (w0 < c.nwords) ? __ldcs(reinterpret_cast<const uint4 *>(cw)) : make_uint4(0u, 0u, 0u, 0u);
+                            w[kk][0] = q.x; w[kk][1] = q.y; w[kk][2] = q.z; w[kk][3] = q.w;
+                        } else if constexpr (ANW == 2) {
+                            const uint2 q = (w0 < c.nwords) ? __ldcs(reinterpret_cast<const uint2 *>(cw)) : make_uint2(0u, 0u);
+                            w[kk][0] = q.x; w[kk][1] = q.y;
+                        } else {
 #pragma unroll
-                    for (int j = 0; j < LU; ++j)
-                        x[j] = __fmaf_rn(c.s, decode_exact<F>(get_code_at<F, NW>(win, j * F::B)), c.b);
-                } else {
-                    const float *r = reinterpret_cast<const float *>(c.base) + e0;
+                            for (int j = 0; j < ANW; ++j) w[kk][j] = (w0 + j < c.nwords) ? __ldcs(cw + j) : 0u;
+                        }
+                    } else {
+                        const float *r = reinterpret_cast<const float *>(c.base) + e0;
 #pragma unroll
-                    for (int j = 0; j < LU / 4; ++j) {
-                        const float4 q = (e0 + 4 * j < n_pad) ? __ldcs(reinterpret_cast<const float4 *>(r) + j)
-                                                              : make_float4(0.f, 0.f, 0.f, 0.f);
-                        x[4 * j] = q.x; x[4 * j + 1] = q.y; x[4 * j + 2] = q.z; x[4 * j + 3] = q.w;
+                        for (int j = 0; j < AL / 4; ++j) {
+                            const float4 q = (e0 + 4 * j < n_pad) ? __ldcs(reinterpret_cast<const float4 *>(r) + j)
+                                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+                            w[kk][4 * j] = __float_as_uint(q.x); w[kk][4 * j + 1] = __float_as_uint(q.y);
+                            w[kk][4 * j + 2] = __float_as_uint(q.z); w[kk][4 * j + 3] = __float_as_uint(q.w);
+                        }
                     }
                 }
 #pragma unroll
-                for (int j = 0; j < LU; ++j) acc[j] = (k == 0) ? x[j] : __fadd_rn(acc[j], x[j]);
+                for (int kk = 0; kk < KB; ++kk) {
+                    if (k0 + kk >= p.nclients) break;
+                    const ClientVar c = cv[k0 + kk];
+                    float x[AL];
+                    if (c.quantised) {
+                        uint32_t win[ANW];
+#pragma unroll
+                        for (int j = 0; j < ANW; ++j) win[j] = w[kk][j];
+#pragma unroll
+                        for (int j = 0; j < AL; ++j)
+                            x[j] = __fmaf_rn(c.s, decode_exact<F>(get_code_at<F, ANW>(win, j * F::B)), c.b);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < AL; ++j) x[j] = __uint_as_float(w[kk][j]);
+                    }
+#pragma unroll
+                    for (int j = 0; j < AL; ++j) acc[j] = (k0 + kk == 0) ? x[j] : __fadd_rn(acc[j], x[j]);
+                }
             }
             float *o = p.out + var.full_off + e0;
 #pragma unroll
-            for (int j = 0; j < LU / 4; ++j)
+            for (int j = 0; j < AL / 4; ++j)
                 if (e0 + 4 * j < n_pad)
-                    reinterpret_cast<float4 *>(o)[j] = make_float4(__fdiv_rn(acc[4 * j], kf), __fdiv_rn(acc[4 * j + 1], kf),
-                                                                   __fdiv_rn(acc[4 * j + 2], kf), __fdiv_rn(acc[4 * j + 3], kf));
+                    reinterpret_cast<float4 *>(o)[j] = make_float4(mean_of(acc[4 * j]), mean_of(acc[4 * j + 1]),
+                                                                   mean_of(acc[4 * j + 2]), mean_of(acc[4 * j + 3]));
         }
         t += cnt;
         ++v;

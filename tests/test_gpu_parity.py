@@ -354,14 +354,14 @@ def test_transition_refuses_mismatched_plans():
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("K", [5, 8], ids=lambda k: "K%d" % k)
 @pytest.mark.parametrize("fmt", [(5, 2), (5, 6), (5, 10), (3, 7), (4, 14)], ids=lambda f: "E%dM%d" % f)
-def test_aggregate_client_replicas(fmt):
+def test_aggregate_client_replicas(fmt, K):
     """Server-side mean of K clients that each quantised their own random subset (Sec. 2.5): the
     oracle decompresses every client and averages in FP32, clients in index order, one division."""
     rng = np.random.default_rng(7)
     numel = [3000, 1, 1024, 5121, 333, 40000, 12289, 77]
     kinds = [0, 0, 0, 0, 1, 0, 0, 2]
-    K = 5
     base = [(rng.standard_normal(n) * 0.1).astype(np.float32) for n in numel]
     clients = []
     for k in range(K):
