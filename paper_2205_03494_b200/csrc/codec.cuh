@@ -187,6 +187,39 @@ __device__ __forceinline__ bool needs_exact_encode(float w)
     return a >= F::OVF_BITS;
 }
 
+// The same two tests for four elements at once, on values instead of bit patterns: one maximum
+// of magnitudes (a NaN among them wins) and one comparison replace four integer comparisons.
+__device__ __forceinline__ float absmax4(float a, float b, float c, float d)
+{
+    float r;
+    asm("{\n\t.reg .f32 t0, t1, t2, t3;\n\t"
+        "abs.f32 t0, %1;\n\tabs.f32 t1, %2;\n\tabs.f32 t2, %3;\n\tabs.f32 t3, %4;\n\t"
+        "max.NaN.f32 t2, t2, t3;\n\t"
+        "max.NaN.f32 %0, t0, t1, t2;\n\t}"
+        : "=f"(r) : "f"(a), "f"(b), "f"(c), "f"(d));
+    return r;
+}
+
+// dec = decode_fast of four codes: a code with an all-ones exponent field decodes to a magnitude
+// of at least 2^(EMAX+1), every other code to less.
+template <class F>
+__device__ __forceinline__ bool any_code_special4(const float (&dec)[4])
+{
+    if constexpr (F::E == 8 || HalfPath<F>::value) return false;
+    else return absmax4(dec[0], dec[1], dec[2], dec[3]) >= u2f(F::pow2_bits(F::EMAX + 1));
+}
+
+template <class F, bool KEEP_PAYLOAD>
+__device__ __forceinline__ bool any_needs_exact_encode4(const float (&w)[4])
+{
+    if constexpr (HalfPath<F>::value && F::M == 10 && !KEEP_PAYLOAD) return false;
+    else {
+        const float m = absmax4(w[0], w[1], w[2], w[3]);
+        if constexpr ((HalfPath<F>::value && F::M == 10) || F::E == 8) return m != m;      // NaN only
+        else return !(m < u2f(F::OVF_BITS));                                               // overflow, Inf, NaN
+    }
+}
+
 // NaN -> sign, all-ones exponent, top M payload bits (a quiet bit is forced if those are zero;
 // with M == 0 there is no NaN code and infinity is written).
 template <class F>

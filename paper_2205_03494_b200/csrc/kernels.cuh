@@ -59,19 +59,19 @@ template <class F, int MODE, bool WOUT>
 struct Smem {
     static constexpr int SUB = Unit<F>::SUB;
     static constexpr int OUTBUFS = Unit<F>::OUTBUFS;
-    static constexpr bool ROWS = (Unit<F>::LU == 32);   // FP32 data in padded rows, one per lane
+    static constexpr bool ROWS = (Unit<F>::LU == 32);   // a lane reads and writes FP32 data as one 128-byte row
     static constexpr int CB = SUB * F::B / 8;     // bytes of one granule's codes
-    static constexpr int FB = ROWS ? 32 * 144 : SUB * 4;   // shared-memory bytes of one granule's FP32 data
-    static constexpr int FB_GLOBAL = SUB * 4;     // ... and its bytes in global memory
+    static constexpr int FB = SUB * 4;            // bytes of one granule's FP32 data
     static constexpr int IN_C = (MODE != COMPRESS) ? CB : 0;
     static constexpr int IN_F = (MODE != DECOMPRESS) ? FB : 0;
     static constexpr int STAGE = IN_C + IN_F;
-    static constexpr int TX_BYTES = IN_C + (IN_F ? FB_GLOBAL : 0);   // what the stage's copies bring in
+    static constexpr int TX_BYTES = STAGE;        // what the stage's copies bring in
     static constexpr int DIST = STAGES - 1;       // granules fetched ahead
     static constexpr int OUT_C = (MODE != DECOMPRESS) ? CB : 0;
     static constexpr int OUT_F = (MODE == DECOMPRESS || WOUT) ? FB : 0;
     static constexpr int OUT = OUT_C + OUT_F;
     static constexpr int PER_WARP = STAGES * STAGE + OUTBUFS * OUT;
+    static_assert(!ROWS || (STAGE % 128 == 0 && OUT % 128 == 0 && CB % 128 == 0), "row layout: FP32 granules stay 128-byte aligned");
     static constexpr int BAR_PAD = (8 * STAGES * WARPS_PER_CTA + 127) / 128 * 128;   // the mbarriers
     static constexpr int TOTAL = BAR_PAD + WARPS_PER_CTA * PER_WARP;
     static_assert(STAGE % 16 == 0 && CB % 16 == 0, "bulk copies move multiples of 16 bytes");
@@ -287,18 +287,21 @@ __device__ __forceinline__ void compute_group(const uint32_t (&win)[NWI], int g,
     uint32_t cin[4], cout[4];
     float vt[4];
     bool bad = false;
+    if constexpr (HAS_CIN) {
+        float dec[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        if constexpr (HAS_CIN) {
+        for (int j = 0; j < 4; ++j) {
             cin[j] = get_code_at<F, NWI>(win, (4 * g + j) * F::B - bitbase);
-            bad |= code_is_special<F>(cin[j]);
-            const float vbar = __fmaf_rn(s, decode_fast<F>(cin[j]), b);
+            dec[j] = decode_fast<F>(cin[j]);
+            const float vbar = __fmaf_rn(s, dec[j], b);
             w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
-        } else {
-            w[j] = fin4[j];
         }
-        if constexpr (MODE != DECOMPRESS) bad |= needs_exact_encode<F, KEEP_PAYLOAD>(w[j]);
+        bad = any_code_special4<F>(dec);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) w[j] = fin4[j];
     }
+    if constexpr (MODE != DECOMPRESS) bad |= any_needs_exact_encode4<F, KEEP_PAYLOAD>(w);
     if constexpr (MODE != DECOMPRESS) {
         encode_fast2<F>(w[0], w[1], cout[0], cout[1], vt[0], vt[1]);
         encode_fast2<F>(w[2], w[3], cout[2], cout[3], vt[2], vt[3]);
@@ -358,7 +361,30 @@ __device__ __forceinline__ void compute_unit(const uint32_t (&win)[Unit<F>::NWOR
 // A full unit of 32 elements per lane (odd code widths) whose FP32 operand and FP32 result live in
 // shared-memory rows: the operand is fetched four elements at a time right where it is used and
 // the result is stored at once, so that a lane never holds 32 values in registers.
-constexpr int ROW_FLOATS = 36;     // 32 values + 16 bytes: lanes 144 bytes apart hit different banks
+//
+// Row layout of a granule of 1024 FP32 values (4 KB, 128-byte aligned): lane l owns values
+// 32 l .. 32 l + 31, a 128-byte row, and its 16-byte chunk c sits at chunk c xor (l mod 8) of
+// the row, so that the eight lanes of a quarter warp touch all 32 banks.  The bulk copies move
+// dense granules; the warp swizzles them in place (eight 16-byte loads, eight stores per lane).
+__device__ __forceinline__ void rows_swizzle_in_place(float *granule, int lane, bool to_rows)
+{
+    float4 *g4 = reinterpret_cast<float4 *>(granule);
+    float4 v[8];
+    // float4 number 32 i + lane of the dense granule is chunk lane mod 8 of row 4 i + lane / 8
+    const int c = lane & 7;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + (lane >> 3);
+        v[i] = g4[to_rows ? 32 * i + lane : r * 8 + (c ^ (r & 7))];
+    }
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + (lane >> 3);
+        g4[to_rows ? r * 8 + (c ^ (r & 7)) : 32 * i + lane] = v[i];
+    }
+    __syncwarp();
+}
 
 __device__ __forceinline__ uint32_t lds_volatile(uint32_t shared_addr)
 {
@@ -372,13 +398,16 @@ __device__ __forceinline__ uint32_t lds_volatile(uint32_t shared_addr)
 // top), finished output words are stored at once, and a word shared by two groups is carried in
 // one register.  `cin` / `cout` / `fin_row` / `fout_row` are this lane's slices in shared memory.
 template <class F, int MODE, bool WOUT>
-__device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const float *fin_row, uint32_t *cout,
-                                                  float *fout_row, float s, float b, float neg_lr, Acc &acc)
+__device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const float *fin_granule, uint32_t *cout,
+                                                  float *fout_granule, float s, float b, float neg_lr, Acc &acc, int lane)
 {
     constexpr int LU = Unit<F>::LU, B = F::B;
     constexpr int GW = (4 * B + 31) / 32 + 1;      // words a group of four codes can touch
     uint32_t ref = 0u, diff = 0u, carry = 0u;
-    const uint32_t cin_a = smem_addr(cin), fin_a = smem_addr(fin_row);     // shared-window addresses, once
+    const uint32_t cin_a = smem_addr(cin);                                 // shared-window addresses, once
+    // chunk g of this lane's row: (row | swizzle) xor 16 g, the granule being 128-byte aligned
+    const uint32_t row_sw = (uint32_t)lane * 128u + (((uint32_t)lane & 7u) << 4);
+    const uint32_t fin_a = smem_addr(fin_granule) + row_sw, fout_a = smem_addr(fout_granule) + row_sw;
     StaticFor<0, LU / 4>::run([&](auto gi) {
         constexpr int g = decltype(gi)::value;
         constexpr int bit0 = 4 * g * B, f0 = bit0 >> 5, cnt = ((bit0 + 4 * B - 1) >> 5) - f0 + 1;
@@ -394,7 +423,7 @@ __device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const flo
         if constexpr (MODE != DECOMPRESS) {
             float4 v;
             asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(fin_a + 16u * g));
+                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(fin_a ^ (16u * g)));
             fin4[0] = v.x; fin4[1] = v.y; fin4[2] = v.z; fin4[3] = v.w;
         }
         float w[4];
@@ -406,7 +435,8 @@ __device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const flo
             carry = ends_on_word ? 0u : ow[cnt - 1];
         }
         if constexpr (MODE == DECOMPRESS || WOUT)
-            reinterpret_cast<float4 *>(fout_row)[g] = make_float4(w[0], w[1], w[2], w[3]);
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};"
+                         ::"r"(fout_a ^ (16u * g)), "f"(w[0]), "f"(w[1]), "f"(w[2]), "f"(w[3]) : "memory");
     });
     if constexpr (MODE != DECOMPRESS) {
         acc.band &= ref & ~diff;
@@ -598,9 +628,8 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
 {
     using U = Unit<F>;
     constexpr int LU = U::LU, NW = U::NWORDS;
-    if constexpr (LU == 32) {       // one unit per lane; FP32 data in rows of ROW_FLOATS
-        compute_unit_rows<F, MODE, WOUT>(s_cin + lane * NW, s_fin + lane * ROW_FLOATS, s_cout + lane * NW,
-                                         s_fout + lane * ROW_FLOATS, s, b, neg_lr, acc);
+    if constexpr (LU == 32) {       // one unit per lane; FP32 data in swizzled 128-byte rows
+        compute_unit_rows<F, MODE, WOUT>(s_cin + lane * NW, s_fin, s_cout + lane * NW, s_fout, s, b, neg_lr, acc, lane);
         return;
     }
     constexpr int G = (U::SUB_STEPS >= 2 && LU == 4) ? 2 : 1;   // steps whose operands are fetched together
@@ -747,8 +776,7 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
     const uint32_t g0 = (uint32_t)(e_begin / SUB);                  // first granule
     const uint32_t ng = (uint32_t)((e_end - e_begin) / SUB);        // whole granules
 
-    constexpr bool ROWS_IN = SM::ROWS && SM::IN_F > 0;      // every lane copies its own row in
-    constexpr bool ROWS_OUT = SM::ROWS && SM::OUT_F > 0;    // ... and stores its own row
+    constexpr bool ROWS_IN = SM::ROWS && SM::IN_F > 0, ROWS_OUT = SM::ROWS && SM::OUT_F > 0;
     auto issue = [&](uint32_t g, uint32_t kk) {           // called by the whole warp
         const uint32_t st = kk % STAGES;
         const uint32_t bar = bar0 + 8u * st;
@@ -757,12 +785,8 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
             mbar_expect_tx(bar, (uint32_t)SM::TX_BYTES);
             if constexpr (SM::IN_C > 0)
                 bulk_load(smem_addr(dst), codes + (size_t)g * SM::CB, SM::CB, bar);
-            if constexpr (SM::IN_F > 0 && !ROWS_IN)
+            if constexpr (SM::IN_F > 0)
                 bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)g * SUB, SM::FB, bar);
-        }
-        if constexpr (ROWS_IN) {
-            __syncwarp();      // the expectation is posted before any of the row copies can complete
-            bulk_load(smem_addr(dst + SM::IN_C + lane * (ROW_FLOATS * 4)), fin + (size_t)g * SUB + lane * 32, 128u, bar);
         }
     };
 
@@ -770,7 +794,7 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
     for (uint32_t i = 0; i < ng; ++i, ++k) {
         const uint32_t g = g0 + i;
         if (i + SM::DIST < ng) issue(g + SM::DIST, k + SM::DIST);   // its stage was consumed last round
-        if (lane == 0 || ROWS_OUT) {
+        if (lane == 0) {
             // the output buffer written next must have left with its last store
             if constexpr (SM::OUTBUFS == 2) bulk_wait_read1(); else bulk_wait_read0();
         }
@@ -784,21 +808,24 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
         if (failed) break;
         uint8_t *stage = wbase + st * SM::STAGE;
         uint8_t *ob = outs + (k % SM::OUTBUFS) * SM::OUT;
-        granule_from_smem<F, MODE, WOUT>(reinterpret_cast<const uint32_t *>(stage),
-                                         reinterpret_cast<const float *>(stage + SM::IN_C),
-                                         reinterpret_cast<uint32_t *>(ob),
-                                         reinterpret_cast<float *>(ob + SM::OUT_C), s, b, neg_lr, acc, lane);
+        const float *fsrc = reinterpret_cast<const float *>(stage + SM::IN_C);
+        float *fdst = reinterpret_cast<float *>(ob + SM::OUT_C);
+        if constexpr (ROWS_IN) rows_swizzle_in_place(const_cast<float *>(fsrc), lane, true);
+        granule_from_smem<F, MODE, WOUT>(reinterpret_cast<const uint32_t *>(stage), fsrc, reinterpret_cast<uint32_t *>(ob),
+                                         fdst, s, b, neg_lr, acc, lane);
+        if constexpr (ROWS_OUT) {
+            __syncwarp();
+            rows_swizzle_in_place(fdst, lane, false);
+        }
         fence_proxy_async();           // make the results visible to the bulk store
         __syncwarp();
         if (lane == 0) {
             if constexpr (MODE != DECOMPRESS)
                 bulk_store(codes + (size_t)g * SM::CB, smem_addr(ob), SM::CB);
-            if constexpr (SM::OUT_F > 0 && !ROWS_OUT)
+            if constexpr (SM::OUT_F > 0)
                 bulk_store(fout + (size_t)g * SUB, smem_addr(ob + SM::OUT_C), SM::FB);
+            bulk_commit();
         }
-        if constexpr (ROWS_OUT)
-            bulk_store(fout + (size_t)g * SUB + lane * 32, smem_addr(ob + SM::OUT_C + lane * (ROW_FLOATS * 4)), 128u);
-        if (lane == 0 || ROWS_OUT) bulk_commit();
     }
     if (failed) { pipe.k = k; pipe.failed = true; return; }
     const uint64_t e_rag = e_begin + (uint64_t)ng * SUB;
