@@ -266,6 +266,25 @@ __device__ __forceinline__ uint32_t get_code_at(const uint32_t (&w)[NW], int pos
     return c & F::CODE_MASK;
 }
 
+// decode_fast of the code at bit position `pos`, without isolating the code first: one shift
+// puts the code's sign at bit 31 (whatever follows the code stays in the low bits), a second one
+// and a mask put exponent and mantissa where FP32 keeps them, and the sign is merged after the
+// rebias multiplication.  Formats on the generic path only (E < 8, not the FP16 family).
+template <class F, int NW>
+__device__ __forceinline__ float decode_fast_at(const uint32_t (&w)[NW], int pos)
+{
+    static_assert(F::E < 8 && !HalfPath<F>::value, "generic path");
+    const int wi = pos >> 5, sh = pos & 31;
+    uint32_t t;      // the code in the top B bits
+    if (sh + F::B <= 32)
+        t = w[wi] << (32 - sh - F::B);
+    else
+        t = __funnelshift_r(w[wi], w[(wi + 1 < NW) ? wi + 1 : wi], sh + F::B - 32);
+    const uint32_t mag = (t >> (8 - F::E)) & (F::MAG_MASK << F::SH);
+    const float v = __fmul_rn(u2f(mag), u2f(F::pow2_bits(127 - F::BIAS)));
+    return u2f(f2u(v) | (t & 0x80000000u));
+}
+
 template <class F, int NW>
 __device__ __forceinline__ void put_code_at(uint32_t (&w)[NW], int pos, uint32_t c)
 {

@@ -67,7 +67,10 @@ struct Smem {
     static constexpr int STAGE = IN_C + IN_F;
     static constexpr int TX_BYTES = STAGE;        // what the stage's copies bring in
     static constexpr int DIST = STAGES - 1;       // granules fetched ahead
-    static constexpr int OUT_C = (MODE != DECOMPRESS) ? CB : 0;
+    // Row layout, fused round: a lane rewrites its own code words behind its reads, so the new codes
+    // take the place of the old ones in the stage and are stored from there.
+    static constexpr bool CODES_IN_PLACE = ROWS && MODE == UPDATE;
+    static constexpr int OUT_C = (MODE != DECOMPRESS && !CODES_IN_PLACE) ? CB : 0;
     static constexpr int OUT_F = (MODE == DECOMPRESS || WOUT) ? FB : 0;
     static constexpr int OUT = OUT_C + OUT_F;
     static constexpr int PER_WARP = STAGES * STAGE + OUTBUFS * OUT;
@@ -284,6 +287,7 @@ __device__ __forceinline__ void compute_group(const uint32_t (&win)[NWI], int g,
 {
     constexpr bool HAS_CIN = (MODE != COMPRESS);
     constexpr bool KEEP_PAYLOAD = (MODE == COMPRESS);    // UPDATE gives arithmetic NaNs one pattern
+    constexpr bool GENERIC = F::E < 8 && !HalfPath<F>::value;   // codes are isolated only on the careful path
     uint32_t cin[4], cout[4];
     float vt[4];
     bool bad = false;
@@ -291,8 +295,12 @@ __device__ __forceinline__ void compute_group(const uint32_t (&win)[NWI], int g,
         float dec[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            cin[j] = get_code_at<F, NWI>(win, (4 * g + j) * F::B - bitbase);
-            dec[j] = decode_fast<F>(cin[j]);
+            if constexpr (GENERIC) {
+                dec[j] = decode_fast_at<F, NWI>(win, (4 * g + j) * F::B - bitbase);
+            } else {
+                cin[j] = get_code_at<F, NWI>(win, (4 * g + j) * F::B - bitbase);
+                dec[j] = decode_fast<F>(cin[j]);
+            }
             const float vbar = __fmaf_rn(s, dec[j], b);
             w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
         }
@@ -310,6 +318,7 @@ __device__ __forceinline__ void compute_group(const uint32_t (&win)[NWI], int g,
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             if constexpr (HAS_CIN) {
+                if constexpr (GENERIC) cin[j] = get_code_at<F, NWI>(win, (4 * g + j) * F::B - bitbase);
                 const float vbar = __fmaf_rn(s, decode_exact<F>(cin[j]), b);
                 w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, fin4[j], vbar) : vbar;
                 // a NaN made by the arithmetic gets one fixed pattern
@@ -793,8 +802,12 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
     for (uint32_t i = 0; i < (uint32_t)SM::DIST && i < ng; ++i) issue(g0 + i, k + i);
     for (uint32_t i = 0; i < ng; ++i, ++k) {
         const uint32_t g = g0 + i;
+        if constexpr (SM::CODES_IN_PLACE) {
+            if (lane == 0) bulk_wait_read0();      // the stage refilled next was stored from last round
+            __syncwarp();
+        }
         if (i + SM::DIST < ng) issue(g + SM::DIST, k + SM::DIST);   // its stage was consumed last round
-        if (lane == 0) {
+        if (lane == 0 && !SM::CODES_IN_PLACE) {
             // the output buffer written next must have left with its last store
             if constexpr (SM::OUTBUFS == 2) bulk_wait_read1(); else bulk_wait_read0();
         }
@@ -811,7 +824,8 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
         const float *fsrc = reinterpret_cast<const float *>(stage + SM::IN_C);
         float *fdst = reinterpret_cast<float *>(ob + SM::OUT_C);
         if constexpr (ROWS_IN) rows_swizzle_in_place(const_cast<float *>(fsrc), lane, true);
-        granule_from_smem<F, MODE, WOUT>(reinterpret_cast<const uint32_t *>(stage), fsrc, reinterpret_cast<uint32_t *>(ob),
+        uint8_t *cdst = SM::CODES_IN_PLACE ? stage : ob;
+        granule_from_smem<F, MODE, WOUT>(reinterpret_cast<const uint32_t *>(stage), fsrc, reinterpret_cast<uint32_t *>(cdst),
                                          fdst, s, b, neg_lr, acc, lane);
         if constexpr (ROWS_OUT) {
             __syncwarp();
@@ -821,7 +835,7 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
         __syncwarp();
         if (lane == 0) {
             if constexpr (MODE != DECOMPRESS)
-                bulk_store(codes + (size_t)g * SM::CB, smem_addr(ob), SM::CB);
+                bulk_store(codes + (size_t)g * SM::CB, smem_addr(cdst), SM::CB);
             if constexpr (SM::OUT_F > 0)
                 bulk_store(fout + (size_t)g * SUB, smem_addr(ob + SM::OUT_C), SM::FB);
             bulk_commit();
