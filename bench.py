@@ -271,6 +271,19 @@ def run_ours(args):
     ms = max_over_ranks(ms, dist, dev)
     ms_per_step = ms / args.steps
 
+    # ---- spread of the same step: ten more chunks, each timed by its own pair of events
+    chunk = max(1, args.steps // 10)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(11)]
+    evs[0].record()
+    for c in range(10):
+        for _ in range(chunk):
+            step()
+        evs[c + 1].record()
+    torch.cuda.synchronize()
+    chunk_ms = sorted(evs[c].elapsed_time(evs[c + 1]) / chunk for c in range(10))
+    spread = {"chunks": 10, "steps_per_chunk": chunk, "best": chunk_ms[0], "median": 0.5 * (chunk_ms[4] + chunk_ms[5]),
+              "worst": chunk_ms[-1]}
+
     # ---- end to end: gradients start in pinned host memory, (s, b) is read back, every step
     host_sb = torch.zeros(max(2 * plan.n_quantised, 1), dtype=torch.float32, pin_memory=True)
     e2e_steps = max(3, min(args.steps, 10))
@@ -420,9 +433,14 @@ def run_ours(args):
         rate, n_s, dt = cpu_oracle_rate(wl, threads, which)
         cpu = {"value": rate, "unit": "params/s", "cores": threads, "kind": "oracle",
                "sample": "1 round over %d variables (%d params) of %s, %.1f s wall" % (len(which), n_s, wl.name, dt)}
+        which1 = sample_vars(wl, 20_000_000)
+        rate1, n1, dt1 = cpu_oracle_rate(wl, 1, which1)
+        cpu["single_thread"] = {"value": rate1, "unit": "params/s", "cores": 1,
+                                "sample": "1 round over %d variables (%d params), %.1f s wall" % (len(which1), n1, dt1)}
     line = {
         "metric": METRIC, "value": replica_value(nparams, world, ms_per_step), "unit": "params/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "ms_per_step_spread": spread,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "%s S1E%dM%d p=%g" % (wl.name, wl.fmt[0], wl.fmt[1], wl.fraction),
                    "params": nparams, "variables": plan.nvars, "quantised_variables": plan.n_quantised,
