@@ -874,7 +874,10 @@ omc_kernel(const KParams p)
 {
     using SM = Smem<F, MODE, WOUT>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    const int lane = threadIdx.x & 31;
+    // read once (volatile): otherwise the compiler re-reads the special register all over the main
+    // loop instead of keeping the lane number in a register
+    int lane;
+    asm volatile("mov.u32 %0, %%laneid;" : "=r"(lane));
     const int wid = threadIdx.x >> 5;
     const uint32_t warp = blockIdx.x * WARPS_PER_CTA + wid;
     if (warp >= p.nwarps) return;
