@@ -36,6 +36,10 @@ constexpr uint32_t WAIT_LIMIT = 1u << 24;   // polls of one mbarrier before givi
 #define OMC_OUTBUFS 0
 #endif
 
+#ifndef OMC_GRANULE_UNROLL
+#define OMC_GRANULE_UNROLL 0          // 0: per format (measured), else the unroll factor of the granule loop
+#endif
+
 // How many consecutive elements one lane takes per step: the smallest run whose codes fill
 // whole 32-bit words.
 template <class F>
@@ -642,7 +646,8 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
         return;
     }
     constexpr int G = (U::SUB_STEPS >= 2 && LU == 4) ? 2 : 1;   // steps whose operands are fetched together
-#pragma unroll 1
+    constexpr int UNROLL = OMC_GRANULE_UNROLL ? OMC_GRANULE_UNROLL : (F::B == 8 ? 4 : 1);
+#pragma unroll UNROLL
     for (int k0 = 0; k0 < U::SUB_STEPS; k0 += G) {
         uint32_t win[G][NW];
         float4 fv[G][LU / 4];
