@@ -50,7 +50,7 @@ typedef struct {
 enum { OMC_KIND_WEIGHT_MATRIX = 0, OMC_KIND_BIAS = 1, OMC_KIND_NORM = 2, OMC_KIND_OTHER = 3 };
 
 typedef struct {
-    uint64_t numel;    /* number of FP32 elements, > 0 */
+    uint64_t numel;    /* number of FP32 elements, 1 .. 2^40 */
     uint32_t kind;     /* OMC_KIND_* */
     uint32_t reserved; /* 0 */
 } omc_var_desc_t;

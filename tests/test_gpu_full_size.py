@@ -67,3 +67,82 @@ def test_large_transformer_1p6b_one_round():
     packed = ls.round(wl.all_grads(0), 2.0, want_w=False)
     ls.check_padding(packed)
     assert ls.sb_ulp_cases <= 1, ls.sb_ulp_cases
+
+
+def test_one_variable_beyond_32_bit_indexing():
+    """A single variable of 2^32 + 1,081,344 elements (8-bit codes, fit on): element and byte offsets
+    no longer fit 32 bits.  The variable is one block of 2^20 + 264 values repeated 4096 times, so the
+    oracle's answer for the block is the answer for the whole: the codes repeat, and the least-squares
+    fit of a repeated sample is the fit of the sample (all sums and n scale by 4096 = 2^12, which the
+    closed form cancels exactly; checked below on the CPU with 4 repeats).  Everything is compared on
+    the device, every byte and every value."""
+    from oracle import omc_oracle as orc
+    from harness import ulp_diff
+    free, _ = torch.cuda.mem_get_info()
+    if free < 80e9:
+        pytest.skip("needs about 70 GB of free device memory")
+    E, M, R, m = 5, 2, 4096, (1 << 20) + 264
+    n_big = R * m
+    assert n_big > (1 << 32)
+    rng = np.random.default_rng(2205)
+    block = (rng.standard_normal(m) * 0.05).astype(np.float32)
+    block[:8] = [0.0, -0.0, 1e-8, -3e-6, 6.1e-5, 0.4375, -3.5, 1e-45]
+    gblock = (rng.standard_normal(m) * 1e-3).astype(np.float32)
+    small = [(rng.standard_normal(k) * 0.05).astype(np.float32) for k in (1000, 77)]
+    # oracle on the block (and the invariance it rests on)
+    pk0, s0, b0 = orc.compress_var(block, E, M)
+    pk4, s4, b4 = orc.compress_var(np.tile(block, 4), E, M)
+    assert (s0, b0) == (s4, b4) and np.array_equal(np.tile(pk0[:m], 4), pk4[:4 * m])
+
+    plan = omc.Plan([1000, n_big, 77], [0, 0, 1], (E, M))
+    dev = torch.device("cuda:0")
+    st = torch.cuda.current_stream().cuda_stream
+    z = lambda k, dt: torch.zeros(max(int(k), 16), dtype=dt, device=dev)
+    full = z(plan.full_elems, torch.float32)
+    off = plan.full_off[1]
+    blk_d = torch.from_numpy(block).to(dev)
+    full[off:off + n_big].view(R, m).copy_(blk_d.unsqueeze(0).expand(R, m))
+    full[plan.full_off[0]:plan.full_off[0] + 1000] = torch.from_numpy(small[0]).to(dev)
+    full[plan.full_off[2]:plan.full_off[2] + 77] = torch.from_numpy(small[1]).to(dev)
+    packed, resid = z(plan.packed_bytes, torch.uint8), z(plan.resid_elems, torch.float32)
+    sb, ws = z(2 * plan.n_quantised, torch.float32), z(plan.workspace_bytes, torch.uint8)
+    plan.prepare(ws.data_ptr(), st)
+    plan.compress(full.data_ptr(), packed.data_ptr(), resid.data_ptr(), sb.data_ptr(), ws.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert plan.status(st) == 0
+
+    def check_codes(pk_block, s_want, b_want):
+        po = plan.packed_off[1]
+        want = torch.from_numpy(pk_block[:m].copy()).to(dev)
+        got = packed[po:po + n_big].view(R, m)
+        assert bool((got == want.unsqueeze(0)).all())
+        assert int(packed[po + n_big:po + plan.var_packed_bytes[1]].max().item() if plan.var_packed_bytes[1] > n_big else 0) == 0
+        k = plan.sb_slot[1]
+        s_got, b_got = np.float32(sb[2 * k].item()), np.float32(sb[2 * k + 1].item())
+        assert ulp_diff(s_got, s_want) <= 1, (s_got, s_want)
+        assert abs(float(b_got) - float(b_want)) <= 4 * n_big * 2.0 ** -53 * float(np.abs(block).mean()) + 2.0 ** -23 * abs(float(b_want))
+        return s_got, b_got
+
+    s_g, b_g = check_codes(pk0, s0, b0)
+    # the small neighbours are untouched by the big one
+    pk_s, s_s, b_s = orc.compress_var(small[0], E, M)
+    assert np.array_equal(packed[plan.packed_off[0]:plan.packed_off[0] + 1000].cpu().numpy(), pk_s[:1000])
+    assert np.array_equal(resid[plan.resid_off[2]:plan.resid_off[2] + 77].cpu().numpy(), small[1])
+
+    # decompress: the oracle's values for the block under the (s, b) the library stored
+    del full
+    out = z(plan.full_elems, torch.float32)
+    plan.decompress(packed.data_ptr(), resid.data_ptr(), sb.data_ptr(), out.data_ptr(), 0, None, st)
+    torch.cuda.synchronize()
+    want = torch.from_numpy(orc.decompress_var(pk0, m, E, M, s_g, b_g)).to(dev)
+    assert bool((out[off:off + n_big].view(R, m).view(torch.int32) == want.view(torch.int32).unsqueeze(0)).all())
+
+    # one fused round with a repeated gradient block
+    out.zero_()
+    out[off:off + n_big].view(R, m).copy_(torch.from_numpy(gblock).to(dev).unsqueeze(0).expand(R, m))
+    plan.update_recompress(packed.data_ptr(), resid.data_ptr(), sb.data_ptr(), out.data_ptr(), 2.0, ws.data_ptr(), None, st)
+    torch.cuda.synchronize()
+    assert plan.status(st) == 0
+    pk1, s1, b1 = orc.update_recompress_var(pk0, m, E, M, s_g, b_g, gblock, 2.0)
+    check_codes(pk1, s1, b1)
+    assert not np.array_equal(pk1[:m], pk0[:m])
