@@ -69,8 +69,9 @@ def test_large_transformer_1p6b_one_round():
     assert ls.sb_ulp_cases <= 1, ls.sb_ulp_cases
 
 
-def test_one_variable_beyond_32_bit_indexing():
-    """A single variable of 2^32 + 1,081,344 elements (8-bit codes, fit on): element and byte offsets
+@pytest.mark.parametrize("fmt", [(5, 2), (3, 7), (5, 10)], ids=lambda f: "E%dM%d" % f)
+def test_one_variable_beyond_32_bit_indexing(fmt):
+    """A single variable of 2^32 + 1,081,344 elements (8-, 11- and 16-bit codes, fit on): element and byte offsets
     no longer fit 32 bits.  The variable is one block of 2^20 + 264 values repeated 4096 times, so the
     oracle's answer for the block is the answer for the whole: the codes repeat, and the least-squares
     fit of a repeated sample is the fit of the sample (all sums and n scale by 4096 = 2^12, which the
@@ -81,7 +82,8 @@ def test_one_variable_beyond_32_bit_indexing():
     free, _ = torch.cuda.mem_get_info()
     if free < 80e9:
         pytest.skip("needs about 70 GB of free device memory")
-    E, M, R, m = 5, 2, 4096, (1 << 20) + 264
+    (E, M), R, m = fmt, 4096, (1 << 20) + 264
+    bb = m * (1 + E + M) // 8                 # bytes of one block's codes (m is a multiple of 8)
     n_big = R * m
     assert n_big > (1 << 32)
     rng = np.random.default_rng(2205)
@@ -92,7 +94,7 @@ def test_one_variable_beyond_32_bit_indexing():
     # oracle on the block (and the invariance it rests on)
     pk0, s0, b0 = orc.compress_var(block, E, M)
     pk4, s4, b4 = orc.compress_var(np.tile(block, 4), E, M)
-    assert (s0, b0) == (s4, b4) and np.array_equal(np.tile(pk0[:m], 4), pk4[:4 * m])
+    assert (s0, b0) == (s4, b4) and np.array_equal(np.tile(pk0[:bb], 4), pk4[:4 * bb])
 
     plan = omc.Plan([1000, n_big, 77], [0, 0, 1], (E, M))
     dev = torch.device("cuda:0")
@@ -113,10 +115,10 @@ def test_one_variable_beyond_32_bit_indexing():
 
     def check_codes(pk_block, s_want, b_want):
         po = plan.packed_off[1]
-        want = torch.from_numpy(pk_block[:m].copy()).to(dev)
-        got = packed[po:po + n_big].view(R, m)
+        want = torch.from_numpy(pk_block[:bb].copy()).to(dev)
+        got = packed[po:po + R * bb].view(R, bb)
         assert bool((got == want.unsqueeze(0)).all())
-        assert int(packed[po + n_big:po + plan.var_packed_bytes[1]].max().item() if plan.var_packed_bytes[1] > n_big else 0) == 0
+        assert plan.var_packed_bytes[1] == R * bb          # a multiple of 16: no padding to check
         k = plan.sb_slot[1]
         s_got, b_got = np.float32(sb[2 * k].item()), np.float32(sb[2 * k + 1].item())
         assert ulp_diff(s_got, s_want) <= 1, (s_got, s_want)
@@ -126,7 +128,7 @@ def test_one_variable_beyond_32_bit_indexing():
     s_g, b_g = check_codes(pk0, s0, b0)
     # the small neighbours are untouched by the big one
     pk_s, s_s, b_s = orc.compress_var(small[0], E, M)
-    assert np.array_equal(packed[plan.packed_off[0]:plan.packed_off[0] + 1000].cpu().numpy(), pk_s[:1000])
+    assert np.array_equal(packed[plan.packed_off[0]:plan.packed_off[0] + pk_s.size].cpu().numpy(), pk_s)
     assert np.array_equal(resid[plan.resid_off[2]:plan.resid_off[2] + 77].cpu().numpy(), small[1])
 
     # decompress: the oracle's values for the block under the (s, b) the library stored
@@ -145,4 +147,4 @@ def test_one_variable_beyond_32_bit_indexing():
     assert plan.status(st) == 0
     pk1, s1, b1 = orc.update_recompress_var(pk0, m, E, M, s_g, b_g, gblock, 2.0)
     check_codes(pk1, s1, b1)
-    assert not np.array_equal(pk1[:m], pk0[:m])
+    assert not np.array_equal(pk1[:bb], pk0[:bb])
