@@ -1110,7 +1110,7 @@ void launch_transition(const KParams &p, int grid, void *stream)
 // 128-bit global accesses; every element is read once per client and written once.
 
 template <class F>
-__global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_aggregate_kernel(const AggParams p)
+__global__ void __launch_bounds__(THREADS, Unit<F>::LU == 32 ? CTAS_PER_SM : 4) omc_aggregate_kernel(const AggParams p)
 {
     using U = Unit<F>;
     constexpr int LU = U::LU, NW = U::NWORDS;
@@ -1206,9 +1206,25 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_aggregate_kernel(con
                         uint32_t win[ANW];
 #pragma unroll
                         for (int j = 0; j < ANW; ++j) win[j] = w[kk][j];
+                        if constexpr (F::E < 8 && !HalfPath<F>::value) {
+                            // generic path: decode from the word, test four values at once for Inf/NaN codes
 #pragma unroll
-                        for (int j = 0; j < AL; ++j)
-                            x[j] = __fmaf_rn(c.s, decode_exact<F>(get_code_at<F, ANW>(win, j * F::B)), c.b);
+                            for (int g = 0; g < AL / 4; ++g) {
+                                float dec[4];
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) dec[j] = decode_fast_at<F, ANW>(win, (4 * g + j) * F::B);
+                                if (any_code_special4<F>(dec)) {
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) dec[j] = decode_exact<F>(get_code_at<F, ANW>(win, (4 * g + j) * F::B));
+                                }
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) x[4 * g + j] = __fmaf_rn(c.s, dec[j], c.b);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < AL; ++j)
+                                x[j] = __fmaf_rn(c.s, decode_exact<F>(get_code_at<F, ANW>(win, j * F::B)), c.b);
+                        }
                     } else {
 #pragma unroll
                         for (int j = 0; j < AL; ++j) x[j] = __uint_as_float(w[kk][j]);
