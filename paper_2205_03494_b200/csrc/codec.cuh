@@ -45,6 +45,15 @@ struct HalfPath {
     static constexpr bool value = (F::E == 5 && F::M <= 10);
 };
 
+// The two 8-bit formats whose codes, below the top of the range, are those of a hardware FP8 type.
+#ifndef OMC_FP8_PATH
+#define OMC_FP8_PATH 1          // 0: build without the FP8 conversion instructions (tuning runs)
+#endif
+template <class F>
+struct Fp8Path {
+    static constexpr bool value = OMC_FP8_PATH && ((F::E == 5 && F::M == 2) || (F::E == 4 && F::M == 3));
+};
+
 __device__ __forceinline__ uint32_t f2u(float x) { return __float_as_uint(x); }
 __device__ __forceinline__ float u2f(uint32_t u) { return __uint_as_float(u); }
 

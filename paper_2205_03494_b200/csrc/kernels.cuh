@@ -198,6 +198,15 @@ static __device__ __noinline__ void flush_and_maybe_finalise(Partial *slots, uin
                                                              int lane)
 {
     acc.warp_reduce();
+    if (nslots == 1) {      // the variable is this warp's alone: nothing to hand over
+        if (lane == 0) {
+            float s, b;
+            fit_from_sums(acc, n, magnitude_mask, s, b);
+            sb[0] = s;
+            sb[1] = b;
+        }
+        return;
+    }
     uint32_t last = 0;
     if (lane == 0) {
         Partial q;
@@ -239,8 +248,8 @@ static __device__ __noinline__ void flush_and_maybe_finalise(Partial *slots, uin
 #endif
 template <class F>
 struct PairPath {
-    static constexpr bool value = HalfPath<F>::value && (F::B == 8 || F::B == 12 || F::B == 16) &&
-                                  (F::B <= OMC_PAIR_PATH_BITS);
+    static constexpr bool value = HalfPath<F>::value && !Fp8Path<F>::value &&
+                                  (F::B == 8 || F::B == 12 || F::B == 16) && (F::B <= OMC_PAIR_PATH_BITS);
 };
 
 // A 32-bit pattern that identifies the value Q^-1(code) up to the sign of zero; the fit only needs
@@ -248,9 +257,11 @@ struct PairPath {
 // both halves (so that two codes can be compared per operation), the others the FP32 pattern.
 template <class F>
 struct ValuePattern {
-    static constexpr uint32_t MAGNITUDE_MASK = PairPath<F>::value ? 0x7FFF7FFFu : 0x7FFFFFFFu;
+    static constexpr uint32_t MAGNITUDE_MASK =
+        Fp8Path<F>::value ? 0x7F7F7F7Fu : PairPath<F>::value ? 0x7FFF7FFFu : 0x7FFFFFFFu;
     __device__ static __forceinline__ uint32_t of(uint32_t code, float vt)
     {
+        if constexpr (Fp8Path<F>::value) return code * 0x01010101u;      // the code in all four bytes
         if constexpr (PairPath<F>::value) return ((code << (10 - F::M)) & 0xFFFFu) * 0x00010001u;
         return f2u(vt);
     }
@@ -594,6 +605,112 @@ __device__ __forceinline__ void compute_unit_pairs(const uint32_t (&win)[Unit<F>
 }
 
 // ---------------------------------------------------------------------------------------------
+// Full units of the two 8-bit formats whose finite codes are the codes of a hardware FP8 type
+// (S1E5M2 = e5m2, S1E4M3 = e4m3 up to exponent field 14): a unit is one word of four codes, and the
+// FP8 conversion instructions do the rounding (to nearest even, gradual underflow) and the
+// unpacking two elements at a time.  The hardware types differ from the paper's family at the top
+// of the range only (saturation instead of infinity; e4m3 has finite values where S1E4M3 has
+// Inf/NaN), and every code that high, read or produced, sends the unit to compute_unit.
+
+// Four codes -> four FP32 values (exact).
+template <class F>
+__device__ __forceinline__ void fp8x4_decode(uint32_t cw, float (&v)[4])
+{
+    uint32_t h01, h23;       // two FP16 pairs
+    if constexpr (F::E == 5) {                   // a code is the top byte of its FP16 pattern
+        h01 = __byte_perm(cw, 0u, 0x1404);
+        h23 = __byte_perm(cw, 0u, 0x3424);
+    } else {
+        asm("{\n\t.reg .b16 lo, hi;\n\t"
+            "mov.b32 {lo, hi}, %2;\n\t"
+            "cvt.rn.f16x2.e4m3x2 %0, lo;\n\t"
+            "cvt.rn.f16x2.e4m3x2 %1, hi;\n\t}"
+            : "=r"(h01), "=r"(h23) : "r"(cw));
+    }
+    const __half2 a = *reinterpret_cast<const __half2 *>(&h01), c = *reinterpret_cast<const __half2 *>(&h23);
+    v[0] = __low2float(a); v[1] = __high2float(a);
+    v[2] = __low2float(c); v[3] = __high2float(c);
+}
+
+// Four FP32 values -> four codes in one word (element 0 in the low byte).  Saturating: a magnitude
+// beyond the type's largest finite value gives that value, a NaN the type's NaN.
+template <class F>
+__device__ __forceinline__ uint32_t fp8x4_encode(const float (&w)[4])
+{
+    uint32_t cw;
+    if constexpr (F::E == 5)
+        asm("{\n\t.reg .b16 lo, hi;\n\t"
+            "cvt.rn.satfinite.e5m2x2.f32 lo, %2, %1;\n\t"
+            "cvt.rn.satfinite.e5m2x2.f32 hi, %4, %3;\n\t"
+            "mov.b32 %0, {lo, hi};\n\t}"
+            : "=r"(cw) : "f"(w[0]), "f"(w[1]), "f"(w[2]), "f"(w[3]));
+    else
+        asm("{\n\t.reg .b16 lo, hi;\n\t"
+            "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+            "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+            "mov.b32 %0, {lo, hi};\n\t}"
+            : "=r"(cw) : "f"(w[0]), "f"(w[1]), "f"(w[2]), "f"(w[3]));
+    return cw;
+}
+
+// Non-zero iff one of the four codes has a magnitude of at least TOP.
+template <uint32_t TOP>
+__device__ __forceinline__ uint32_t fp8x4_any_at_least(uint32_t cw)
+{
+    return ((cw & 0x7F7F7F7Fu) + (0x80u - TOP) * 0x01010101u) & 0x80808080u;
+}
+
+template <class F, int MODE>
+__device__ __forceinline__ void compute_unit_fp8(const uint32_t (&win)[1], const float4 (&fv)[1], uint32_t (&wout)[1],
+                                                 float4 (&fo)[1], float s, float b, float neg_lr, Acc &acc)
+{
+    // Codes from here up are not handled by the hardware type as the format wants them: Inf/NaN
+    // codes of S1E4M3 when read; when written, the largest finite code too (saturation hides an
+    // overflow behind it) and with it every Inf/NaN.
+    constexpr uint32_t TOP_IN = F::INF_MAG, TOP_OUT = F::INF_MAG - 1u;
+    float w[4], vt[4];
+    uint32_t special = 0u, cw = 0u;
+    if constexpr (MODE != COMPRESS) {
+        float dec[4];
+        fp8x4_decode<F>(win[0], dec);
+        if constexpr (F::E != 5) special = fp8x4_any_at_least<TOP_IN>(win[0]);   // e5m2 decodes Inf/NaN as such
+        const float g[4] = {fv[0].x, fv[0].y, fv[0].z, fv[0].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float vbar = __fmaf_rn(s, dec[j], b);
+            w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, g[j], vbar) : vbar;
+        }
+    } else {
+        w[0] = fv[0].x; w[1] = fv[0].y; w[2] = fv[0].z; w[3] = fv[0].w;
+    }
+    if constexpr (MODE != DECOMPRESS) {
+        cw = fp8x4_encode<F>(w);
+        special |= fp8x4_any_at_least<TOP_OUT>(cw);
+        fp8x4_decode<F>(cw, vt);
+    }
+    if (special) {          // rare: redo the unit on copies, so that only they have addresses
+        uint32_t win_c[1] = {(MODE != COMPRESS) ? win[0] : 0u}, wout_c[1];
+        float4 fv_c[1] = {fv[0]}, fo_c[1];
+        Acc acc_c = acc;
+        compute_unit_careful<F, MODE>(win_c, fv_c, wout_c, fo_c, s, b, neg_lr, &acc_c);
+        acc = acc_c;
+        wout[0] = wout_c[0];
+        fo[0] = fo_c[0];
+        return;
+    }
+    if constexpr (MODE != DECOMPRESS) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc.add(w[j], vt[j]);
+        const uint32_t ref = __byte_perm(cw, 0u, 0x0000);     // element 0's code in all four bytes
+        const uint32_t diff = cw ^ ref;
+        acc.band &= ref & ~diff;
+        acc.bor |= ref | diff;
+        wout[0] = cw;
+    }
+    fo[0] = make_float4(w[0], w[1], w[2], w[3]);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Register <-> memory moves of a unit (global or shared: the address space is inferred).
 
 template <int N>
@@ -666,7 +783,9 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
             const int unit = (k0 + g) * 32 + lane;
             uint32_t wout[NW];
             float4 fo[LU / 4];
-            if constexpr (PairPath<F>::value)
+            if constexpr (Fp8Path<F>::value)
+                compute_unit_fp8<F, MODE>(win[g], fv[g], wout, fo, s, b, neg_lr, acc);
+            else if constexpr (PairPath<F>::value)
                 compute_unit_pairs<F, MODE>(win[g], fv[g], wout, fo, s, b, neg_lr, acc);
             else
                 compute_unit<F, MODE, false>(win[g], fv[g], wout, fo, s, b, neg_lr, acc, LU);
@@ -681,42 +800,53 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
 
 // The ragged end of a variable (fewer than SUB elements), straight from and to global memory
 // with predicated accesses.  `n_rem` = elements left in the variable; `w_rem` = 32-bit words left
-// in its padded code stream.  Rare: kept out of line so that it costs the main loop no registers.
+// in its padded code stream.  All loads are issued before the arithmetic starts, so that the warp
+// waits for memory once and not once per step.  Out of line: it runs once per (variable, warp) at
+// most and must cost the main loop no registers.
 template <class F, int MODE, bool WOUT>
 __device__ __noinline__ Acc tile_ragged(uint32_t *cw, const float *fin, float *fout, uint32_t n_rem,
                                         uint32_t w_rem, float s, float b, float neg_lr, Acc acc, int lane)
 {
     using U = Unit<F>;
-    constexpr int LU = U::LU, NW = U::NWORDS;
+    constexpr int LU = U::LU, NW = U::NWORDS, NS = U::SUB_STEPS;
+    static_assert(NS * (NW + LU) <= 64, "the ragged end is held in registers");
     const uint32_t n_pad = (n_rem + 3u) & ~3u;       // floats that exist in the full layout
-#pragma unroll 1
-    for (int k = 0; k < U::SUB_STEPS; ++k) {
-        if ((uint32_t)k * U::STEP >= n_rem) break;
+    uint32_t win[NS][NW];
+    float4 fv[NS][LU / 4];
+#pragma unroll
+    for (int k = 0; k < NS; ++k) {
         const uint32_t unit = (uint32_t)k * 32u + (uint32_t)lane;
         const uint32_t e0 = unit * LU;
-        uint32_t win[NW], wout[NW];
-        float4 fv[LU / 4], fo[LU / 4];
         if constexpr (MODE != COMPRESS) {
 #pragma unroll
-            for (int j = 0; j < NW; ++j) win[j] = (unit * NW + j < w_rem) ? cw[unit * NW + j] : 0u;
+            for (int j = 0; j < NW; ++j) win[k][j] = (unit * NW + j < w_rem) ? cw[unit * NW + j] : 0u;
         }
         if constexpr (MODE != DECOMPRESS) {
 #pragma unroll
             for (int j = 0; j < LU / 4; ++j)
-                fv[j] = (e0 + 4 * j < n_pad) ? reinterpret_cast<const float4 *>(fin + e0)[j]
-                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+                fv[k][j] = (e0 + 4 * j < n_pad) ? reinterpret_cast<const float4 *>(fin + e0)[j]
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        const int valid = e0 >= n_rem ? 0 : (n_rem - e0 < (uint32_t)LU ? (int)(n_rem - e0) : LU);
-        compute_unit<F, MODE, true>(win, fv, wout, fo, s, b, neg_lr, acc, valid);
-        if constexpr (MODE != DECOMPRESS) {
+    }
 #pragma unroll
-            for (int j = 0; j < NW; ++j)
-                if (unit * NW + j < w_rem) cw[unit * NW + j] = wout[j];
-        }
-        if constexpr (MODE == DECOMPRESS || WOUT) {
+    for (int k = 0; k < NS; ++k) {
+        if ((uint32_t)k * U::STEP < n_rem) {         // the same for the whole warp
+            const uint32_t unit = (uint32_t)k * 32u + (uint32_t)lane;
+            const uint32_t e0 = unit * LU;
+            uint32_t wout[NW];
+            float4 fo[LU / 4];
+            const int valid = e0 >= n_rem ? 0 : (n_rem - e0 < (uint32_t)LU ? (int)(n_rem - e0) : LU);
+            compute_unit<F, MODE, true>(win[k], fv[k], wout, fo, s, b, neg_lr, acc, valid);
+            if constexpr (MODE != DECOMPRESS) {
 #pragma unroll
-            for (int j = 0; j < LU / 4; ++j)
-                if (e0 + 4 * j < n_pad) reinterpret_cast<float4 *>(fout + e0)[j] = fo[j];
+                for (int j = 0; j < NW; ++j)
+                    if (unit * NW + j < w_rem) cw[unit * NW + j] = wout[j];
+            }
+            if constexpr (MODE == DECOMPRESS || WOUT) {
+#pragma unroll
+                for (int j = 0; j < LU / 4; ++j)
+                    if (e0 + 4 * j < n_pad) reinterpret_cast<float4 *>(fout + e0)[j] = fo[j];
+            }
         }
     }
     return acc;
