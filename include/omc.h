@@ -228,11 +228,11 @@ int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *packed, cons
  * fragmentation-sensitive service whose buffers are all reserved at start-up, or a plug-in that is
  * handed its input and output buffers and nothing else.  Such a caller cannot use omc_compress,
  * because omc_plan_prepare allocates the plan's device table and the caller would have to provide a
- * workspace.  Here the table entry, the ticket, the status word and the per-warp partial sums of
- * the Sec. 2.3 fit live in a fixed 196,864-byte array inside the library's device image (every GPU
- * that loads the library carries it until the process ends).  The function calls no cudaMalloc,
- * cudaFree or other allocating routine; the result is bit-identical to omc_compress on a
- * one-variable plan.
+ * workspace.  Here the table entry, the ticket, the status word, the division of the work among
+ * warps and the per-warp partial sums of the Sec. 2.3 fit live in a fixed 229,640-byte array inside
+ * the library's device image (every GPU that loads the library carries it until the process ends).
+ * The function calls no cudaMalloc, cudaFree or other allocating routine; the result is
+ * bit-identical to omc_compress on a one-variable plan.
  *
  *   values  device, numel floats (readable up to the next multiple of 4), 16-byte aligned.
  *   numel   1 .. OMC_STATIC_MAX_NUMEL; anything larger returns OMC_ERR_TOO_LARGE and does nothing.

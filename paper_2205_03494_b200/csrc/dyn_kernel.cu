@@ -87,8 +87,8 @@ __global__ void __launch_bounds__(THREADS) omc_dyn_kernel(const KParams p, const
     const int lane = threadIdx.x & 31;
     const uint32_t warp = blockIdx.x * WARPS_PER_CTA + (threadIdx.x >> 5);
     if (warp >= p.nwarps) return;
-    uint64_t t = p.tile_begin + (uint64_t)warp * p.tile_count / p.nwarps;
-    const uint64_t tend = p.tile_begin + (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
+    uint64_t t, tend;
+    warp_tile_range(p, warp, t, tend);
     uint32_t lo = p.var_begin, hi = p.var_end;
     while (hi - lo > 1) {
         const uint32_t mid = (lo + hi) >> 1;

@@ -1032,8 +1032,8 @@ omc_kernel(const KParams p)
     }
     __syncwarp();
 
-    uint64_t t = p.tile_begin + (uint64_t)warp * p.tile_count / p.nwarps;
-    const uint64_t tend = p.tile_begin + (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
+    uint64_t t, tend;
+    warp_tile_range(p, warp, t, tend);
     // variable that holds tile t
     uint32_t lo = p.var_begin, hi = p.var_end;
     while (hi - lo > 1) {
@@ -1156,8 +1156,8 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_transition_kernel(co
     }
     __syncwarp();
 
-    uint64_t t = p.tile_begin + (uint64_t)warp * p.tile_count / p.nwarps;
-    const uint64_t tend = p.tile_begin + (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
+    uint64_t t, tend;
+    warp_tile_range(p, warp, t, tend);
     uint32_t lo = p.var_begin, hi = p.var_end;
     while (hi - lo > 1) {
         const uint32_t mid = (lo + hi) >> 1;

@@ -40,12 +40,16 @@ extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
     if (plan->d_vars && plan->device != dev) return OMC_ERR_PLAN_MISMATCH;
     if (!plan->d_vars) {
         const size_t bytes = sizeof(omc::VarDev) * (size_t)plan->nvars;
-        rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), bytes + 16));
+        const size_t ws_bytes = sizeof(uint64_t) * plan->warp_start.size();
+        rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), bytes + 16 + ws_bytes));
         if (rc) { plan->d_vars = nullptr; return rc; }
-        rc = omc::note_cuda(cudaMemcpy(plan->d_vars, plan->vars.data(), bytes, cudaMemcpyHostToDevice));
-        if (!rc) rc = omc::note_cuda(cudaMemset(plan->d_vars + plan->nvars, 0, 16));
+        char *const base = reinterpret_cast<char *>(plan->d_vars);
+        rc = omc::note_cuda(cudaMemcpy(base, plan->vars.data(), bytes, cudaMemcpyHostToDevice));
+        if (!rc) rc = omc::note_cuda(cudaMemset(base + bytes, 0, 16));
+        if (!rc) rc = omc::note_cuda(cudaMemcpy(base + bytes + 16, plan->warp_start.data(), ws_bytes, cudaMemcpyHostToDevice));
         if (rc) { (void)cudaFree(plan->d_vars); plan->d_vars = nullptr; return rc; }
-        plan->d_status = reinterpret_cast<uint32_t *>(plan->d_vars + plan->nvars);
+        plan->d_status = reinterpret_cast<uint32_t *>(base + bytes);
+        plan->d_warp_start = reinterpret_cast<uint64_t *>(base + bytes + 16);
         plan->device = dev;
     }
     return omc::note_cuda(cudaMemsetAsync(workspace, 0, plan->ws_bytes, static_cast<cudaStream_t>(stream)));
@@ -70,6 +74,7 @@ static KParams whole_model(const omc_plan_t *plan, void *workspace)
     p.tile_begin = 0;
     p.tile_count = plan->ntiles;
     p.nwarps = plan->nwarps;
+    p.warp_start = plan->d_warp_start;
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
     p.dyn_e = plan->fmt.exp_bits;
     p.dyn_m = plan->fmt.man_bits;

@@ -61,6 +61,9 @@ struct KParams {
     uint64_t tile_begin;           // first tile covered
     uint64_t tile_count;           // number of tiles covered
     uint32_t nwarps;               // warps the tiles are divided among (<= tile_count)
+    // Optional: nwarps + 1 tile indices, warp w owns tiles [warp_start[w], warp_start[w + 1]).
+    // NULL: warp w owns [tile_begin + w * tile_count / nwarps, tile_begin + (w + 1) * tile_count / nwarps).
+    const uint64_t *warp_start;
     uint32_t pvt;
     uint32_t dyn_e, dyn_m;         // the format, for the kernels that take it at run time
     uint8_t *packed;
@@ -104,6 +107,25 @@ struct FmtOps {
 };
 const FmtOps *find_ops(int E, int M);
 
+// Divides the tiles of vars[0 .. nvars) (n, quantised, tile_start and ntiles filled in) among
+// nwarps warps: writes warp_start[0 .. nwarps] (warp w owns tiles [warp_start[w], warp_start[w+1]))
+// and each variable's first_warp, nslots and slot_base; returns the number of partial-sum slots.
+uint32_t divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nwarps, uint64_t *warp_start);
+
+// The tiles [t, tend) of warp `warp` under the launch's division of the work.
+#ifdef __CUDACC__
+__device__ __forceinline__ void warp_tile_range(const KParams &p, uint32_t warp, uint64_t &t, uint64_t &tend)
+{
+    if (p.warp_start) {
+        t = __ldg(p.warp_start + warp);
+        tend = __ldg(p.warp_start + warp + 1);
+    } else {
+        t = p.tile_begin + (uint64_t)warp * p.tile_count / p.nwarps;
+        tend = p.tile_begin + (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
+    }
+}
+#endif
+
 }  // namespace omc
 
 struct omc_plan {
@@ -119,7 +141,9 @@ struct omc_plan {
     uint64_t ws_tickets_off, ws_slots_off, ws_bytes;
     const omc::FmtOps *ops;
     // device side
-    omc::VarDev *d_vars;               // one allocation: the tables, then the status word
+    std::vector<uint64_t> warp_start;  // nwarps + 1 entries: the cost-balanced division of the tiles
+    omc::VarDev *d_vars;               // one allocation: the variable table, the status word, warp_start
     uint32_t *d_status;
+    uint64_t *d_warp_start;
     int device;                        // device the tables live on, -1 before prepare
 };

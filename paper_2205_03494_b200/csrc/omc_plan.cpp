@@ -51,6 +51,18 @@ static uint64_t splitmix64(uint64_t &state)
 
 static uint64_t round_up(uint64_t x, uint64_t m) { return (x + m - 1) / m * m; }
 
+// Estimated cost of a warp's work, in sixteenths of the time of one tile of codes (measured on
+// B200 with the fused round; overridable at build time for tuning runs).
+#ifndef OMC_COST_TILE
+#define OMC_COST_TILE 16
+#endif
+#ifndef OMC_COST_FP32_TILE
+#define OMC_COST_FP32_TILE 16
+#endif
+#ifndef OMC_COST_VARIABLE
+#define OMC_COST_VARIABLE 48
+#endif
+
 static uint32_t query_sm_count()
 {
     int dev = 0, sms = 0;
@@ -60,6 +72,55 @@ static uint32_t query_sm_count()
         return omc::DEFAULT_SMS;
     }
     return (uint32_t)sms;
+}
+
+// Division of the tiles among warps: contiguous runs of equal estimated cost.  A warp pays for a
+// tile and, on top, for every quantised variable it enters (pipeline restart, ragged end,
+// hand-over of the fit's sums).  A tile goes to warp floor(cost before it * nwarps / total cost):
+// monotone in the tile index, and inside a variable consecutive owners differ by at most one, so
+// the warps first_warp .. first_warp + nslots - 1 of a variable all own one of its tiles.
+uint32_t omc::divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nwarps, uint64_t *warp_start)
+{
+    const uint64_t NW = nwarps;
+    auto var_cost = [](const VarDev &v) {
+        return v.quantised ? (uint64_t)OMC_COST_TILE * v.ntiles + OMC_COST_VARIABLE
+                           : (uint64_t)OMC_COST_FP32_TILE * v.ntiles;
+    };
+    uint64_t total_cost = 0, tiles = 0;
+    for (uint32_t i = 0; i < nvars; ++i) {
+        total_cost += var_cost(vars[i]);
+        tiles += vars[i].ntiles;
+    }
+    // 128-bit products: the cost of 2^40-element variables times the warp count overflows 64 bits
+    auto warp_of = [&](uint64_t cost) { return (uint32_t)(((unsigned __int128)cost * NW) / total_cost); };
+    warp_start[0] = 0;
+    uint32_t slots = 0, w = 0;
+    uint64_t before = 0;
+    for (uint32_t i = 0; i < nvars; ++i) {
+        VarDev &v = vars[i];
+        const uint64_t per_tile = v.quantised ? OMC_COST_TILE : OMC_COST_FP32_TILE;
+        const uint64_t c = before + (v.quantised ? OMC_COST_VARIABLE : 0);     // cost before tile 0 of v
+        v.first_warp = warp_of(c);
+        // the tiles of v at which the owner changes, solved for instead of walking every tile
+        uint64_t k = 0;
+        while (k < v.ntiles) {
+            const uint32_t own = warp_of(c + per_tile * k);
+            while (w < own) warp_start[++w] = v.tile_start + k;
+            // smallest cost that belongs to the next warp, and the first tile of v that reaches it
+            const unsigned __int128 need = ((unsigned __int128)(own + 1) * total_cost + NW - 1) / NW;
+            uint64_t k2 = (uint64_t)((need - c + per_tile - 1) / per_tile);
+            if (k2 <= k) k2 = k + 1;
+            k = k2 < v.ntiles ? k2 : v.ntiles;
+        }
+        v.nslots = warp_of(c + per_tile * (v.ntiles - 1)) - v.first_warp + 1;
+        if (v.quantised) {
+            v.slot_base = slots;
+            slots += v.nslots;
+        }
+        before += var_cost(v);
+    }
+    while (w < NW) warp_start[++w] = tiles;
+    return slots;
 }
 
 extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t fmt, double fraction,
@@ -88,6 +149,7 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         pl->ops = ops;
         pl->d_vars = nullptr;
         pl->d_status = nullptr;
+        pl->d_warp_start = nullptr;
         pl->device = -1;
         const uint32_t B = 1u + fmt.exp_bits + fmt.man_bits;
 
@@ -150,23 +212,13 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         pl->closed_form_bytes = closed;
         pl->ntiles = tiles;
 
-        // ---- division of the tiles among warps: warp w owns tiles [w*T/NW, (w+1)*T/NW)
+        // ---- division of the tiles among warps
         pl->n_sm = query_sm_count();
         pl->n_cta = pl->n_sm * omc::CTAS_PER_SM;
         const uint64_t max_warps = (uint64_t)pl->n_cta * omc::WARPS_PER_CTA;
         pl->nwarps = (uint32_t)(tiles < max_warps ? tiles : max_warps);
-        const uint64_t T = tiles, NW = pl->nwarps;
-        auto owner = [&](uint64_t t) { return (uint32_t)(((t + 1) * NW - 1) / T); };
-        uint32_t slots = 0;
-        for (uint32_t i = 0; i < nvars; ++i) {
-            VarDev &v = pl->vars[i];
-            v.first_warp = owner(v.tile_start);
-            v.nslots = owner(v.tile_start + v.ntiles - 1) - v.first_warp + 1;
-            if (v.quantised) {
-                v.slot_base = slots;
-                slots += v.nslots;
-            }
-        }
+        pl->warp_start.assign((size_t)pl->nwarps + 1, 0);
+        const uint32_t slots = omc::divide_tiles(pl->vars.data(), nvars, pl->nwarps, pl->warp_start.data());
         pl->nslots = slots;
         pl->ws_tickets_off = omc::WS_HEADER_BYTES;
         pl->ws_slots_off = round_up(pl->ws_tickets_off + 4ull * (nq ? nq : 1), 256);

@@ -1,8 +1,9 @@
 // omc_compress_var_static: compression of one variable for callers that may not allocate.
 //
 // Everything omc_compress keeps in caller- or plan-owned device memory besides the inputs and
-// outputs (the one-entry variable table, the ticket, the per-warp partial-sum records of the fit
-// and the status word) lives here in a fixed array inside the library's own device image.
+// outputs (the one-entry variable table, the ticket, the status word, the division of the tiles
+// among warps and the per-warp partial-sum records of the fit) lives here in a fixed array inside
+// the library's own device image.
 #include <cuda_runtime.h>
 
 #include "omc_internal.h"
@@ -18,7 +19,8 @@ constexpr size_t OFF_VAR = 0;                            // omc::VarDev, 64 byte
 constexpr size_t OFF_TICKET = 64;                        // uint32_t
 constexpr size_t OFF_STATUS = 68;                        // uint32_t
 constexpr size_t OFF_SLOTS = 256;                        // omc::Partial[MAX_SLOTS]
-constexpr size_t SCRATCH_BYTES = OFF_SLOTS + sizeof(omc::Partial) * MAX_SLOTS;   // 196,864 bytes
+constexpr size_t OFF_WARP_START = OFF_SLOTS + sizeof(omc::Partial) * MAX_SLOTS;   // uint64_t[MAX_SLOTS + 1]
+constexpr size_t SCRATCH_BYTES = OFF_WARP_START + sizeof(uint64_t) * (MAX_SLOTS + 1);   // 229,640 bytes
 
 // Held by every GPU that loads the library until the process exits.  In host code this name is
 // only a handle for cudaGetSymbolAddress; it is never passed to a kernel.
@@ -88,13 +90,17 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     v.quantised = 1;
     v.sb_slot = 0;
     v.slot_base = 0;
-    v.first_warp = 0;
-    v.nslots = nwarps;            // every warp owns at least one tile because nwarps <= tiles
+    uint64_t warp_start[MAX_SLOTS + 1];        // host copy; the same division omc_plan makes
+    omc::divide_tiles(&v, 1, nwarps, warp_start);
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // The array keeps what the last call left: the table entry is rewritten, the ticket and the
-    // status word are cleared; the records are all rewritten by the kernel before they are read.
+    // The array keeps what the last call left: the table entry and the division are rewritten, the
+    // ticket and the status word are cleared; the records are all rewritten by the kernel before
+    // they are read.  Both host buffers are pageable, so each copy has left them when it returns.
     rc = omc::note_cuda(cudaMemcpyAsync(scratch + OFF_VAR, &v, sizeof v, cudaMemcpyHostToDevice, st));
+    if (rc) return rc;
+    rc = omc::note_cuda(cudaMemcpyAsync(scratch + OFF_WARP_START, warp_start, sizeof(uint64_t) * (nwarps + 1),
+                                        cudaMemcpyHostToDevice, st));
     if (rc) return rc;
     rc = omc::note_cuda(cudaMemsetAsync(scratch + OFF_TICKET, 0, 8, st));
     if (rc) return rc;
@@ -106,6 +112,7 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     p.tile_begin = 0;
     p.tile_count = tiles;
     p.nwarps = nwarps;
+    p.warp_start = reinterpret_cast<const uint64_t *>(scratch + OFF_WARP_START);
     p.pvt = (flags & OMC_PLAN_PVT) ? 1u : 0u;
     p.dyn_e = fmt.exp_bits;
     p.dyn_m = fmt.man_bits;
