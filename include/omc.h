@@ -114,6 +114,19 @@ int omc_plan_var(const omc_plan_t *plan, uint32_t i, int *quantised, uint64_t *f
                  uint32_t *sb_slot);
 
 /*
+ * omc_plan_division -- how the plan divides the work among the warps of one launch (host only).
+ * The model's variables are cut into tiles of 1024 elements, numbered in variable order (a
+ * variable's last tile may be short); warp w of omc_compress / omc_update_recompress /
+ * omc_transition processes tiles [warp_start[w], warp_start[w + 1]), contiguous runs of about
+ * equal estimated cost.  *warp_start points at n_warps + 1 non-decreasing entries owned by the
+ * plan (valid until omc_plan_destroy), the first 0 and the last *n_tiles.  Any output pointer may
+ * be NULL.  Sec. 2.3's sums are taken per variable whatever the division; it only decides which
+ * warp adds which elements, and so the order of the fp64 additions.
+ */
+int omc_plan_division(const omc_plan_t *plan, uint32_t *n_warps, uint64_t *n_tiles,
+                      const uint64_t **warp_start);
+
+/*
  * omc_plan_prepare -- copy the plan's tables to the current device (the one allocation the
  * library makes; synchronous) and clear `workspace` (device, workspace_bytes) on `stream`.
  * Must precede the first device call with this plan; the workspace then stays valid from call

@@ -19,7 +19,7 @@ PLAN_PVT, PLAN_WEIGHTS_ONLY = 1, 2
 PLAN_DEFAULT = PLAN_PVT | PLAN_WEIGHTS_ONLY
 
 EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_sizes",
-           "omc_plan_var", "omc_plan_prepare", "omc_plan_status", "omc_compress", "omc_decompress",
+           "omc_plan_var", "omc_plan_division", "omc_plan_prepare", "omc_plan_status", "omc_compress", "omc_decompress",
            "omc_update_recompress", "omc_update_recompress_host", "omc_transition", "omc_aggregate", "omc_matmul",
            "omc_compress_var_static"]
 STATIC_MAX_NUMEL = 1 << 28
@@ -63,6 +63,7 @@ def lib():
         L.omc_plan_destroy.argtypes = [vp]
         L.omc_plan_sizes.argtypes = [vp, u64p, u64p, u64p, u32p, u64p, u64p]
         L.omc_plan_var.argtypes = [vp, C.c_uint32, C.POINTER(C.c_int), u64p, u64p, u64p, u64p, u32p]
+        L.omc_plan_division.argtypes = [vp, u32p, u64p, C.POINTER(u64p)]
         L.omc_plan_prepare.argtypes = [vp, vp, vp]
         L.omc_plan_status.argtypes = [vp, vp, u32p]
         L.omc_compress.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -134,6 +135,12 @@ class Plan:
             self.close()
         except Exception:
             pass
+
+    def division(self):
+        """omc_plan_division: (n_tiles, [warp_start[0], ..., warp_start[n_warps]])."""
+        nw, nt, tab = C.c_uint32(), C.c_uint64(), C.POINTER(C.c_uint64)()
+        _check(lib().omc_plan_division(self._h, C.byref(nw), C.byref(nt), C.byref(tab)), "omc_plan_division")
+        return nt.value, [tab[i] for i in range(nw.value + 1)]
 
     # ---- device calls (addresses are ints; 0/None = NULL) -----------------------------------
     def prepare(self, workspace, stream=0):

@@ -260,6 +260,16 @@ extern "C" int omc_plan_sizes(const omc_plan_t *plan, uint64_t *full_elems, uint
     return OMC_OK;
 }
 
+extern "C" int omc_plan_division(const omc_plan_t *plan, uint32_t *n_warps, uint64_t *n_tiles,
+                                 const uint64_t **warp_start)
+{
+    if (!plan) return OMC_ERR_NULL_PTR;
+    if (n_warps) *n_warps = plan->nwarps;
+    if (n_tiles) *n_tiles = plan->ntiles;
+    if (warp_start) *warp_start = plan->warp_start.data();
+    return OMC_OK;
+}
+
 extern "C" int omc_plan_var(const omc_plan_t *plan, uint32_t i, int *quantised, uint64_t *full_off_elems,
                             uint64_t *resid_off_elems, uint64_t *packed_off_bytes, uint64_t *packed_bytes,
                             uint32_t *sb_slot)
