@@ -258,7 +258,7 @@ struct PairPath {
 template <class F>
 struct ValuePattern {
     static constexpr uint32_t MAGNITUDE_MASK =
-        Fp8Path<F>::value ? 0x7F7F7F7Fu : PairPath<F>::value ? 0x7FFF7FFFu : 0x7FFFFFFFu;
+        Fp8Path<F>::value ? F::MAG_MASK * 0x01010101u : PairPath<F>::value ? 0x7FFF7FFFu : 0x7FFFFFFFu;
     __device__ static __forceinline__ uint32_t of(uint32_t code, float vt)
     {
         if constexpr (Fp8Path<F>::value) return code * 0x01010101u;      // the code in all four bytes
@@ -605,14 +605,15 @@ __device__ __forceinline__ void compute_unit_pairs(const uint32_t (&win)[Unit<F>
 }
 
 // ---------------------------------------------------------------------------------------------
-// Full units of the two 8-bit formats whose finite codes are the codes of a hardware FP8 type
-// (S1E5M2 = e5m2, S1E4M3 = e4m3 up to exponent field 14): a unit is one word of four codes, and the
-// FP8 conversion instructions do the rounding (to nearest even, gradual underflow) and the
-// unpacking two elements at a time.  The hardware types differ from the paper's family at the top
-// of the range only (saturation instead of infinity; e4m3 has finite values where S1E4M3 has
-// Inf/NaN), and every code that high, read or produced, sends the unit to compute_unit.
+// Full units of the formats whose finite codes are the codes of a hardware narrow-float type
+// (S1E5M2 = e5m2, S1E4M3 = e4m3 up to exponent field 14, S1E2M3 = e2m3 up to field 2).  The
+// conversion instructions keep one code per byte and do the rounding (to nearest even, gradual
+// underflow) and the unpacking two elements at a time; four codes travel in one register.  The
+// hardware types differ from the paper's family at the top of the range only (saturation instead
+// of infinity; e4m3 and e2m3 have finite values where the family has Inf/NaN), and every code that
+// high, read or produced, sends the unit to compute_unit.
 
-// Four codes -> four FP32 values (exact).
+// Four codes, one per byte -> four FP32 values (exact).
 template <class F>
 __device__ __forceinline__ void fp8x4_decode(uint32_t cw, float (&v)[4])
 {
@@ -620,11 +621,17 @@ __device__ __forceinline__ void fp8x4_decode(uint32_t cw, float (&v)[4])
     if constexpr (F::E == 5) {                   // a code is the top byte of its FP16 pattern
         h01 = __byte_perm(cw, 0u, 0x1404);
         h23 = __byte_perm(cw, 0u, 0x3424);
-    } else {
+    } else if constexpr (F::E == 4) {
         asm("{\n\t.reg .b16 lo, hi;\n\t"
             "mov.b32 {lo, hi}, %2;\n\t"
             "cvt.rn.f16x2.e4m3x2 %0, lo;\n\t"
             "cvt.rn.f16x2.e4m3x2 %1, hi;\n\t}"
+            : "=r"(h01), "=r"(h23) : "r"(cw));
+    } else {
+        asm("{\n\t.reg .b16 lo, hi;\n\t"
+            "mov.b32 {lo, hi}, %2;\n\t"
+            "cvt.rn.f16x2.e2m3x2 %0, lo;\n\t"
+            "cvt.rn.f16x2.e2m3x2 %1, hi;\n\t}"
             : "=r"(h01), "=r"(h23) : "r"(cw));
     }
     const __half2 a = *reinterpret_cast<const __half2 *>(&h01), c = *reinterpret_cast<const __half2 *>(&h23);
@@ -632,8 +639,9 @@ __device__ __forceinline__ void fp8x4_decode(uint32_t cw, float (&v)[4])
     v[2] = __low2float(c); v[3] = __high2float(c);
 }
 
-// Four FP32 values -> four codes in one word (element 0 in the low byte).  Saturating: a magnitude
-// beyond the type's largest finite value gives that value, a NaN the type's NaN.
+// Four FP32 values -> four codes, one per byte (element 0 in the low byte).  Saturating: a
+// magnitude beyond the type's largest finite value gives that value; a NaN gives the type's NaN,
+// or, in e2m3, which has none, its largest value.
 template <class F>
 __device__ __forceinline__ uint32_t fp8x4_encode(const float (&w)[4])
 {
@@ -644,70 +652,154 @@ __device__ __forceinline__ uint32_t fp8x4_encode(const float (&w)[4])
             "cvt.rn.satfinite.e5m2x2.f32 hi, %4, %3;\n\t"
             "mov.b32 %0, {lo, hi};\n\t}"
             : "=r"(cw) : "f"(w[0]), "f"(w[1]), "f"(w[2]), "f"(w[3]));
-    else
+    else if constexpr (F::E == 4)
         asm("{\n\t.reg .b16 lo, hi;\n\t"
             "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
             "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
             "mov.b32 %0, {lo, hi};\n\t}"
             : "=r"(cw) : "f"(w[0]), "f"(w[1]), "f"(w[2]), "f"(w[3]));
+    else
+        asm("{\n\t.reg .b16 lo, hi;\n\t"
+            "cvt.rn.satfinite.e2m3x2.f32 lo, %2, %1;\n\t"
+            "cvt.rn.satfinite.e2m3x2.f32 hi, %4, %3;\n\t"
+            "mov.b32 %0, {lo, hi};\n\t}"
+            : "=r"(cw) : "f"(w[0]), "f"(w[1]), "f"(w[2]), "f"(w[3]));
     return cw;
 }
 
-// Non-zero iff one of the four codes has a magnitude of at least TOP.
-template <uint32_t TOP>
+// Non-zero iff one of the four codes (one per byte) has a magnitude of at least TOP.
+template <class F, uint32_t TOP>
 __device__ __forceinline__ uint32_t fp8x4_any_at_least(uint32_t cw)
 {
-    return ((cw & 0x7F7F7F7Fu) + (0x80u - TOP) * 0x01010101u) & 0x80808080u;
+    return ((cw & (F::MAG_MASK * 0x01010101u)) + (0x80u - TOP) * 0x01010101u) & 0x80808080u;
+}
+
+// 6-bit codes: 24 bits of the packed stream <-> four codes, one per byte.
+__device__ __forceinline__ uint32_t spread6(uint32_t t)
+{
+    return (t & 0x3Fu) | ((t << 2) & 0x3F00u) | ((t << 4) & 0x3F0000u) | ((t << 6) & 0x3F000000u);
+}
+__device__ __forceinline__ uint32_t gather6(uint32_t c)
+{
+    return (c & 0x3Fu) | ((c >> 2) & 0xFC0u) | ((c >> 4) & 0x3F000u) | ((c >> 6) & 0xFC0000u);
+}
+
+// Out-of-line compute_group for the rare group of four that holds a code from the top of the
+// range: `g` is a run-time value here and everything lives behind pointers, so that the main path
+// keeps its registers.  New codes are OR-ed into wout_p (as compute_group does).
+template <class F, int MODE>
+__device__ __noinline__ void compute_group_careful(const uint32_t *win_p, int g, float4 f4, uint32_t *wout_p,
+                                                   float *w_p, float s, float b, float neg_lr, Acc *acc_p,
+                                                   uint32_t *ref_p, uint32_t *diff_p)
+{
+    constexpr int NW = Unit<F>::NWORDS;
+    uint32_t win[NW], wout[NW];
+#pragma unroll
+    for (int j = 0; j < NW; ++j) {
+        win[j] = win_p[j];
+        wout[j] = wout_p[j];
+    }
+    const float fin4[4] = {f4.x, f4.y, f4.z, f4.w};
+    float w[4];
+    Acc acc = *acc_p;
+    uint32_t ref = *ref_p, diff = *diff_p;
+    if (g == 0)     // compute_group takes element 0's pattern as the reference when g is 0
+        compute_group<F, MODE, false, NW, NW>(win, 0, fin4, wout, w, s, b, neg_lr, acc, ref, diff, Unit<F>::LU);
+    else
+        compute_group<F, MODE, false, NW, NW>(win, g, fin4, wout, w, s, b, neg_lr, acc, ref, diff, Unit<F>::LU);
+    *acc_p = acc;
+    *ref_p = ref;
+    *diff_p = diff;
+#pragma unroll
+    for (int j = 0; j < NW; ++j) wout_p[j] = wout[j];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) w_p[j] = w[j];
 }
 
 template <class F, int MODE>
-__device__ __forceinline__ void compute_unit_fp8(const uint32_t (&win)[1], const float4 (&fv)[1], uint32_t (&wout)[1],
-                                                 float4 (&fo)[1], float s, float b, float neg_lr, Acc &acc)
+__device__ __forceinline__ void compute_unit_fp8(const uint32_t (&win)[Unit<F>::NWORDS],
+                                                 const float4 (&fv)[Unit<F>::LU / 4],
+                                                 uint32_t (&wout)[Unit<F>::NWORDS], float4 (&fo)[Unit<F>::LU / 4],
+                                                 float s, float b, float neg_lr, Acc &acc)
 {
+    constexpr int LU = Unit<F>::LU, NW = Unit<F>::NWORDS, NG = LU / 4;
+    static_assert((F::B == 8 && NG == 1) || (F::B == 6 && NG == 4 && NW == 3), "one byte or six bits per code");
     // Codes from here up are not handled by the hardware type as the format wants them: Inf/NaN
-    // codes of S1E4M3 when read; when written, the largest finite code too (saturation hides an
-    // overflow behind it) and with it every Inf/NaN.
+    // codes when read (e5m2 alone decodes them as such); when written, the largest finite code
+    // too (saturation hides an overflow behind it) and with it every Inf/NaN.
     constexpr uint32_t TOP_IN = F::INF_MAG, TOP_OUT = F::INF_MAG - 1u;
-    float w[4], vt[4];
-    uint32_t special = 0u, cw = 0u;
+    uint32_t cin[NG], cout[NG];
     if constexpr (MODE != COMPRESS) {
-        float dec[4];
-        fp8x4_decode<F>(win[0], dec);
-        if constexpr (F::E != 5) special = fp8x4_any_at_least<TOP_IN>(win[0]);   // e5m2 decodes Inf/NaN as such
-        const float g[4] = {fv[0].x, fv[0].y, fv[0].z, fv[0].w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float vbar = __fmaf_rn(s, dec[j], b);
-            w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, g[j], vbar) : vbar;
+        if constexpr (F::B == 8) {
+            cin[0] = win[0];
+        } else {            // group g is bits [24 g, 24 g + 24) of the unit's three words
+            cin[0] = spread6(win[0]);
+            cin[1] = spread6(__funnelshift_r(win[0], win[1], 24));
+            cin[2] = spread6(__funnelshift_r(win[1], win[2], 16));
+            cin[3] = spread6(win[2] >> 8);
         }
-    } else {
-        w[0] = fv[0].x; w[1] = fv[0].y; w[2] = fv[0].z; w[3] = fv[0].w;
     }
-    if constexpr (MODE != DECOMPRESS) {
-        cw = fp8x4_encode<F>(w);
-        special |= fp8x4_any_at_least<TOP_OUT>(cw);
-        fp8x4_decode<F>(cw, vt);
-    }
-    if (special) {          // rare: redo the unit on copies, so that only they have addresses
-        uint32_t win_c[1] = {(MODE != COMPRESS) ? win[0] : 0u}, wout_c[1];
-        float4 fv_c[1] = {fv[0]}, fo_c[1];
-        Acc acc_c = acc;
-        compute_unit_careful<F, MODE>(win_c, fv_c, wout_c, fo_c, s, b, neg_lr, &acc_c);
-        acc = acc_c;
-        wout[0] = wout_c[0];
-        fo[0] = fo_c[0];
-        return;
-    }
-    if constexpr (MODE != DECOMPRESS) {
+    uint32_t diff = 0u, ref = 0u;
+    uint32_t wout_sp[NW];       // codes written by the careful path, already at their place in the stream
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc.add(w[j], vt[j]);
-        const uint32_t ref = __byte_perm(cw, 0u, 0x0000);     // element 0's code in all four bytes
-        const uint32_t diff = cw ^ ref;
+    for (int j = 0; j < NW; ++j) wout_sp[j] = 0u;
+#pragma unroll
+    for (int g = 0; g < NG; ++g) {
+        float w[4], vt[4];
+        uint32_t special = 0u;
+        if constexpr (MODE != COMPRESS) {
+            float dec[4];
+            fp8x4_decode<F>(cin[g], dec);
+            if constexpr (F::E != 5) special = fp8x4_any_at_least<F, TOP_IN>(cin[g]);
+            const float gr[4] = {fv[g].x, fv[g].y, fv[g].z, fv[g].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float vbar = __fmaf_rn(s, dec[j], b);
+                w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, gr[j], vbar) : vbar;
+            }
+        } else {
+            w[0] = fv[g].x; w[1] = fv[g].y; w[2] = fv[g].z; w[3] = fv[g].w;
+        }
+        if constexpr (MODE != DECOMPRESS) {
+            cout[g] = fp8x4_encode<F>(w);
+            special |= fp8x4_any_at_least<F, TOP_OUT>(cout[g]);
+            fp8x4_decode<F>(cout[g], vt);
+        }
+        if (special) {
+            // on copies, so that only they (and not the registers of the main path) have addresses
+            uint32_t win_c[NW];
+            float w_c[4];
+            Acc acc_c = acc;
+            uint32_t ref_c = ref, diff_c = diff;
+#pragma unroll
+            for (int j = 0; j < NW; ++j) win_c[j] = (MODE != COMPRESS) ? win[j] : 0u;
+            compute_group_careful<F, MODE>(win_c, g, fv[g], wout_sp, w_c, s, b, neg_lr, &acc_c, &ref_c, &diff_c);
+            acc = acc_c;
+            ref = ref_c;
+            diff = diff_c;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) w[j] = w_c[j];
+            if constexpr (MODE != DECOMPRESS) cout[g] = 0u;
+        } else if constexpr (MODE != DECOMPRESS) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc.add(w[j], vt[j]);
+            if (g == 0) ref = __byte_perm(cout[0], 0u, 0x0000);     // element 0's code in all four bytes
+            diff |= cout[g] ^ ref;
+        }
+        fo[g] = make_float4(w[0], w[1], w[2], w[3]);
+    }
+    if constexpr (MODE != DECOMPRESS) {
         acc.band &= ref & ~diff;
         acc.bor |= ref | diff;
-        wout[0] = cw;
+        if constexpr (F::B == 8) {
+            wout[0] = cout[0] | wout_sp[0];
+        } else {
+            const uint32_t t0 = gather6(cout[0]), t1 = gather6(cout[1]), t2 = gather6(cout[2]), t3 = gather6(cout[3]);
+            wout[0] = t0 | (t1 << 24) | wout_sp[0];
+            wout[1] = (t1 >> 8) | (t2 << 16) | wout_sp[1];
+            wout[2] = (t2 >> 16) | (t3 << 8) | wout_sp[2];
+        }
     }
-    fo[0] = make_float4(w[0], w[1], w[2], w[3]);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1336,7 +1428,24 @@ __global__ void __launch_bounds__(THREADS, Unit<F>::LU == 32 ? CTAS_PER_SM : 4) 
                         uint32_t win[ANW];
 #pragma unroll
                         for (int j = 0; j < ANW; ++j) win[j] = w[kk][j];
-                        if constexpr (F::E < 8 && !HalfPath<F>::value) {
+                        if constexpr (Fp8Path<F>::value) {
+                            // four codes at a time through the narrow-float conversions; Inf/NaN codes redone
+#pragma unroll
+                            for (int g = 0; g < AL / 4; ++g) {
+                                float dec[4];
+                                uint32_t c4;            // the group's codes, one per byte
+                                if constexpr (F::B == 8) c4 = win[g];
+                                else c4 = spread6(g == 0 ? win[0] : g == 1 ? __funnelshift_r(win[0], win[1], 24)
+                                                  : g == 2 ? __funnelshift_r(win[1], win[2], 16) : win[2] >> 8);
+                                fp8x4_decode<F>(c4, dec);
+                                if (F::E != 5 && fp8x4_any_at_least<F, F::INF_MAG>(c4)) {
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) dec[j] = decode_exact<F>((c4 >> (8 * j)) & 0xFFu);
+                                }
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) x[4 * g + j] = __fmaf_rn(c.s, dec[j], c.b);
+                            }
+                        } else if constexpr (F::E < 8 && !HalfPath<F>::value) {
                             // generic path: decode from the word, test four values at once for Inf/NaN codes
 #pragma unroll
                             for (int g = 0; g < AL / 4; ++g) {

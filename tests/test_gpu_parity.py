@@ -240,6 +240,48 @@ def test_special_values(fmt):
     ls.check_decompress()
 
 
+@pytest.mark.parametrize("fmt", [(5, 2), (4, 3), (2, 3), (5, 6), (3, 7), (5, 10), (4, 8), (8, 7)],
+                         ids=lambda f: "E%dM%d" % f)
+def test_rounding_boundaries_through_the_fast_path(fmt):
+    """Every midpoint between neighbouring values of the format (up to 4096 of them, the lowest
+    and the highest always included), each with its two FP32 neighbours and in both signs, and a
+    log-uniform sweep from below the smallest subnormal to beyond the overflow threshold, laid out
+    as variables of whole tiles so that the kernels take their full-granule path (hardware
+    narrow-float and FP16 conversions where the format has them) and not the careful one.
+    Compress and one update round (zero gradient: decode, then encode again) against the oracle."""
+    E, M = fmt
+    bias = (1 << (E - 1)) - 1
+    emin, emax = 1 - bias, bias
+    # finite magnitudes of the format, ascending: m * 2^(emin - M) for the subnormals, then the binades
+    mags = [m * 2.0 ** (emin - M) for m in range(1 << M)]
+    for e in range(emin, emax + 1):
+        mags += [(1 + m / 2.0 ** M) * 2.0 ** e for m in range(1 << M)]
+    mags = np.array(mags, np.float64)
+    mids = 0.5 * (mags[:-1] + mags[1:])
+    mids = np.append(mids, 2.0 ** emax * (2 - 2.0 ** -(M + 1)))      # the overflow threshold
+    mids = mids[mids < 3.4e38]
+    if mids.size > 4096:
+        keep = np.unique(np.concatenate([np.arange(64), np.arange(mids.size - 64, mids.size),
+                                         np.linspace(0, mids.size - 1, 3968).astype(np.int64)]))
+        mids = mids[keep]
+    m32 = mids.astype(np.float32)
+    near = np.concatenate([m32, np.nextafter(m32, np.float32(0)), np.nextafter(m32, np.float32(np.inf))])
+    rng = np.random.default_rng(E * 31 + M)
+    lo, hi = np.log(max(2.0 ** (emin - M - 3), 1e-44)), np.log(min(2.0 ** (emax + 2), 3e38))
+    sweep = np.exp(rng.uniform(lo, hi, 60000)).astype(np.float32) * rng.choice([-1.0, 1.0], 60000).astype(np.float32)
+    vals = np.concatenate([near, -near, sweep])
+    n = (vals.size + 4095) // 4096 * 4096                       # whole tiles, whatever the granule size
+    vals = np.concatenate([vals, np.resize(m32, n - vals.size)])
+    rng.shuffle(vals)
+    in_range = vals[np.abs(vals) < 2.0 ** emax]                 # a second variable with no overflow: finite fit
+    in_range = in_range[:in_range.size // 4096 * 4096]
+    params = [vals, in_range]
+    ls = Lockstep([p.size for p in params], [0, 0], fmt, params)
+    ls.check_decompress()
+    ls.round([np.zeros(p.size, np.float32) for p in params], 1.0)
+    ls.check_decompress()
+
+
 def test_plan_switches():
     """Per-variable transformation off (s = 1, b = 0 stay put), weights-only off, explicit mask."""
     wl = workloads.tiny()
