@@ -114,17 +114,19 @@ int omc_plan_var(const omc_plan_t *plan, uint32_t i, int *quantised, uint64_t *f
                  uint32_t *sb_slot);
 
 /*
- * omc_plan_division -- how the plan divides the work among the warps of one launch (host only).
+ * omc_plan_division -- how the plan divides the work of one launch (host only).
  * The model's variables are cut into tiles of 1024 elements, numbered in variable order (a
- * variable's last tile may be short); warp w of omc_compress / omc_update_recompress /
- * omc_transition processes tiles [warp_start[w], warp_start[w + 1]), contiguous runs of about
- * equal estimated cost.  *warp_start points at n_warps + 1 non-decreasing entries owned by the
- * plan (valid until omc_plan_destroy), the first 0 and the last *n_tiles.  Any output pointer may
- * be NULL.  Sec. 2.3's sums are taken per variable whatever the division; it only decides which
- * warp adds which elements, and so the order of the fp64 additions.
+ * variable's last tile may be short), and the tiles into *n_runs contiguous runs of about equal
+ * estimated cost: run r = tiles [run_start[r], run_start[r + 1]).  Warp w of omc_compress /
+ * omc_update_recompress / omc_transition (and of omc_decompress over the whole model) takes runs
+ * w, w + *n_warps, w + 2 * *n_warps, ...: the warps that run at the same time work on neighbouring
+ * memory.  *run_start points at *n_runs + 1 non-decreasing entries owned by the plan (valid until
+ * omc_plan_destroy), the first 0 and the last *n_tiles; *n_runs is a multiple of *n_warps.  Any
+ * output pointer may be NULL.  Sec. 2.3's sums are taken per variable whatever the division; it
+ * only decides which warp adds which elements, and so the order of the fp64 additions.
  */
-int omc_plan_division(const omc_plan_t *plan, uint32_t *n_warps, uint64_t *n_tiles,
-                      const uint64_t **warp_start);
+int omc_plan_division(const omc_plan_t *plan, uint32_t *n_warps, uint32_t *n_runs, uint64_t *n_tiles,
+                      const uint64_t **run_start);
 
 /*
  * omc_plan_prepare -- copy the plan's tables to the current device (the one allocation the
@@ -241,8 +243,8 @@ int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *packed, cons
  * fragmentation-sensitive service whose buffers are all reserved at start-up, or a plug-in that is
  * handed its input and output buffers and nothing else.  Such a caller cannot use omc_compress,
  * because omc_plan_prepare allocates the plan's device table and the caller would have to provide a
- * workspace.  Here the table entry, the ticket, the status word, the division of the work among
- * warps and the per-warp partial sums of the Sec. 2.3 fit live in a fixed 229,640-byte array inside
+ * workspace.  Here the table entry, the ticket, the status word, the division of the work into
+ * runs and the per-run partial sums of the Sec. 2.3 fit live in a fixed 246,024-byte array inside
  * the library's device image (every GPU that loads the library carries it until the process ends).
  * The function calls no cudaMalloc, cudaFree or other allocating routine; the result is
  * bit-identical to omc_compress on a one-variable plan.

@@ -63,7 +63,7 @@ def lib():
         L.omc_plan_destroy.argtypes = [vp]
         L.omc_plan_sizes.argtypes = [vp, u64p, u64p, u64p, u32p, u64p, u64p]
         L.omc_plan_var.argtypes = [vp, C.c_uint32, C.POINTER(C.c_int), u64p, u64p, u64p, u64p, u32p]
-        L.omc_plan_division.argtypes = [vp, u32p, u64p, C.POINTER(u64p)]
+        L.omc_plan_division.argtypes = [vp, u32p, u32p, u64p, C.POINTER(u64p)]
         L.omc_plan_prepare.argtypes = [vp, vp, vp]
         L.omc_plan_status.argtypes = [vp, vp, u32p]
         L.omc_compress.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -137,10 +137,11 @@ class Plan:
             pass
 
     def division(self):
-        """omc_plan_division: (n_tiles, [warp_start[0], ..., warp_start[n_warps]])."""
-        nw, nt, tab = C.c_uint32(), C.c_uint64(), C.POINTER(C.c_uint64)()
-        _check(lib().omc_plan_division(self._h, C.byref(nw), C.byref(nt), C.byref(tab)), "omc_plan_division")
-        return nt.value, [tab[i] for i in range(nw.value + 1)]
+        """omc_plan_division: (n_warps, n_tiles, [run_start[0], ..., run_start[n_runs]])."""
+        nw, nr, nt, tab = C.c_uint32(), C.c_uint32(), C.c_uint64(), C.POINTER(C.c_uint64)()
+        _check(lib().omc_plan_division(self._h, C.byref(nw), C.byref(nr), C.byref(nt), C.byref(tab)),
+               "omc_plan_division")
+        return nw.value, nt.value, [tab[i] for i in range(nr.value + 1)]
 
     # ---- device calls (addresses are ints; 0/None = NULL) -----------------------------------
     def prepare(self, workspace, stream=0):

@@ -87,89 +87,86 @@ __global__ void __launch_bounds__(THREADS) omc_dyn_kernel(const KParams p, const
     const int lane = threadIdx.x & 31;
     const uint32_t warp = blockIdx.x * WARPS_PER_CTA + (threadIdx.x >> 5);
     if (warp >= p.nwarps) return;
-    uint64_t t, tend;
-    warp_tile_range(p, warp, t, tend);
-    uint32_t lo = p.var_begin, hi = p.var_end;
-    while (hi - lo > 1) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (__ldg(&p.vars[mid].tile_start) <= t) lo = mid; else hi = mid;
-    }
-    uint32_t v = lo;
     const uint32_t code_mask = f.B == 32 ? 0xFFFFFFFFu : ((1u << f.B) - 1u);
-    while (t < tend) {
-        const VarDev var = p.vars[v];
-        const uint32_t local = (uint32_t)(t - var.tile_start);
-        const uint64_t left = tend - t;
-        const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
-        if (var.quantised) {
-            float s = 1.f, b = 0.f;
-            if (MODE != COMPRESS) { s = __ldcg(p.sb + 2 * var.sb_slot); b = __ldcg(p.sb + 2 * var.sb_slot + 1); }
-            Acc acc;
-            acc.reset();
-            uint32_t *const cw = reinterpret_cast<uint32_t *>(p.packed + var.store_off);
-            const uint64_t nwords = var.packed_bytes / 4;
-            for (uint32_t i = 0; i < cnt; ++i) {
-                // this lane's 32 elements of the tile and the B words that hold exactly their codes
-                const uint64_t e0 = (uint64_t)(local + i) * TILE + (uint64_t)lane * 32;
-                const uint64_t w0 = e0 / 32 * f.B;
-                const int valid = e0 >= var.n ? 0 : (var.n - e0 < 32 ? (int)(var.n - e0) : 32);
-                uint64_t rbuf = 0, wbuf = 0;      // bit reader / writer over consecutive words
-                int rfill = 0, wfill = 0;
-                uint64_t rw = w0, ww = w0;
-                uint32_t ref = 0u, diff = 0u;
-                for (int k = 0; k < valid; ++k) {
-                    float w;
-                    if (MODE != COMPRESS) {
-                        if (rfill < f.B) { rbuf |= (uint64_t)cw[rw++] << rfill; rfill += 32; }
-                        const uint32_t c = (uint32_t)rbuf & code_mask;
-                        rbuf >>= f.B; rfill -= f.B;
-                        const float vbar = __fmaf_rn(s, dyn_decode(f, c), b);
-                        w = vbar;
-                        if (MODE == UPDATE) {
-                            w = __fmaf_rn(p.neg_lr, p.fin[var.full_off + e0 + k], vbar);
-                            if (w != w) w = u2f(0x7FFFFFFFu);     // arithmetic NaNs get one pattern
+    for (uint32_t run = warp; run < p.nruns; run += p.nwarps) {
+        uint64_t t, tend;
+        run_tile_range(p, run, t, tend);
+        uint32_t v = run_first_var(p, run, t);
+        while (t < tend) {
+            const VarDev var = p.vars[v];
+            const uint32_t local = (uint32_t)(t - var.tile_start);
+            const uint64_t left = tend - t;
+            const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
+            if (var.quantised) {
+                float s = 1.f, b = 0.f;
+                if (MODE != COMPRESS) { s = __ldcg(p.sb + 2 * var.sb_slot); b = __ldcg(p.sb + 2 * var.sb_slot + 1); }
+                Acc acc;
+                acc.reset();
+                uint32_t *const cw = reinterpret_cast<uint32_t *>(p.packed + var.store_off);
+                const uint64_t nwords = var.packed_bytes / 4;
+                for (uint32_t i = 0; i < cnt; ++i) {
+                    // this lane's 32 elements of the tile and the B words that hold exactly their codes
+                    const uint64_t e0 = (uint64_t)(local + i) * TILE + (uint64_t)lane * 32;
+                    const uint64_t w0 = e0 / 32 * f.B;
+                    const int valid = e0 >= var.n ? 0 : (var.n - e0 < 32 ? (int)(var.n - e0) : 32);
+                    uint64_t rbuf = 0, wbuf = 0;      // bit reader / writer over consecutive words
+                    int rfill = 0, wfill = 0;
+                    uint64_t rw = w0, ww = w0;
+                    uint32_t ref = 0u, diff = 0u;
+                    for (int k = 0; k < valid; ++k) {
+                        float w;
+                        if (MODE != COMPRESS) {
+                            if (rfill < f.B) { rbuf |= (uint64_t)cw[rw++] << rfill; rfill += 32; }
+                            const uint32_t c = (uint32_t)rbuf & code_mask;
+                            rbuf >>= f.B; rfill -= f.B;
+                            const float vbar = __fmaf_rn(s, dyn_decode(f, c), b);
+                            w = vbar;
+                            if (MODE == UPDATE) {
+                                w = __fmaf_rn(p.neg_lr, p.fin[var.full_off + e0 + k], vbar);
+                                if (w != w) w = u2f(0x7FFFFFFFu);     // arithmetic NaNs get one pattern
+                            }
+                        } else {
+                            w = p.fin[var.full_off + e0 + k];
                         }
-                    } else {
-                        w = p.fin[var.full_off + e0 + k];
+                        if (MODE != DECOMPRESS) {
+                            float vt;
+                            const uint32_t c = dyn_encode(f, w, vt);
+                            acc.add(w, vt);
+                            if (k == 0) ref = f2u(vt); else diff |= f2u(vt) ^ ref;
+                            wbuf |= (uint64_t)c << wfill; wfill += f.B;
+                            if (wfill >= 32) { cw[ww++] = (uint32_t)wbuf; wbuf >>= 32; wfill -= 32; }
+                        }
+                        if (MODE == DECOMPRESS || WOUT) p.fout[var.full_off + e0 + k] = w;
                     }
                     if (MODE != DECOMPRESS) {
-                        float vt;
-                        const uint32_t c = dyn_encode(f, w, vt);
-                        acc.add(w, vt);
-                        if (k == 0) ref = f2u(vt); else diff |= f2u(vt) ^ ref;
-                        wbuf |= (uint64_t)c << wfill; wfill += f.B;
-                        if (wfill >= 32) { cw[ww++] = (uint32_t)wbuf; wbuf >>= 32; wfill -= 32; }
+                        if (valid > 0) { acc.band &= ref & ~diff; acc.bor |= ref | diff; }
+                        if (wfill > 0) { cw[ww++] = (uint32_t)wbuf; }
+                        // words of this lane's share that hold no code any more: zero padding
+                        for (; ww < w0 + (uint64_t)f.B && ww < nwords; ++ww) cw[ww] = 0u;
                     }
-                    if (MODE == DECOMPRESS || WOUT) p.fout[var.full_off + e0 + k] = w;
                 }
                 if (MODE != DECOMPRESS) {
-                    if (valid > 0) { acc.band &= ref & ~diff; acc.bor |= ref | diff; }
-                    if (wfill > 0) { cw[ww++] = (uint32_t)wbuf; }
-                    // words of this lane's share that hold no code any more: zero padding
-                    for (; ww < w0 + (uint64_t)f.B && ww < nwords; ++ww) cw[ww] = 0u;
+                    if (p.pvt) {
+                        flush_and_maybe_finalise(p.slots + var.slot_base, run - var.first_run, var.nslots,
+                                                 p.tickets + var.sb_slot, cnt, var.ntiles, var.n, 0x7FFFFFFFu,
+                                                 p.sb + 2 * var.sb_slot, acc, lane);
+                    } else if (MODE == COMPRESS && local == 0 && lane == 0) {
+                        p.sb[2 * var.sb_slot] = 1.f;
+                        p.sb[2 * var.sb_slot + 1] = 0.f;
+                    }
+                }
+            } else {
+                for (uint32_t i = 0; i < cnt; ++i) {
+                    const uint64_t e0 = (uint64_t)(local + i) * TILE;
+                    tile_resid<MODE, WOUT>(p.resid + var.store_off + e0,
+                                           (MODE != DECOMPRESS) ? p.fin + var.full_off + e0 : nullptr,
+                                           ((MODE == DECOMPRESS) || WOUT) ? p.fout + var.full_off + e0 : nullptr,
+                                           var.n - e0, p.neg_lr, lane);
                 }
             }
-            if (MODE != DECOMPRESS) {
-                if (p.pvt) {
-                    flush_and_maybe_finalise(p.slots + var.slot_base, warp - var.first_warp, var.nslots,
-                                             p.tickets + var.sb_slot, cnt, var.ntiles, var.n, 0x7FFFFFFFu,
-                                             p.sb + 2 * var.sb_slot, acc, lane);
-                } else if (MODE == COMPRESS && local == 0 && lane == 0) {
-                    p.sb[2 * var.sb_slot] = 1.f;
-                    p.sb[2 * var.sb_slot + 1] = 0.f;
-                }
-            }
-        } else {
-            for (uint32_t i = 0; i < cnt; ++i) {
-                const uint64_t e0 = (uint64_t)(local + i) * TILE;
-                tile_resid<MODE, WOUT>(p.resid + var.store_off + e0,
-                                       (MODE != DECOMPRESS) ? p.fin + var.full_off + e0 : nullptr,
-                                       ((MODE == DECOMPRESS) || WOUT) ? p.fout + var.full_off + e0 : nullptr,
-                                       var.n - e0, p.neg_lr, lane);
-            }
+            t += cnt;
+            ++v;
         }
-        t += cnt;
-        ++v;
     }
 }
 

@@ -25,7 +25,22 @@ namespace omc {
 
 enum Mode { COMPRESS = 0, DECOMPRESS = 1, UPDATE = 2 };
 
-constexpr int STAGES = 2;                   // input stages per warp
+// Input stages per warp (granules fetched ahead = stages - 1), per kind of kernel.  The decoder
+// spends little time on a granule, so it needs more granules in flight to cover the load latency.
+#ifndef OMC_STAGES_COMPRESS
+#define OMC_STAGES_COMPRESS 2
+#endif
+#ifndef OMC_STAGES_DECOMPRESS
+#define OMC_STAGES_DECOMPRESS 2
+#endif
+#ifndef OMC_STAGES_UPDATE
+#define OMC_STAGES_UPDATE 2
+#endif
+constexpr int MAX_STAGES = 4;               // mbarriers reserved per warp
+constexpr int stages_for(int mode)
+{
+    return mode == 0 ? OMC_STAGES_COMPRESS : mode == 1 ? OMC_STAGES_DECOMPRESS : OMC_STAGES_UPDATE;
+}
 constexpr uint32_t WAIT_LIMIT = 1u << 24;   // polls of one mbarrier before giving up
 
 // Build-time overrides for tuning runs: granule size and number of output buffers for all formats.
@@ -58,7 +73,7 @@ struct Unit {
     static_assert(LU != 32 || SUB == STEP, "row layout: one 32-element row per lane and granule");
 };
 
-// Shared-memory budget of one warp: STAGES input stages and OUTBUFS output buffers of one granule.
+// Shared-memory budget of one warp: NSTAGES input stages and OUTBUFS output buffers of one granule.
 template <class F, int MODE, bool WOUT>
 struct Smem {
     static constexpr int SUB = Unit<F>::SUB;
@@ -70,16 +85,18 @@ struct Smem {
     static constexpr int IN_F = (MODE != DECOMPRESS) ? FB : 0;
     static constexpr int STAGE = IN_C + IN_F;
     static constexpr int TX_BYTES = STAGE;        // what the stage's copies bring in
-    static constexpr int DIST = STAGES - 1;       // granules fetched ahead
+    static constexpr int NSTAGES = stages_for(MODE);
+    static_assert(NSTAGES >= 2 && NSTAGES <= MAX_STAGES, "");
+    static constexpr int DIST = NSTAGES - 1;      // granules fetched ahead
     // Row layout, fused round: a lane rewrites its own code words behind its reads, so the new codes
     // take the place of the old ones in the stage and are stored from there.
     static constexpr bool CODES_IN_PLACE = ROWS && MODE == UPDATE;
     static constexpr int OUT_C = (MODE != DECOMPRESS && !CODES_IN_PLACE) ? CB : 0;
     static constexpr int OUT_F = (MODE == DECOMPRESS || WOUT) ? FB : 0;
     static constexpr int OUT = OUT_C + OUT_F;
-    static constexpr int PER_WARP = STAGES * STAGE + OUTBUFS * OUT;
+    static constexpr int PER_WARP = NSTAGES * STAGE + OUTBUFS * OUT;
     static_assert(!ROWS || (STAGE % 128 == 0 && OUT % 128 == 0 && CB % 128 == 0), "row layout: FP32 granules stay 128-byte aligned");
-    static constexpr int BAR_PAD = (8 * STAGES * WARPS_PER_CTA + 127) / 128 * 128;   // the mbarriers
+    static constexpr int BAR_PAD = (8 * MAX_STAGES * WARPS_PER_CTA + 127) / 128 * 128;   // the mbarriers
     static constexpr int TOTAL = BAR_PAD + WARPS_PER_CTA * PER_WARP;
     static_assert(STAGE % 16 == 0 && CB % 16 == 0, "bulk copies move multiples of 16 bytes");
 };
@@ -990,6 +1007,7 @@ struct WarpPipe {
     uint8_t *wbase;
     uint32_t bar0;
     uint32_t k;
+    uint32_t phases;      // bit i: the parity the next wait on mbarrier i looks for
     bool failed;
 };
 
@@ -1004,7 +1022,7 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
 {
     using SM = Smem<F, MODE, WOUT>;
     uint8_t *const wbase = pipe.wbase;
-    uint8_t *const outs = wbase + STAGES * SM::STAGE;
+    uint8_t *const outs = wbase + SM::NSTAGES * SM::STAGE;
     const uint32_t bar0 = pipe.bar0;
     uint32_t k = pipe.k;
     bool failed = false;
@@ -1014,7 +1032,7 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
 
     constexpr bool ROWS_IN = SM::ROWS && SM::IN_F > 0, ROWS_OUT = SM::ROWS && SM::OUT_F > 0;
     auto issue = [&](uint32_t g, uint32_t kk) {           // called by the whole warp
-        const uint32_t st = kk % STAGES;
+        const uint32_t st = kk % SM::NSTAGES;
         const uint32_t bar = bar0 + 8u * st;
         uint8_t *dst = wbase + st * SM::STAGE;
         if (lane == 0) {
@@ -1040,7 +1058,8 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
         }
         __syncwarp();
         // wait for this granule's bytes (bounded)
-        const uint32_t st = k % STAGES, bar = bar0 + 8u * st, parity = (k / STAGES) & 1u;
+        const uint32_t st = k % SM::NSTAGES, bar = bar0 + 8u * st, parity = (pipe.phases >> st) & 1u;
+        pipe.phases ^= 1u << st;
         uint32_t polls = 0;
         while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) {
             if (++polls > WAIT_LIMIT) { failed = true; break; }
@@ -1091,7 +1110,7 @@ __device__ __forceinline__ VarDev load_var(const VarDev *src)
     var.n = a.x; var.full_off = a.y; var.store_off = c.x; var.packed_bytes = c.y;
     var.tile_start = ((uint64_t)d.y << 32) | d.x;
     var.ntiles = d.z; var.quantised = d.w;
-    var.sb_slot = e.x; var.slot_base = e.y; var.first_warp = e.z; var.nslots = e.w;
+    var.sb_slot = e.x; var.slot_base = e.y; var.first_run = e.z; var.nslots = e.w;
     return var;
 }
 
@@ -1109,72 +1128,69 @@ omc_kernel(const KParams p)
     const uint32_t warp = blockIdx.x * WARPS_PER_CTA + wid;
     if (warp >= p.nwarps) return;
 
-    // this warp's slice of shared memory: STAGES input stages, then the output buffers
+    // this warp's slice of shared memory: the input stages, then the output buffers
     WarpPipe pipe;
     pipe.wbase = smem_raw + SM::BAR_PAD + wid * SM::PER_WARP;
-    pipe.bar0 = smem_addr(smem_raw) + (uint32_t)wid * STAGES * 8u;
+    pipe.bar0 = smem_addr(smem_raw) + (uint32_t)wid * MAX_STAGES * 8u;
     pipe.k = 0;
+    pipe.phases = 0u;
     pipe.failed = false;
     const uint32_t bar0 = pipe.bar0;
     if (lane == 0) {
 #pragma unroll
-        for (int i = 0; i < STAGES; ++i) mbar_init(bar0 + 8u * i, 1u);
+        for (int i = 0; i < MAX_STAGES; ++i) mbar_init(bar0 + 8u * i, 1u);
         fence_mbar_init();
         fence_proxy_async();
     }
     __syncwarp();
 
-    uint64_t t, tend;
-    warp_tile_range(p, warp, t, tend);
-    // variable that holds tile t
-    uint32_t lo = p.var_begin, hi = p.var_end;
-    while (hi - lo > 1) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (__ldg(&p.vars[mid].tile_start) <= t) lo = mid; else hi = mid;
-    }
-    uint32_t v = lo;
-    while (t < tend && !pipe.failed) {
-        const VarDev var = load_var(p.vars + v);
-        const uint32_t local = (uint32_t)(t - var.tile_start);
-        const uint64_t left = tend - t;
-        const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
-        if (var.quantised) {
-            float s = 1.f, b = 0.f;
-            if constexpr (MODE != COMPRESS) {
-                s = __ldcg(p.sb + 2 * var.sb_slot);
-                b = __ldcg(p.sb + 2 * var.sb_slot + 1);
-            }
-            Acc acc;
-            acc.reset();
-            uint8_t *const codes = p.packed + var.store_off;
-            const float *const fin = (MODE != DECOMPRESS) ? p.fin + var.full_off : nullptr;
-            float *const fout = (MODE == DECOMPRESS || WOUT) ? p.fout + var.full_off : nullptr;
-            const uint64_t e_begin = (uint64_t)local * TILE;
-            const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
-            run_elements<F, MODE, WOUT>(pipe, codes, fin, fout, e_begin, e_end, var.n, var.packed_bytes, s, b,
-                                        p.neg_lr, acc, lane);
-            if (pipe.failed) break;
-            if constexpr (MODE != DECOMPRESS) {
-                if (p.pvt) {
-                    flush_and_maybe_finalise(p.slots + var.slot_base, warp - var.first_warp, var.nslots,
-                                             p.tickets + var.sb_slot, cnt, var.ntiles, var.n,
-                                             ValuePattern<F>::MAGNITUDE_MASK, p.sb + 2 * var.sb_slot, acc, lane);
-                } else if (MODE == COMPRESS && local == 0 && lane == 0) {
-                    p.sb[2 * var.sb_slot] = 1.f;
-                    p.sb[2 * var.sb_slot + 1] = 0.f;
+    for (uint32_t run = warp; run < p.nruns && !pipe.failed; run += p.nwarps) {
+        uint64_t t, tend;
+        run_tile_range(p, run, t, tend);
+        uint32_t v = run_first_var(p, run, t);
+        while (t < tend && !pipe.failed) {
+            const VarDev var = load_var(p.vars + v);
+            const uint32_t local = (uint32_t)(t - var.tile_start);
+            const uint64_t left = tend - t;
+            const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
+            if (var.quantised) {
+                float s = 1.f, b = 0.f;
+                if constexpr (MODE != COMPRESS) {
+                    s = __ldcg(p.sb + 2 * var.sb_slot);
+                    b = __ldcg(p.sb + 2 * var.sb_slot + 1);
+                }
+                Acc acc;
+                acc.reset();
+                uint8_t *const codes = p.packed + var.store_off;
+                const float *const fin = (MODE != DECOMPRESS) ? p.fin + var.full_off : nullptr;
+                float *const fout = (MODE == DECOMPRESS || WOUT) ? p.fout + var.full_off : nullptr;
+                const uint64_t e_begin = (uint64_t)local * TILE;
+                const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
+                run_elements<F, MODE, WOUT>(pipe, codes, fin, fout, e_begin, e_end, var.n, var.packed_bytes, s, b,
+                                            p.neg_lr, acc, lane);
+                if (pipe.failed) break;
+                if constexpr (MODE != DECOMPRESS) {
+                    if (p.pvt) {
+                        flush_and_maybe_finalise(p.slots + var.slot_base, run - var.first_run, var.nslots,
+                                                 p.tickets + var.sb_slot, cnt, var.ntiles, var.n,
+                                                 ValuePattern<F>::MAGNITUDE_MASK, p.sb + 2 * var.sb_slot, acc, lane);
+                    } else if (MODE == COMPRESS && local == 0 && lane == 0) {
+                        p.sb[2 * var.sb_slot] = 1.f;
+                        p.sb[2 * var.sb_slot + 1] = 0.f;
+                    }
+                }
+            } else {
+                for (uint32_t i = 0; i < cnt; ++i) {
+                    const uint64_t e0 = (uint64_t)(local + i) * TILE;
+                    tile_resid<MODE, WOUT>(p.resid + var.store_off + e0,
+                                           (MODE != DECOMPRESS) ? p.fin + var.full_off + e0 : nullptr,
+                                           ((MODE == DECOMPRESS) || WOUT) ? p.fout + var.full_off + e0 : nullptr,
+                                           var.n - e0, p.neg_lr, lane);
                 }
             }
-        } else {
-            for (uint32_t i = 0; i < cnt; ++i) {
-                const uint64_t e0 = (uint64_t)(local + i) * TILE;
-                tile_resid<MODE, WOUT>(p.resid + var.store_off + e0,
-                                       (MODE != DECOMPRESS) ? p.fin + var.full_off + e0 : nullptr,
-                                       ((MODE == DECOMPRESS) || WOUT) ? p.fout + var.full_off + e0 : nullptr,
-                                       var.n - e0, p.neg_lr, lane);
-            }
+            t += cnt;
+            ++v;
         }
-        t += cnt;
-        ++v;
     }
     if (pipe.failed && lane == 0) atomicExch(p.status, 1u);   // a bulk load never arrived
     bulk_wait_all();                                     // stores must finish before the CTA's memory goes
@@ -1237,73 +1253,71 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_transition_kernel(co
     if (warp >= p.nwarps) return;
     WarpPipe pipe;
     pipe.wbase = smem_raw + TS::C::BAR_PAD + wid * TS::PER_WARP;
-    pipe.bar0 = smem_addr(smem_raw) + (uint32_t)wid * STAGES * 8u;
+    pipe.bar0 = smem_addr(smem_raw) + (uint32_t)wid * MAX_STAGES * 8u;
     pipe.k = 0;
+    pipe.phases = 0u;
     pipe.failed = false;
     if (lane == 0) {
 #pragma unroll
-        for (int i = 0; i < STAGES; ++i) mbar_init(pipe.bar0 + 8u * i, 1u);
+        for (int i = 0; i < MAX_STAGES; ++i) mbar_init(pipe.bar0 + 8u * i, 1u);
         fence_mbar_init();
         fence_proxy_async();
     }
     __syncwarp();
 
-    uint64_t t, tend;
-    warp_tile_range(p, warp, t, tend);
-    uint32_t lo = p.var_begin, hi = p.var_end;
-    while (hi - lo > 1) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (__ldg(&p.vars[mid].tile_start) <= t) lo = mid; else hi = mid;
-    }
-    uint32_t v = lo;
-    while (t < tend && !pipe.failed) {
-        const VarDev var = load_var(p.vars + v);            // where the variable goes
-        const VarDev src = load_var(p.vars_from + v);       // where it is now
-        const uint32_t local = (uint32_t)(t - var.tile_start);
-        const uint64_t left = tend - t;
-        const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
-        const uint64_t e_begin = (uint64_t)local * TILE;
-        const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
-        if (var.quantised && src.quantised) {
-            // same codes, other place: this run's share of the padded stream
-            const uint64_t b0 = e_begin / 8 * F::B;
-            const uint64_t b1 = (uint64_t)(local + cnt) == var.ntiles ? var.packed_bytes : e_end / 8 * F::B;
-            warp_copy16(reinterpret_cast<uint4 *>(p.packed + var.store_off + b0),
-                        reinterpret_cast<const uint4 *>(p.packed_from + src.store_off + b0), (b1 - b0) / 16, lane);
-            if (local == 0 && lane == 0) {
-                p.sb[2 * var.sb_slot] = p.sb_from[2 * src.sb_slot];
-                p.sb[2 * var.sb_slot + 1] = p.sb_from[2 * src.sb_slot + 1];
+    for (uint32_t run = warp; run < p.nruns && !pipe.failed; run += p.nwarps) {
+        uint64_t t, tend;
+        run_tile_range(p, run, t, tend);
+        uint32_t v = run_first_var(p, run, t);
+        while (t < tend && !pipe.failed) {
+            const VarDev var = load_var(p.vars + v);            // where the variable goes
+            const VarDev src = load_var(p.vars_from + v);       // where it is now
+            const uint32_t local = (uint32_t)(t - var.tile_start);
+            const uint64_t left = tend - t;
+            const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
+            const uint64_t e_begin = (uint64_t)local * TILE;
+            const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
+            if (var.quantised && src.quantised) {
+                // same codes, other place: this run's share of the padded stream
+                const uint64_t b0 = e_begin / 8 * F::B;
+                const uint64_t b1 = (uint64_t)(local + cnt) == var.ntiles ? var.packed_bytes : e_end / 8 * F::B;
+                warp_copy16(reinterpret_cast<uint4 *>(p.packed + var.store_off + b0),
+                            reinterpret_cast<const uint4 *>(p.packed_from + src.store_off + b0), (b1 - b0) / 16, lane);
+                if (local == 0 && lane == 0) {
+                    p.sb[2 * var.sb_slot] = p.sb_from[2 * src.sb_slot];
+                    p.sb[2 * var.sb_slot + 1] = p.sb_from[2 * src.sb_slot + 1];
+                }
+            } else if (!var.quantised && !src.quantised) {
+                warp_copy16(reinterpret_cast<uint4 *>(p.resid + var.store_off + e_begin),
+                            reinterpret_cast<const uint4 *>(p.resid_from + src.store_off + e_begin),
+                            (e_end - e_begin + 3) / 4, lane);
+            } else if (src.quantised) {
+                // released: decompress into the FP32 arena
+                const float s = __ldcg(p.sb_from + 2 * src.sb_slot), b = __ldcg(p.sb_from + 2 * src.sb_slot + 1);
+                Acc none;
+                none.reset();
+                run_elements<F, DECOMPRESS, false>(pipe, const_cast<uint8_t *>(p.packed_from) + src.store_off, nullptr,
+                                                   p.resid + var.store_off, e_begin, e_end, var.n, src.packed_bytes,
+                                                   s, b, 0.f, none, lane);
+            } else {
+                // newly selected: quantise the FP32 values, fit (s, b)
+                Acc acc;
+                acc.reset();
+                run_elements<F, COMPRESS, false>(pipe, p.packed + var.store_off, p.resid_from + src.store_off, nullptr,
+                                                 e_begin, e_end, var.n, var.packed_bytes, 1.f, 0.f, 0.f, acc, lane);
+                if (pipe.failed) break;
+                if (p.pvt) {
+                    flush_and_maybe_finalise(p.slots + var.slot_base, run - var.first_run, var.nslots,
+                                             p.tickets + var.sb_slot, cnt, var.ntiles, var.n,
+                                             ValuePattern<F>::MAGNITUDE_MASK, p.sb + 2 * var.sb_slot, acc, lane);
+                } else if (local == 0 && lane == 0) {
+                    p.sb[2 * var.sb_slot] = 1.f;
+                    p.sb[2 * var.sb_slot + 1] = 0.f;
+                }
             }
-        } else if (!var.quantised && !src.quantised) {
-            warp_copy16(reinterpret_cast<uint4 *>(p.resid + var.store_off + e_begin),
-                        reinterpret_cast<const uint4 *>(p.resid_from + src.store_off + e_begin),
-                        (e_end - e_begin + 3) / 4, lane);
-        } else if (src.quantised) {
-            // released: decompress into the FP32 arena
-            const float s = __ldcg(p.sb_from + 2 * src.sb_slot), b = __ldcg(p.sb_from + 2 * src.sb_slot + 1);
-            Acc none;
-            none.reset();
-            run_elements<F, DECOMPRESS, false>(pipe, const_cast<uint8_t *>(p.packed_from) + src.store_off, nullptr,
-                                               p.resid + var.store_off, e_begin, e_end, var.n, src.packed_bytes,
-                                               s, b, 0.f, none, lane);
-        } else {
-            // newly selected: quantise the FP32 values, fit (s, b)
-            Acc acc;
-            acc.reset();
-            run_elements<F, COMPRESS, false>(pipe, p.packed + var.store_off, p.resid_from + src.store_off, nullptr,
-                                             e_begin, e_end, var.n, var.packed_bytes, 1.f, 0.f, 0.f, acc, lane);
-            if (pipe.failed) break;
-            if (p.pvt) {
-                flush_and_maybe_finalise(p.slots + var.slot_base, warp - var.first_warp, var.nslots,
-                                         p.tickets + var.sb_slot, cnt, var.ntiles, var.n,
-                                         ValuePattern<F>::MAGNITUDE_MASK, p.sb + 2 * var.sb_slot, acc, lane);
-            } else if (local == 0 && lane == 0) {
-                p.sb[2 * var.sb_slot] = 1.f;
-                p.sb[2 * var.sb_slot + 1] = 0.f;
-            }
+            t += cnt;
+            ++v;
         }
-        t += cnt;
-        ++v;
     }
     if (pipe.failed && lane == 0) atomicExch(p.status, 1u);
     bulk_wait_all();

@@ -40,16 +40,22 @@ extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
     if (plan->d_vars && plan->device != dev) return OMC_ERR_PLAN_MISMATCH;
     if (!plan->d_vars) {
         const size_t bytes = sizeof(omc::VarDev) * (size_t)plan->nvars;
-        const size_t ws_bytes = sizeof(uint64_t) * plan->warp_start.size();
-        rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), bytes + 16 + ws_bytes));
+        const size_t rs_bytes = sizeof(uint64_t) * plan->run_start.size();
+        const size_t rv_bytes = sizeof(uint32_t) * plan->run_var.size();
+        const size_t dv_bytes = sizeof(uint32_t) * plan->dec_run_var.size();
+        rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), bytes + 16 + rs_bytes + rv_bytes + dv_bytes));
         if (rc) { plan->d_vars = nullptr; return rc; }
         char *const base = reinterpret_cast<char *>(plan->d_vars);
         rc = omc::note_cuda(cudaMemcpy(base, plan->vars.data(), bytes, cudaMemcpyHostToDevice));
         if (!rc) rc = omc::note_cuda(cudaMemset(base + bytes, 0, 16));
-        if (!rc) rc = omc::note_cuda(cudaMemcpy(base + bytes + 16, plan->warp_start.data(), ws_bytes, cudaMemcpyHostToDevice));
+        if (!rc) rc = omc::note_cuda(cudaMemcpy(base + bytes + 16, plan->run_start.data(), rs_bytes, cudaMemcpyHostToDevice));
+        if (!rc) rc = omc::note_cuda(cudaMemcpy(base + bytes + 16 + rs_bytes, plan->run_var.data(), rv_bytes, cudaMemcpyHostToDevice));
+        if (!rc) rc = omc::note_cuda(cudaMemcpy(base + bytes + 16 + rs_bytes + rv_bytes, plan->dec_run_var.data(), dv_bytes, cudaMemcpyHostToDevice));
         if (rc) { (void)cudaFree(plan->d_vars); plan->d_vars = nullptr; return rc; }
         plan->d_status = reinterpret_cast<uint32_t *>(base + bytes);
-        plan->d_warp_start = reinterpret_cast<uint64_t *>(base + bytes + 16);
+        plan->d_run_start = reinterpret_cast<uint64_t *>(base + bytes + 16);
+        plan->d_run_var = reinterpret_cast<uint32_t *>(base + bytes + 16 + rs_bytes);
+        plan->d_dec_run_var = reinterpret_cast<uint32_t *>(base + bytes + 16 + rs_bytes + rv_bytes);
         plan->device = dev;
     }
     return omc::note_cuda(cudaMemsetAsync(workspace, 0, plan->ws_bytes, static_cast<cudaStream_t>(stream)));
@@ -74,7 +80,9 @@ static KParams whole_model(const omc_plan_t *plan, void *workspace)
     p.tile_begin = 0;
     p.tile_count = plan->ntiles;
     p.nwarps = plan->nwarps;
-    p.warp_start = plan->d_warp_start;
+    p.nruns = plan->nruns;
+    p.run_start = plan->d_run_start;
+    p.run_var = plan->d_run_var;
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
     p.dyn_e = plan->fmt.exp_bits;
     p.dyn_m = plan->fmt.man_bits;
@@ -124,6 +132,14 @@ extern "C" int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, con
     p.tile_count = lastv.tile_start + lastv.ntiles - p.tile_begin;
     const uint64_t max_warps = (uint64_t)plan->n_sm * omc::DECOMPRESS_CTAS_PER_SM * omc::WARPS_PER_CTA;
     p.nwarps = (uint32_t)(p.tile_count < max_warps ? p.tile_count : max_warps);
+    // short runs of equal length, dealt out to the warps in turn
+    if (n_vars == plan->nvars) {      // the whole model: the plan knows where each run starts
+        p.nwarps = plan->dec_nwarps;
+        p.nruns = plan->dec_nruns;
+        p.run_var = plan->d_dec_run_var;
+    } else {
+        p.nruns = omc::runs_for(p.tile_count, p.nwarps, plan->dec_tiles_per_run, omc::DECODE_MAX_RUNS);
+    }
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
     p.dyn_e = plan->fmt.exp_bits;
     p.dyn_m = plan->fmt.man_bits;

@@ -39,8 +39,8 @@ struct VarDev {
     uint32_t quantised;
     uint32_t sb_slot;       // index into sb[] and the ticket array
     uint32_t slot_base;     // first partial-sum slot of this variable in the workspace
-    uint32_t first_warp;    // the warp (of the plan-wide partition) that owns the first tile
-    uint32_t nslots;        // number of warps that own at least one tile of this variable
+    uint32_t first_run;     // the run (of the plan-wide division) that holds the first tile
+    uint32_t nslots;        // number of runs that hold at least one tile of this variable
 };
 static_assert(sizeof(VarDev) == 64, "VarDev is laid out for 16-byte loads");
 
@@ -60,10 +60,15 @@ struct KParams {
     uint32_t var_begin, var_end;   // variables covered by this launch
     uint64_t tile_begin;           // first tile covered
     uint64_t tile_count;           // number of tiles covered
-    uint32_t nwarps;               // warps the tiles are divided among (<= tile_count)
-    // Optional: nwarps + 1 tile indices, warp w owns tiles [warp_start[w], warp_start[w + 1]).
-    // NULL: warp w owns [tile_begin + w * tile_count / nwarps, tile_begin + (w + 1) * tile_count / nwarps).
-    const uint64_t *warp_start;
+    uint32_t nwarps;               // warps launched (<= tile_count)
+    // The tiles are divided into nruns contiguous runs; warp w takes runs w, w + nwarps, ... so that
+    // the warps running at the same time work on neighbouring memory.
+    // run_start: nruns + 1 tile indices, run r = tiles [run_start[r], run_start[r + 1]); if NULL, run r =
+    // tiles [tile_begin + r * tile_count / nruns, tile_begin + (r + 1) * tile_count / nruns).
+    // run_var[r] = the variable that holds the run's first tile; if NULL, the kernel searches for it.
+    uint32_t nruns;
+    const uint64_t *run_start;
+    const uint32_t *run_var;
     uint32_t pvt;
     uint32_t dyn_e, dyn_m;         // the format, for the kernels that take it at run time
     uint8_t *packed;
@@ -107,22 +112,47 @@ struct FmtOps {
 };
 const FmtOps *find_ops(int E, int M);
 
-// Divides the tiles of vars[0 .. nvars) (n, quantised, tile_start and ntiles filled in) among
-// nwarps warps: writes warp_start[0 .. nwarps] (warp w owns tiles [warp_start[w], warp_start[w+1]))
-// and each variable's first_warp, nslots and slot_base; returns the number of partial-sum slots.
-uint32_t divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nwarps, uint64_t *warp_start);
-
-// The tiles [t, tend) of warp `warp` under the launch's division of the work.
-#ifdef __CUDACC__
-__device__ __forceinline__ void warp_tile_range(const KParams &p, uint32_t warp, uint64_t &t, uint64_t &tend)
+// Divides the tiles of vars[0 .. nvars) (n, quantised, tile_start and ntiles filled in) into nruns
+// contiguous runs of about equal estimated cost: writes run_start[0 .. nruns], run_var[0 .. nruns)
+// and each variable's first_run, nslots and slot_base; returns the number of partial-sum slots.
+uint32_t divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nruns, uint64_t *run_start, uint32_t *run_var);
+// How many runs of about tiles_per_run tiles a launch of nwarps warps over `tiles` tiles is cut
+// into: a multiple of nwarps, at most max_runs (but at least nwarps).
+uint32_t runs_for(uint64_t tiles, uint32_t nwarps, uint32_t tiles_per_run, uint32_t max_runs);
+// The decoder's runs, in tiles (measured on B200 with 8-, 12- and 16-bit codes: best at about four
+// pipeline granules per run; one-tile runs are slower than none at all).
+#ifndef OMC_DECODE_TILES_PER_RUN
+#define OMC_DECODE_TILES_PER_RUN 0          // 0: by code width; otherwise this many tiles for every format
+#endif
+constexpr uint32_t decode_tiles_per_run(uint32_t code_bits)
 {
-    if (p.warp_start) {
-        t = __ldg(p.warp_start + warp);
-        tend = __ldg(p.warp_start + warp + 1);
+    return OMC_DECODE_TILES_PER_RUN ? OMC_DECODE_TILES_PER_RUN : (code_bits >= 16 ? 4u : 2u);
+}
+constexpr uint32_t DECODE_MAX_RUNS = 1u << 22;
+
+#ifdef __CUDACC__
+// The tiles [t, tend) of run `run`.
+__device__ __forceinline__ void run_tile_range(const KParams &p, uint32_t run, uint64_t &t, uint64_t &tend)
+{
+    if (p.run_start) {
+        t = __ldg(p.run_start + run);
+        tend = __ldg(p.run_start + run + 1);
     } else {
-        t = p.tile_begin + (uint64_t)warp * p.tile_count / p.nwarps;
-        tend = p.tile_begin + (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
+        // tile_count < 2^40 and nruns <= 2^22: the products fit 64 bits
+        t = p.tile_begin + (uint64_t)run * p.tile_count / p.nruns;
+        tend = p.tile_begin + (uint64_t)(run + 1) * p.tile_count / p.nruns;
     }
+}
+// The variable that holds tile t, the first tile of run `run`.
+__device__ __forceinline__ uint32_t run_first_var(const KParams &p, uint32_t run, uint64_t t)
+{
+    if (p.run_var) return __ldg(p.run_var + run);
+    uint32_t lo = p.var_begin, hi = p.var_end;
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (__ldg(&p.vars[mid].tile_start) <= t) lo = mid; else hi = mid;
+    }
+    return lo;
 }
 #endif
 
@@ -136,14 +166,21 @@ struct omc_plan {
     std::vector<uint64_t> resid_off;   // per variable (valid iff !quantised)
     uint64_t full_elems, resid_elems, packed_bytes, closed_form_bytes;
     uint64_t ntiles;                   // all tiles
-    uint32_t n_sm, n_cta, nwarps;      // launch geometry the partition was made for
+    uint32_t n_sm, n_cta, nwarps;      // launch geometry the division was made for
+    uint32_t nruns;
+    uint32_t dec_nwarps, dec_nruns;    // the decoder's launch: equal runs, dealt out in turn
+    uint32_t dec_tiles_per_run;
     uint32_t nslots;
     uint64_t ws_tickets_off, ws_slots_off, ws_bytes;
     const omc::FmtOps *ops;
     // device side
-    std::vector<uint64_t> warp_start;  // nwarps + 1 entries: the cost-balanced division of the tiles
-    omc::VarDev *d_vars;               // one allocation: the variable table, the status word, warp_start
+    std::vector<uint64_t> run_start;   // nruns + 1 entries: the cost-balanced division of the tiles
+    std::vector<uint32_t> run_var;     // nruns entries: the variable each run starts in
+    std::vector<uint32_t> dec_run_var; // dec_nruns entries: the same for the decoder's runs
+    omc::VarDev *d_vars;               // one allocation: the variable table, the status word, the two run tables
     uint32_t *d_status;
-    uint64_t *d_warp_start;
+    uint64_t *d_run_start;
+    uint32_t *d_run_var;
+    uint32_t *d_dec_run_var;
     int device;                        // device the tables live on, -1 before prepare
 };

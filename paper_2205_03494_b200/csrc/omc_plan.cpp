@@ -74,14 +74,14 @@ static uint32_t query_sm_count()
     return (uint32_t)sms;
 }
 
-// Division of the tiles among warps: contiguous runs of equal estimated cost.  A warp pays for a
-// tile and, on top, for every quantised variable it enters (pipeline restart, ragged end,
-// hand-over of the fit's sums).  A tile goes to warp floor(cost before it * nwarps / total cost):
-// monotone in the tile index, and inside a variable consecutive owners differ by at most one, so
-// the warps first_warp .. first_warp + nslots - 1 of a variable all own one of its tiles.
-uint32_t omc::divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nwarps, uint64_t *warp_start)
+// Division of the tiles into contiguous runs of equal estimated cost.  A run pays for a tile and,
+// on top, for every quantised variable it enters (pipeline restart, ragged end, hand-over of the
+// fit's sums).  A tile goes to run floor(cost before it * nruns / total cost): monotone in the tile
+// index, and inside a variable consecutive tiles' runs differ by at most one, so the runs
+// first_run .. first_run + nslots - 1 of a variable all hold one of its tiles.
+uint32_t omc::divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nruns, uint64_t *run_start, uint32_t *run_var)
 {
-    const uint64_t NW = nwarps;
+    const uint64_t NR = nruns;
     auto var_cost = [](const VarDev &v) {
         return v.quantised ? (uint64_t)OMC_COST_TILE * v.ntiles + OMC_COST_VARIABLE
                            : (uint64_t)OMC_COST_FP32_TILE * v.ntiles;
@@ -91,36 +91,54 @@ uint32_t omc::divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nwarps, uint64
         total_cost += var_cost(vars[i]);
         tiles += vars[i].ntiles;
     }
-    // 128-bit products: the cost of 2^40-element variables times the warp count overflows 64 bits
-    auto warp_of = [&](uint64_t cost) { return (uint32_t)(((unsigned __int128)cost * NW) / total_cost); };
-    warp_start[0] = 0;
-    uint32_t slots = 0, w = 0;
+    // 128-bit products: the cost of 2^40-element variables times the run count overflows 64 bits
+    auto run_of = [&](uint64_t cost) { return (uint32_t)(((unsigned __int128)cost * NR) / total_cost); };
+    run_start[0] = 0;
+    run_var[0] = 0;
+    uint32_t slots = 0, r = 0;
     uint64_t before = 0;
     for (uint32_t i = 0; i < nvars; ++i) {
         VarDev &v = vars[i];
         const uint64_t per_tile = v.quantised ? OMC_COST_TILE : OMC_COST_FP32_TILE;
         const uint64_t c = before + (v.quantised ? OMC_COST_VARIABLE : 0);     // cost before tile 0 of v
-        v.first_warp = warp_of(c);
-        // the tiles of v at which the owner changes, solved for instead of walking every tile
+        v.first_run = run_of(c);
+        // the tiles of v at which the run changes, solved for instead of walking every tile
         uint64_t k = 0;
         while (k < v.ntiles) {
-            const uint32_t own = warp_of(c + per_tile * k);
-            while (w < own) warp_start[++w] = v.tile_start + k;
-            // smallest cost that belongs to the next warp, and the first tile of v that reaches it
-            const unsigned __int128 need = ((unsigned __int128)(own + 1) * total_cost + NW - 1) / NW;
+            const uint32_t own = run_of(c + per_tile * k);
+            while (r < own) {
+                run_start[++r] = v.tile_start + k;
+                run_var[r] = i;
+            }
+            // smallest cost that belongs to the next run, and the first tile of v that reaches it
+            const unsigned __int128 need = ((unsigned __int128)(own + 1) * total_cost + NR - 1) / NR;
             uint64_t k2 = (uint64_t)((need - c + per_tile - 1) / per_tile);
             if (k2 <= k) k2 = k + 1;
             k = k2 < v.ntiles ? k2 : v.ntiles;
         }
-        v.nslots = warp_of(c + per_tile * (v.ntiles - 1)) - v.first_warp + 1;
+        v.nslots = run_of(c + per_tile * (v.ntiles - 1)) - v.first_run + 1;
         if (v.quantised) {
             v.slot_base = slots;
             slots += v.nslots;
         }
         before += var_cost(v);
     }
-    while (w < NW) warp_start[++w] = tiles;
+    while (r < NR) {
+        run_start[++r] = tiles;
+        if (r < NR) run_var[r] = nvars - 1;      // an empty run at the end
+    }
     return slots;
+}
+
+// Runs of about tiles_per_run tiles, a whole number of them per warp (at least one, at most max_runs
+// in all).
+uint32_t omc::runs_for(uint64_t tiles, uint32_t nwarps, uint32_t tiles_per_run, uint32_t max_runs)
+{
+    const uint64_t per_round = (uint64_t)nwarps * tiles_per_run;
+    uint64_t rounds = (tiles + per_round - 1) / per_round;
+    if (rounds * nwarps > max_runs) rounds = max_runs / nwarps;
+    if (rounds < 1) rounds = 1;
+    return (uint32_t)(rounds * nwarps);
 }
 
 extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t fmt, double fraction,
@@ -149,7 +167,9 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         pl->ops = ops;
         pl->d_vars = nullptr;
         pl->d_status = nullptr;
-        pl->d_warp_start = nullptr;
+        pl->d_run_start = nullptr;
+        pl->d_run_var = nullptr;
+        pl->d_dec_run_var = nullptr;
         pl->device = -1;
         const uint32_t B = 1u + fmt.exp_bits + fmt.man_bits;
 
@@ -217,9 +237,27 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         pl->n_cta = pl->n_sm * omc::CTAS_PER_SM;
         const uint64_t max_warps = (uint64_t)pl->n_cta * omc::WARPS_PER_CTA;
         pl->nwarps = (uint32_t)(tiles < max_warps ? tiles : max_warps);
-        pl->warp_start.assign((size_t)pl->nwarps + 1, 0);
-        const uint32_t slots = omc::divide_tiles(pl->vars.data(), nvars, pl->nwarps, pl->warp_start.data());
+        // Kernels that fit (s, b) take one run per warp: a run ends with a hand-over of the sums,
+        // which costs more than working side by side with the other warps gains.
+        pl->nruns = pl->nwarps;
+        pl->run_start.assign((size_t)pl->nruns + 1, 0);
+        pl->run_var.assign((size_t)pl->nruns, 0);
+        const uint32_t slots = omc::divide_tiles(pl->vars.data(), nvars, pl->nruns, pl->run_start.data(),
+                                                 pl->run_var.data());
         pl->nslots = slots;
+
+        // ---- the decoder's own division (it keeps no sums): short runs of equal length, dealt out
+        // to the warps in turn, so that the warps of a launch sweep through memory side by side
+        const uint64_t max_dec_warps = (uint64_t)pl->n_sm * omc::DECOMPRESS_CTAS_PER_SM * omc::WARPS_PER_CTA;
+        pl->dec_nwarps = (uint32_t)(tiles < max_dec_warps ? tiles : max_dec_warps);
+        pl->dec_tiles_per_run = omc::decode_tiles_per_run(B);
+        pl->dec_nruns = omc::runs_for(tiles, pl->dec_nwarps, pl->dec_tiles_per_run, omc::DECODE_MAX_RUNS);
+        pl->dec_run_var.assign(pl->dec_nruns, 0);
+        for (uint32_t r = 0, i = 0; r < pl->dec_nruns; ++r) {
+            const uint64_t t = (uint64_t)(((unsigned __int128)r * tiles) / pl->dec_nruns);   // the run's first tile
+            while (i + 1 < nvars && pl->vars[i + 1].tile_start <= t) ++i;
+            pl->dec_run_var[r] = i;
+        }
         pl->ws_tickets_off = omc::WS_HEADER_BYTES;
         pl->ws_slots_off = round_up(pl->ws_tickets_off + 4ull * (nq ? nq : 1), 256);
         pl->ws_bytes = round_up(pl->ws_slots_off + sizeof(omc::Partial) * (uint64_t)(slots ? slots : 1), 256);
@@ -260,13 +298,14 @@ extern "C" int omc_plan_sizes(const omc_plan_t *plan, uint64_t *full_elems, uint
     return OMC_OK;
 }
 
-extern "C" int omc_plan_division(const omc_plan_t *plan, uint32_t *n_warps, uint64_t *n_tiles,
-                                 const uint64_t **warp_start)
+extern "C" int omc_plan_division(const omc_plan_t *plan, uint32_t *n_warps, uint32_t *n_runs, uint64_t *n_tiles,
+                                 const uint64_t **run_start)
 {
     if (!plan) return OMC_ERR_NULL_PTR;
     if (n_warps) *n_warps = plan->nwarps;
+    if (n_runs) *n_runs = plan->nruns;
     if (n_tiles) *n_tiles = plan->ntiles;
-    if (warp_start) *warp_start = plan->warp_start.data();
+    if (run_start) *run_start = plan->run_start.data();
     return OMC_OK;
 }
 

@@ -14,13 +14,14 @@ int note_cuda(cudaError_t e);
 
 namespace {
 
-constexpr uint32_t MAX_SLOTS = 4096;                     // warps that may each leave one record
+constexpr uint32_t MAX_SLOTS = 4096;                     // runs, each of which leaves one record
 constexpr size_t OFF_VAR = 0;                            // omc::VarDev, 64 bytes
 constexpr size_t OFF_TICKET = 64;                        // uint32_t
 constexpr size_t OFF_STATUS = 68;                        // uint32_t
 constexpr size_t OFF_SLOTS = 256;                        // omc::Partial[MAX_SLOTS]
-constexpr size_t OFF_WARP_START = OFF_SLOTS + sizeof(omc::Partial) * MAX_SLOTS;   // uint64_t[MAX_SLOTS + 1]
-constexpr size_t SCRATCH_BYTES = OFF_WARP_START + sizeof(uint64_t) * (MAX_SLOTS + 1);   // 229,640 bytes
+constexpr size_t OFF_RUN_START = OFF_SLOTS + sizeof(omc::Partial) * MAX_SLOTS;   // uint64_t[MAX_SLOTS + 1]
+constexpr size_t OFF_RUN_VAR = OFF_RUN_START + sizeof(uint64_t) * (MAX_SLOTS + 1);    // uint32_t[MAX_SLOTS], all zero
+constexpr size_t SCRATCH_BYTES = OFF_RUN_VAR + sizeof(uint32_t) * MAX_SLOTS;   // 246,024 bytes
 
 // Held by every GPU that loads the library until the process exits.  In host code this name is
 // only a handle for cudaGetSymbolAddress; it is never passed to a kernel.
@@ -79,6 +80,7 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     const uint64_t max_warps = (uint64_t)sms * omc::CTAS_PER_SM * omc::WARPS_PER_CTA;
     const uint32_t nwarps = (uint32_t)(tiles < max_warps ? tiles : max_warps);
     if (nwarps > MAX_SLOTS) return OMC_ERR_TOO_LARGE;
+    const uint32_t nruns = nwarps;          // one run per warp, as in omc_compress
 
     omc::VarDev v{};
     v.n = numel;
@@ -90,8 +92,9 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     v.quantised = 1;
     v.sb_slot = 0;
     v.slot_base = 0;
-    uint64_t warp_start[MAX_SLOTS + 1];        // host copy; the same division omc_plan makes
-    omc::divide_tiles(&v, 1, nwarps, warp_start);
+    uint64_t run_start[MAX_SLOTS + 1];         // host copy; the same division omc_plan makes
+    uint32_t run_var[MAX_SLOTS];               // all zero: there is one variable
+    omc::divide_tiles(&v, 1, nruns, run_start, run_var);
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // The array keeps what the last call left: the table entry and the division are rewritten, the
@@ -99,7 +102,10 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     // they are read.  Both host buffers are pageable, so each copy has left them when it returns.
     rc = omc::note_cuda(cudaMemcpyAsync(scratch + OFF_VAR, &v, sizeof v, cudaMemcpyHostToDevice, st));
     if (rc) return rc;
-    rc = omc::note_cuda(cudaMemcpyAsync(scratch + OFF_WARP_START, warp_start, sizeof(uint64_t) * (nwarps + 1),
+    rc = omc::note_cuda(cudaMemcpyAsync(scratch + OFF_RUN_START, run_start, sizeof(uint64_t) * (nruns + 1),
+                                        cudaMemcpyHostToDevice, st));
+    if (rc) return rc;
+    rc = omc::note_cuda(cudaMemcpyAsync(scratch + OFF_RUN_VAR, run_var, sizeof(uint32_t) * nruns,
                                         cudaMemcpyHostToDevice, st));
     if (rc) return rc;
     rc = omc::note_cuda(cudaMemsetAsync(scratch + OFF_TICKET, 0, 8, st));
@@ -112,7 +118,9 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     p.tile_begin = 0;
     p.tile_count = tiles;
     p.nwarps = nwarps;
-    p.warp_start = reinterpret_cast<const uint64_t *>(scratch + OFF_WARP_START);
+    p.nruns = nruns;
+    p.run_start = reinterpret_cast<const uint64_t *>(scratch + OFF_RUN_START);
+    p.run_var = reinterpret_cast<const uint32_t *>(scratch + OFF_RUN_VAR);
     p.pvt = (flags & OMC_PLAN_PVT) ? 1u : 0u;
     p.dyn_e = fmt.exp_bits;
     p.dyn_m = fmt.man_bits;

@@ -131,10 +131,11 @@ def test_workload_shapes():
     assert not np.array_equal(g, workloads.tiny().grads(0, 0)) and abs(g.std() - 1e-3) < 1e-4
 
 
-def test_division_of_the_tiles_among_warps():
-    """Every tile belongs to exactly one warp, runs are contiguous and in order, and no warp's
-    run is much longer than an equal share: at most the share plus three tiles for every
-    quantised variable that starts inside it (what the plan charges a warp for entering one)."""
+def test_division_of_the_tiles_into_runs():
+    """Every tile belongs to exactly one run, runs are contiguous and in order, their number is a
+    whole multiple of the warps launched, and no run is much longer than an equal share: at most
+    the share plus three tiles for every quantised variable that starts inside it (what the plan
+    charges a run for entering one)."""
     rag = workloads.ragged()
     conf = workloads.conformer_like()
     cases = [(rag.numel, rag.kinds, rag.fmt, 1.0), (conf.numel, conf.kinds, conf.fmt, 1.0),
@@ -142,22 +143,20 @@ def test_division_of_the_tiles_among_warps():
              ([1], [0], (5, 10), 1.0), ([1 << 40], [0], (5, 2), 1.0), ([3] * 5000, [0] * 5000, (4, 3), 1.0)]
     for numel, kinds, fmt, frac in cases:
         p = omc.Plan(numel, kinds, fmt, fraction=frac)
-        ntiles, ws = p.division()
+        nwarps, ntiles, rs = p.division()
         tiles = [(n + 1023) // 1024 for n in numel]
         assert ntiles == sum(tiles)
-        assert ws[0] == 0 and ws[-1] == ntiles and all(a <= b for a, b in zip(ws, ws[1:]))
-        nwarps = len(ws) - 1
-        assert 1 <= nwarps <= ntiles
-        if len(numel) > 10000 or ntiles > 1 << 24:
+        assert rs[0] == 0 and rs[-1] == ntiles and all(a <= b for a, b in zip(rs, rs[1:]))
+        nruns = len(rs) - 1
+        assert 1 <= nwarps <= ntiles and nruns % nwarps == 0 and nruns // nwarps <= 64
+        if ntiles > 1 << 24:
             continue
         # tile index at which each variable starts, to count the variables a run enters
         starts = np.cumsum([0] + tiles[:-1])
         qstarts = np.array([t for t, q in zip(starts, p.quantised) if q])
-        share = ntiles / nwarps
-        for w in range(nwarps):
-            run = ws[w + 1] - ws[w]
-            entered = int(np.searchsorted(qstarts, ws[w + 1]) - np.searchsorted(qstarts, ws[w]))
-            cost_share = share + 3 * len(qstarts) / nwarps
-            assert run <= cost_share + 2, (w, run, cost_share)
-            assert run + 3 * entered >= cost_share - 5, (w, run, entered, cost_share)
-
+        cost_share = (ntiles + 3 * len(qstarts)) / nruns
+        for r in range(nruns):
+            run = rs[r + 1] - rs[r]
+            entered = int(np.searchsorted(qstarts, rs[r + 1]) - np.searchsorted(qstarts, rs[r]))
+            assert run <= cost_share + 2, (r, run, cost_share)
+            assert run + 3 * entered >= cost_share - 5, (r, run, entered, cost_share)
