@@ -257,29 +257,15 @@ static __device__ __noinline__ void flush_and_maybe_finalise(Partial *slots, uin
     }
 }
 
-// Formats whose full units take compute_unit_pairs (two elements per register) instead of
-// compute_unit.  Measured on B200: a gain for 8-bit codes only (the 12- and 16-bit kernels are
-// no faster with it), so only S1E5M2 uses it; the switch lets a tuning build change that.
-#ifndef OMC_PAIR_PATH_BITS
-#define OMC_PAIR_PATH_BITS 8
-#endif
-template <class F>
-struct PairPath {
-    static constexpr bool value = HalfPath<F>::value && !Fp8Path<F>::value &&
-                                  (F::B == 8 || F::B == 12 || F::B == 16) && (F::B <= OMC_PAIR_PATH_BITS);
-};
-
 // A 32-bit pattern that identifies the value Q^-1(code) up to the sign of zero; the fit only needs
-// to know whether all of a variable's values are equal.  Pair-path formats use the FP16 pattern in
-// both halves (so that two codes can be compared per operation), the others the FP32 pattern.
+// to know whether all of a variable's values are equal.  The narrow-float formats use the code in
+// all four bytes (so that four codes can be compared per operation), the others the FP32 pattern.
 template <class F>
 struct ValuePattern {
-    static constexpr uint32_t MAGNITUDE_MASK =
-        Fp8Path<F>::value ? F::MAG_MASK * 0x01010101u : PairPath<F>::value ? 0x7FFF7FFFu : 0x7FFFFFFFu;
+    static constexpr uint32_t MAGNITUDE_MASK = Fp8Path<F>::value ? F::MAG_MASK * 0x01010101u : 0x7FFFFFFFu;
     __device__ static __forceinline__ uint32_t of(uint32_t code, float vt)
     {
-        if constexpr (Fp8Path<F>::value) return code * 0x01010101u;      // the code in all four bytes
-        if constexpr (PairPath<F>::value) return ((code << (10 - F::M)) & 0xFFFFu) * 0x00010001u;
+        if constexpr (Fp8Path<F>::value) return code * 0x01010101u;
         return f2u(vt);
     }
 };
@@ -483,142 +469,6 @@ __device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const flo
         acc.band &= ref & ~diff;
         acc.bor |= ref | diff;
     }
-}
-
-// ---------------------------------------------------------------------------------------------
-// The same arithmetic for full units of the half-path formats with 8-, 12- and 16-bit codes, two
-// elements at a time: a pair lives in one register as two FP16 patterns (code << (10-M), element
-// 2p in the low half).  Byte permutes unpack and pack, and Inf/NaN/overflow are detected on the
-// packed result (exponent field 31) once per unit, which then goes to compute_unit out of line.
-// Results are identical to compute_unit.
-
-// Out-of-line entry to compute_unit for the rare unit that holds a special value, so that the
-// careful path costs the main loop neither registers nor instruction-cache space.
-template <class F, int MODE>
-__device__ __noinline__ void compute_unit_careful(const uint32_t *win_p, const float4 *fv_p, uint32_t *wout_p,
-                                                  float4 *fo_p, float s, float b, float neg_lr, Acc *acc_p)
-{
-    constexpr int LU = Unit<F>::LU, NW = Unit<F>::NWORDS;
-    uint32_t win[NW], wout[NW];
-    float4 fv[LU / 4], fo[LU / 4];
-#pragma unroll
-    for (int j = 0; j < NW; ++j) win[j] = win_p[j];
-#pragma unroll
-    for (int j = 0; j < LU / 4; ++j) fv[j] = fv_p[j];
-    Acc acc = *acc_p;
-    compute_unit<F, MODE, false>(win, fv, wout, fo, s, b, neg_lr, acc, LU);
-    *acc_p = acc;
-#pragma unroll
-    for (int j = 0; j < NW; ++j) wout_p[j] = wout[j];
-#pragma unroll
-    for (int j = 0; j < LU / 4; ++j) fo_p[j] = fo[j];
-}
-
-template <class F>
-__device__ __forceinline__ void unpack_pairs(const uint32_t (&w)[Unit<F>::NWORDS], uint32_t (&X)[Unit<F>::LU / 2])
-{
-    if constexpr (F::B == 16) {
-        X[0] = w[0]; X[1] = w[1];
-    } else if constexpr (F::B == 8) {            // a code is the top byte of its FP16 pattern
-        X[0] = __byte_perm(w[0], 0u, 0x1404);
-        X[1] = __byte_perm(w[0], 0u, 0x3424);
-    } else {                                     // B == 12: pair p is bytes 3p .. 3p+2 of the unit
-        const uint32_t t[4] = {__byte_perm(w[0], 0u, 0x2110), __byte_perm(w[0], w[1], 0x5443),
-                               __byte_perm(w[1], w[2], 0x4332), __byte_perm(w[2], 0u, 0x3221)};
-#pragma unroll
-        for (int p = 0; p < 4; ++p)              // low half: code << 4; high half: already in place
-            X[p] = ((t[p] << 4) & 0x0000FFF0u) | (t[p] & 0xFFF00000u);
-    }
-}
-
-template <class F>
-__device__ __forceinline__ void pack_pairs(const uint32_t (&Y)[Unit<F>::LU / 2], uint32_t (&w)[Unit<F>::NWORDS])
-{
-    if constexpr (F::B == 16) {
-        w[0] = Y[0]; w[1] = Y[1];
-    } else if constexpr (F::B == 8) {
-        w[0] = __byte_perm(Y[0], Y[1], 0x7531);
-    } else {                                     // B == 12: 24 bits per pair, four pairs in three words
-        uint32_t q[4];
-#pragma unroll
-        for (int p = 0; p < 4; ++p) q[p] = ((Y[p] >> 4) & 0x00000FFFu) | ((Y[p] >> 8) & 0x00FFF000u);
-        w[0] = __byte_perm(q[0], q[1], 0x4210);
-        w[1] = __byte_perm(q[1], q[2], 0x5421);
-        w[2] = __byte_perm(q[2], q[3], 0x6542);
-    }
-}
-
-template <class F, int MODE>
-__device__ __forceinline__ void compute_unit_pairs(const uint32_t (&win)[Unit<F>::NWORDS],
-                                                   const float4 (&fv)[Unit<F>::LU / 4],
-                                                   uint32_t (&wout)[Unit<F>::NWORDS], float4 (&fo)[Unit<F>::LU / 4],
-                                                   float s, float b, float neg_lr, Acc &acc)
-{
-    constexpr int LU = Unit<F>::LU, NP = LU / 2;
-    uint32_t X[NP], Y[NP];
-    float w[LU], vt[LU];
-    if constexpr (MODE != COMPRESS) unpack_pairs<F>(win, X);
-    uint32_t special = 0u;
-#pragma unroll
-    for (int p = 0; p < NP; ++p) {
-        const float g0 = (p & 1) ? fv[p / 2].z : fv[p / 2].x, g1 = (p & 1) ? fv[p / 2].w : fv[p / 2].y;
-        if constexpr (MODE != COMPRESS) {
-            const __half2 hx = *reinterpret_cast<const __half2 *>(&X[p]);
-            const float v0 = __low2float(hx), v1 = __high2float(hx);     // exact, all codes
-            const float vb0 = __fmaf_rn(s, v0, b), vb1 = __fmaf_rn(s, v1, b);
-            w[2 * p] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, g0, vb0) : vb0;
-            w[2 * p + 1] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, g1, vb1) : vb1;
-        } else {
-            w[2 * p] = g0;
-            w[2 * p + 1] = g1;
-        }
-        if constexpr (MODE != DECOMPRESS) {
-            __half2 h;
-            if constexpr (F::M == 10) {
-                h = __floats2half2_rn(w[2 * p], w[2 * p + 1]);
-                vt[2 * p] = __low2float(h);
-                vt[2 * p + 1] = __high2float(h);
-            } else {
-                uint32_t c0, c1;                              // unused: the codes are read off Y
-                encode_fast2<F>(w[2 * p], w[2 * p + 1], c0, c1, vt[2 * p], vt[2 * p + 1]);
-                h = __floats2half2_rn(vt[2 * p], vt[2 * p + 1]);   // exact unless out of range
-            }
-            Y[p] = *reinterpret_cast<const uint32_t *>(&h);
-            special |= (Y[p] & 0x7FFF7FFFu) + 0x04000400u;    // bit 15 of a half set <=> exponent field 31
-        }
-    }
-    if constexpr (MODE != DECOMPRESS) {
-        if (special & 0x80008000u) {      // Inf, NaN or overflow in this unit: take the careful path,
-            // on copies, so that only they (and not the registers of the main path) have addresses
-            uint32_t win_c[Unit<F>::NWORDS], wout_c[Unit<F>::NWORDS];
-            float4 fv_c[LU / 4], fo_c[LU / 4];
-            Acc acc_c = acc;
-#pragma unroll
-            for (int j = 0; j < Unit<F>::NWORDS; ++j) win_c[j] = (MODE != COMPRESS) ? win[j] : 0u;
-#pragma unroll
-            for (int j = 0; j < LU / 4; ++j) fv_c[j] = fv[j];
-            compute_unit_careful<F, MODE>(win_c, fv_c, wout_c, fo_c, s, b, neg_lr, &acc_c);
-            acc = acc_c;
-#pragma unroll
-            for (int j = 0; j < Unit<F>::NWORDS; ++j) wout[j] = wout_c[j];
-#pragma unroll
-            for (int j = 0; j < LU / 4; ++j) fo[j] = fo_c[j];
-            return;
-        }
-        const uint32_t ref = __byte_perm(Y[0], 0u, 0x1010);   // element 0's pattern in both halves
-        uint32_t diff = 0u;
-#pragma unroll
-        for (int p = 0; p < NP; ++p) {
-            acc.add(w[2 * p], vt[2 * p]);
-            acc.add(w[2 * p + 1], vt[2 * p + 1]);
-            diff |= Y[p] ^ ref;
-        }
-        acc.band &= ref & ~diff;
-        acc.bor |= ref | diff;
-        pack_pairs<F>(Y, wout);
-    }
-#pragma unroll
-    for (int g = 0; g < LU / 4; ++g) fo[g] = make_float4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -894,8 +744,6 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
             float4 fo[LU / 4];
             if constexpr (Fp8Path<F>::value)
                 compute_unit_fp8<F, MODE>(win[g], fv[g], wout, fo, s, b, neg_lr, acc);
-            else if constexpr (PairPath<F>::value)
-                compute_unit_pairs<F, MODE>(win[g], fv[g], wout, fo, s, b, neg_lr, acc);
             else
                 compute_unit<F, MODE, false>(win[g], fv[g], wout, fo, s, b, neg_lr, acc, LU);
             if constexpr (MODE != DECOMPRESS) store_words<NW>(wout, s_cout + unit * NW);
