@@ -223,9 +223,10 @@ int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint
  *     Y = X * Wbar^T,  Wbar = s*Wt + b (Sec. 2.3),  computed as  s * (X * Wt^T) + b * rowsum(X)
  * with X and the codes as FP16 operands of the tensor cores and FP32 accumulation (the paper
  * computes "in full precision or other hardware-supported formats").
- *   S1E5M10 (the codes are IEEE halves and feed the tensor cores as they are), S1E5M6 and S1E5M2
- *   (expanded to halves inside the kernel, on the way into the operand tile); other formats return
- *   OMC_ERR_BAD_FORMAT.
+ *   S1E5M10 (the codes are IEEE halves and feed the tensor cores as they are); S1E5M6, S1E5M2,
+ *   S1E4M3 and S1E2M3 (every value of these formats is an FP16 value: the codes are expanded to
+ *   halves inside the kernel, on the way into the operand tile; Inf and NaN codes included); other
+ *   formats return OMC_ERR_BAD_FORMAT.
  *   var must be quantised and N*K == its numel; N % 128 == 0, K % 64 == 0 (else OMC_ERR_INVALID_ARG).
  *   packed, sb      device, the model state (read only).
  *   x_half          device, M x K IEEE halves, K contiguous, 16-byte aligned.

@@ -35,10 +35,13 @@ constexpr int TILE_A_BYTES = BM * BK * 2, TILE_B_BYTES = BN * BK * 2;
 constexpr int TMEM_COLS = 512;                   // two accumulators of 128 lanes x 256 FP32 columns
 constexpr uint32_t WAIT_LIMIT = 1u << 20;        // polls of one mbarrier before giving up
 
-// B = bits per code.  16: no decode stage, four stages of 48 KB.  12 / 8: three stages of
-// 72 / 64 KB (X tile, operand tile, packed bytes of the tile) and eight decoder warps.
-template <int B>
+// B = bits per code, E = exponent bits.  16: no decode stage, four stages of 48 KB.  12 / 8 / 6:
+// three stages of 72 / 64 / 60 KB (X tile, operand tile, packed bytes of the tile) and eight
+// decoder warps.  E = 5 codes are FP16 patterns with the low mantissa bits dropped; S1E4M3 and
+// S1E2M3 codes go through the narrow-float conversion instructions.
+template <int B, int E>
 struct Cfg {
+    static_assert((E == 5 && (B == 16 || B == 12 || B == 8)) || (E == 4 && B == 8) || (E == 2 && B == 6), "");
     static constexpr bool DECODE = B != 16;
     static constexpr int ROW_BYTES = BK * B / 8;                 // one tile row of codes
     static constexpr int RAW_BYTES = DECODE ? BN * ROW_BYTES : 0;
@@ -122,16 +125,67 @@ __global__ void rowsum_kernel(const __half *__restrict__ x, uint32_t M, uint32_t
     if (lane == 0) out[row] = acc;
 }
 
-// Eight codes (one 16-byte chunk of halves) from their packed words.
-template <int B>
-__device__ __forceinline__ uint4 expand_chunk(const uint32_t *raw)
+// Four codes of a narrow-float type, one per byte, as two FP16 pairs.  MAG_MASK / INF_MAG: the
+// magnitude bits of a code and the magnitude of the family's infinity; the hardware type has
+// finite values (or its own NaN) from there on, the family has Inf (INF_MAG) and NaNs (above),
+// which are patched in afterwards (rare: a weight would have to be Inf or NaN).
+template <int E>
+__device__ __forceinline__ void narrow_to_halves(uint32_t c4, uint32_t &h01, uint32_t &h23)
 {
-    if constexpr (B == 8) {                  // a code is the top byte of its half
+    constexpr uint32_t MAG_MASK = E == 4 ? 0x7Fu : 0x1Fu, INF_MAG = E == 4 ? 0x78u : 0x18u;
+    constexpr uint32_t SIGN_SHIFT = E == 4 ? 7u : 5u;
+    if constexpr (E == 4)
+        asm("{\n\t.reg .b16 lo, hi;\n\t"
+            "mov.b32 {lo, hi}, %2;\n\t"
+            "cvt.rn.f16x2.e4m3x2 %0, lo;\n\t"
+            "cvt.rn.f16x2.e4m3x2 %1, hi;\n\t}"
+            : "=r"(h01), "=r"(h23) : "r"(c4));
+    else
+        asm("{\n\t.reg .b16 lo, hi;\n\t"
+            "mov.b32 {lo, hi}, %2;\n\t"
+            "cvt.rn.f16x2.e2m3x2 %0, lo;\n\t"
+            "cvt.rn.f16x2.e2m3x2 %1, hi;\n\t}"
+            : "=r"(h01), "=r"(h23) : "r"(c4));
+    if (((c4 & (MAG_MASK * 0x01010101u)) + (0x80u - INF_MAG) * 0x01010101u) & 0x80808080u) {
+        uint32_t h[4] = {h01 & 0xFFFFu, h01 >> 16, h23 & 0xFFFFu, h23 >> 16};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t c = (c4 >> (8 * j)) & 0xFFu, mag = c & MAG_MASK;
+            if (mag >= INF_MAG) h[j] = (((c >> SIGN_SHIFT) & 1u) << 15) | (mag == INF_MAG ? 0x7C00u : 0x7E00u);
+        }
+        h01 = h[0] | (h[1] << 16);
+        h23 = h[2] | (h[3] << 16);
+    }
+}
+
+// Eight codes (one 16-byte chunk of halves) from their B packed bytes.
+template <int B, int E>
+__device__ __forceinline__ uint4 expand_chunk(const uint8_t *raw)
+{
+    if constexpr (B == 8 && E == 5) {        // a code is the top byte of its half
         const uint2 w = *reinterpret_cast<const uint2 *>(raw);
         return make_uint4(__byte_perm(w.x, 0u, 0x1404), __byte_perm(w.x, 0u, 0x3424),
                           __byte_perm(w.y, 0u, 0x1404), __byte_perm(w.y, 0u, 0x3424));
+    } else if constexpr (B == 8) {           // S1E4M3
+        const uint2 w = *reinterpret_cast<const uint2 *>(raw);
+        uint4 o;
+        narrow_to_halves<E>(w.x, o.x, o.y);
+        narrow_to_halves<E>(w.y, o.z, o.w);
+        return o;
+    } else if constexpr (B == 6) {           // S1E2M3: 48 bits, spread to one code per byte
+        const uint16_t *r16 = reinterpret_cast<const uint16_t *>(raw);
+        const uint32_t a = r16[0], m = r16[1], z = r16[2];
+        const uint32_t lo24 = a | ((m & 0xFFu) << 16), hi24 = (m >> 8) | (z << 8);
+        auto spread = [](uint32_t t) {
+            return (t & 0x3Fu) | ((t << 2) & 0x3F00u) | ((t << 4) & 0x3F0000u) | ((t << 6) & 0x3F000000u);
+        };
+        uint4 o;
+        narrow_to_halves<E>(spread(lo24), o.x, o.y);
+        narrow_to_halves<E>(spread(hi24), o.z, o.w);
+        return o;
     } else {                                 // 12-bit codes: pair p is bytes 3p .. 3p+2, half = code << 4
-        const uint32_t w0 = raw[0], w1 = raw[1], w2 = raw[2];
+        const uint32_t *rw = reinterpret_cast<const uint32_t *>(raw);
+        const uint32_t w0 = rw[0], w1 = rw[1], w2 = rw[2];
         const uint32_t t0 = __byte_perm(w0, 0u, 0x2110), t1 = __byte_perm(w0, w1, 0x5443);
         const uint32_t t2 = __byte_perm(w1, w2, 0x4332), t3 = __byte_perm(w2, 0u, 0x3221);
         return make_uint4(((t0 << 4) & 0x0000FFF0u) | (t0 & 0xFFF00000u), ((t1 << 4) & 0x0000FFF0u) | (t1 & 0xFFF00000u),
@@ -139,13 +193,13 @@ __device__ __forceinline__ uint4 expand_chunk(const uint32_t *raw)
     }
 }
 
-template <int B>
-__global__ void __launch_bounds__(Cfg<B>::THREADS, 1)
+template <int B, int E>
+__global__ void __launch_bounds__(Cfg<B, E>::THREADS, 1)
 matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
               const float *__restrict__ sb, const float *__restrict__ rowsum, float *__restrict__ y,
               uint32_t M, uint32_t N, uint32_t K, uint32_t *status)
 {
-    using C = Cfg<B>;
+    using C = Cfg<B, E>;
     constexpr int NS = C::NSTAGES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (saddr(smem_raw) + 1023u) & ~1023u;      // tiles need 1024-byte alignment
@@ -277,12 +331,12 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                     ok = mbar_wait(full(s), (it / NS) & 1u);
                     if (!ok) break;
                     uint8_t *stage = base_ptr + s * C::STAGE;
-                    const uint32_t *raw = reinterpret_cast<const uint32_t *>(stage + TILE_A_BYTES + TILE_B_BYTES) + t * (B / 4);
+                    const uint8_t *raw = stage + TILE_A_BYTES + TILE_B_BYTES + t * B;      // 8 codes = B bytes
                     uint8_t *dst = stage + TILE_A_BYTES;
 #pragma unroll
                     for (int i = 0; i < BN * 8 / C::DEC_THREADS; ++i) {
                         const int r = i * (C::DEC_THREADS / 8) + (t >> 3);
-                        const uint4 o = expand_chunk<B>(raw + i * C::DEC_THREADS * (B / 4));
+                        const uint4 o = expand_chunk<B, E>(raw + i * C::DEC_THREADS * B);
                         // 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r mod 8)
                         *reinterpret_cast<uint4 *>(dst + r * 128 + ((c ^ (r & 7)) << 4)) = o;
                     }
@@ -346,11 +400,11 @@ bool make_raw_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t row_b
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int B>
+template <int B, int E>
 int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const float *rowsum, float *y,
            uint32_t M, uint32_t N, uint32_t K, uint32_t n_sm, uint32_t *status, cudaStream_t st)
 {
-    using C = Cfg<B>;
+    using C = Cfg<B, E>;
     CUtensorMap map_w;
     if (C::DECODE ? !make_raw_map(&map_w, codes, N, (uint64_t)K * B / 8, C::ROW_BYTES) : !make_map(&map_w, codes, N, K, BN))
         return OMC_ERR_CUDA;
@@ -358,13 +412,13 @@ int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const f
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        int rc = omc::note_cuda(cudaFuncSetAttribute(matmul_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+        int rc = omc::note_cuda(cudaFuncSetAttribute(matmul_kernel<B, E>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
         if (rc) return rc;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const uint32_t ntiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
     const uint32_t grid = ntiles < n_sm ? ntiles : n_sm;
-    matmul_kernel<B><<<grid, C::THREADS, C::SMEM, st>>>(map_x, map_w, sb, rowsum, y, M, N, K, status);
+    matmul_kernel<B, E><<<grid, C::THREADS, C::SMEM, st>>>(map_x, map_w, sb, rowsum, y, M, N, K, status);
     return omc::note_cuda(cudaGetLastError());
 }
 
@@ -378,8 +432,10 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     if (!plan->d_vars) return OMC_ERR_PLAN_MISMATCH;
     if (!packed || !sb || !x_half || !y || !rowsum_scratch) return OMC_ERR_NULL_PTR;
     if (var >= plan->nvars || !plan->vars[var].quantised) return OMC_ERR_INVALID_ARG;
-    const int man = plan->fmt.man_bits;
-    if (plan->fmt.exp_bits != 5 || (man != 10 && man != 6 && man != 2)) return OMC_ERR_BAD_FORMAT;
+    const int exp = plan->fmt.exp_bits, man = plan->fmt.man_bits;
+    const bool half_family = exp == 5 && (man == 10 || man == 6 || man == 2);
+    const bool narrow = (exp == 4 && man == 3) || (exp == 2 && man == 3);
+    if (!half_family && !narrow) return OMC_ERR_BAD_FORMAT;
     if (M == 0 || N == 0 || K == 0 || N % 128 != 0 || K % BK != 0 || (uint64_t)N * K != plan->vars[var].n)
         return OMC_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(packed) | reinterpret_cast<uintptr_t>(x_half) | reinterpret_cast<uintptr_t>(y)) & 15u)
@@ -392,9 +448,11 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     const uint8_t *codes = packed + v.store_off;
     const float *sbv = sb + 2 * v.sb_slot;
     const uint32_t n_sm = plan->n_sm ? plan->n_sm : 1;
+    if (exp == 4) return launch<8, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
+    if (exp == 2) return launch<6, 2>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
     switch (man) {
-    case 10: return launch<16>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
-    case 6: return launch<12>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
-    default: return launch<8>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
+    case 10: return launch<16, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
+    case 6: return launch<12, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
+    default: return launch<8, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
     }
 }

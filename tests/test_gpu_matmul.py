@@ -15,13 +15,15 @@ from harness import DeviceModel
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("fmt", [(5, 10), (5, 6), (5, 2)], ids=lambda f: "E%dM%d" % f)
+@pytest.mark.parametrize("fmt", [(5, 10), (5, 6), (5, 2), (4, 3), (2, 3)], ids=lambda f: "E%dM%d" % f)
 @pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 256, 192), (1000, 384, 512), (64, 128, 1024)])
 def test_matmul_from_codes_matches_definition(M, N, K, fmt):
     rng = np.random.default_rng(M + N + K)
     numel = [777, N * K, 64, 128 * 64]
     kinds = [0, 0, 1, 0]
-    params = [(rng.standard_normal(n) * 0.05 + 0.01).astype(np.float32) for n in numel]
+    scale = 1.0 if fmt == (2, 3) else 0.05          # S1E2M3 resolves nothing below 1/8 ...
+    params = [np.clip(rng.standard_normal(n) * scale + 0.2 * scale, -3.5, 3.5).astype(np.float32)
+              for n in numel]                        # ... and overflows from 3.875 on
     plan = omc.Plan(numel, kinds, fmt)
     dm = DeviceModel(plan)
     dm.compress(dm.upload_full(params))
@@ -46,7 +48,7 @@ def test_matmul_from_codes_matches_definition(M, N, K, fmt):
 def test_matmul_argument_checks():
     plan = omc.Plan([128 * 64, 100], [0, 1], (5, 10))
     dm = DeviceModel(plan)
-    p8 = omc.Plan([128 * 64], [0], (4, 3))
+    p8 = omc.Plan([128 * 64], [0], (3, 7))
     d8 = DeviceModel(p8)
     x = torch.zeros(128 * 64, dtype=torch.float16, device="cuda")
     y = torch.zeros(128 * 128, dtype=torch.float32, device="cuda")
@@ -60,3 +62,35 @@ def test_matmul_argument_checks():
                         y.data_ptr(), None) == -2
     assert L.omc_matmul(plan._h, 0, *a, 128, 128, 64, None, y.data_ptr(), None) == -3
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("fmt", [(4, 3), (2, 3)], ids=lambda f: "E%dM%d" % f)
+def test_matmul_weights_at_the_top_of_the_range(fmt):
+    """Weights that are infinite, NaN or the largest finite value of S1E4M3 / S1E2M3: the hardware
+    narrow-float types have other values at those codes, so the decoder patches them.  A row of W
+    with an infinity gives an infinite or NaN output column, a row with the largest finite value
+    the exact product."""
+    E, M = fmt
+    N, K, Mr = 128, 64, 128
+    top = 2.0 ** ((1 << (E - 1)) - 1) * (2 - 2.0 ** -M)
+    w = np.full((N, K), 0.5 * top, np.float32)           # a value of the format in both cases
+    w[3, 5] = np.inf
+    w[7, 9] = -np.inf
+    w[11, 0] = np.nan
+    w[20, :] = top
+    w[21, :] = -top
+    plan = omc.Plan([N * K], [0], fmt, flags=omc.PLAN_WEIGHTS_ONLY)       # no transformation: s = 1, b = 0
+    dm = DeviceModel(plan)
+    dm.compress(dm.upload_full([w.reshape(-1)]))
+    x = np.ones((Mr, K), np.float16)
+    xd = torch.from_numpy(x).cuda()
+    y = torch.zeros((Mr, N), dtype=torch.float32, device="cuda")
+    scratch = torch.zeros(Mr, dtype=torch.float32, device="cuda")
+    omc.matmul(plan, 0, dm.packed.data_ptr(), dm.sb.data_ptr(), xd.data_ptr(), Mr, N, K, y.data_ptr(),
+               scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    got = y.cpu().numpy()
+    assert np.all(got[:, 3] == np.inf) and np.all(got[:, 7] == -np.inf) and np.all(np.isnan(got[:, 11]))
+    assert np.all(got[:, 20] == np.float32(top * K)) and np.all(got[:, 21] == np.float32(-top * K))
+    assert np.all(got[:, 0] == np.float32(0.5 * top * K))
+
