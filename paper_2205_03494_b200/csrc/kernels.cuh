@@ -2,15 +2,18 @@
 // template.
 //
 // Work is a flat list of 1024-element tiles over all variables; the tiles are divided into
-// contiguous runs, one per warp, so that ragged variable lists load-balance and a warp keeps the
-// fit's running sums in registers across the tiles of a variable.  Every warp is its own
+// contiguous runs and warp w takes runs w, w + nwarps, ...  The kernels that fit (s, b) get one
+// run per warp, of equal estimated cost, so that ragged variable lists load-balance and a warp
+// keeps the fit's running sums in registers across the tiles of a variable; the decoder, which
+// keeps no sums, gets short runs of equal length, so that the warps running at the same time
+// work on neighbouring memory.  Every warp is its own
 // producer/consumer pipeline: lane 0 streams the next granule (a tile or half a tile: packed codes
 // and FP32 operand) into one of the warp's shared-memory stages with 1-D TMA bulk copies that
 // complete on an mbarrier while the warp computes on the current stage; results go to an output
 // buffer and leave through a bulk store.  There is no block-wide barrier anywhere.  Ragged ends of
 // variables and FP32-only variables take a plain path with predicated vector loads and stores.
 //
-// Per (variable, warp) one partial-sum record goes to the workspace; the warp that completes a
+// Per (variable, run) one partial-sum record goes to the workspace; the warp that completes a
 // variable's last tile adds the records in a fixed order and finalises (s, b): deterministic, no
 // floating-point atomics, and no warp ever waits for another.  The only waits are on the warp's
 // own copies; they are bounded, and a wait that runs out sets the plan's status word and ends
