@@ -1116,7 +1116,8 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_transition_kernel(co
     }
     __syncwarp();
 
-    for (uint32_t run = warp; run < p.nruns && !pipe.failed; run += p.nwarps) {
+    const uint32_t nruns = __ldg(p.nruns_dev);      // this launch's own division (transition_division.cu)
+    for (uint32_t run = warp; run < nruns && !pipe.failed; run += p.nwarps) {
         uint64_t t, tend;
         run_tile_range(p, run, t, tend);
         uint32_t v = run_first_var(p, run, t);
@@ -1158,9 +1159,10 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_transition_kernel(co
                                                  e_begin, e_end, var.n, var.packed_bytes, 1.f, 0.f, 0.f, acc, lane);
                 if (pipe.failed) break;
                 if (p.pvt) {
-                    flush_and_maybe_finalise(p.slots + var.slot_base, run - var.first_run, var.nslots,
-                                             p.tickets + var.sb_slot, cnt, var.ntiles, var.n,
-                                             ValuePattern<F>::MAGNITUDE_MASK, p.sb + 2 * var.sb_slot, acc, lane);
+                    const uint4 tv = __ldg(reinterpret_cast<const uint4 *>(p.trans_vars) + v);   // first_run, nslots, slot_base
+                    flush_and_maybe_finalise(p.slots + tv.z, run - tv.x, tv.y, p.tickets + var.sb_slot, cnt,
+                                             var.ntiles, var.n, ValuePattern<F>::MAGNITUDE_MASK,
+                                             p.sb + 2 * var.sb_slot, acc, lane);
                 } else if (local == 0 && lane == 0) {
                     p.sb[2 * var.sb_slot] = 1.f;
                     p.sb[2 * var.sb_slot + 1] = 0.f;

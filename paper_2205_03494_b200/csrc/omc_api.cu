@@ -1,6 +1,8 @@
 // Device-side C-ABI entry points: argument checks, launch geometry, dispatch on the format.
 #include <cuda_runtime.h>
 
+#include <algorithm>
+
 #include "omc_internal.h"
 
 namespace omc {
@@ -28,6 +30,15 @@ const FmtOps *find_ops(int E, int M)
 
 using omc::KParams;
 
+// omc_transition's cost model (sixteenths of a tile; overridable at build time for tuning runs):
+// an FP32 tile copied, and the fixed part of a tile converted.
+#ifndef OMC_TCOST_COPY
+#define OMC_TCOST_COPY 16
+#endif
+#ifndef OMC_TCOST_CONVERT
+#define OMC_TCOST_CONVERT 12
+#endif
+
 static bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
 extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
@@ -43,7 +54,11 @@ extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
         const size_t rs_bytes = sizeof(uint64_t) * plan->run_start.size();
         const size_t rv_bytes = sizeof(uint32_t) * plan->run_var.size();
         const size_t dv_bytes = sizeof(uint32_t) * plan->dec_run_var.size();
-        rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), bytes + 16 + rs_bytes + rv_bytes + dv_bytes));
+        // omc_transition's tables (filled on the device before each launch)
+        const size_t nv = plan->nvars, nw = plan->nwarps;
+        const size_t tables = (bytes + 16 + rs_bytes + rv_bytes + dv_bytes + 15) / 16 * 16;
+        const size_t tr_bytes = 16 * nv + 8 * (nw + 1) + sizeof(omc::TransitionVar) * nv + 4 * nw + 16;
+        rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), tables + tr_bytes));
         if (rc) { plan->d_vars = nullptr; return rc; }
         char *const base = reinterpret_cast<char *>(plan->d_vars);
         rc = omc::note_cuda(cudaMemcpy(base, plan->vars.data(), bytes, cudaMemcpyHostToDevice));
@@ -56,6 +71,13 @@ extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
         plan->d_run_start = reinterpret_cast<uint64_t *>(base + bytes + 16);
         plan->d_run_var = reinterpret_cast<uint32_t *>(base + bytes + 16 + rs_bytes);
         plan->d_dec_run_var = reinterpret_cast<uint32_t *>(base + bytes + 16 + rs_bytes + rv_bytes);
+        char *tr = base + tables;                    // 16-byte entries first, then 8-byte ones, then 4-byte ones
+        plan->d_trans.vars = reinterpret_cast<omc::TransitionVar *>(tr);
+        plan->d_trans.before = reinterpret_cast<uint64_t *>(tr + sizeof(omc::TransitionVar) * nv);
+        plan->d_trans.last = plan->d_trans.before + nv;
+        plan->d_trans.run_start = plan->d_trans.last + nv;
+        plan->d_trans.run_var = reinterpret_cast<uint32_t *>(plan->d_trans.run_start + nw + 1);
+        plan->d_trans.nruns = plan->d_trans.run_var + nw;
         plan->device = dev;
     }
     return omc::note_cuda(cudaMemsetAsync(workspace, 0, plan->ws_bytes, static_cast<cudaStream_t>(stream)));
@@ -228,10 +250,27 @@ extern "C" int omc_transition(const omc_plan_t *from, const omc_plan_t *to, cons
     if (misaligned(packed_from) || misaligned(resid_from) || misaligned(sb_from) || misaligned(packed_to) ||
         misaligned(resid_to) || misaligned(sb_to) || misaligned(workspace_to))
         return OMC_ERR_MISALIGNED;
+    // The launch's own division of the work, by what each tile costs given both plans: copying codes
+    // moves B/4 bytes per element, copying FP32 values 8, converting 4 + B/8 plus the arithmetic; a
+    // variable that is fitted costs three tiles more (as in omc_plan).
+    const uint32_t B = 1u + to->fmt.exp_bits + to->fmt.man_bits;
+    omc::TransitionCosts costs;
+    costs.copy_codes = (B + 1) / 2 * OMC_TCOST_COPY / 16;
+    costs.copy_fp32 = OMC_TCOST_COPY;
+    costs.convert = OMC_TCOST_CONVERT + B / 4;
+    costs.fit_entry = 48;
+    if (costs.copy_codes < 1) costs.copy_codes = 1;
+    costs.max_tile = std::max(std::max(costs.copy_codes, costs.copy_fp32), costs.convert);
+    omc::launch_transition_division(to->d_vars, from->d_vars, to->nvars, to->ntiles, to->nwarps, costs, to->d_trans,
+                                    stream);
     KParams p = whole_model(to, workspace_to);
     p.packed = packed_to; p.resid = resid_to; p.sb = sb_to;
     p.vars_from = from->d_vars;
     p.packed_from = packed_from; p.resid_from = resid_from; p.sb_from = sb_from;
+    p.run_start = to->d_trans.run_start;
+    p.run_var = to->d_trans.run_var;
+    p.trans_vars = to->d_trans.vars;
+    p.nruns_dev = to->d_trans.nruns;
     to->ops->transition(p, grid_for(p.nwarps), stream);
     return omc::note_cuda(cudaGetLastError());
 }

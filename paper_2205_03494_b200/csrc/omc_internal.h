@@ -54,6 +54,8 @@ static_assert(sizeof(Partial) == 48, "");
 
 constexpr uint64_t WS_HEADER_BYTES = 256;
 
+struct TransitionVar;
+
 // Arguments of one kernel launch.
 struct KParams {
     const VarDev *vars;
@@ -84,8 +86,29 @@ struct KParams {
     const uint8_t *packed_from;
     const float *resid_from;
     const float *sb_from;
+    const TransitionVar *trans_vars;   // the launch's own record numbering
+    const uint32_t *nruns_dev;         // the launch's run count (replaces nruns)
     uint32_t *status;              // the plan's device status word: set non-zero if a copy never arrived
 };
+
+// omc_transition's own division of the work, made on the device before each launch.
+struct TransitionVar {          // for a variable that gets a fresh fit: its partial-sum records
+    uint32_t first_run, nslots, slot_base, pad;
+};
+struct TransitionTables {       // device memory owned by the destination plan
+    uint64_t *before;           // nvars: estimated cost of all variables before this one
+    uint64_t *last;             // nvars: estimated cost of everything before this variable's last tile
+    TransitionVar *vars;        // nvars
+    uint64_t *run_start;        // max_runs + 1
+    uint32_t *run_var;          // max_runs
+    uint32_t *nruns;            // 1: how many runs this launch has
+};
+struct TransitionCosts {        // per tile, in sixteenths of a tile that is quantised and fitted
+    uint32_t copy_codes, copy_fp32, convert, fit_entry, max_tile;
+};
+void launch_transition_division(const VarDev *to, const VarDev *from, uint32_t nvars, uint64_t ntiles,
+                                uint32_t max_runs, const TransitionCosts &c, const TransitionTables &out,
+                                void *stream);
 
 // Arguments of the aggregation kernel: the states of up to MAX_CLIENTS replicas of one model.
 constexpr int MAX_CLIENTS = 16;
@@ -182,5 +205,6 @@ struct omc_plan {
     uint64_t *d_run_start;
     uint32_t *d_run_var;
     uint32_t *d_dec_run_var;
+    omc::TransitionTables d_trans;     // omc_transition's tables (this plan as the destination)
     int device;                        // device the tables live on, -1 before prepare
 };

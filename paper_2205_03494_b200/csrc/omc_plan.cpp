@@ -2,6 +2,7 @@
 // tiles are divided among warps) and the C-ABI entry points that need no kernel.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -170,6 +171,7 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         pl->d_run_start = nullptr;
         pl->d_run_var = nullptr;
         pl->d_dec_run_var = nullptr;
+        pl->d_trans = omc::TransitionTables{};
         pl->device = -1;
         const uint32_t B = 1u + fmt.exp_bits + fmt.man_bits;
 
@@ -260,7 +262,10 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         }
         pl->ws_tickets_off = omc::WS_HEADER_BYTES;
         pl->ws_slots_off = round_up(pl->ws_tickets_off + 4ull * (nq ? nq : 1), 256);
-        pl->ws_bytes = round_up(pl->ws_slots_off + sizeof(omc::Partial) * (uint64_t)(slots ? slots : 1), 256);
+        // omc_transition numbers the records anew for each launch: at most one per run and one more
+        // per variable that is fitted
+        const uint64_t slots_cap = std::max<uint64_t>(slots ? slots : 1, (uint64_t)pl->nwarps + nq);
+        pl->ws_bytes = round_up(pl->ws_slots_off + sizeof(omc::Partial) * slots_cap, 256);
     } catch (const std::bad_alloc &) {
         delete pl;
         return OMC_ERR_NO_MEMORY;

@@ -69,6 +69,33 @@ def test_large_transformer_1p6b_one_round():
     assert ls.sb_ulp_cases <= 1, ls.sb_ulp_cases
 
 
+@pytest.mark.parametrize("fmt", [(5, 10), (5, 2)], ids=lambda f: "E%dM%d" % f)
+def test_conformer_like_100m_transition_between_90pct_subsets(fmt):
+    """omc_transition at the size bench.py times it: the whole 100M set from one random 90 % of the
+    matrices to another (its division of the work is made on the device by several thread blocks
+    and has thousands of runs here), every variable against the oracle, then one more round."""
+    from test_gpu_parity import oracle_transition
+    wl = workloads.conformer_like()
+    params = wl.all_params()
+    ls = Lockstep(wl.numel, wl.kinds, fmt, params, fraction=0.9, seed=21, threads=8)
+    del params
+    plan_to = omc.Plan(wl.numel, wl.kinds, fmt, fraction=0.9, seed=22)
+    changing = sum(a != b for a, b in zip(ls.plan.quantised, plan_to.quantised))
+    assert changing >= 10
+    from harness import DeviceModel
+    dm_to = DeviceModel(plan_to)
+    a, b = ls.dm, dm_to
+    omc.transition(ls.plan, plan_to, a.packed.data_ptr(), a.resid.data_ptr(), a.sb.data_ptr(),
+                   b.packed.data_ptr(), b.resid.data_ptr(), b.sb.data_ptr(), b.ws.data_ptr(),
+                   torch.cuda.current_stream().cuda_stream)
+    ls.st = oracle_transition(ls.st, plan_to.quantised)
+    ls.plan, ls.dm = plan_to, dm_to
+    packed = ls.check_state("transition")
+    ls.check_padding(packed)
+    ls.round(wl.all_grads(0), 5.0, want_w=False)
+    assert ls.sb_ulp_cases <= 1, ls.sb_ulp_cases
+
+
 @pytest.mark.parametrize("fmt", [(5, 2), (3, 7), (5, 10)], ids=lambda f: "E%dM%d" % f)
 def test_one_variable_beyond_32_bit_indexing(fmt):
     """A single variable of 2^32 + 1,081,344 elements (8-, 11- and 16-bit codes, fit on): element and byte offsets
