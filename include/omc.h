@@ -117,13 +117,15 @@ int omc_plan_var(const omc_plan_t *plan, uint32_t i, int *quantised, uint64_t *f
  * omc_plan_division -- how the plan divides the work of one launch (host only).
  * The model's variables are cut into tiles of 1024 elements, numbered in variable order (a
  * variable's last tile may be short), and the tiles into *n_runs contiguous runs of about equal
- * estimated cost: run r = tiles [run_start[r], run_start[r + 1]).  Warp w of omc_compress /
- * omc_update_recompress / omc_transition (and of omc_decompress over the whole model) takes runs
- * w, w + *n_warps, w + 2 * *n_warps, ...: the warps that run at the same time work on neighbouring
- * memory.  *run_start points at *n_runs + 1 non-decreasing entries owned by the plan (valid until
+ * estimated cost: run r = tiles [run_start[r], run_start[r + 1]).  Warp w of omc_compress and
+ * omc_update_recompress takes runs w, w + *n_warps, ... (one run per warp as the plans are made
+ * today: *n_runs == *n_warps), so that a warp adds up a variable's elements in its registers.
+ * *run_start points at *n_runs + 1 non-decreasing entries owned by the plan (valid until
  * omc_plan_destroy), the first 0 and the last *n_tiles; *n_runs is a multiple of *n_warps.  Any
  * output pointer may be NULL.  Sec. 2.3's sums are taken per variable whatever the division; it
  * only decides which warp adds which elements, and so the order of the fp64 additions.
+ * (omc_decompress keeps no sums and deals out short runs of equal length to its warps instead;
+ * omc_transition makes a division of its own for each call.)
  */
 int omc_plan_division(const omc_plan_t *plan, uint32_t *n_warps, uint32_t *n_runs, uint64_t *n_tiles,
                       const uint64_t **run_start);
@@ -188,7 +190,10 @@ int omc_update_recompress_host(const omc_plan_t *plan, uint8_t *packed, float *r
 /*
  * omc_transition -- re-selection (Sec. 2.5, Sec. 3.1: the quantised subset of weight matrices
  * changes from round to round and from client to client).  Takes a model's state under plan `from`
- * to its state under plan `to` in one launch.  Both plans must be prepared on the current device
+ * to its state under plan `to` in one call (a small kernel that divides the work by what each
+ * variable needs, given both plans, and the kernel that does it; `to`'s device tables are
+ * rewritten by the first, so calls with the same `to` must not overlap on the GPU).  Both plans
+ * must be prepared on the current device
  * and describe the same variables (count, sizes) in the same format, else OMC_ERR_PLAN_MISMATCH.
  * Per variable: quantised in both -> codes and (s, b) copied; FP32 in both -> copied; quantised only
  * in `from` -> decompressed into resid_to (fma(s, Vt, b)); quantised only in `to` -> quantised from

@@ -1116,7 +1116,11 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_transition_kernel(co
     }
     __syncwarp();
 
-    const uint32_t nruns = __ldg(p.nruns_dev);      // this launch's own division (transition_division.cu)
+    // This launch's own division (transition_division.cu) is written by the kernel before it on the
+    // stream; launched as its programmatic dependent, this kernel may start while that one ends,
+    // and waits here for its results.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const uint32_t nruns = *reinterpret_cast<const volatile uint32_t *>(p.nruns_dev);
     for (uint32_t run = warp; run < nruns && !pipe.failed; run += p.nwarps) {
         uint64_t t, tend;
         run_tile_range(p, run, t, tend);
@@ -1187,7 +1191,17 @@ void launch_transition(const KParams &p, int grid, void *stream)
                              TransitionSmem<F>::TOTAL);
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    omc_transition_kernel<F><<<grid, THREADS, TransitionSmem<F>::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = TransitionSmem<F>::TOTAL;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, omc_transition_kernel<F>, p);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -74,6 +74,8 @@ __global__ void __launch_bounds__(DIV_THREADS) transition_division_kernel(const 
     __shared__ uint64_t s_last[LAST_IN_SMEM];      // out.last for the searches below, if it fits
     const uint32_t tid = threadIdx.x;
     const bool cached = nvars <= LAST_IN_SMEM;
+    // omc_transition's main kernel may be scheduled now; it waits for this grid's results itself
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- cost before each variable
     uint64_t carry = 0;
