@@ -381,6 +381,31 @@ def test_transition_between_selections(fmt):
     assert ls.sb_ulp_cases <= 2
 
 
+@pytest.mark.parametrize("fmt", [(5, 10), (4, 3)], ids=lambda f: "E%dM%d" % f)
+def test_transition_extreme_selections(fmt):
+    """Selections at the ends: nothing quantised -> everything -> the same again -> nothing, and a
+    model of one single-element variable.  The launch's own division of the work then has only
+    copies, only conversions, or fewer tiles than one warp's share."""
+    rng = np.random.default_rng(5)
+    for numel in ([3000, 1, 1024, 70001, 2048, 12289, 64], [1]):
+        kinds = [0] * len(numel)
+        params = [(rng.standard_normal(n) * 0.1).astype(np.float32) for n in numel]
+        none, every = [0] * len(numel), [1] * len(numel)
+        ls = Lockstep(numel, kinds, fmt, params, mask=none)
+        for mask in (every, every, none, none):
+            plan_to = omc.Plan(numel, kinds, fmt, mask=mask)
+            dm_to = DeviceModel(plan_to)
+            a, b = ls.dm, dm_to
+            omc.transition(ls.plan, plan_to, a.packed.data_ptr(), a.resid.data_ptr(), a.sb.data_ptr(),
+                           b.packed.data_ptr(), b.resid.data_ptr(), b.sb.data_ptr(), b.ws.data_ptr(),
+                           torch.cuda.current_stream().cuda_stream)
+            ls.st = oracle_transition(ls.st, plan_to.quantised)
+            ls.plan, ls.dm = plan_to, dm_to
+            ls.check_padding(ls.check_state("transition"))
+            ls.round([(rng.standard_normal(n) * 0.05).astype(np.float32) for n in numel], 0.5)
+        assert ls.plan.status() == 0
+
+
 def test_transition_refuses_mismatched_plans():
     a = omc.Plan([100, 200], [0, 0], (5, 2))
     b = omc.Plan([100, 201], [0, 0], (5, 2))
