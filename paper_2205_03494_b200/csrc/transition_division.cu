@@ -6,8 +6,8 @@
 // list into runs of equal cost (the rule omc_plan uses: a tile goes to run
 // floor(cost before it * runs / total cost)) and numbers the partial-sum records of the
 // variables that get a fresh fit.  Everything stays on the stream: no host copy, no wait.
-// A few blocks share the runs; each of them adds up the costs for itself (the tables they write
-// that way hold the same values), block 0 numbers the records.
+// A few blocks share the runs and the last one numbers the records; each of them adds up the costs
+// for itself (the tables they write that way hold the same values).
 #include <cuda_runtime.h>
 
 #include "omc_internal.h"
@@ -123,7 +123,9 @@ __global__ void __launch_bounds__(DIV_THREADS) transition_division_kernel(const 
     auto last_cbt = [&](uint32_t i) { return cached ? s_last[i] : out.last[i]; };
 
     // ---- where each run starts: the first tile whose cost-before reaches ceil(r * total / nruns)
-    for (uint32_t r = blockIdx.x * DIV_THREADS + tid; r <= nruns; r += gridDim.x * DIV_THREADS) {
+    const uint32_t run_blocks = gridDim.x - 1;        // the last block numbers the records instead
+    for (uint32_t r = blockIdx.x * DIV_THREADS + tid; blockIdx.x < run_blocks && r <= nruns;
+         r += run_blocks * DIV_THREADS) {
         if (r == nruns) {
             out.run_start[r] = ntiles;
             continue;
@@ -147,7 +149,7 @@ __global__ void __launch_bounds__(DIV_THREADS) transition_division_kernel(const 
     }
 
     // ---- partial-sum records of the variables that get a fresh fit
-    if (blockIdx.x != 0) return;
+    if (blockIdx.x != run_blocks) return;
     uint32_t slot_carry = 0;
     for (uint32_t base = 0; base < nvars; base += DIV_THREADS) {
         const uint32_t i = base + tid;
@@ -181,6 +183,7 @@ void launch_transition_division(const VarDev *to, const VarDev *from, uint32_t n
 {
     uint32_t grid = (max_runs + DIV_THREADS) / DIV_THREADS;      // one thread per run, within reason
     if (grid > 32) grid = 32;
+    grid += 1;                                                   // and one block for the records
     transition_division_kernel<<<grid, DIV_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(to, from, nvars, ntiles,
                                                                                           max_runs, c, out);
 }
