@@ -27,6 +27,10 @@ namespace omc {
 int note_cuda(cudaError_t e);
 }
 
+#ifndef OMC_MATMUL_DECODER_THREADS
+#define OMC_MATMUL_DECODER_THREADS 512      // sixteen decoder warps (measured against eight)
+#endif
+
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;       // CTA tile; BK halves = one 128-byte swizzle row
@@ -36,7 +40,7 @@ constexpr int TMEM_COLS = 512;                   // two accumulators of 128 lane
 constexpr uint32_t WAIT_LIMIT = 1u << 20;        // polls of one mbarrier before giving up
 
 // B = bits per code, E = exponent bits.  16: no decode stage, four stages of 48 KB.  12 / 8 / 6:
-// three stages of 72 / 64 / 60 KB (X tile, operand tile, packed bytes of the tile) and eight
+// three stages of 72 / 64 / 60 KB (X tile, operand tile, packed bytes of the tile) and sixteen
 // decoder warps.  E = 5 codes are FP16 patterns with the low mantissa bits dropped; S1E4M3 and
 // S1E2M3 codes go through the narrow-float conversion instructions.
 template <int B, int E>
@@ -48,7 +52,7 @@ struct Cfg {
     static constexpr int STAGE = TILE_A_BYTES + TILE_B_BYTES + RAW_BYTES;
     static constexpr int NSTAGES = DECODE ? 3 : 4;
     static constexpr int SMEM = NSTAGES * STAGE + 1024 /* alignment slack */ + 256 /* barriers, tmem slot */;
-    static constexpr int DEC_THREADS = DECODE ? 256 : 0;
+    static constexpr int DEC_THREADS = DECODE ? OMC_MATMUL_DECODER_THREADS : 0;
     static constexpr int THREADS = 192 + DEC_THREADS;
     static constexpr uint32_t TX_BYTES = TILE_A_BYTES + (DECODE ? RAW_BYTES : TILE_B_BYTES);
     static_assert(STAGE % 1024 == 0, "operand tiles stay 1024-byte aligned");
