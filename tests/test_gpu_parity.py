@@ -282,6 +282,34 @@ def test_rounding_boundaries_through_the_fast_path(fmt):
     ls.check_decompress()
 
 
+@pytest.mark.parametrize("fmt", [(5, 10), (5, 2), (3, 7)], ids=lambda f: "E%dM%d" % f)
+def test_twenty_rounds_free_running(fmt):
+    """The GPU and the oracle each run twenty rounds on their own, neither seeing the other's
+    (s, b) in between; afterwards the decompressed models agree to 1e-6 relative.  A one-ulp
+    difference in some (s, b) along the way (fp64 sums in another order, about once in 2^16
+    fits) could flip a few codes in later rounds, so a 1e-5 share of the elements may differ."""
+    wl = workloads.conformer_like(blocks=1)
+    wl.fmt = fmt
+    params = wl.all_params()
+    plan = omc.Plan(wl.numel, wl.kinds, fmt)
+    dm = DeviceModel(plan)
+    dm.compress(dm.upload_full(params))
+    st = orc.compress(params, plan.quantised, fmt[0], fmt[1], True, 8)
+    for r in range(20):
+        grads = wl.all_grads(r)
+        dm.update(dm.upload_full(grads), 50.0)          # large steps: the codes keep moving
+        orc.update_recompress(st, grads, 50.0, 8)
+    got = dm.decompress().cpu().numpy()
+    want = orc.decompress(st, 8)
+    bad = total = 0
+    for i in range(plan.nvars):
+        g, w = from_full(plan, got, i), want[i]
+        bad += int(np.count_nonzero(~np.isclose(g, w, rtol=1e-6, atol=0.0, equal_nan=True)))
+        total += w.size
+    assert bad <= 1e-5 * total, (bad, total)
+    assert plan.status() == 0
+
+
 def test_plan_switches():
     """Per-variable transformation off (s = 1, b = 0 stay put), weights-only off, explicit mask."""
     wl = workloads.tiny()
