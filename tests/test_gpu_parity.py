@@ -161,6 +161,10 @@ def test_partial_quantisation_sweep(wl):
         nz = v != 0
         bound = np.exp2(np.maximum(np.floor(np.log2(np.abs(v[nz]))), emin) - M - 1)
         assert np.all(np.abs(vt[nz] - v[nz]) <= bound)
+        # uniform-noise model: the error in units of the local spacing is spread evenly over
+        # [-1/2, 1/2], so its RMS is 1/sqrt(12) (sanity check, 10 %)
+        rms = float(np.sqrt(np.mean(((vt[nz] - v[nz]) / (2 * bound)) ** 2)))
+        assert 0.9 / np.sqrt(12) <= rms <= 1.1 / np.sqrt(12), (i, rms)
         rec = from_full(ls.plan, out, i).astype(np.float64)
         assert np.linalg.norm(rec - v) <= np.linalg.norm(vt - v) * (1 + 1e-6)
     for r in range(2):
