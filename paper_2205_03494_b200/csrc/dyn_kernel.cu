@@ -156,13 +156,9 @@ __global__ void __launch_bounds__(THREADS) omc_dyn_kernel(const KParams p, const
                     }
                 }
             } else {
-                for (uint32_t i = 0; i < cnt; ++i) {
-                    const uint64_t e0 = (uint64_t)(local + i) * TILE;
-                    tile_resid<MODE, WOUT>(p.resid + var.store_off + e0,
-                                           (MODE != DECOMPRESS) ? p.fin + var.full_off + e0 : nullptr,
-                                           ((MODE == DECOMPRESS) || WOUT) ? p.fout + var.full_off + e0 : nullptr,
-                                           var.n - e0, p.neg_lr, lane);
-                }
+                resid_tiles<MODE, WOUT>(p.resid + var.store_off, (MODE != DECOMPRESS) ? p.fin + var.full_off : nullptr,
+                                        ((MODE == DECOMPRESS) || WOUT) ? p.fout + var.full_off : nullptr, var.n, local,
+                                        cnt, p.neg_lr, lane);
             }
             t += cnt;
             ++v;
@@ -177,6 +173,6 @@ static void launch_dyn(const KParams &p, int grid, void *stream)
 }
 
 extern const FmtOps ops_dynamic = {-1, -1, launch_dyn<COMPRESS, false>, launch_dyn<DECOMPRESS, false>,
-                                   launch_dyn<UPDATE, false>, launch_dyn<UPDATE, true>, nullptr, nullptr};
+                                   launch_dyn<UPDATE, false>, launch_dyn<UPDATE, true>, nullptr, nullptr, nullptr};
 
 }  // namespace omc

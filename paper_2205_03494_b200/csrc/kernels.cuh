@@ -54,6 +54,13 @@ constexpr uint32_t WAIT_LIMIT = 1u << 24;   // polls of one mbarrier before givi
 #define OMC_OUTBUFS 0
 #endif
 
+#ifndef OMC_RESID_PREFETCH
+#define OMC_RESID_PREFETCH 1
+#endif
+#ifndef OMC_RESID_PER
+#define OMC_RESID_PER 4
+#endif
+
 #ifndef OMC_GRANULE_UNROLL
 #define OMC_GRANULE_UNROLL 0          // 0: per format (measured), else the unroll factor of the granule loop
 #endif
@@ -812,40 +819,69 @@ __device__ __noinline__ Acc tile_ragged(uint32_t *cw, const float *fin, float *f
     return acc;
 }
 
-// One tile of a variable that stays FP32 (Sec. 2.4): copy in / copy out / plain SGD step.
+// `cnt` consecutive tiles of a variable that stays FP32 (Sec. 2.4), from tile `local` on: copy in / copy out / plain SGD
+// step, in chunks of 512 elements with the next chunk's loads issued before the current chunk's
+// arithmetic and stores.  Out of line: the values in flight take 32 to 64 registers per lane, which
+// the kernels of the narrower codes, already at their register limit, can only afford in a frame of
+// its own (inlined and tile by tile, the fused round of the 100M set with a tenth of the matrices
+// in FP32 took 0.19 ms with 12-bit codes).
 template <int MODE, bool WOUT>
-__device__ __forceinline__ void tile_resid(float *__restrict__ r, const float *__restrict__ fin,
-                                           float *__restrict__ fout, uint64_t n_rem, float neg_lr,
-                                           int lane)
+__device__ __noinline__ void resid_tiles(float *__restrict__ r, const float *__restrict__ fin, float *__restrict__ fout,
+                                         uint64_t n, uint32_t local, uint32_t cnt, float neg_lr, int lane)
 {
-    const uint32_t n4 = (uint32_t)(((n_rem < (uint64_t)TILE ? n_rem : (uint64_t)TILE) + 3) / 4);   // float4s
-    float4 a[TILE / 128], g[TILE / 128];
+    constexpr int PER = OMC_RESID_PER;             // 16-byte values per lane and chunk
+    const uint64_t e_begin = (uint64_t)local * TILE;
+    const uint64_t e_end = (uint64_t)(local + cnt) * TILE < n ? (uint64_t)(local + cnt) * TILE : n;
+    const uint32_t n4 = (uint32_t)((e_end - e_begin + 3) / 4);          // at most cnt * 256
+    float4 *const r4 = reinterpret_cast<float4 *>(r + e_begin);
+    const float4 *const g4 = (MODE != DECOMPRESS) ? reinterpret_cast<const float4 *>(fin + e_begin) : nullptr;
+    float4 *const o4 = (MODE == DECOMPRESS || WOUT) ? reinterpret_cast<float4 *>(fout + e_begin) : nullptr;
+    float4 a[PER], g[PER], an[PER], gn[PER];
+    auto load = [&](uint32_t base, float4 (&av)[PER], float4 (&gv)[PER]) {
 #pragma unroll
-    for (int j = 0; j < TILE / 128; ++j) {
-        const uint32_t i = j * 32 + lane;
-        if (i < n4) {
-            if constexpr (MODE != COMPRESS) a[j] = reinterpret_cast<const float4 *>(r)[i];
-            if constexpr (MODE != DECOMPRESS) g[j] = __ldcs(reinterpret_cast<const float4 *>(fin) + i);
-        }
-    }
-#pragma unroll
-    for (int j = 0; j < TILE / 128; ++j) {
-        const uint32_t i = j * 32 + lane;
-        if (i < n4) {
-            if constexpr (MODE == COMPRESS) {
-                reinterpret_cast<float4 *>(r)[i] = g[j];
-            } else if constexpr (MODE == DECOMPRESS) {
-                reinterpret_cast<float4 *>(fout)[i] = a[j];
-            } else {
-                float4 w;
-                w.x = __fmaf_rn(neg_lr, g[j].x, a[j].x);
-                w.y = __fmaf_rn(neg_lr, g[j].y, a[j].y);
-                w.z = __fmaf_rn(neg_lr, g[j].z, a[j].z);
-                w.w = __fmaf_rn(neg_lr, g[j].w, a[j].w);
-                reinterpret_cast<float4 *>(r)[i] = w;
-                if constexpr (WOUT) reinterpret_cast<float4 *>(fout)[i] = w;
+        for (int j = 0; j < PER; ++j) {
+            const uint32_t i = base + j * 32 + lane;
+            if (i < n4) {
+                if constexpr (MODE != COMPRESS) av[j] = r4[i];
+                if constexpr (MODE != DECOMPRESS) gv[j] = __ldcs(g4 + i);
             }
         }
+    };
+#if OMC_RESID_PREFETCH
+    load(0, a, g);
+#endif
+    for (uint32_t base = 0; base < n4; base += PER * 32) {
+#if OMC_RESID_PREFETCH
+        if (base + PER * 32 < n4) load(base + PER * 32, an, gn);
+#else
+        load(base, a, g);
+#endif
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const uint32_t i = base + j * 32 + lane;
+            if (i < n4) {
+                if constexpr (MODE == COMPRESS) {
+                    r4[i] = g[j];
+                } else if constexpr (MODE == DECOMPRESS) {
+                    o4[i] = a[j];
+                } else {
+                    float4 w;
+                    w.x = __fmaf_rn(neg_lr, g[j].x, a[j].x);
+                    w.y = __fmaf_rn(neg_lr, g[j].y, a[j].y);
+                    w.z = __fmaf_rn(neg_lr, g[j].z, a[j].z);
+                    w.w = __fmaf_rn(neg_lr, g[j].w, a[j].w);
+                    r4[i] = w;
+                    if constexpr (WOUT) o4[i] = w;
+                }
+            }
+        }
+#if OMC_RESID_PREFETCH
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            a[j] = an[j];
+            g[j] = gn[j];
+        }
+#endif
     }
 }
 
@@ -965,7 +1001,60 @@ __device__ __forceinline__ VarDev load_var(const VarDev *src)
     return var;
 }
 
-template <class F, int MODE, bool WOUT>
+// The FP32 variables' tiles of a launch form one list, taken in chunks by whichever warp is through
+// with its run of quantised tiles: FP32 tiles cost a warp more or less than tiles of codes
+// depending on how many other warps move FP32 data at the same time, which no fixed division can
+// know, and they need no sums, so any warp can take any of them.  queue[0] hands out chunks,
+// queue[1] counts the warps that are through; the last of them clears both for the next launch.
+constexpr uint32_t FP32_CHUNK_TILES = 4;
+
+template <int MODE, bool WOUT>
+__device__ __noinline__ void fp32_queue(const KParams &p, int lane)
+{
+    // the first three quarters of the list go out in chunks of FP32_CHUNK_TILES tiles, the rest tile
+    // by tile, so that the warps finish within a tile of each other
+    const uint64_t total = __ldg(p.fp32_tile_start + p.n_fp32);
+    const uint64_t big = total * 3 / 4 / FP32_CHUNK_TILES;
+    const uint64_t nchunks = big + (total - big * FP32_CHUNK_TILES);
+    uint32_t next = 0;
+    if (lane == 0) next = atomicAdd(p.queue, 1u);
+    next = __shfl_sync(0xFFFFFFFFu, next, 0);
+    while (next < nchunks) {
+        const uint32_t c = next;
+        if (lane == 0) next = atomicAdd(p.queue, 1u);       // the following chunk, asked for ahead of the work
+        uint64_t t = c < big ? (uint64_t)c * FP32_CHUNK_TILES : big * FP32_CHUNK_TILES + (c - big);
+        const uint64_t tend = c < big ? t + FP32_CHUNK_TILES : t + 1;
+        uint32_t lo = 0, hi = p.n_fp32;                     // the FP32 variable that holds tile t
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (__ldg(p.fp32_tile_start + mid) <= t) lo = mid; else hi = mid;
+        }
+        while (t < tend) {
+            const uint64_t first = __ldg(p.fp32_tile_start + lo), after = __ldg(p.fp32_tile_start + lo + 1);
+            const VarDev var = load_var(p.vars + __ldg(p.fp32_var + lo));
+            const uint32_t local = (uint32_t)(t - first);
+            const uint32_t cnt = (uint32_t)((after < tend ? after : tend) - t);
+            resid_tiles<MODE, WOUT>(p.resid + var.store_off, p.fin + var.full_off, WOUT ? p.fout + var.full_off : nullptr,
+                                    var.n, local, cnt, p.neg_lr, lane);
+            t += cnt;
+            ++lo;
+        }
+        next = __shfl_sync(0xFFFFFFFFu, next, 0);
+    }
+    if (lane == 0) {
+        __threadfence();
+        if (atomicAdd(p.queue + 1, 1u) == p.nwarps - 1) {   // every warp has taken its last chunk number
+            p.queue[0] = 0u;
+            p.queue[1] = 0u;
+        }
+    }
+}
+
+
+// QUEUE (fused round only): the FP32 variables' tiles are taken from the queue (fp32_queue above)
+// instead of the runs; a separate instantiation, because the call costs the kernels of
+// all-quantised models 3 to 8 %.
+template <class F, int MODE, bool WOUT, bool QUEUE = false>
 __global__ void __launch_bounds__(THREADS, MODE == DECOMPRESS ? DECOMPRESS_CTAS_PER_SM : CTAS_PER_SM)
 omc_kernel(const KParams p)
 {
@@ -1030,24 +1119,23 @@ omc_kernel(const KParams p)
                         p.sb[2 * var.sb_slot + 1] = 0.f;
                     }
                 }
-            } else {
-                for (uint32_t i = 0; i < cnt; ++i) {
-                    const uint64_t e0 = (uint64_t)(local + i) * TILE;
-                    tile_resid<MODE, WOUT>(p.resid + var.store_off + e0,
-                                           (MODE != DECOMPRESS) ? p.fin + var.full_off + e0 : nullptr,
-                                           ((MODE == DECOMPRESS) || WOUT) ? p.fout + var.full_off + e0 : nullptr,
-                                           var.n - e0, p.neg_lr, lane);
-                }
-            }
+            } else if (!QUEUE) {
+                resid_tiles<MODE, WOUT>(p.resid + var.store_off, (MODE != DECOMPRESS) ? p.fin + var.full_off : nullptr,
+                                        ((MODE == DECOMPRESS) || WOUT) ? p.fout + var.full_off : nullptr, var.n, local,
+                                        cnt, p.neg_lr, lane);
+            }       // else: FP32 tiles are taken from the queue below
             t += cnt;
             ++v;
         }
+    }
+    if constexpr (QUEUE) {
+        if (!pipe.failed) fp32_queue<MODE, WOUT>(p, lane);
     }
     if (pipe.failed && lane == 0) atomicExch(p.status, 1u);   // a bulk load never arrived
     bulk_wait_all();                                     // stores must finish before the CTA's memory goes
 }
 
-template <class F, int MODE, bool WOUT>
+template <class F, int MODE, bool WOUT, bool QUEUE = false>
 void launch(const KParams &p, int grid, void *stream)
 {
     using SM = Smem<F, MODE, WOUT>;
@@ -1055,10 +1143,10 @@ void launch(const KParams &p, int grid, void *stream)
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        cudaFuncSetAttribute(omc_kernel<F, MODE, WOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL);
+        cudaFuncSetAttribute(omc_kernel<F, MODE, WOUT, QUEUE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL);
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    omc_kernel<F, MODE, WOUT><<<grid, THREADS, SM::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
+    omc_kernel<F, MODE, WOUT, QUEUE><<<grid, THREADS, SM::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1376,6 +1464,7 @@ void launch_aggregate(const AggParams &p, int grid, void *stream)
                                             launch<Fmt<E_, M_>, DECOMPRESS, false>,             \
                                             launch<Fmt<E_, M_>, UPDATE, false>,                 \
                                             launch<Fmt<E_, M_>, UPDATE, true>,                  \
+                                            launch<Fmt<E_, M_>, UPDATE, false, true>,           \
                                             launch_transition<Fmt<E_, M_>>,                     \
                                             launch_aggregate<Fmt<E_, M_>>};
 

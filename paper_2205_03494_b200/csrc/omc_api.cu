@@ -57,7 +57,9 @@ extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
         // omc_transition's tables (filled on the device before each launch)
         const size_t nv = plan->nvars, nw = plan->nwarps;
         const size_t tables = (bytes + 16 + rs_bytes + rv_bytes + dv_bytes + 15) / 16 * 16;
-        const size_t tr_bytes = 16 * nv + 8 * (nw + 1) + sizeof(omc::TransitionVar) * nv + 4 * nw + 16;
+        const size_t nf = plan->fp32_var.size();
+        const size_t tr_bytes = 16 * nv + 8 * (nw + 1) + sizeof(omc::TransitionVar) * nv + 4 * nw + 16 +
+                                8 * (nf + 1) + 4 * nf + 16;
         rc = omc::note_cuda(cudaMalloc(reinterpret_cast<void **>(&plan->d_vars), tables + tr_bytes));
         if (rc) { plan->d_vars = nullptr; return rc; }
         char *const base = reinterpret_cast<char *>(plan->d_vars);
@@ -78,6 +80,13 @@ extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
         plan->d_trans.run_start = plan->d_trans.last + nv;
         plan->d_trans.run_var = reinterpret_cast<uint32_t *>(plan->d_trans.run_start + nw + 1);
         plan->d_trans.nruns = plan->d_trans.run_var + nw;
+        // the FP32 variables' tile list, behind the transition tables (8-byte aligned)
+        char *fl = reinterpret_cast<char *>(plan->d_trans.run_var) + (4 * nw + 4 + 7) / 8 * 8;
+        plan->d_fp32_tile_start = reinterpret_cast<uint64_t *>(fl);
+        plan->d_fp32_var = reinterpret_cast<uint32_t *>(fl + 8 * (nf + 1));
+        rc = omc::note_cuda(cudaMemcpy(plan->d_fp32_tile_start, plan->fp32_tile_start.data(), 8 * (nf + 1), cudaMemcpyHostToDevice));
+        if (!rc && nf) rc = omc::note_cuda(cudaMemcpy(plan->d_fp32_var, plan->fp32_var.data(), 4 * nf, cudaMemcpyHostToDevice));
+        if (rc) { (void)cudaFree(plan->d_vars); plan->d_vars = nullptr; return rc; }
         plan->device = dev;
     }
     return omc::note_cuda(cudaMemsetAsync(workspace, 0, plan->ws_bytes, static_cast<cudaStream_t>(stream)));
@@ -109,9 +118,26 @@ static KParams whole_model(const omc_plan_t *plan, void *workspace)
     p.dyn_e = plan->fmt.exp_bits;
     p.dyn_m = plan->fmt.man_bits;
     p.status = plan->d_status;
+    p.queue = static_cast<uint32_t *>(workspace);       // the workspace header
     p.tickets = reinterpret_cast<uint32_t *>(static_cast<char *>(workspace) + plan->ws_tickets_off);
     p.slots = reinterpret_cast<omc::Partial *>(static_cast<char *>(workspace) + plan->ws_slots_off);
     return p;
+}
+
+// Whether the fused round takes the FP32 variables' tiles from the queue: the format has such a
+// kernel and the FP32 tiles are a real share of the work.  Measured on the 100M set, against FP32
+// tiles inside the runs: 8 to 28 % faster with 8- and 12-bit codes from a tenth of the matrices in
+// FP32 on, 8 % faster with 16-bit codes at a half, 4 % slower with 16-bit codes at a tenth (where
+// the runs already moved 6.3 TB/s).  A few small vectors (a fiftieth of the tiles or less) are
+// cheaper inside the runs than one more round trip to the counter for every warp.
+static bool use_fp32_queue(const omc_plan_t *plan, KParams &p)
+{
+    if (!plan->ops->update_q || plan->fp32_var.empty()) return false;
+    if (plan->fp32_tile_start.back() * 50 < plan->ntiles) return false;
+    p.fp32_tile_start = plan->d_fp32_tile_start;
+    p.fp32_var = plan->d_fp32_var;
+    p.n_fp32 = (uint32_t)plan->fp32_var.size();
+    return true;
 }
 
 static int grid_for(uint32_t nwarps) { return (int)((nwarps + omc::WARPS_PER_CTA - 1) / omc::WARPS_PER_CTA); }
@@ -191,6 +217,8 @@ extern "C" int omc_update_recompress(const omc_plan_t *plan, uint8_t *packed, fl
     p.neg_lr = -lr;
     if (debug_w_out)
         plan->ops->update_w(p, grid_for(p.nwarps), stream);
+    else if (use_fp32_queue(plan, p))
+        plan->ops->update_q(p, grid_for(p.nwarps), stream);
     else
         plan->ops->update(p, grid_for(p.nwarps), stream);
     return omc::note_cuda(cudaGetLastError());

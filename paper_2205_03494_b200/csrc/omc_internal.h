@@ -86,6 +86,14 @@ struct KParams {
     const uint8_t *packed_from;
     const float *resid_from;
     const float *sb_from;
+    // FP32 variables in omc_update_recompress (where they are a real share of the work): their tiles
+    // are not processed with the runs but as one list that the warps take chunks from as they finish
+    // their runs (a counter in the workspace header).  fp32_tile_start: n_fp32 + 1 entries, the tiles before each FP32 variable
+    // among the FP32 variables' tiles; fp32_var: the variables' indices.  NULL: none.
+    const uint64_t *fp32_tile_start;
+    const uint32_t *fp32_var;
+    uint32_t n_fp32;
+    uint32_t *queue;                   // [0] next chunk, [1] warps that are through
     const TransitionVar *trans_vars;   // the launch's own record numbering
     const uint32_t *nruns_dev;         // the launch's run count (replaces nruns)
     uint32_t *status;              // the plan's device status word: set non-zero if a copy never arrived
@@ -130,6 +138,7 @@ struct FmtOps {
     void (*decompress)(const KParams &, int grid, void *stream);
     void (*update)(const KParams &, int grid, void *stream);     // W not stored
     void (*update_w)(const KParams &, int grid, void *stream);   // W stored to fout
+    void (*update_q)(const KParams &, int grid, void *stream);   // FP32 variables' tiles from the queue; NULL if unsupported
     void (*transition)(const KParams &, int grid, void *stream); // plan-to-plan; NULL if unsupported
     void (*aggregate)(const AggParams &, int grid, void *stream); // mean of replicas; NULL if unsupported
 };
@@ -200,11 +209,15 @@ struct omc_plan {
     std::vector<uint64_t> run_start;   // nruns + 1 entries: the cost-balanced division of the tiles
     std::vector<uint32_t> run_var;     // nruns entries: the variable each run starts in
     std::vector<uint32_t> dec_run_var; // dec_nruns entries: the same for the decoder's runs
+    std::vector<uint64_t> fp32_tile_start;   // n_fp32 + 1: tiles before each FP32 variable among the FP32 tiles
+    std::vector<uint32_t> fp32_var;          // n_fp32: their indices
     omc::VarDev *d_vars;               // one allocation: the variable table, the status word, the two run tables
     uint32_t *d_status;
     uint64_t *d_run_start;
     uint32_t *d_run_var;
     uint32_t *d_dec_run_var;
+    uint64_t *d_fp32_tile_start;
+    uint32_t *d_fp32_var;
     omc::TransitionTables d_trans;     // omc_transition's tables (this plan as the destination)
     int device;                        // device the tables live on, -1 before prepare
 };

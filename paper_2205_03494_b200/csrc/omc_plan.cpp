@@ -171,6 +171,8 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         pl->d_run_start = nullptr;
         pl->d_run_var = nullptr;
         pl->d_dec_run_var = nullptr;
+        pl->d_fp32_tile_start = nullptr;
+        pl->d_fp32_var = nullptr;
         pl->d_trans = omc::TransitionTables{};
         pl->device = -1;
         const uint32_t B = 1u + fmt.exp_bits + fmt.man_bits;
@@ -247,6 +249,14 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         const uint32_t slots = omc::divide_tiles(pl->vars.data(), nvars, pl->nruns, pl->run_start.data(),
                                                  pl->run_var.data());
         pl->nslots = slots;
+
+        // ---- the FP32 variables' tiles as one list (taken in chunks by whichever warp is free)
+        pl->fp32_tile_start.assign(1, 0);
+        for (uint32_t i = 0; i < nvars; ++i)
+            if (!pl->vars[i].quantised) {
+                pl->fp32_var.push_back(i);
+                pl->fp32_tile_start.push_back(pl->fp32_tile_start.back() + pl->vars[i].ntiles);
+            }
 
         // ---- the decoder's own division (it keeps no sums): short runs of equal length, dealt out
         // to the warps in turn, so that the warps of a launch sweep through memory side by side
