@@ -54,13 +54,6 @@ constexpr uint32_t WAIT_LIMIT = 1u << 24;   // polls of one mbarrier before givi
 #define OMC_OUTBUFS 0
 #endif
 
-#ifndef OMC_RESID_PREFETCH
-#define OMC_RESID_PREFETCH 1
-#endif
-#ifndef OMC_RESID_PER
-#define OMC_RESID_PER 4
-#endif
-
 #ifndef OMC_GRANULE_UNROLL
 #define OMC_GRANULE_UNROLL 0          // 0: per format (measured), else the unroll factor of the granule loop
 #endif
@@ -820,16 +813,17 @@ __device__ __noinline__ Acc tile_ragged(uint32_t *cw, const float *fin, float *f
 }
 
 // `cnt` consecutive tiles of a variable that stays FP32 (Sec. 2.4), from tile `local` on: copy in / copy out / plain SGD
-// step, in chunks of 512 elements with the next chunk's loads issued before the current chunk's
-// arithmetic and stores.  Out of line: the values in flight take 32 to 64 registers per lane, which
+// step.  Out of line: the values in flight take 32 to 64 registers per lane, which
 // the kernels of the narrower codes, already at their register limit, can only afford in a frame of
 // its own (inlined and tile by tile, the fused round of the 100M set with a tenth of the matrices
 // in FP32 took 0.19 ms with 12-bit codes).
-template <int MODE, bool WOUT>
+// AHEAD: chunks of 512 elements with the next chunk's loads in flight (best for the queue, where
+// a warp does nothing else); otherwise whole tiles one after the other (best inside the runs).
+template <int MODE, bool WOUT, bool AHEAD = false>
 __device__ __noinline__ void resid_tiles(float *__restrict__ r, const float *__restrict__ fin, float *__restrict__ fout,
                                          uint64_t n, uint32_t local, uint32_t cnt, float neg_lr, int lane)
 {
-    constexpr int PER = OMC_RESID_PER;             // 16-byte values per lane and chunk
+    constexpr int PER = AHEAD ? 4 : 8;             // 16-byte values per lane and chunk
     const uint64_t e_begin = (uint64_t)local * TILE;
     const uint64_t e_end = (uint64_t)(local + cnt) * TILE < n ? (uint64_t)(local + cnt) * TILE : n;
     const uint32_t n4 = (uint32_t)((e_end - e_begin + 3) / 4);          // at most cnt * 256
@@ -847,15 +841,13 @@ __device__ __noinline__ void resid_tiles(float *__restrict__ r, const float *__r
             }
         }
     };
-#if OMC_RESID_PREFETCH
-    load(0, a, g);
-#endif
+    if constexpr (AHEAD) load(0, a, g);
     for (uint32_t base = 0; base < n4; base += PER * 32) {
-#if OMC_RESID_PREFETCH
-        if (base + PER * 32 < n4) load(base + PER * 32, an, gn);
-#else
-        load(base, a, g);
-#endif
+        if constexpr (AHEAD) {
+            if (base + PER * 32 < n4) load(base + PER * 32, an, gn);
+        } else {
+            load(base, a, g);
+        }
 #pragma unroll
         for (int j = 0; j < PER; ++j) {
             const uint32_t i = base + j * 32 + lane;
@@ -875,13 +867,13 @@ __device__ __noinline__ void resid_tiles(float *__restrict__ r, const float *__r
                 }
             }
         }
-#if OMC_RESID_PREFETCH
+        if constexpr (AHEAD) {
 #pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            a[j] = an[j];
-            g[j] = gn[j];
+            for (int j = 0; j < PER; ++j) {
+                a[j] = an[j];
+                g[j] = gn[j];
+            }
         }
-#endif
     }
 }
 
@@ -1034,8 +1026,8 @@ __device__ __noinline__ void fp32_queue(const KParams &p, int lane)
             const VarDev var = load_var(p.vars + __ldg(p.fp32_var + lo));
             const uint32_t local = (uint32_t)(t - first);
             const uint32_t cnt = (uint32_t)((after < tend ? after : tend) - t);
-            resid_tiles<MODE, WOUT>(p.resid + var.store_off, p.fin + var.full_off, WOUT ? p.fout + var.full_off : nullptr,
-                                    var.n, local, cnt, p.neg_lr, lane);
+            resid_tiles<MODE, WOUT, true>(p.resid + var.store_off, p.fin + var.full_off,
+                                          WOUT ? p.fout + var.full_off : nullptr, var.n, local, cnt, p.neg_lr, lane);
             t += cnt;
             ++lo;
         }

@@ -128,12 +128,14 @@ static KParams whole_model(const omc_plan_t *plan, void *workspace)
 // kernel and the FP32 tiles are a real share of the work.  Measured on the 100M set, against FP32
 // tiles inside the runs: 8 to 28 % faster with 8- and 12-bit codes from a tenth of the matrices in
 // FP32 on, 8 % faster with 16-bit codes at a half, 4 % slower with 16-bit codes at a tenth (where
-// the runs already moved 6.3 TB/s).  A few small vectors (a fiftieth of the tiles or less) are
-// cheaper inside the runs than one more round trip to the counter for every warp.
+// the runs already move 6.3 TB/s): hence a quarter of the tiles as the threshold for 16 bits and
+// more, a fiftieth below (a few small vectors are cheaper inside the runs than one more round trip
+// to the counter for every warp).
 static bool use_fp32_queue(const omc_plan_t *plan, KParams &p)
 {
     if (!plan->ops->update_q || plan->fp32_var.empty()) return false;
-    if (plan->fp32_tile_start.back() * 50 < plan->ntiles) return false;
+    const uint32_t B = 1u + plan->fmt.exp_bits + plan->fmt.man_bits;
+    if (plan->fp32_tile_start.back() * (B < 16 ? 50 : 4) < plan->ntiles) return false;
     p.fp32_tile_start = plan->d_fp32_tile_start;
     p.fp32_var = plan->d_fp32_var;
     p.n_fp32 = (uint32_t)plan->fp32_var.size();
