@@ -126,16 +126,16 @@ static KParams whole_model(const omc_plan_t *plan, void *workspace)
 
 // Whether the fused round takes the FP32 variables' tiles from the queue: the format has such a
 // kernel and the FP32 tiles are a real share of the work.  Measured on the 100M set, against FP32
-// tiles inside the runs: 8 to 28 % faster with 8- and 12-bit codes from a tenth of the matrices in
-// FP32 on, 8 % faster with 16-bit codes at a half, 4 % slower with 16-bit codes at a tenth (where
-// the runs already move 6.3 TB/s): hence a quarter of the tiles as the threshold for 16 bits and
-// more, a fiftieth below (a few small vectors are cheaper inside the runs than one more round trip
-// to the counter for every warp).
+// tiles inside the runs: 8 to 28 % faster from a tenth of the matrices in FP32 on (S1E4M14 at a
+// tenth: 0.232 -> 0.167 ms), except with S1E5M10, whose kernel already moves 6.3 TB/s at a tenth
+// (the queue is 4 % slower there) and gains 8 % at a half: hence a quarter of the tiles as its
+// threshold and a fiftieth for the other formats (a few small vectors are cheaper inside the runs
+// than one more round trip to the counter for every warp).
 static bool use_fp32_queue(const omc_plan_t *plan, KParams &p)
 {
     if (!plan->ops->update_q || plan->fp32_var.empty()) return false;
-    const uint32_t B = 1u + plan->fmt.exp_bits + plan->fmt.man_bits;
-    if (plan->fp32_tile_start.back() * (B < 16 ? 50 : 4) < plan->ntiles) return false;
+    const bool fp16 = plan->fmt.exp_bits == 5 && plan->fmt.man_bits == 10;
+    if (plan->fp32_tile_start.back() * (fp16 ? 4 : 50) < plan->ntiles) return false;
     p.fp32_tile_start = plan->d_fp32_tile_start;
     p.fp32_var = plan->d_fp32_var;
     p.n_fp32 = (uint32_t)plan->fp32_var.size();
