@@ -27,10 +27,33 @@ METRIC = "params/s, fused decode->update->re-encode"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes per launch of the fused kernel from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by workload name; None until a capture of the current kernel exists.
-# The capture is of the default configuration (format, fraction and plan switches as the workload sets them).
-NCU_TRAFFIC_BYTES = {"conformer_like_17b_d512": 797_592_576}   # profiles/fused_update_conformer_100m_e5m10.md
+KERNEL_SOURCES = ("kernels.cuh", "codec.cuh", "omc_internal.h", "omc_api.cu", "omc_plan.cpp")
+
+
+def kernel_source_hash() -> str:
+    """Hash of the sources the fused kernel and its launch are built from."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2205_03494_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload_key: str):
+    """DRAM bytes per launch of the fused kernel (dram__bytes_read.sum + dram__bytes_write.sum of
+    one ncu capture), from profiles/dram_traffic.txt: lines of `workload-key bytes source-hash`.
+    None when no capture exists for the workload or the kernel's sources changed since it was taken."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    except OSError:
+        return None
+    now = kernel_source_hash()
+    for r in rows:
+        if len(r) >= 3 and r[0] == workload_key and r[2] == now:
+            return int(r[1])
+    return None
 
 
 def make_workload(name):
@@ -197,6 +220,111 @@ def replica_value(nparams: int, world: int, ms_per_step: float) -> float:
     return world * nparams / (ms_per_step * 1e-3)
 
 
+class FusedRun:
+    """One workload resident on the device, ready for rounds of the fused update-recompress."""
+
+    def __init__(self, wl, plan, dev, stream):
+        import numpy as np
+        import torch
+        self.wl, self.plan, self.dev, self.stream = wl, plan, dev, stream
+        z = lambda n, dt: torch.zeros(max(int(n), 16), dtype=dt, device=dev)
+        self.packed, self.resid = z(plan.packed_bytes, torch.uint8), z(plan.resid_elems, torch.float32)
+        self.sb, self.ws = z(2 * plan.n_quantised, torch.float32), z(plan.workspace_bytes, torch.uint8)
+        plan.prepare(self.ws.data_ptr(), stream)
+        params = self.upload(wl.params)
+        plan.compress(params.data_ptr(), self.packed.data_ptr(), self.resid.data_ptr(), self.sb.data_ptr(),
+                      self.ws.data_ptr(), stream)
+        torch.cuda.synchronize()
+        del params
+        self.grads = self.upload(lambda i: wl.grads(i, 0))
+        self.nparams = wl.total
+        self.step_bytes = algorithmic_bytes(plan)
+
+    def upload(self, make):
+        """The seeded variables `make(i)`, generated on the host cores a few at a time and copied to
+        their places in a device array in the plan's full layout (never the whole model on the host)."""
+        import torch
+        from concurrent.futures import ThreadPoolExecutor
+        from paper_2205_03494_b200.workloads import default_threads
+        plan = self.plan
+        out = torch.zeros(plan.full_elems, dtype=torch.float32, device=self.dev)
+        idx = list(range(plan.nvars))
+        group = max(1, default_threads())
+        with ThreadPoolExecutor(max_workers=group) as ex:
+            for g0 in range(0, len(idx), 4 * group):
+                chunk = idx[g0:g0 + 4 * group]
+                for i, x in zip(chunk, ex.map(make, chunk)):
+                    out[plan.full_off[i]:plan.full_off[i] + plan.numel[i]].copy_(torch.from_numpy(x))
+        return out
+
+    def step(self):
+        self.plan.update_recompress(self.packed.data_ptr(), self.resid.data_ptr(), self.sb.data_ptr(),
+                                    self.grads.data_ptr(), self.wl.lr, self.ws.data_ptr(), None, self.stream)
+
+    def timed(self, steps):
+        """Milliseconds for `steps` back-to-back rounds (CUDA events on the launching stream)."""
+        import torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            self.step()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    def roofline(self, ms_per_step, traffic_key=None):
+        peak, peak_kind = measured_peak()
+        achieved = self.step_bytes / (ms_per_step * 1e6)       # GB/s
+        return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+                "peak_source": peak_kind + " copy bandwidth", "kernel": "omc_kernel<UPDATE>",
+                "traffic": ncu_traffic(traffic_key) if traffic_key else None}
+
+    def sustained(self, seconds, local, est_ms):
+        """A run of at least `seconds` of back-to-back rounds with the clocks sampled: long enough for
+        the power cap to act on the SM clock, which the short timed region never sees."""
+        steps = max(10, int(seconds * 1e3 / est_ms) + 1)
+        sampler = ClockSampler(local)
+        sampler.start()
+        time.sleep(0.25)
+        ms = self.timed(steps)
+        clocks = sampler.stop()
+        per = ms / steps
+        out = {"steps": steps, "seconds": ms * 1e-3, "ms_per_step": per, "params_per_s": self.nparams / (per * 1e-3),
+               "roofline": self.roofline(per), "clocks": clocks}
+        if clocks.get("sm_mhz"):
+            out["ms_x_sm_ghz"] = per * clocks["sm_mhz"] * 1e-3       # time x clock: compares runs at different clocks
+        return out
+
+
+def config_label(wl):
+    return "%s S1E%dM%d p=%g" % (wl.name, wl.fmt[0], wl.fmt[1], wl.fraction)
+
+
+def bench_other_config(name, local, dev, stream, seconds):
+    """A sub-record for one of the other target configurations: its own rounds as the configuration
+    states them, the spread, and a sustained run, each with its roofline fraction."""
+    import torch
+    import paper_2205_03494_b200 as omc
+    wl = make_workload(name)
+    plan = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=wl.fraction, seed=wl.sel_seed)
+    run = FusedRun(wl, plan, dev, stream)
+    for _ in range(3):
+        run.step()
+    rounds = max(wl.rounds, 10)
+    chunks = sorted(run.timed(rounds) / rounds for _ in range(5))
+    per = chunks[len(chunks) // 2]
+    rec = {"config": config_label(wl), "params": run.nparams, "variables": plan.nvars,
+           "bytes_per_step": run.step_bytes, "rounds_per_timing": rounds,
+           "ms_per_step": per, "ms_per_step_spread": {"chunks": 5, "best": chunks[0], "median": per, "worst": chunks[-1]},
+           "params_per_s": run.nparams / (per * 1e-3), "roofline": run.roofline(per),
+           "sustained": run.sustained(seconds, local, per), "status": plan.status(stream)}
+    del run
+    torch.cuda.empty_cache()
+    return rec
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -223,42 +351,23 @@ def run_ours(args):
     flags = (0 if args.no_pvt else omc.PLAN_PVT) | (0 if args.all_variables else omc.PLAN_WEIGHTS_ONLY)
     plan = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=wl.fraction, seed=wl.sel_seed, flags=flags)
     stream = torch.cuda.current_stream().cuda_stream
-
-    def full_array(arrays, pinned=False):
-        t = torch.zeros(plan.full_elems, dtype=torch.float32, pin_memory=pinned)
-        a = t.numpy()
-        for i, x in enumerate(arrays):
-            a[plan.full_off[i]:plan.full_off[i] + plan.numel[i]] = x
-        return t
-
+    run = FusedRun(wl, plan, dev, stream)
+    packed, resid, sb, ws, grads = run.packed, run.resid, run.sb, run.ws, run.grads
+    nparams, step_bytes = run.nparams, run.step_bytes
+    step = run.step
     z = lambda n, dt: torch.zeros(max(int(n), 16), dtype=dt, device=dev)
-    packed, resid = z(plan.packed_bytes, torch.uint8), z(plan.resid_elems, torch.float32)
-    sb, ws = z(2 * plan.n_quantised, torch.float32), z(plan.workspace_bytes, torch.uint8)
-    plan.prepare(ws.data_ptr(), stream)
-    params = full_array(wl.all_params()).to(dev)
-    plan.compress(params.data_ptr(), packed.data_ptr(), resid.data_ptr(), sb.data_ptr(), ws.data_ptr(), stream)
-    torch.cuda.synchronize()
-    del params
-    host_grads = full_array(wl.all_grads(0), pinned=True)
-    grads = host_grads.to(dev)
-    nparams = wl.total
-    step_bytes = algorithmic_bytes(plan)
-
-    def step():
-        plan.update_recompress(packed.data_ptr(), resid.data_ptr(), sb.data_ptr(), grads.data_ptr(), wl.lr,
-                               ws.data_ptr(), None, stream)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()          # before the warm-up, so that a short timed region still has samples around it
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
@@ -284,7 +393,12 @@ def run_ours(args):
     spread = {"chunks": 10, "steps_per_chunk": chunk, "best": chunk_ms[0], "median": 0.5 * (chunk_ms[4] + chunk_ms[5]),
               "worst": chunk_ms[-1]}
 
+    # ---- the same step for two seconds and more, clocks sampled (rank 0 reports its own GPU)
+    sustained = run.sustained(args.sustain, local, ms_per_step) if (rank == 0 and args.sustain > 0) else None
+
     # ---- end to end: gradients start in pinned host memory, (s, b) is read back, every step
+    host_grads = torch.empty(plan.full_elems, dtype=torch.float32, pin_memory=True)
+    host_grads.copy_(grads)
     host_sb = torch.zeros(max(2 * plan.n_quantised, 1), dtype=torch.float32, pin_memory=True)
     e2e_steps = max(3, min(args.steps, 10))
 
@@ -301,6 +415,7 @@ def run_ours(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
     e2e_ms = max_over_ranks(e2e_ms, dist, dev)
+    del host_grads
 
     # ---- the two other kernels, for context (not part of the step)
     extra = {}
@@ -443,6 +558,19 @@ def run_ours(args):
                 extra[key] = {"unavailable": str(err)}
         del wsrc, xh, yo
 
+    # ---- the other target configurations as sub-records (default workload, one GPU only)
+    other_configs = []
+    if rank == 0 and world == 1 and args.workload == "conformer" and not args.no_other_configs and \
+            not (args.format or args.fraction or args.no_pvt or args.all_variables):
+        del packed, resid, sb, ws, grads
+        run.packed = run.resid = run.sb = run.ws = run.grads = None
+        torch.cuda.empty_cache()
+        for name in ("large", "ragged"):
+            try:
+                other_configs.append(bench_other_config(name, local, dev, stream, args.sustain or 2.0))
+            except (RuntimeError, MemoryError) as err:      # e.g. a GPU with less free memory than the set needs
+                other_configs.append({"config": name, "unavailable": str(err).splitlines()[0][:200]})
+
     if dist is not None:
         dist.barrier()
     if rank != 0:
@@ -450,7 +578,6 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peak()
     achieved = step_bytes / (ms_per_step * 1e6)       # GB/s
     threads = default_threads()
     cpu = None
@@ -468,7 +595,7 @@ def run_ours(args):
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "ms_per_step_spread": spread,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "%s S1E%dM%d p=%g" % (wl.name, wl.fmt[0], wl.fmt[1], wl.fraction),
+        "config": {"workload": config_label(wl),
                    "params": nparams, "variables": plan.nvars, "quantised_variables": plan.n_quantised,
                    "bytes_per_step": step_bytes, "lr": wl.lr, "pvt": not args.no_pvt, "weights_only": not args.all_variables, "gradients": "one seeded buffer reused every step",
                    "l2": "inputs per step (%.0f MB) exceed the 126 MB L2; no flush" % (step_bytes / 1e6),
@@ -479,10 +606,10 @@ def run_ours(args):
                 "h2d_bytes_per_step": 4 * plan.full_elems, "d2h_bytes_per_step": 8 * plan.n_quantised,
                 "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
         "gpu_launches": args.steps,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_source": peak_kind + " copy bandwidth", "kernel": "omc_kernel<UPDATE>",
-                     "traffic": None if (args.format or args.fraction or args.no_pvt or args.all_variables)
-                     else NCU_TRAFFIC_BYTES.get(wl.name)},
+        "roofline": run.roofline(ms_per_step, None if (args.format or args.fraction or args.no_pvt or args.all_variables)
+                                 else wl.name),
+        "sustained": sustained,
+        "other_configs": other_configs,
         "cpu_baseline": cpu,
         "other_kernels": extra,
     }
@@ -504,6 +631,10 @@ def main():
     ap.add_argument("--all-variables", action="store_true", help="ablation: biases and norms are eligible too")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-extra", action="store_true", help="skip timing the decompress / compress kernels")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the sub-records of the large transformer and the ragged set")
+    ap.add_argument("--sustain", type=float, default=2.0,
+                    help="seconds of back-to-back steps in the sustained sub-record (0 = skip)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

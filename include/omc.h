@@ -227,7 +227,7 @@ int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint
  * FP32 at all).  For variable `var` of the plan, read as an N x K matrix W (K contiguous):
  *     Y = X * Wbar^T,  Wbar = s*Wt + b (Sec. 2.3),  computed as  s * (X * Wt^T) + b * rowsum(X)
  * with X and the codes as FP16 operands of the tensor cores and FP32 accumulation (the paper
- * computes "in full precision or other hardware-supported formats").
+ * leaves the precision of the layer arithmetic open: full precision or a format the hardware supports).
  *   S1E5M10 (the codes are IEEE halves and feed the tensor cores as they are); S1E5M6, S1E5M2,
  *   S1E4M3 and S1E2M3 (every value of these formats is an FP16 value: the codes are expanded to
  *   halves inside the kernel, on the way into the operand tile; Inf and NaN codes included); other
@@ -262,15 +262,26 @@ int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *packed, cons
  *   sb      device, 2 floats (s, b), 8-byte aligned; written.
  *
  * The first call on a device looks up the array's address on that device (with that device
- * current); make that first call outside any stream capture.  All calls share the one array, which
- * keeps the previous call's contents: each call rewrites the table entry and clears the counters it
- * needs on `stream` before its kernel runs, so back-to-back calls on one stream are fine, but two
- * calls whose work overlaps on the same GPU (different streams or host threads) race on the array
- * and give wrong results.  Asynchronous like the other device calls.
+ * current; safe when several host threads make it at once); make that first call outside any
+ * stream capture.  All calls share the one array, which keeps the previous call's contents: each
+ * call queues a small kernel on `stream` that rewrites the table entry and the division and clears
+ * the counters, then the compression kernel (two launches, no copies from host memory), so
+ * back-to-back calls on one stream are fine, but two calls whose work overlaps on the same GPU
+ * (different streams or host threads) race on the array and give wrong results.  Asynchronous like
+ * the other device calls.
  */
 #define OMC_STATIC_MAX_NUMEL (1ull << 28)
 int omc_compress_var_static(const float *values, uint64_t numel, omc_format_t fmt, uint32_t flags,
                             uint8_t *packed, float *sb, void *stream);
+/*
+ * omc_static_status -- the status word of omc_compress_var_static on the current device (it lives
+ * in the same fixed array, so no plan can report it; the paper has no counterpart either).  Waits
+ * for `stream`, then writes to *host_status (host) 0 if the most recent call's kernel ran to
+ * completion, non-zero if it gave up waiting for one of its own copies (its outputs are then
+ * incomplete).  Each call of omc_compress_var_static clears the word, so ask before the next one.
+ * Allocates nothing.
+ */
+int omc_static_status(void *stream, uint32_t *host_status);
 
 #ifdef __cplusplus
 }

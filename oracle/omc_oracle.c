@@ -339,6 +339,23 @@ void orc_sgd_var(float *v, const float *g, uint64_t n, float lr)
     for (uint64_t k = 0; k < n; ++k) v[k] = fmaf(-lr, g[k], v[k]);
 }
 
+/*
+ * Server side (Sec. 1: the clients' trained models are sent back and aggregated; Sec. 2.5: each
+ * client compresses its own subset, so for one parameter some clients deliver decompressed values
+ * and others full-precision ones).  The paper says only "aggregated"; the reading here is the
+ * plain mean in FP32: x[0][e] + x[1][e] + ... in client order, every addition rounded to FP32,
+ * then one correctly rounded division by K ("parity unpinned" by the paper beyond "mean").
+ * x[k] = client k's values of the variable (already decompressed where it held codes).
+ */
+void orc_aggregate_var(const float *const *x, uint32_t K, uint64_t n, float *out)
+{
+    for (uint64_t e = 0; e < n; ++e) {
+        float acc = x[0][e];
+        for (uint32_t k = 1; k < K; ++k) acc = acc + x[k][e];
+        out[e] = acc / (float)K;
+    }
+}
+
 /* ------------------------------------------------------------------------------------------ */
 /* Selection (Sec. 2.4, 2.5, 3.1) and size accounting (Tables 1 and 2).                         */
 

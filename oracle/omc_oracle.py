@@ -64,6 +64,7 @@ def lib():
         L.orc_update_recompress_var.argtypes = [u8p, C.c_uint64, C.c_int, C.c_int, C.c_int, f32p,
                                                 f32p, f32p, C.c_float, f32p]
         L.orc_sgd_var.argtypes = [f32p, f32p, C.c_uint64, C.c_float]
+        L.orc_aggregate_var.argtypes = [C.POINTER(f32p), C.c_uint32, C.c_uint64, f32p]
         L.orc_splitmix64.argtypes = [C.c_uint64, C.c_uint32]
         L.orc_splitmix64.restype = C.c_uint64
         L.orc_select.argtypes = [u8p, C.c_uint32, C.c_double, C.c_uint64, u8p]
@@ -172,6 +173,24 @@ def sgd_var(v, g, lr: float) -> np.ndarray:
     g = _f32(g).ravel()
     lib().orc_sgd_var(_p(v, C.c_float), _p(g, C.c_float), v.size, C.c_float(lr))
     return v
+
+
+def aggregate_var(client_values) -> np.ndarray:
+    """FP32 mean of one variable over the clients (their decompressed or FP32 values), clients
+    added in index order, one division at the end."""
+    xs = [_f32(x).ravel() for x in client_values]
+    n = xs[0].size
+    ptrs = (C.POINTER(C.c_float) * len(xs))(*[_p(x, C.c_float) for x in xs])
+    out = np.empty(n, np.float32)
+    lib().orc_aggregate_var(ptrs, len(xs), n, _p(out, C.c_float))
+    return out
+
+
+def aggregate(states, threads: int = 1) -> list:
+    """Server-side mean of the clients' models: every client's state is decompressed, then each
+    variable is averaged by :func:`aggregate_var`."""
+    dec = [decompress(st, threads) for st in states]
+    return _map(lambda i: aggregate_var([d[i] for d in dec]), range(len(dec[0])), threads)
 
 
 # --------------------------------------------------------------------------------------------

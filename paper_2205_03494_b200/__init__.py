@@ -21,7 +21,7 @@ PLAN_DEFAULT = PLAN_PVT | PLAN_WEIGHTS_ONLY
 EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_sizes",
            "omc_plan_var", "omc_plan_division", "omc_plan_prepare", "omc_plan_status", "omc_compress", "omc_decompress",
            "omc_update_recompress", "omc_update_recompress_host", "omc_transition", "omc_aggregate", "omc_matmul",
-           "omc_compress_var_static"]
+           "omc_compress_var_static", "omc_static_status"]
 STATIC_MAX_NUMEL = 1 << 28
 
 
@@ -74,6 +74,7 @@ def lib():
         L.omc_matmul.argtypes = [vp, C.c_uint32, vp, vp, vp, C.c_uint32, C.c_uint32, C.c_uint32, vp, vp, vp]
         L.omc_aggregate.argtypes = [C.POINTER(vp), C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp, vp]
         L.omc_compress_var_static.argtypes = [vp, C.c_uint64, Format, C.c_uint32, vp, vp, vp]
+        L.omc_static_status.argtypes = [vp, u32p]
         _lib = L
     return _lib
 
@@ -198,3 +199,10 @@ def compress_var_static(values, numel, fmt, packed, sb, flags=PLAN_PVT, stream=0
     S, E, M = (1, fmt[0], fmt[1]) if len(fmt) == 2 else fmt
     _check(lib().omc_compress_var_static(values, int(numel), Format(S, E, M, 0), int(flags), packed, sb,
                                          stream), "omc_compress_var_static")
+
+
+def static_status(stream=0) -> int:
+    """omc_static_status: the status word of the most recent compress_var_static on this device."""
+    st = C.c_uint32(0)
+    _check(lib().omc_static_status(stream, C.byref(st)), "omc_static_status")
+    return st.value

@@ -44,8 +44,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(OBJ, os.path.basename(src) + ".o")
         objs.append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), newest_dep):
-            cmd = [_nvcc(), *NVCC_FLAGS, *os.environ.get("OMC_NVCC_FLAGS", "").split(), "-x", "cu", "-c", src,
-                   "-o", obj]
+            cmd = [_nvcc(), *NVCC_FLAGS, "-x", "cu", "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)

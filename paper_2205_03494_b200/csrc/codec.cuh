@@ -47,13 +47,10 @@ struct HalfPath {
 
 // Formats whose codes, below the top of the range, are those of a hardware narrow-float type
 // (e5m2, e4m3 and the 6-bit e2m3, each held in one byte by the conversion instructions).
-#ifndef OMC_FP8_PATH
-#define OMC_FP8_PATH 1          // 0: build without the narrow-float conversion instructions (tuning runs)
-#endif
 template <class F>
 struct Fp8Path {
     static constexpr bool value =
-        OMC_FP8_PATH && ((F::E == 5 && F::M == 2) || (F::E == 4 && F::M == 3) || (F::E == 2 && F::M == 3));
+        (F::E == 5 && F::M == 2) || (F::E == 4 && F::M == 3) || (F::E == 2 && F::M == 3);
 };
 
 __device__ __forceinline__ uint32_t f2u(float x) { return __float_as_uint(x); }

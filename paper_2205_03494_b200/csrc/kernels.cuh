@@ -28,35 +28,11 @@ namespace omc {
 
 enum Mode { COMPRESS = 0, DECOMPRESS = 1, UPDATE = 2 };
 
-// Input stages per warp (granules fetched ahead = stages - 1), per kind of kernel.  The decoder
-// spends little time on a granule, so it needs more granules in flight to cover the load latency.
-#ifndef OMC_STAGES_COMPRESS
-#define OMC_STAGES_COMPRESS 2
-#endif
-#ifndef OMC_STAGES_DECOMPRESS
-#define OMC_STAGES_DECOMPRESS 2
-#endif
-#ifndef OMC_STAGES_UPDATE
-#define OMC_STAGES_UPDATE 2
-#endif
+// Input stages per warp (granules fetched ahead = stages - 1), per kind of kernel: two for each
+// (three and four were measured: no gain for the decoder, slower for the others, fewer CTAs fit).
 constexpr int MAX_STAGES = 4;               // mbarriers reserved per warp
-constexpr int stages_for(int mode)
-{
-    return mode == 0 ? OMC_STAGES_COMPRESS : mode == 1 ? OMC_STAGES_DECOMPRESS : OMC_STAGES_UPDATE;
-}
+constexpr int stages_for(int /*mode*/) { return 2; }
 constexpr uint32_t WAIT_LIMIT = 1u << 24;   // polls of one mbarrier before giving up
-
-// Build-time overrides for tuning runs: granule size and number of output buffers for all formats.
-#ifndef OMC_SUB
-#define OMC_SUB 0
-#endif
-#ifndef OMC_OUTBUFS
-#define OMC_OUTBUFS 0
-#endif
-
-#ifndef OMC_GRANULE_UNROLL
-#define OMC_GRANULE_UNROLL 0          // 0: per format (measured), else the unroll factor of the granule loop
-#endif
 
 // How many consecutive elements one lane takes per step: the smallest run whose codes fill
 // whole 32-bit words.
@@ -69,9 +45,9 @@ struct Unit {
     // 16-bit codes run best with half-tile granules and two output buffers (measured); the narrower
     // codes, which spend more instructions per byte, with whole tiles and one buffer.
     static constexpr int SUB_DEFAULT = (F::B == 16) ? 512 : TILE;
-    static constexpr int SUB = (OMC_SUB ? OMC_SUB : SUB_DEFAULT) > STEP ? (OMC_SUB ? OMC_SUB : SUB_DEFAULT) : STEP;
+    static constexpr int SUB = SUB_DEFAULT > STEP ? SUB_DEFAULT : STEP;
     static constexpr int SUB_STEPS = SUB / STEP;
-    static constexpr int OUTBUFS = OMC_OUTBUFS ? OMC_OUTBUFS : (SUB < TILE ? 2 : 1);
+    static constexpr int OUTBUFS = SUB < TILE ? 2 : 1;
     static_assert(TILE % SUB == 0 && (OUTBUFS == 1 || OUTBUFS == 2), "");
     static_assert(LU != 32 || SUB == STEP, "row layout: one 32-element row per lane and granule");
 };
@@ -725,7 +701,7 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
         return;
     }
     constexpr int G = (U::SUB_STEPS >= 2 && LU == 4) ? 2 : 1;   // steps whose operands are fetched together
-    constexpr int UNROLL = OMC_GRANULE_UNROLL ? OMC_GRANULE_UNROLL : (F::B == 8 ? 4 : 1);
+    constexpr int UNROLL = F::B == 8 ? 4 : 1;
 #pragma unroll UNROLL
     for (int k0 = 0; k0 < U::SUB_STEPS; k0 += G) {
         uint32_t win[G][NW];

@@ -30,14 +30,9 @@ const FmtOps *find_ops(int E, int M)
 
 using omc::KParams;
 
-// omc_transition's cost model (sixteenths of a tile; overridable at build time for tuning runs):
-// an FP32 tile copied, and the fixed part of a tile converted.
-#ifndef OMC_TCOST_COPY
-#define OMC_TCOST_COPY 16
-#endif
-#ifndef OMC_TCOST_CONVERT
-#define OMC_TCOST_CONVERT 12
-#endif
+// omc_transition's cost model (sixteenths of a tile; swept on B200, flat around these values): an
+// FP32 tile copied, and the fixed part of a tile converted.
+constexpr uint32_t TCOST_COPY = 16, TCOST_CONVERT = 12;
 
 static bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -285,9 +280,9 @@ extern "C" int omc_transition(const omc_plan_t *from, const omc_plan_t *to, cons
     // variable that is fitted costs three tiles more (as in omc_plan).
     const uint32_t B = 1u + to->fmt.exp_bits + to->fmt.man_bits;
     omc::TransitionCosts costs;
-    costs.copy_codes = (B + 1) / 2 * OMC_TCOST_COPY / 16;
-    costs.copy_fp32 = OMC_TCOST_COPY;
-    costs.convert = OMC_TCOST_CONVERT + B / 4;
+    costs.copy_codes = (B + 1) / 2 * TCOST_COPY / 16;
+    costs.copy_fp32 = TCOST_COPY;
+    costs.convert = TCOST_CONVERT + B / 4;
     costs.fit_entry = 48;
     if (costs.copy_codes < 1) costs.copy_codes = 1;
     costs.max_tile = std::max(std::max(costs.copy_codes, costs.copy_fp32), costs.convert);

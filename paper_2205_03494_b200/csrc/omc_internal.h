@@ -8,24 +8,13 @@
 
 namespace omc {
 
-// Launch shape (overridable at build time for tuning runs).
-#ifndef OMC_WARPS_PER_CTA
-#define OMC_WARPS_PER_CTA 8
-#endif
-#ifndef OMC_CTAS_PER_SM
-#define OMC_CTAS_PER_SM 2
-#endif
-
+// Launch shape (measured best on B200 among 4 / 8 / 16 warps and 1 to 4 CTAs per SM).
 constexpr int TILE = 1024;         // elements per tile: the unit of work a warp takes
-constexpr int WARPS_PER_CTA = OMC_WARPS_PER_CTA;
+constexpr int WARPS_PER_CTA = 8;
 constexpr int THREADS = 32 * WARPS_PER_CTA;
-constexpr int CTAS_PER_SM = OMC_CTAS_PER_SM;
-#ifndef OMC_DECOMPRESS_CTAS_PER_SM
-#define OMC_DECOMPRESS_CTAS_PER_SM 2
-#endif
-// The decompress kernel keeps no running sums and needs fewer registers: it may run more CTAs per SM
-// (it divides its tiles at launch, so its grid is independent of the plan's partition).
-constexpr int DECOMPRESS_CTAS_PER_SM = OMC_DECOMPRESS_CTAS_PER_SM;
+constexpr int CTAS_PER_SM = 2;
+// The decompress kernel divides its tiles at launch, so its grid is independent of the plan's division.
+constexpr int DECOMPRESS_CTAS_PER_SM = 2;
 constexpr int DEFAULT_SMS = 148;   // B200; used when no device can be queried at plan time
 
 // One per variable, in the caller's order; lives in device memory after omc_plan_prepare.
@@ -53,6 +42,12 @@ struct Partial {
 static_assert(sizeof(Partial) == 48, "");
 
 constexpr uint64_t WS_HEADER_BYTES = 256;
+
+// Estimated cost of a warp's work in the division of the tiles, in sixteenths of the time of one
+// tile of codes (measured on B200 with the fused round): a tile of codes, a tile of FP32 values,
+// and what entering a quantised variable costs on top (pipeline restart, ragged end, hand-over of
+// the fit's sums).
+constexpr uint64_t COST_TILE = 16, COST_FP32_TILE = 16, COST_VARIABLE = 48;
 
 struct TransitionVar;
 
@@ -153,13 +148,7 @@ uint32_t divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nruns, uint64_t *ru
 uint32_t runs_for(uint64_t tiles, uint32_t nwarps, uint32_t tiles_per_run, uint32_t max_runs);
 // The decoder's runs, in tiles (measured on B200 with 8-, 12- and 16-bit codes: best at about four
 // pipeline granules per run; one-tile runs are slower than none at all).
-#ifndef OMC_DECODE_TILES_PER_RUN
-#define OMC_DECODE_TILES_PER_RUN 0          // 0: by code width; otherwise this many tiles for every format
-#endif
-constexpr uint32_t decode_tiles_per_run(uint32_t code_bits)
-{
-    return OMC_DECODE_TILES_PER_RUN ? OMC_DECODE_TILES_PER_RUN : (code_bits >= 16 ? 4u : 2u);
-}
+constexpr uint32_t decode_tiles_per_run(uint32_t code_bits) { return code_bits >= 16 ? 4u : 2u; }
 constexpr uint32_t DECODE_MAX_RUNS = 1u << 22;
 
 #ifdef __CUDACC__

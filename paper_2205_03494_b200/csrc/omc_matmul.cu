@@ -27,9 +27,7 @@ namespace omc {
 int note_cuda(cudaError_t e);
 }
 
-#ifndef OMC_MATMUL_DECODER_THREADS
-#define OMC_MATMUL_DECODER_THREADS 512      // sixteen decoder warps (measured against eight)
-#endif
+constexpr int MATMUL_DECODER_THREADS = 512;      // sixteen decoder warps (measured against eight)
 
 namespace {
 
@@ -52,7 +50,7 @@ struct Cfg {
     static constexpr int STAGE = TILE_A_BYTES + TILE_B_BYTES + RAW_BYTES;
     static constexpr int NSTAGES = DECODE ? 3 : 4;
     static constexpr int SMEM = NSTAGES * STAGE + 1024 /* alignment slack */ + 256 /* barriers, tmem slot */;
-    static constexpr int DEC_THREADS = DECODE ? OMC_MATMUL_DECODER_THREADS : 0;
+    static constexpr int DEC_THREADS = DECODE ? MATMUL_DECODER_THREADS : 0;
     static constexpr int THREADS = 192 + DEC_THREADS;
     static constexpr uint32_t TX_BYTES = TILE_A_BYTES + (DECODE ? RAW_BYTES : TILE_B_BYTES);
     static_assert(STAGE % 1024 == 0, "operand tiles stay 1024-byte aligned");
@@ -434,6 +432,12 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
 {
     if (!plan) return OMC_ERR_NULL_PTR;
     if (!plan->d_vars) return OMC_ERR_PLAN_MISMATCH;
+    {   // the plan's tables and status word live on the device it was prepared on
+        int dev = 0;
+        const int rc = omc::note_cuda(cudaGetDevice(&dev));
+        if (rc) return rc;
+        if (dev != plan->device) return OMC_ERR_PLAN_MISMATCH;
+    }
     if (!packed || !sb || !x_half || !y || !rowsum_scratch) return OMC_ERR_NULL_PTR;
     if (var >= plan->nvars || !plan->vars[var].quantised) return OMC_ERR_INVALID_ARG;
     const int exp = plan->fmt.exp_bits, man = plan->fmt.man_bits;
@@ -442,8 +446,10 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     if (!half_family && !narrow) return OMC_ERR_BAD_FORMAT;
     if (M == 0 || N == 0 || K == 0 || N % 128 != 0 || K % BK != 0 || (uint64_t)N * K != plan->vars[var].n)
         return OMC_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(packed) | reinterpret_cast<uintptr_t>(x_half) | reinterpret_cast<uintptr_t>(y)) & 15u)
+    if ((reinterpret_cast<uintptr_t>(packed) | reinterpret_cast<uintptr_t>(x_half) | reinterpret_cast<uintptr_t>(y) |
+         reinterpret_cast<uintptr_t>(sb)) & 15u)
         return OMC_ERR_MISALIGNED;
+    if (reinterpret_cast<uintptr_t>(rowsum_scratch) & 3u) return OMC_ERR_MISALIGNED;
     const omc::VarDev &v = plan->vars[var];
     CUtensorMap map_x;
     if (!make_map(&map_x, x_half, M, K, BM)) return OMC_ERR_CUDA;

@@ -52,18 +52,6 @@ static uint64_t splitmix64(uint64_t &state)
 
 static uint64_t round_up(uint64_t x, uint64_t m) { return (x + m - 1) / m * m; }
 
-// Estimated cost of a warp's work, in sixteenths of the time of one tile of codes (measured on
-// B200 with the fused round; overridable at build time for tuning runs).
-#ifndef OMC_COST_TILE
-#define OMC_COST_TILE 16
-#endif
-#ifndef OMC_COST_FP32_TILE
-#define OMC_COST_FP32_TILE 16
-#endif
-#ifndef OMC_COST_VARIABLE
-#define OMC_COST_VARIABLE 48
-#endif
-
 static uint32_t query_sm_count()
 {
     int dev = 0, sms = 0;
@@ -84,8 +72,8 @@ uint32_t omc::divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nruns, uint64_
 {
     const uint64_t NR = nruns;
     auto var_cost = [](const VarDev &v) {
-        return v.quantised ? (uint64_t)OMC_COST_TILE * v.ntiles + OMC_COST_VARIABLE
-                           : (uint64_t)OMC_COST_FP32_TILE * v.ntiles;
+        return v.quantised ? omc::COST_TILE * v.ntiles + omc::COST_VARIABLE
+                           : omc::COST_FP32_TILE * v.ntiles;
     };
     uint64_t total_cost = 0, tiles = 0;
     for (uint32_t i = 0; i < nvars; ++i) {
@@ -100,8 +88,8 @@ uint32_t omc::divide_tiles(VarDev *vars, uint32_t nvars, uint32_t nruns, uint64_
     uint64_t before = 0;
     for (uint32_t i = 0; i < nvars; ++i) {
         VarDev &v = vars[i];
-        const uint64_t per_tile = v.quantised ? OMC_COST_TILE : OMC_COST_FP32_TILE;
-        const uint64_t c = before + (v.quantised ? OMC_COST_VARIABLE : 0);     // cost before tile 0 of v
+        const uint64_t per_tile = v.quantised ? omc::COST_TILE : omc::COST_FP32_TILE;
+        const uint64_t c = before + (v.quantised ? omc::COST_VARIABLE : 0);     // cost before tile 0 of v
         v.first_run = run_of(c);
         // the tiles of v at which the run changes, solved for instead of walking every tile
         uint64_t k = 0;

@@ -6,6 +6,8 @@
 // the library's own device image.
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "omc_internal.h"
 
 namespace omc {
@@ -28,29 +30,83 @@ constexpr size_t SCRATCH_BYTES = OFF_RUN_VAR + sizeof(uint32_t) * MAX_SLOTS;   /
 static __device__ __align__(256) unsigned char g_static_scratch[SCRATCH_BYTES];
 
 constexpr int MAX_DEVICES = 64;
-unsigned char *g_scratch_addr[MAX_DEVICES] = {};         // device address of the array, per device
-int g_sm_count[MAX_DEVICES] = {};
+struct DeviceScratch {
+    std::once_flag once;
+    int rc = OMC_OK;
+    unsigned char *addr = nullptr;      // device address of the array on this device
+    int sms = 0;
+};
+DeviceScratch g_dev[MAX_DEVICES];
 
-// First use on the current device: look up where the array lives there.
+// First use on the current device: look up where the array lives there (once per device, also
+// when several host threads make their first call at the same time).
 int scratch_for_current_device(unsigned char **out, int *sms)
 {
     int dev = 0;
     int rc = omc::note_cuda(cudaGetDevice(&dev));
     if (rc) return rc;
     if (dev < 0 || dev >= MAX_DEVICES) return OMC_ERR_INVALID_ARG;
-    if (!g_scratch_addr[dev]) {
+    DeviceScratch &d = g_dev[dev];
+    std::call_once(d.once, [&d, dev]() {
         void *p = nullptr;
-        rc = omc::note_cuda(cudaGetSymbolAddress(&p, g_static_scratch));
-        if (rc) return rc;
+        d.rc = omc::note_cuda(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (d.rc) return;
         int n = 0;
-        rc = omc::note_cuda(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
-        if (rc) return rc;
-        g_sm_count[dev] = n;
-        g_scratch_addr[dev] = static_cast<unsigned char *>(p);
-    }
-    *out = g_scratch_addr[dev];
-    *sms = g_sm_count[dev];
+        d.rc = omc::note_cuda(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+        if (d.rc) return;
+        d.sms = n;
+        d.addr = static_cast<unsigned char *>(p);
+    });
+    if (d.rc) return d.rc;
+    *out = d.addr;
+    *sms = d.sms;
     return OMC_OK;
+}
+
+// What the call needs in the array before the compression kernel starts, written on the device
+// (the host hands over nothing that lives in its own memory, only kernel arguments): the
+// one-entry variable table, the cleared ticket and status word, and the division of the tiles into
+// runs -- the rule of omc_plan's division for a single quantised variable, solved per run: a tile
+// costs T, entering the variable V, and tile k belongs to run floor((V + T k) * nruns / total),
+// so run r starts at the first tile k with V + T k >= ceil(r * total / nruns).
+// numel <= 2^28 and nruns <= 4096 keep every product below 2^36.
+__global__ void static_setup_kernel(unsigned char *scratch, uint64_t numel, uint64_t packed_bytes, uint32_t ntiles,
+                                    uint32_t nruns)
+{
+    constexpr uint64_t TILE_COST = omc::COST_TILE, VAR_COST = omc::COST_VARIABLE;
+    const uint64_t total = TILE_COST * ntiles + VAR_COST;
+    auto run_of = [&](uint64_t cost) { return (uint32_t)(cost * nruns / total); };
+    uint64_t *run_start = reinterpret_cast<uint64_t *>(scratch + OFF_RUN_START);
+    uint32_t *run_var = reinterpret_cast<uint32_t *>(scratch + OFF_RUN_VAR);
+    for (uint32_t r = blockIdx.x * blockDim.x + threadIdx.x; r <= nruns; r += gridDim.x * blockDim.x) {
+        uint64_t k;
+        if (r == nruns) {
+            k = ntiles;
+        } else {
+            const uint64_t need = ((uint64_t)r * total + nruns - 1) / nruns;
+            k = need <= VAR_COST ? 0 : (need - VAR_COST + TILE_COST - 1) / TILE_COST;
+            if (k > ntiles) k = ntiles;
+            run_var[r] = 0u;
+        }
+        run_start[r] = k;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        omc::VarDev v;
+        v.n = numel;
+        v.full_off = 0;
+        v.store_off = 0;
+        v.packed_bytes = packed_bytes;
+        v.tile_start = 0;
+        v.ntiles = ntiles;
+        v.quantised = 1;
+        v.sb_slot = 0;
+        v.slot_base = 0;
+        v.first_run = run_of(VAR_COST);
+        v.nslots = run_of(VAR_COST + TILE_COST * (ntiles - 1)) - v.first_run + 1;
+        *reinterpret_cast<omc::VarDev *>(scratch + OFF_VAR) = v;
+        *reinterpret_cast<uint32_t *>(scratch + OFF_TICKET) = 0u;
+        *reinterpret_cast<uint32_t *>(scratch + OFF_STATUS) = 0u;
+    }
 }
 
 }  // namespace
@@ -81,34 +137,15 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     const uint32_t nwarps = (uint32_t)(tiles < max_warps ? tiles : max_warps);
     if (nwarps > MAX_SLOTS) return OMC_ERR_TOO_LARGE;
     const uint32_t nruns = nwarps;          // one run per warp, as in omc_compress
+    const uint64_t packed_bytes = ((numel * B + 7) / 8 + 15) / 16 * 16;
 
-    omc::VarDev v{};
-    v.n = numel;
-    v.full_off = 0;
-    v.store_off = 0;
-    v.packed_bytes = ((numel * B + 7) / 8 + 15) / 16 * 16;
-    v.tile_start = 0;
-    v.ntiles = (uint32_t)tiles;
-    v.quantised = 1;
-    v.sb_slot = 0;
-    v.slot_base = 0;
-    uint64_t run_start[MAX_SLOTS + 1];         // host copy; the same division omc_plan makes
-    uint32_t run_var[MAX_SLOTS];               // all zero: there is one variable
-    omc::divide_tiles(&v, 1, nruns, run_start, run_var);
-
+    // The array keeps what the last call left.  A small kernel on `stream` rewrites the table entry
+    // and the division and clears the ticket and the status word; the records are all rewritten by
+    // the compression kernel before they are read.  Nothing is copied from host memory, so the call
+    // leaves no pointer to the caller's stack or heap behind on the stream.
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // The array keeps what the last call left: the table entry and the division are rewritten, the
-    // ticket and the status word are cleared; the records are all rewritten by the kernel before
-    // they are read.  Both host buffers are pageable, so each copy has left them when it returns.
-    rc = omc::note_cuda(cudaMemcpyAsync(scratch + OFF_VAR, &v, sizeof v, cudaMemcpyHostToDevice, st));
-    if (rc) return rc;
-    rc = omc::note_cuda(cudaMemcpyAsync(scratch + OFF_RUN_START, run_start, sizeof(uint64_t) * (nruns + 1),
-                                        cudaMemcpyHostToDevice, st));
-    if (rc) return rc;
-    rc = omc::note_cuda(cudaMemcpyAsync(scratch + OFF_RUN_VAR, run_var, sizeof(uint32_t) * nruns,
-                                        cudaMemcpyHostToDevice, st));
-    if (rc) return rc;
-    rc = omc::note_cuda(cudaMemsetAsync(scratch + OFF_TICKET, 0, 8, st));
+    static_setup_kernel<<<(nruns + 1 + 255) / 256, 256, 0, st>>>(scratch, numel, packed_bytes, (uint32_t)tiles, nruns);
+    rc = omc::note_cuda(cudaGetLastError());
     if (rc) return rc;
 
     omc::KParams p{};
@@ -133,4 +170,17 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     p.slots = reinterpret_cast<omc::Partial *>(scratch + OFF_SLOTS);
     ops->compress(p, (int)((nwarps + omc::WARPS_PER_CTA - 1) / omc::WARPS_PER_CTA), stream);
     return omc::note_cuda(cudaGetLastError());
+}
+
+extern "C" int omc_static_status(void *stream, uint32_t *host_status)
+{
+    if (!host_status) return OMC_ERR_NULL_PTR;
+    unsigned char *scratch = nullptr;
+    int sms = 0;
+    int rc = scratch_for_current_device(&scratch, &sms);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = omc::note_cuda(cudaMemcpyAsync(host_status, scratch + OFF_STATUS, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    if (rc) return rc;
+    return omc::note_cuda(cudaStreamSynchronize(st));
 }

@@ -21,18 +21,56 @@ def from_full(plan, full: np.ndarray, i: int) -> np.ndarray:
     return full[plan.full_off[i]:plan.full_off[i] + plan.numel[i]]
 
 
+GUARD_BYTES = 1024
+GUARD_BYTE = 0xA5
+
+
+class Guarded:
+    """A device buffer followed by canary bytes: no race detector or sanitizer is available for the
+    GPU runs, so every buffer a kernel writes is followed by a known pattern that the tests check
+    after the calls (a store past the end of an arena shows up here)."""
+
+    def __init__(self, n: int, dtype, dev, fill=None):
+        self.n = max(int(n), 16)
+        item = torch.empty(0, dtype=dtype).element_size()
+        nbytes = (self.n * item + 15) // 16 * 16
+        self.raw = torch.empty(nbytes + GUARD_BYTES, dtype=torch.uint8, device=dev)
+        self.raw[nbytes:] = GUARD_BYTE
+        self.t = self.raw[:self.n * item].view(dtype)
+        if fill is None:
+            self.t.zero_()
+            self.raw[self.n * item:nbytes] = 0
+        else:
+            self.t.fill_(fill)
+            self.raw[self.n * item:nbytes] = GUARD_BYTE
+        self._tail = self.n * item if fill is not None else nbytes
+
+    def intact(self) -> bool:
+        return bool((self.raw[self._tail:] == GUARD_BYTE).all())
+
+
 class DeviceModel:
     """Device buffers of one compressed model plus helpers to move variables in and out."""
 
     def __init__(self, plan: omc.Plan, device="cuda:0"):
         self.plan = plan
         self.dev = torch.device(device)
-        z = lambda n, dt: torch.zeros(max(int(n), 16), dtype=dt, device=self.dev)
-        self.packed = z(plan.packed_bytes, torch.uint8)
-        self.resid = z(plan.resid_elems, torch.float32)
-        self.sb = z(2 * plan.n_quantised, torch.float32)
-        self.ws = z(plan.workspace_bytes, torch.uint8)
+        self.guards = {}
+
+        def z(name, n, dt):
+            g = Guarded(n, dt, self.dev)
+            self.guards[name] = g
+            return g.t
+        self.packed = z("packed", plan.packed_bytes, torch.uint8)
+        self.resid = z("resid", plan.resid_elems, torch.float32)
+        self.sb = z("sb", 2 * plan.n_quantised, torch.float32)
+        self.ws = z("workspace", plan.workspace_bytes, torch.uint8)
         plan.prepare(self.ws.data_ptr(), torch.cuda.current_stream().cuda_stream)
+
+    def check_guards(self):
+        """The canary bytes behind every arena are untouched."""
+        for name, g in self.guards.items():
+            assert g.intact(), "a kernel wrote past the end of the %s arena" % name
 
     def _s(self):
         return torch.cuda.current_stream().cuda_stream
@@ -40,13 +78,19 @@ class DeviceModel:
     def upload_full(self, arrays) -> torch.Tensor:
         return torch.from_numpy(to_full(self.plan, arrays)).to(self.dev)
 
+    def full_buffer(self, name: str) -> torch.Tensor:
+        """A zeroed FP32 buffer in the full layout with canary bytes behind it (for outputs)."""
+        g = Guarded(self.plan.full_elems, torch.float32, self.dev)
+        self.guards[name] = g
+        return g.t[:self.plan.full_elems]
+
     def compress(self, params_full: torch.Tensor):
         self.plan.compress(params_full.data_ptr(), self.packed.data_ptr(), self.resid.data_ptr(),
                            self.sb.data_ptr(), self.ws.data_ptr(), self._s())
 
     def decompress(self, first_var=0, n_vars=None, out=None) -> torch.Tensor:
         if out is None:
-            out = torch.zeros(self.plan.full_elems, dtype=torch.float32, device=self.dev)
+            out = self.full_buffer("decompress output")
         self.plan.decompress(self.packed.data_ptr(), self.resid.data_ptr(), self.sb.data_ptr(),
                              out.data_ptr(), first_var, n_vars, self._s())
         return out
@@ -60,6 +104,7 @@ class DeviceModel:
     def host_state(self):
         torch.cuda.synchronize()
         assert self.plan.status(self._s()) == 0, "a kernel gave up waiting for one of its copies"
+        self.check_guards()
         return (self.packed.cpu().numpy(), self.resid.cpu().numpy(), self.sb.cpu().numpy())
 
     def var_packed(self, packed_host, i):

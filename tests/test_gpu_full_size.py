@@ -1,8 +1,8 @@
 """Parity at the benchmark configurations' full sizes, in the launch configuration bench.py times
-(whole-model plans, one kernel launch per call).  The GPU processes every variable; the oracle
-recomputes a sample of variables (largest, smallest, first, last, FP32-only ones) completely, so
-every code, (s, b) and W of those variables is compared; the rest is covered by the status word and
-by the zero-padding and determinism checks."""
+(whole-model plans, one kernel launch per call).  On the 100M and the ragged set every variable is
+compared with the oracle; on the 1.6-billion-parameter set the oracle recomputes a sample of
+variables completely (every code, (s, b) and W of those), the rest is covered by the status word
+and the zero-padding check."""
 import numpy as np
 import pytest
 import torch
@@ -14,43 +14,49 @@ from test_gpu_parity import Lockstep
 pytestmark = pytest.mark.gpu
 
 
-def pick(wl, extra=()):
-    n = np.array(wl.numel)
-    q = [i for i, k in enumerate(wl.kinds) if k == 0]
-    o = [i for i, k in enumerate(wl.kinds) if k != 0]
-    s = {q[0], q[-1], q[int(np.argmax(n[q]))], q[int(np.argmin(n[q]))], *extra}
-    if o:
-        s |= {o[0], o[-1]}
-    return sorted(s)
-
-
 def test_conformer_like_100m_three_rounds():
+    """The bench workload, every variable compared in every round; the last round is the launch
+    bench.py times (W not stored) with a step large enough to move most codes."""
     wl = workloads.conformer_like()
-    sample = pick(wl, extra=(2, 20, 300, 301))
     params = wl.all_params()
-    ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params, sample=sample, threads=8)
+    ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params, threads=8)
     del params
     ls.check_decompress()
     for r in range(3):
-        packed = ls.round(wl.all_grads(r), wl.lr if r < 2 else 30.0)
+        packed = ls.round(wl.all_grads(r), wl.lr if r < 2 else 30.0, want_w=(r < 2))
+    ls.check_padding(packed)
+    ls.check_decompress()
+    assert ls.sb_ulp_cases <= 1, ls.sb_ulp_cases
+
+
+@pytest.mark.parametrize("fmt,fraction", [((5, 6), 1.0), ((3, 7), 0.9), ((4, 14), 0.9), ((5, 2), 0.5)],
+                         ids=lambda v: str(v).replace(" ", ""))
+def test_conformer_like_100m_other_formats(fmt, fraction):
+    """The 100M set in the formats of Tables 1-2 and with a share of the matrices left in FP32 (the
+    launch that takes FP32 tiles from the queue), every variable compared, W not stored."""
+    wl = workloads.conformer_like()
+    params = wl.all_params()
+    ls = Lockstep(wl.numel, wl.kinds, fmt, params, fraction=fraction, seed=5, threads=8)
+    del params
+    for r in range(2):
+        packed = ls.round(wl.all_grads(r), 30.0, want_w=False)
     ls.check_padding(packed)
     ls.check_decompress()
     assert ls.sb_ulp_cases <= 1, ls.sb_ulp_cases
 
 
 def test_ragged_4096_variables_two_rounds():
+    """The ragged set, every one of its 4096 variables compared; the second round is the launch a
+    training loop makes (W not stored) with a large step."""
     wl = workloads.ragged()
-    n = np.array(wl.numel)
-    order = np.argsort(n)
-    sample = sorted({int(i) for i in list(order[:6]) + list(order[-3:]) + list(order[::400])} | {0, 4095})
     params = wl.all_params()
-    ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params, sample=sample, threads=8)
+    ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params, threads=8)
     del params
     ls.check_decompress()
     for r in range(2):
-        packed = ls.round(wl.all_grads(r), 0.01 if r == 0 else 20.0, want_w=(r == 1))
+        packed = ls.round(wl.all_grads(r), 0.01 if r == 0 else 20.0, want_w=(r == 0))
     ls.check_padding(packed)
-    assert ls.sb_ulp_cases <= 2, ls.sb_ulp_cases
+    assert ls.sb_ulp_cases <= 4, ls.sb_ulp_cases
 
 
 def test_large_transformer_1p6b_one_round():
@@ -59,7 +65,7 @@ def test_large_transformer_1p6b_one_round():
     if free < 24e9:
         pytest.skip("needs about 24 GB of free device memory")
     wl = workloads.large_transformer()
-    sample = [0, 4, 95, 191]          # two attention matrices, a 2048x8192 and the last 8192x2048
+    sample = list(range(0, 6)) + [95, 100] + list(range(186, 192))     # the first and the last layer whole, two in the middle
     params = wl.all_params()
     ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params, sample=sample, threads=4)
     del params
@@ -94,6 +100,34 @@ def test_conformer_like_100m_transition_between_90pct_subsets(fmt):
     ls.check_padding(packed)
     ls.round(wl.all_grads(0), 5.0, want_w=False)
     assert ls.sb_ulp_cases <= 1, ls.sb_ulp_cases
+
+
+@pytest.mark.parametrize("fmt,K", [((5, 10), 3), ((5, 6), 4), ((3, 7), 3)], ids=lambda v: str(v).replace(" ", ""))
+def test_conformer_like_100m_aggregate(fmt, K):
+    """omc_aggregate at the size bench.py times it: K clients of the 100M set, each with its own
+    random 90 % of the matrices, every element of the mean against the oracle.  The launch has
+    about a hundred tiles per warp here, so every warp walks over many tiles and across variable
+    boundaries."""
+    from oracle import omc_oracle as orc
+    from harness import from_full, same_f32
+    wl = workloads.conformer_like()
+    base = wl.all_params()
+    clients = []
+    for k in range(K):
+        rng = np.random.default_rng(500 + k)
+        params = [p + np.float32(0.003 * (k + 1)) * rng.standard_normal(p.size, dtype=np.float32) for p in base]
+        clients.append(Lockstep(wl.numel, wl.kinds, fmt, params, fraction=0.9, seed=40 + k, threads=8))
+        del params
+    assert len({tuple(c.plan.quantised) for c in clients}) == K
+    out = torch.full((clients[0].plan.full_elems,), float("nan"), dtype=torch.float32, device="cuda")
+    omc.aggregate([c.plan for c in clients], [c.dm.packed.data_ptr() for c in clients],
+                  [c.dm.resid.data_ptr() for c in clients], [c.dm.sb.data_ptr() for c in clients],
+                  out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    want = orc.aggregate([c.st for c in clients], threads=8)
+    for i in range(len(wl.numel)):
+        assert same_f32(from_full(clients[0].plan, got, i), want[i]), i
 
 
 @pytest.mark.parametrize("fmt", [(5, 2), (3, 7), (5, 10)], ids=lambda f: "E%dM%d" % f)

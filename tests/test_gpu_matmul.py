@@ -1,23 +1,29 @@
 """omc_matmul: the forward-path product computed straight from the codes (tensor cores) against
 the definition: decompress the variable with the oracle, then Y = X Wbar^T in fp64 (numpy matmul).
 Tolerance: X and the codes are exact FP16 inputs and their products are exact in FP32, so the only
-errors are the FP32 accumulation over K (<= K 2^-23 of sum |x||w|) and the epilogue's two roundings;
-the test allows 1e-3 of sum_k |x||w| (+ the same for the b*rowsum term), four orders of magnitude
-below what a wrong tile, swizzle or index would produce."""
+errors are the FP32 accumulation over K in the tensor cores (at most one unit in the last place per
+addition, i.e. K 2^-23 of sum |x||w|, if the accumulator truncates), the same for rowsum(X), the
+rounding of Wbar = s*Wt + b in the definition and the epilogue's two roundings: the bound is
+(4 K + 8) 2^-24 (|s| sum_k |x||wt| + |b| sum_k |x|), a factor two above that worst case."""
 import numpy as np
 import pytest
 import torch
 
 import paper_2205_03494_b200 as omc
 from oracle import omc_oracle as orc
-from harness import DeviceModel
+from harness import DeviceModel, Guarded
 
 pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("fmt", [(5, 10), (5, 6), (5, 2), (4, 3), (2, 3)], ids=lambda f: "E%dM%d" % f)
-@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 256, 192), (1000, 384, 512), (64, 128, 1024)])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 256, 192), (1000, 384, 512), (64, 128, 1024),
+                                   (4000, 4224, 192)])
 def test_matmul_from_codes_matches_definition(M, N, K, fmt):
+    """The last shape has 32 x 17 = 544 tiles of 128 x 256 (M and N not multiples of the tile), so
+    every persistent CTA walks over three or four tiles: both accumulators in tensor memory are
+    reused, the producer runs ahead across tile boundaries, and the epilogue of one tile overlaps
+    the products of the next."""
     rng = np.random.default_rng(M + N + K)
     numel = [777, N * K, 64, 128 * 64]
     kinds = [0, 0, 1, 0]
@@ -30,16 +36,22 @@ def test_matmul_from_codes_matches_definition(M, N, K, fmt):
     st = orc.compress(params, plan.quantised, *fmt)
     x = (rng.standard_normal((M, K)) * 0.5).astype(np.float16)
     xd = torch.from_numpy(x).cuda()
-    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    yg = Guarded(M * N, torch.float32, "cuda", fill=float("nan"))
+    y = yg.t[:M * N].view(M, N)
     scratch = torch.zeros(M, dtype=torch.float32, device="cuda")
     omc.matmul(plan, 1, dm.packed.data_ptr(), dm.sb.data_ptr(), xd.data_ptr(), M, N, K, y.data_ptr(),
                scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
     assert plan.status() == 0
-    wbar = orc.decompress_var(st["packed"][1], N * K, fmt[0], fmt[1], st["s"][1], st["b"][1]).reshape(N, K).astype(np.float64)
+    assert yg.intact()
+    E_, M_ = fmt
+    s_, b_ = float(st["s"][1]), float(st["b"][1])
+    wbar = orc.decompress_var(st["packed"][1], N * K, E_, M_, st["s"][1], st["b"][1]).reshape(N, K).astype(np.float64)
+    wt = orc.decode(orc.unpack(st["packed"][1], N * K, 1 + E_ + M_), E_, M_).reshape(N, K).astype(np.float64)
     x64 = x.astype(np.float64)
     want = x64 @ wbar.T
-    bound = 1e-3 * (np.abs(x64) @ np.abs(wbar).T + abs(float(st["b"][1])) * np.abs(x64).sum(1, keepdims=True)) + 1e-7
+    bound = (4 * K + 8) * 2.0 ** -24 * (abs(s_) * (np.abs(x64) @ np.abs(wt).T)
+                                        + abs(b_) * np.abs(x64).sum(1, keepdims=True)) + 1e-30
     got = y.cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()
     assert np.all(np.abs(got - want) <= bound), float(np.max(np.abs(got - want) / bound))

@@ -97,6 +97,7 @@ class Lockstep:
     def check_decompress(self, first=0, count=None):
         out = self.dm.decompress(first, count)
         torch.cuda.synchronize()
+        self.dm.check_guards()
         out = out.cpu().numpy()
         want = orc.decompress(self.st, self.threads)
         hi = self.plan.nvars if count is None else first + count
@@ -108,7 +109,7 @@ class Lockstep:
     def round(self, grads, lr, want_w=True):
         """grads: list over all variables (GPU) -- the oracle takes the sampled ones."""
         gfull = self.dm.upload_full(grads)
-        w_out = torch.zeros(self.plan.full_elems, dtype=torch.float32, device=self.dm.dev) if want_w else None
+        w_out = self.dm.full_buffer("W output") if want_w else None
         self.dm.update(gfull, lr, w_out)
         ws = orc.update_recompress(self.st, [grads[i] for i in self.idx], lr, self.threads, want_w=True)
         packed = self.check_state("update")
@@ -121,16 +122,22 @@ class Lockstep:
 
 # ---------------------------------------------------------------------------------------------
 
+WANT_W = pytest.mark.parametrize("want_w", [True, False], ids=["w_out", "production"])
+
+
+@WANT_W
 @pytest.mark.parametrize("lr", [0.01, 10.0])
-def test_tiny_set_one_round(lr):
+def test_tiny_set_one_round(lr, want_w):
     """Tiny set, 1/5/2, all four matrices: compress, decompress, one update round.  lr = 10 makes
-    the step larger than the code spacing so that the re-encode path really changes codes."""
+    the step larger than the code spacing so that the re-encode path really changes codes.
+    want_w = False is the launch a training loop makes (W is never stored); want_w = True the
+    instantiation that also writes W, so that W itself is compared."""
     wl = workloads.tiny()
     params = wl.all_params()
     ls = Lockstep(wl.numel, wl.kinds, wl.fmt, params)
     before = ls.dm.packed.cpu().numpy().copy()
     ls.check_decompress()
-    packed = ls.round(wl.all_grads(0), lr)
+    packed = ls.round(wl.all_grads(0), lr, want_w=want_w)
     ls.check_padding(packed)
     ls.check_decompress()
     changed = np.count_nonzero(before != packed[:before.size])
@@ -172,8 +179,9 @@ def test_partial_quantisation_sweep(wl):
     ls.check_decompress()
 
 
+@WANT_W
 @pytest.mark.parametrize("fmt", ALL_FORMATS, ids=lambda f: "E%dM%d" % f)
-def test_ragged_small_all_formats(fmt):
+def test_ragged_small_all_formats(fmt, want_w):
     """Ragged list (sizes 1 .. a few tiles, not multiples of anything), mixed kinds, three rounds
     with a step large enough to move codes across binades and into the subnormal range."""
     rng = np.random.default_rng(fmt[0] * 100 + fmt[1])
@@ -196,7 +204,7 @@ def test_ragged_small_all_formats(fmt):
     for r in range(3):
         grads = [(rng.standard_normal(n) * 0.3 * span * 10.0 ** (-(j % 6))).astype(np.float32)
                  for j, n in enumerate(numel)]
-        packed = ls.round(grads, [0.01, 1.0, 0.5][r])
+        packed = ls.round(grads, [0.01, 1.0, 0.5][r], want_w=want_w)
         ls.check_padding(packed)
     ls.check_decompress()
     assert ls.sb_ulp_cases <= 3, ls.sb_ulp_cases
@@ -204,7 +212,8 @@ def test_ragged_small_all_formats(fmt):
 
 @pytest.mark.parametrize("fmt", [(5, 2), (5, 6), (5, 10), (4, 3), (3, 7), (8, 7), (2, 3), (6, 5), (8, 10), (3, 0)],
                          ids=lambda f: "E%dM%d" % f)
-def test_special_values(fmt):
+@WANT_W
+def test_special_values(fmt, want_w):
     """Zeros of both signs, FP32 subnormals, ties, the overflow threshold, infinities and NaNs with
     payloads, a constant variable, a one-element variable."""
     E, M = fmt
@@ -237,16 +246,17 @@ def test_special_values(fmt):
     ls.check_decompress()
     grads = [(rng.standard_normal(n) * 0.05).astype(np.float32) for n in numel]
     grads[0][:8] = [np.inf, -np.inf, np.nan, 1e38, -1e38, 0.0, -0.0, 1e-45]
-    ls.round(grads, 1.0)
+    ls.round(grads, 1.0, want_w=want_w)
     ls.check_decompress()
     grads = [(rng.standard_normal(n) * 0.05).astype(np.float32) for n in numel]
-    ls.round(grads, 0.5)
+    ls.round(grads, 0.5, want_w=want_w)
     ls.check_decompress()
 
 
 @pytest.mark.parametrize("fmt", [(5, 2), (4, 3), (2, 3), (5, 6), (3, 7), (5, 10), (4, 8), (8, 7)],
                          ids=lambda f: "E%dM%d" % f)
-def test_rounding_boundaries_through_the_fast_path(fmt):
+@WANT_W
+def test_rounding_boundaries_through_the_fast_path(fmt, want_w):
     """Every midpoint between neighbouring values of the format (up to 4096 of them, the lowest
     and the highest always included), each with its two FP32 neighbours and in both signs, and a
     log-uniform sweep from below the smallest subnormal to beyond the overflow threshold, laid out
@@ -282,7 +292,7 @@ def test_rounding_boundaries_through_the_fast_path(fmt):
     params = [vals, in_range]
     ls = Lockstep([p.size for p in params], [0, 0], fmt, params)
     ls.check_decompress()
-    ls.round([np.zeros(p.size, np.float32) for p in params], 1.0)
+    ls.round([np.zeros(p.size, np.float32) for p in params], 1.0, want_w=want_w)
     ls.check_decompress()
 
 
@@ -457,8 +467,8 @@ def test_transition_refuses_mismatched_plans():
 @pytest.mark.parametrize("K", [5, 8], ids=lambda k: "K%d" % k)
 @pytest.mark.parametrize("fmt", [(5, 2), (5, 6), (5, 10), (3, 7), (4, 14)], ids=lambda f: "E%dM%d" % f)
 def test_aggregate_client_replicas(fmt, K):
-    """Server-side mean of K clients that each quantised their own random subset (Sec. 2.5): the
-    oracle decompresses every client and averages in FP32, clients in index order, one division."""
+    """Server-side mean of K clients that each quantised their own random subset (Sec. 2.5) against
+    the oracle's aggregate (every client decompressed, FP32 mean in client order, one division)."""
     rng = np.random.default_rng(7)
     numel = [3000, 1, 1024, 5121, 333, 40000, 12289, 77]
     kinds = [0, 0, 0, 0, 1, 0, 0, 2]
@@ -478,13 +488,9 @@ def test_aggregate_client_replicas(fmt, K):
     torch.cuda.synchronize()
     got = out.cpu().numpy()
     dec = [orc.decompress(c.st) for c in clients]
-    with np.errstate(all="ignore"):
-        for i, n in enumerate(numel):
-            acc = dec[0][i].copy()
-            for k in range(1, K):
-                acc = acc + dec[k][i]                     # FP32 adds, client order
-            want = acc / np.float32(K)
-            assert same_f32(from_full(clients[0].plan, got, i), want), i
+    want = orc.aggregate([c.st for c in clients])
+    for i in range(len(numel)):
+        assert same_f32(from_full(clients[0].plan, got, i), want[i]), i
     # one client alone: the mean is its decompressed model
     omc.aggregate([clients[1].plan], [clients[1].dm.packed.data_ptr()], [clients[1].dm.resid.data_ptr()],
                   [clients[1].dm.sb.data_ptr()], out.data_ptr(), torch.cuda.current_stream().cuda_stream)

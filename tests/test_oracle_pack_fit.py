@@ -271,3 +271,72 @@ def test_update_nan_is_canonical():
     assert np.all(W.view(np.uint32)[nanmask] == 0x7FFFFFFF)
     codes = orc.unpack(new_packed, 4, 8)
     assert np.all(codes[nanmask] == 0x7F)
+
+
+# ---------------------------------------------------------------------------------------------
+# server-side mean of the clients' models (Sec. 1, Sec. 2.5)
+
+@pytest.mark.parametrize("K", [1, 2, 3, 5, 8, 16])
+def test_aggregate_var_is_the_sequentially_rounded_mean(K):
+    """FP32 additions in client order, one rounded division: every step in exact rationals."""
+    rng = np.random.default_rng(K)
+    n = 60
+    xs = [(rng.standard_normal(n) * 10.0 ** rng.integers(-3, 3)).astype(np.float32) for _ in range(K)]
+    xs[0][:4] = [1e30, 1.0, -0.0, 3.0]
+    if K >= 3:
+        xs[1][:4] = [1.0, 1e-8, 0.0, 1e-45]
+        xs[2][:4] = [-1e30, -1.0, -0.0, 2e-45]      # order matters: (1e30 + 1) - 1e30 = 0, not 1
+    got = orc.aggregate_var(xs)
+    for e in range(n):
+        acc = np.float32(xs[0][e])
+        for k in range(1, K):
+            acc = f32_round(Fraction(float(acc)) + Fraction(float(xs[k][e])))
+        want = f32_round(Fraction(float(acc)) / K)
+        assert got[e] == want, (e, got[e], want)
+    if K >= 3:
+        assert got[0] == 0.0 or K > 3                 # the cancellation case above, clients in order
+    if K == 1:
+        assert np.array_equal(got.view(np.uint32), xs[0].view(np.uint32))
+
+
+def test_aggregate_var_invariants():
+    rng = np.random.default_rng(3)
+    x = (rng.standard_normal(500)).astype(np.float32)
+    # identical clients: x + x and its half are exact; with few significant bits every partial
+    # sum k x is exact too, and so is the division for any K
+    assert np.array_equal(orc.aggregate_var([x, x]), x)
+    coarse = np.round(x * 1024).astype(np.float32) / np.float32(1024)
+    for K in (3, 4, 7, 16):
+        assert np.array_equal(orc.aggregate_var([coarse] * K), coarse)
+    # the mean lies between the smallest and the largest client value
+    xs = [(x + rng.standard_normal(500).astype(np.float32) * np.float32(0.1)) for _ in range(7)]
+    m = orc.aggregate_var(xs)
+    lo, hi = np.min(xs, axis=0), np.max(xs, axis=0)
+    tol = 7 * 2.0 ** -23 * np.max(np.abs(xs), axis=0)        # six additions and a division, each within half an ulp
+    assert np.all(m >= lo - tol) and np.all(m <= hi + tol)
+    # non-finite values follow IEEE-754: Inf + (-Inf) = NaN, Inf stays Inf
+    a = np.array([np.inf, np.inf, 1.0], np.float32)
+    b = np.array([-np.inf, 1.0, np.nan], np.float32)
+    got = orc.aggregate_var([a, b])
+    assert np.isnan(got[0]) and got[1] == np.inf and np.isnan(got[2])
+
+
+def test_aggregate_models_decompresses_each_client_first():
+    """aggregate(states) = aggregate_var over the clients' decompressed variables; a client that
+    kept a variable in FP32 contributes its precise values (Sec. 2.5)."""
+    rng = np.random.default_rng(11)
+    numel = [300, 17, 1000]
+    base = [(rng.standard_normal(n) * 0.1).astype(np.float32) for n in numel]
+    sels = [[True, False, True], [False, False, True], [True, True, False]]
+    states = [orc.compress([p + np.float32(0.01 * k) for p in base], sel, 5, 2) for k, sel in enumerate(sels)]
+    got = orc.aggregate(states)
+    for i, n in enumerate(numel):
+        xs = []
+        for st in states:
+            xs.append(orc.decompress_var(st["packed"][i], n, 5, 2, st["s"][i], st["b"][i]) if st["sel"][i]
+                      else st["fp32"][i])
+        want = xs[0].copy()
+        for x in xs[1:]:
+            want = want + x
+        assert np.array_equal(got[i], want / np.float32(3))
+    assert np.array_equal(states[1]["fp32"][0], base[0] + np.float32(0.01))

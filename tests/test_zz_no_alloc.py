@@ -2,7 +2,8 @@
 running inside another framework's memory pool, services with all buffers reserved up front,
 plug-ins handed only their inputs and outputs).  Its scratch is a fixed array inside the library,
 so the test checks what such a caller relies on: the output equals omc_compress's on a one-variable
-plan, bit for bit, on two calls in a row that share the array (different sizes and formats, so the
+plan, bit for bit (and the CPU oracle's: codes bit for bit, (s, b) within one FP32 unit in the
+last place, the tolerance of every other parity test), on two calls in a row that share the array (different sizes and formats, so the
 second call meets whatever the first one left), and oversize requests are refused untouched.
 Collected last on purpose (file name), and self-contained so it also passes in a fresh process."""
 import numpy as np
@@ -10,6 +11,8 @@ import pytest
 import torch
 
 import paper_2205_03494_b200 as omc
+from oracle import omc_oracle as orc
+from harness import ulp_diff
 
 pytestmark = pytest.mark.gpu
 
@@ -40,6 +43,7 @@ def static_call(values: torch.Tensor, fmt, flags):
     omc.compress_var_static(values.data_ptr(), n, fmt, packed.data_ptr(), sb.data_ptr(), flags=flags,
                             stream=torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
+    assert omc.static_status(torch.cuda.current_stream().cuda_stream) == 0
     return packed.cpu().numpy(), sb.cpu().numpy()
 
 
@@ -63,6 +67,10 @@ def test_two_calls_in_a_row_match_omc_compress():
         want_p, want_sb = reference(v, fmt, flags)
         assert np.array_equal(got_p, want_p), (n, fmt)
         assert np.array_equal(got_sb.view(np.uint32), want_sb.view(np.uint32)), (n, fmt, got_sb, want_sb)
+        # and against the CPU oracle itself, so that a defect shared by both entry points shows
+        orc_p, orc_s, orc_b = orc.compress_var(v.cpu().numpy(), fmt[0], fmt[1], bool(flags & omc.PLAN_PVT))
+        assert np.array_equal(got_p, orc_p), (n, fmt)
+        assert ulp_diff(got_sb[0], orc_s) <= 1 and ulp_diff(got_sb[1], orc_b) <= 1, (n, fmt, got_sb, orc_s, orc_b)
     # same input twice through the shared array: identical bytes
     v = padded(200_000, gen, 0.1)
     a = static_call(v, (5, 10), omc.PLAN_PVT)
