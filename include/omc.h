@@ -100,6 +100,17 @@ int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t fmt, doubl
 int omc_plan_destroy(omc_plan_t *plan); /* also frees the plan's device tables, if any */
 
 /*
+ * omc_plan_seed -- one seed per (round, client) from one seed for the whole job (host only).
+ * Sec. 3.1 varies the selection from round to round and from client to client; the paper does
+ * not say how the draws are seeded, so the rule is this library's: the seed of (round, client) is
+ * output number round * 2^32 + client (counted from 0) of the SplitMix64 stream seeded with
+ * base_seed.  Pass the result to omc_plan as `seed`.  The generator's state is a counter, so the
+ * call costs the same for every (round, client).  base_seed = 0, round = 0 gives the generator's
+ * published check values for client = 0, 1, 2, ...
+ */
+uint64_t omc_plan_seed(uint64_t base_seed, uint32_t round, uint32_t client);
+
+/*
  * Sizes the caller must allocate (any output pointer may be NULL).
  *   closed_form_bytes: the stored size of the model as the paper counts it (Tables 1 and 2):
  *   sum over quantised variables of ceil(numel*B/8) + 8, plus 4*numel for the others.
@@ -135,6 +146,8 @@ int omc_plan_division(const omc_plan_t *plan, uint32_t *n_warps, uint32_t *n_run
  * library makes; synchronous) and clear `workspace` (device, workspace_bytes) on `stream`.
  * Must precede the first device call with this plan; the workspace then stays valid from call
  * to call (each kernel leaves it cleared) as long as calls using it do not overlap on the GPU.
+ * Calling it again re-clears the workspace and the plan's status word (the way back to a usable
+ * state after omc_plan_status reported a kernel that gave up).
  */
 int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream);
 
@@ -146,6 +159,19 @@ int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream);
  * is not expected to happen; the bounded wait exists so that a fault cannot hang the GPU.
  */
 int omc_plan_status(const omc_plan_t *plan, void *stream, uint32_t *host_status);
+
+/*
+ * omc_plan_inject_wait_timeout -- diagnostics for the bounded waits (the paper has no counterpart).
+ * The next kernel launched with this plan (omc_compress, omc_decompress, omc_update_recompress,
+ * omc_transition with the plan as destination, omc_matmul) announces its asynchronous loads to
+ * their barriers without issuing them and gives up each wait after `polls` polls (1 .. 2^24):
+ * every wait runs out with no copy in flight, the kernel sets the status word and returns, its
+ * outputs are garbage.  Afterwards omc_plan_status reports non-zero; call omc_plan_prepare again
+ * (it clears the status word and the workspace, whose counters the kernel left mid-count) before
+ * the next real call.  Host only; applies to one launch.  For tests of the give-up path: nothing
+ * faults, hangs or reads out of bounds.
+ */
+int omc_plan_inject_wait_timeout(omc_plan_t *plan, uint32_t polls);
 
 /*
  * omc_compress -- initial compression of a full-precision model (Sec. 2.2, 2.3).

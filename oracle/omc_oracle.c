@@ -375,6 +375,24 @@ uint64_t orc_splitmix64(uint64_t seed, uint32_t nth) /* the nth (0-based) output
 }
 
 /*
+ * Sec. 3.1: the selection varies "from round to round and from client to client", so every
+ * (round, client) pair needs a selection seed of its own, derived from one seed for the whole job.
+ * The rule is this library's (the paper says only that the selections vary): the seed of
+ * (round, client) is output number round * 2^32 + client, counted from 0, of the SplitMix64 stream
+ * seeded with `base`.  The generator's state is a counter (it advances by a fixed odd constant per
+ * output), so output number k is the output function applied to base + (k + 1) * constant: no
+ * stepping through the stream is needed.
+ */
+uint64_t orc_plan_seed(uint64_t base, uint32_t round, uint32_t client)
+{
+    const uint64_t k = ((uint64_t)round << 32) | (uint64_t)client;
+    uint64_t z = base + (k + 1u) * 0x9E3779B97F4A7C15ull;      /* the state after k + 1 steps */
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+/*
  * Which variables are quantised.  eligible[i] != 0 marks the weight matrices (Sec. 2.4);
  * k = floor(p*W + 1/2) of the W eligible ones are chosen at random (Sec. 2.5, Sec. 3.1): the
  * eligible indices in ascending order are shuffled by Fisher-Yates (i from W-1 down to 1,

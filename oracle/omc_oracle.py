@@ -67,6 +67,8 @@ def lib():
         L.orc_aggregate_var.argtypes = [C.POINTER(f32p), C.c_uint32, C.c_uint64, f32p]
         L.orc_splitmix64.argtypes = [C.c_uint64, C.c_uint32]
         L.orc_splitmix64.restype = C.c_uint64
+        L.orc_plan_seed.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32]
+        L.orc_plan_seed.restype = C.c_uint64
         L.orc_select.argtypes = [u8p, C.c_uint32, C.c_double, C.c_uint64, u8p]
         L.orc_model_bytes.argtypes = [u64p, u8p, C.c_uint32, C.c_int]
         L.orc_model_bytes.restype = C.c_uint64
@@ -198,6 +200,11 @@ def aggregate(states, threads: int = 1) -> list:
 
 def splitmix64(seed: int, nth: int) -> int:
     return int(lib().orc_splitmix64(seed, nth))
+
+
+def plan_seed(base: int, round_: int, client: int) -> int:
+    """Selection seed of (round, client) under one job seed (Sec. 3.1)."""
+    return int(lib().orc_plan_seed(base, round_, client))
 
 
 def select(kinds, fraction: float, seed: int, weights_only: bool = True) -> np.ndarray:

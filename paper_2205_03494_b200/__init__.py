@@ -18,8 +18,8 @@ KIND_WEIGHT_MATRIX, KIND_BIAS, KIND_NORM, KIND_OTHER = 0, 1, 2, 3
 PLAN_PVT, PLAN_WEIGHTS_ONLY = 1, 2
 PLAN_DEFAULT = PLAN_PVT | PLAN_WEIGHTS_ONLY
 
-EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_sizes",
-           "omc_plan_var", "omc_plan_division", "omc_plan_prepare", "omc_plan_status", "omc_compress", "omc_decompress",
+EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_seed", "omc_plan_sizes",
+           "omc_plan_var", "omc_plan_division", "omc_plan_prepare", "omc_plan_status", "omc_plan_inject_wait_timeout", "omc_compress", "omc_decompress",
            "omc_update_recompress", "omc_update_recompress_host", "omc_transition", "omc_aggregate", "omc_matmul",
            "omc_compress_var_static", "omc_static_status"]
 STATIC_MAX_NUMEL = 1 << 28
@@ -61,11 +61,14 @@ def lib():
         L.omc_plan.argtypes = [C.POINTER(VarDesc), C.c_uint32, Format, C.c_double, C.c_uint64,
                                C.POINTER(C.c_uint8), C.c_uint32, C.POINTER(vp)]
         L.omc_plan_destroy.argtypes = [vp]
+        L.omc_plan_seed.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32]
+        L.omc_plan_seed.restype = C.c_uint64
         L.omc_plan_sizes.argtypes = [vp, u64p, u64p, u64p, u32p, u64p, u64p]
         L.omc_plan_var.argtypes = [vp, C.c_uint32, C.POINTER(C.c_int), u64p, u64p, u64p, u64p, u32p]
         L.omc_plan_division.argtypes = [vp, u32p, u32p, u64p, C.POINTER(u64p)]
         L.omc_plan_prepare.argtypes = [vp, vp, vp]
         L.omc_plan_status.argtypes = [vp, vp, u32p]
+        L.omc_plan_inject_wait_timeout.argtypes = [vp, C.c_uint32]
         L.omc_compress.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.omc_decompress.argtypes = [vp, vp, vp, vp, C.c_uint32, C.c_uint32, vp, vp]
         L.omc_update_recompress.argtypes = [vp, vp, vp, vp, vp, C.c_float, vp, vp, vp]
@@ -148,6 +151,10 @@ class Plan:
     def prepare(self, workspace, stream=0):
         _check(lib().omc_plan_prepare(self._h, workspace, stream), "omc_plan_prepare")
 
+    def inject_wait_timeout(self, polls: int):
+        """omc_plan_inject_wait_timeout: the next launch gives up its waits (diagnostics)."""
+        _check(lib().omc_plan_inject_wait_timeout(self._h, int(polls)), "omc_plan_inject_wait_timeout")
+
     def status(self, stream=0) -> int:
         st = C.c_uint32(0)
         _check(lib().omc_plan_status(self._h, stream, C.byref(st)), "omc_plan_status")
@@ -172,6 +179,11 @@ class Plan:
         _check(lib().omc_update_recompress_host(self._h, packed, resid, sb, host_grads, float(lr),
                                                 grads_staging, host_sb_out, workspace, stream),
                "omc_update_recompress_host")
+
+
+def plan_seed(base_seed: int, round_: int, client: int) -> int:
+    """omc_plan_seed: the selection seed of (round, client) under one job seed (Sec. 3.1)."""
+    return int(lib().omc_plan_seed(int(base_seed), int(round_), int(client)))
 
 
 def transition(plan_from: Plan, plan_to: Plan, packed_from, resid_from, sb_from, packed_to, resid_to, sb_to,

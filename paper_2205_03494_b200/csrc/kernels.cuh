@@ -240,12 +240,72 @@ static __device__ __noinline__ void flush_and_maybe_finalise(Partial *slots, uin
 // to know whether all of a variable's values are equal.  The narrow-float formats use the code in
 // all four bytes (so that four codes can be compared per operation), the others the FP32 pattern.
 template <class F>
+struct WordPath {      // full units are handled a unit's code words at a time (compute_unit_b12)
+    static constexpr bool value = (F::B == 12 && HalfPath<F>::value);
+};
+template <class F>
 struct ValuePattern {
-    static constexpr uint32_t MAGNITUDE_MASK = Fp8Path<F>::value ? F::MAG_MASK * 0x01010101u : 0x7FFFFFFFu;
+    static constexpr bool BY_CODE = Fp8Path<F>::value || WordPath<F>::value;
+    static constexpr uint32_t MAGNITUDE_MASK = Fp8Path<F>::value ? F::MAG_MASK * 0x01010101u
+                                               : WordPath<F>::value ? F::MAG_MASK : 0x7FFFFFFFu;
     __device__ static __forceinline__ uint32_t of(uint32_t code, float vt)
     {
         if constexpr (Fp8Path<F>::value) return code * 0x01010101u;
+        if constexpr (WordPath<F>::value) return code;
         return f2u(vt);
+    }
+};
+
+// Equality of all the codes a lane has produced in full units since reset(), kept on whole code
+// words (every unit starts at a multiple of LU elements, so equal codes mean equal words from unit
+// to unit): one logic operation per word instead of one per element.  fold() hands the result to
+// the running sums' AND / OR trackers.
+template <class F>
+struct EqTracker {
+    static constexpr bool USED = WordPath<F>::value;
+    static constexpr int NW = USED ? Unit<F>::NWORDS : 1;
+    uint32_t ref[NW], diff, seen;
+    __device__ __forceinline__ void reset()
+    {
+        diff = 0u;
+        seen = 0u;
+#pragma unroll
+        for (int j = 0; j < NW; ++j) ref[j] = 0u;
+    }
+    // `first`: this is the warp's first unit since reset().  A lane whose first unit took the careful
+    // path instead keeps the reference 0 and reports "different" from then on, which is the truth:
+    // that unit held an Inf or NaN code and the units that come here never do.
+    __device__ __forceinline__ void unit(const uint32_t (&w)[NW], bool first)
+    {
+        if (first) {
+#pragma unroll
+            for (int j = 0; j < NW; ++j) ref[j] = w[j];
+        }
+#pragma unroll
+        for (int j = 0; j < NW; ++j) diff |= w[j] ^ ref[j];
+        seen = 1u;
+    }
+    __device__ __forceinline__ void fold(Acc &acc) const
+    {
+        if constexpr (USED) {
+            if (!seen) return;
+            // the reference unit itself: LU equal codes c give these words
+            const uint32_t c = ref[0] & F::CODE_MASK;
+            uint32_t d = diff;
+#pragma unroll
+            for (int j = 0; j < NW; ++j) {
+                uint32_t e = 0u;
+#pragma unroll
+                for (int k = 0; k < Unit<F>::LU; ++k) {
+                    const int pos = k * F::B - 32 * j;
+                    if (pos > -F::B && pos < 32) e |= pos >= 0 ? c << pos : c >> -pos;
+                }
+                d |= e ^ ref[j];
+            }
+            const uint32_t all = d ? 0xFFFFFFFFu : 0u;
+            acc.band &= c & ~all;
+            acc.bor |= c | all;
+        }
     }
 };
 
@@ -649,6 +709,123 @@ __device__ __forceinline__ void compute_unit_fp8(const uint32_t (&win)[Unit<F>::
 }
 
 // ---------------------------------------------------------------------------------------------
+// Full units of S1E5M6: eight 12-bit codes in three words.  A code << 4 is an IEEE half, and the
+// half-to-float conversion reads either half of a register, so a code is moved to bits 4..15 (or
+// 20..31) of a register with one or two operations and everything above or beside it is ignored;
+// new codes leave the packed conversion as pairs of halves and are squeezed into 24 bits per pair
+// and byte-permuted into the three words.  A unit in which a value overflows (the fast rounding
+// would keep it finite) is redone by compute_unit.
+
+// A whole unit on the careful path, out of line, from and to the unit's places in shared memory, so
+// that the main path keeps its registers and prepares nothing for it.
+template <class F, int MODE, bool WOUT>
+__device__ __noinline__ Acc compute_unit_careful(const uint32_t *cin, const float *fin, uint32_t *cout, float *fout,
+                                                 float s, float b, float neg_lr, Acc acc)
+{
+    constexpr int LU = Unit<F>::LU, NW = Unit<F>::NWORDS;
+    uint32_t win[NW], wout[NW];
+    float4 fv[LU / 4], fo[LU / 4];
+#pragma unroll
+    for (int j = 0; j < NW; ++j) win[j] = (MODE != COMPRESS) ? cin[j] : 0u;
+#pragma unroll
+    for (int j = 0; j < LU / 4; ++j)
+        fv[j] = (MODE != DECOMPRESS) ? reinterpret_cast<const float4 *>(fin)[j] : make_float4(0.f, 0.f, 0.f, 0.f);
+    compute_unit<F, MODE, false>(win, fv, wout, fo, s, b, neg_lr, acc, LU);
+    if constexpr (MODE != DECOMPRESS) {
+#pragma unroll
+        for (int j = 0; j < NW; ++j) cout[j] = wout[j];
+    }
+    if constexpr (MODE == DECOMPRESS || WOUT) {
+#pragma unroll
+        for (int j = 0; j < LU / 4; ++j) reinterpret_cast<float4 *>(fout)[j] = fo[j];
+    }
+    return acc;
+}
+
+__device__ __forceinline__ float half_lo(uint32_t r)
+{
+    return __low2float(*reinterpret_cast<const __half2 *>(&r));
+}
+__device__ __forceinline__ float half_hi(uint32_t r)
+{
+    return __high2float(*reinterpret_cast<const __half2 *>(&r));
+}
+__device__ __forceinline__ float max3_nan(float a, float b, float c)
+{
+    float r;
+    asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// Returns false, with nothing accumulated or produced, when the unit has to take the careful path.
+template <class F, int MODE>
+__device__ __forceinline__ bool compute_unit_b12(const uint32_t (&win)[3], const float4 (&fv)[2], uint32_t (&wout)[3],
+                                                 float4 (&fo)[2], float s, float b, float neg_lr, Acc &acc,
+                                                 EqTracker<F> &eq, bool first)
+{
+    static_assert(F::B == 12 && HalfPath<F>::value && Unit<F>::LU == 8, "S1E5M6");
+    float w[8];
+    if constexpr (MODE != COMPRESS) {
+        const uint32_t w0 = win[0], w1 = win[1], w2 = win[2];
+        float dec[8];
+        dec[0] = half_lo(w0 << 4);                                   // code 0: bits 0..11
+        dec[1] = half_lo((w0 >> 8) & 0xFFF0u);                       // code 1: bits 12..23
+        dec[2] = half_lo(__funnelshift_r(w0, w1, 24) << 4);          // code 2: bits 24..35
+        dec[3] = half_lo(w1 & 0xFFF0u);                              // code 3: bits 4..15 of word 1
+        dec[4] = half_lo((w1 >> 12) & 0xFFF0u);                      // code 4: bits 16..27 of word 1
+        dec[5] = half_lo(__funnelshift_r(w1, w2, 28) << 4);          // code 5: bits 28..39 of word 1
+        dec[6] = half_lo((w2 >> 4) & 0xFFF0u);                       // code 6: bits 8..19 of word 2
+        dec[7] = half_hi(w2 & 0xFFF00000u);                          // code 7: bits 20..31 of word 2
+        const float g[8] = {fv[0].x, fv[0].y, fv[0].z, fv[0].w, fv[1].x, fv[1].y, fv[1].z, fv[1].w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float vbar = __fmaf_rn(s, dec[j], b);
+            w[j] = (MODE == UPDATE) ? __fmaf_rn(neg_lr, g[j], vbar) : vbar;
+        }
+    } else {
+        w[0] = fv[0].x; w[1] = fv[0].y; w[2] = fv[0].z; w[3] = fv[0].w;
+        w[4] = fv[1].x; w[5] = fv[1].y; w[6] = fv[1].z; w[7] = fv[1].w;
+    }
+    fo[0] = make_float4(w[0], w[1], w[2], w[3]);
+    fo[1] = make_float4(w[4], w[5], w[6], w[7]);
+    if constexpr (MODE != DECOMPRESS) {
+        // Inf, NaN or a value that rounds to infinity among the eight: the careful path
+        const float m = max3_nan(max3_nan(fabsf(w[0]), fabsf(w[1]), fabsf(w[2])),
+                                 max3_nan(fabsf(w[3]), fabsf(w[4]), fabsf(w[5])), max3_nan(fabsf(w[6]), fabsf(w[7]), 0.f));
+        if (!(m < u2f(F::OVF_BITS))) return false;
+        float vt[8];
+        uint32_t pr[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            // The software rounding of encode_fast2 with the adder's constant 2^(max(e, EMIN) + 23 - M)
+            // written as 2^max(e, EMIN) * 2^(23 - M): the product is exact, so each fused
+            // multiply-add rounds exactly what the addition and the subtraction would.
+            const float w0_ = w[2 * k], w1_ = w[2 * k + 1];
+            const uint32_t u0 = f2u(w0_), u1 = f2u(w1_);
+            const float m0 = u2f(max(u0 & 0x7F800000u, F::pow2_bits(F::EMIN)));
+            const float m1 = u2f(max(u1 & 0x7F800000u, F::pow2_bits(F::EMIN)));
+            constexpr float K = (float)(1u << F::SH);
+            const float r0 = __fmaf_rn(m0, -K, __fmaf_rn(m0, K, fabsf(w0_)));
+            const float r1 = __fmaf_rn(m1, -K, __fmaf_rn(m1, K, fabsf(w1_)));
+            vt[2 * k] = u2f(f2u(r0) | (u0 & 0x80000000u));
+            vt[2 * k + 1] = u2f(f2u(r1) | (u1 & 0x80000000u));
+            const __half2 h = __floats2half2_rn(vt[2 * k], vt[2 * k + 1]);   // exact: both are FP16 values
+            const uint32_t x = *reinterpret_cast<const uint32_t *>(&h);      // code 2k << 4 | code 2k+1 << 20
+            // the pair's 24 bits; what is left above them is never selected by the byte permutes below
+            const uint32_t lo = x >> 4, hi = x >> 8;
+            pr[k] = (lo & 0xFFFu) | (hi & ~0xFFFu);
+        }
+        wout[0] = __byte_perm(pr[0], pr[1], 0x4210);
+        wout[1] = __byte_perm(pr[1], pr[2], 0x5421);
+        wout[2] = __byte_perm(pr[2], pr[3], 0x6542);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc.add(w[j], vt[j]);
+        eq.unit(wout, first);
+    }
+    return true;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Register <-> memory moves of a unit (global or shared: the address space is inferred).
 
 template <int N>
@@ -692,7 +869,7 @@ __device__ __forceinline__ void store_words(const uint32_t (&w)[N], uint32_t *p)
 template <class F, int MODE, bool WOUT>
 __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const float *s_fin, uint32_t *s_cout,
                                                   float *s_fout, float s, float b, float neg_lr, Acc &acc,
-                                                  int lane)
+                                                  EqTracker<F> &eq, bool first_granule, int lane)
 {
     using U = Unit<F>;
     constexpr int LU = U::LU, NW = U::NWORDS;
@@ -701,7 +878,7 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
         return;
     }
     constexpr int G = (U::SUB_STEPS >= 2 && LU == 4) ? 2 : 1;   // steps whose operands are fetched together
-    constexpr int UNROLL = F::B == 8 ? 4 : 1;
+    constexpr int UNROLL = (F::B == 8 || F::B == 12) ? 4 : 1;     // measured
 #pragma unroll UNROLL
     for (int k0 = 0; k0 < U::SUB_STEPS; k0 += G) {
         uint32_t win[G][NW];
@@ -723,7 +900,14 @@ __device__ __forceinline__ void granule_from_smem(const uint32_t *s_cin, const f
             float4 fo[LU / 4];
             if constexpr (Fp8Path<F>::value)
                 compute_unit_fp8<F, MODE>(win[g], fv[g], wout, fo, s, b, neg_lr, acc);
-            else
+            else if constexpr (WordPath<F>::value) {
+                if (!compute_unit_b12<F, MODE>(win[g], fv[g], wout, fo, s, b, neg_lr, acc, eq,
+                                               first_granule && k0 + g == 0)) {
+                    acc = compute_unit_careful<F, MODE, WOUT>(s_cin + unit * NW, s_fin + unit * LU, s_cout + unit * NW,
+                                                              s_fout + unit * LU, s, b, neg_lr, acc);
+                    continue;
+                }
+            } else
                 compute_unit<F, MODE, false>(win[g], fv[g], wout, fo, s, b, neg_lr, acc, LU);
             if constexpr (MODE != DECOMPRESS) store_words<NW>(wout, s_cout + unit * NW);
             if constexpr (MODE == DECOMPRESS || WOUT) {
@@ -863,8 +1047,19 @@ struct WarpPipe {
     uint32_t bar0;
     uint32_t k;
     uint32_t phases;      // bit i: the parity the next wait on mbarrier i looks for
+    uint32_t wait_limit;  // polls of one mbarrier before giving up
+    bool skip_loads;      // diagnostics: announce the loads, do not issue them
     bool failed;
 };
+
+__device__ __forceinline__ void pipe_init(WarpPipe &pipe, const KParams &p)
+{
+    pipe.k = 0;
+    pipe.phases = 0u;
+    pipe.wait_limit = p.wait_limit ? p.wait_limit : WAIT_LIMIT;
+    pipe.skip_loads = p.skip_loads != 0u;
+    pipe.failed = false;
+}
 
 // Elements [e_begin, e_end) of one quantised variable (e_begin on a tile boundary, e_end on a tile
 // boundary or at the variable's end): whole granules through the warp's pipeline, the rest (only
@@ -892,13 +1087,17 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
         uint8_t *dst = wbase + st * SM::STAGE;
         if (lane == 0) {
             mbar_expect_tx(bar, (uint32_t)SM::TX_BYTES);
-            if constexpr (SM::IN_C > 0)
-                bulk_load(smem_addr(dst), codes + (size_t)g * SM::CB, SM::CB, bar);
-            if constexpr (SM::IN_F > 0)
-                bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)g * SUB, SM::FB, bar);
+            if (!pipe.skip_loads) {
+                if constexpr (SM::IN_C > 0)
+                    bulk_load(smem_addr(dst), codes + (size_t)g * SM::CB, SM::CB, bar);
+                if constexpr (SM::IN_F > 0)
+                    bulk_load(smem_addr(dst + SM::IN_C), fin + (size_t)g * SUB, SM::FB, bar);
+            }
         }
     };
 
+    EqTracker<F> eq;
+    eq.reset();
     for (uint32_t i = 0; i < (uint32_t)SM::DIST && i < ng; ++i) issue(g0 + i, k + i);
     for (uint32_t i = 0; i < ng; ++i, ++k) {
         const uint32_t g = g0 + i;
@@ -917,7 +1116,7 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
         pipe.phases ^= 1u << st;
         uint32_t polls = 0;
         while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) {
-            if (++polls > WAIT_LIMIT) { failed = true; break; }
+            if (++polls > pipe.wait_limit) { failed = true; break; }
         }
         if (failed) break;
         uint8_t *stage = wbase + st * SM::STAGE;
@@ -927,7 +1126,7 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
         if constexpr (ROWS_IN) rows_swizzle_in_place(const_cast<float *>(fsrc), lane, true);
         uint8_t *cdst = SM::CODES_IN_PLACE ? stage : ob;
         granule_from_smem<F, MODE, WOUT>(reinterpret_cast<const uint32_t *>(stage), fsrc, reinterpret_cast<uint32_t *>(cdst),
-                                         fdst, s, b, neg_lr, acc, lane);
+                                         fdst, s, b, neg_lr, acc, eq, i == 0, lane);
         if constexpr (ROWS_OUT) {
             __syncwarp();
             rows_swizzle_in_place(fdst, lane, false);
@@ -943,6 +1142,7 @@ __device__ __forceinline__ void run_elements(WarpPipe &pipe, uint8_t *codes, con
         }
     }
     if (failed) { pipe.k = k; pipe.failed = true; return; }
+    if constexpr (MODE != DECOMPRESS) eq.fold(acc);
     const uint64_t e_rag = e_begin + (uint64_t)ng * SUB;
     if (e_rag < e_end) {     // the variable's ragged end
         const uint64_t w0 = e_rag / 32 * F::B;
@@ -1040,9 +1240,7 @@ omc_kernel(const KParams p)
     WarpPipe pipe;
     pipe.wbase = smem_raw + SM::BAR_PAD + wid * SM::PER_WARP;
     pipe.bar0 = smem_addr(smem_raw) + (uint32_t)wid * MAX_STAGES * 8u;
-    pipe.k = 0;
-    pipe.phases = 0u;
-    pipe.failed = false;
+    pipe_init(pipe, p);
     const uint32_t bar0 = pipe.bar0;
     if (lane == 0) {
 #pragma unroll
@@ -1161,9 +1359,7 @@ __global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_transition_kernel(co
     WarpPipe pipe;
     pipe.wbase = smem_raw + TS::C::BAR_PAD + wid * TS::PER_WARP;
     pipe.bar0 = smem_addr(smem_raw) + (uint32_t)wid * MAX_STAGES * 8u;
-    pipe.k = 0;
-    pipe.phases = 0u;
-    pipe.failed = false;
+    pipe_init(pipe, p);
     if (lane == 0) {
 #pragma unroll
         for (int i = 0; i < MAX_STAGES; ++i) mbar_init(pipe.bar0 + 8u * i, 1u);

@@ -84,6 +84,10 @@ extern "C" int omc_plan_prepare(omc_plan_t *plan, void *workspace, void *stream)
         if (rc) { (void)cudaFree(plan->d_vars); plan->d_vars = nullptr; return rc; }
         plan->device = dev;
     }
+    // a repeated call also clears the status word (after a kernel gave up, the workspace's counters
+    // are left mid-count and the caller prepares again)
+    rc = omc::note_cuda(cudaMemsetAsync(plan->d_status, 0, sizeof(uint32_t), static_cast<cudaStream_t>(stream)));
+    if (rc) return rc;
     return omc::note_cuda(cudaMemsetAsync(workspace, 0, plan->ws_bytes, static_cast<cudaStream_t>(stream)));
 }
 
@@ -97,9 +101,18 @@ static int check_ready(const omc_plan_t *plan)
     return dev == plan->device ? OMC_OK : OMC_ERR_PLAN_MISMATCH;
 }
 
+// The diagnostic of omc_plan_inject_wait_timeout applies to one launch.
+static void take_injection(const omc_plan_t *plan, KParams &p)
+{
+    p.wait_limit = plan->inject_polls;
+    p.skip_loads = plan->inject_polls ? 1u : 0u;
+    plan->inject_polls = 0;
+}
+
 static KParams whole_model(const omc_plan_t *plan, void *workspace)
 {
     KParams p{};
+    take_injection(plan, p);
     p.vars = plan->d_vars;
     p.var_begin = 0;
     p.var_end = plan->nvars;
@@ -169,6 +182,7 @@ extern "C" int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, con
     if (any_r && !resid) return OMC_ERR_NULL_PTR;
     if (misaligned(packed) || misaligned(resid) || misaligned(sb) || misaligned(out)) return OMC_ERR_MISALIGNED;
     KParams p{};
+    take_injection(plan, p);
     p.vars = plan->d_vars;
     p.var_begin = first_var;
     p.var_end = first_var + n_vars;
@@ -252,6 +266,14 @@ extern "C" int omc_plan_status(const omc_plan_t *plan, void *stream, uint32_t *h
     rc = omc::note_cuda(cudaMemcpyAsync(host_status, plan->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     if (rc) return rc;
     return omc::note_cuda(cudaStreamSynchronize(st));
+}
+
+extern "C" int omc_plan_inject_wait_timeout(omc_plan_t *plan, uint32_t polls)
+{
+    if (!plan) return OMC_ERR_NULL_PTR;
+    if (polls == 0 || polls > (1u << 24)) return OMC_ERR_INVALID_ARG;
+    plan->inject_polls = polls;
+    return OMC_OK;
 }
 
 extern "C" int omc_transition(const omc_plan_t *from, const omc_plan_t *to, const uint8_t *packed_from,

@@ -92,6 +92,11 @@ struct KParams {
     const TransitionVar *trans_vars;   // the launch's own record numbering
     const uint32_t *nruns_dev;         // the launch's run count (replaces nruns)
     uint32_t *status;              // the plan's device status word: set non-zero if a copy never arrived
+    // Diagnostics (omc_plan_inject_wait_timeout): polls of one mbarrier before a warp gives up (0 = the
+    // default), and whether the warps announce their bulk loads to the mbarrier without issuing them,
+    // so that the waits run out with nothing in flight.
+    uint32_t wait_limit;
+    uint32_t skip_loads;
 };
 
 // omc_transition's own division of the work, made on the device before each launch.
@@ -208,5 +213,6 @@ struct omc_plan {
     uint64_t *d_fp32_tile_start;
     uint32_t *d_fp32_var;
     omc::TransitionTables d_trans;     // omc_transition's tables (this plan as the destination)
+    mutable uint32_t inject_polls;     // omc_plan_inject_wait_timeout: applies to the next launch, then 0
     int device;                        // device the tables live on, -1 before prepare
 };

@@ -72,9 +72,9 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Bounded wait for the phase with the given parity; false if it never completed.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit)
 {
-    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -199,10 +199,14 @@ template <int B, int E>
 __global__ void __launch_bounds__(Cfg<B, E>::THREADS, 1)
 matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
               const float *__restrict__ sb, const float *__restrict__ rowsum, float *__restrict__ y,
-              uint32_t M, uint32_t N, uint32_t K, uint32_t *status)
+              uint32_t M, uint32_t N, uint32_t K, uint32_t *status, uint32_t inject_polls)
 {
     using C = Cfg<B, E>;
     constexpr int NS = C::NSTAGES;
+    // diagnostics (omc_plan_inject_wait_timeout): the producer announces its loads without issuing
+    // them and every wait gives up after inject_polls polls, with no copy in flight
+    const uint32_t limit = inject_polls ? inject_polls : WAIT_LIMIT;
+    const bool skip_loads = inject_polls != 0u;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (saddr(smem_raw) + 1023u) & ~1023u;      // tiles need 1024-byte alignment
     const uint32_t bars = base + NS * C::STAGE;     // full[NS], decoded[NS], empty[NS], acc_full[2], acc_empty[2], tmem slot
@@ -243,9 +247,10 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
             const int tm = t % tiles_m, tn = t / tiles_m;
             for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % NS;
-                if (it >= (uint32_t)NS) ok = mbar_wait(empty(s), ((it / NS) - 1) & 1u);
+                if (it >= (uint32_t)NS) ok = mbar_wait(empty(s), ((it / NS) - 1) & 1u, limit);
                 if (!ok) break;
                 mbar_expect_tx(full(s), C::TX_BYTES);
+                if (skip_loads) continue;
                 const uint32_t a = base + s * C::STAGE;
                 tma_load_2d(a, &map_x, (int)(kb * BK), tm * BM, full(s));
                 if constexpr (C::DECODE)
@@ -259,14 +264,14 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         uint32_t it = 0, lt = 0;
         for (uint32_t t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++lt) {
             const uint32_t buf = lt & 1u;
-            if (lt >= 2) ok = mbar_wait(acc_empty(buf), ((lt >> 1) - 1) & 1u);   // the epilogue has drained it
+            if (lt >= 2) ok = mbar_wait(acc_empty(buf), ((lt >> 1) - 1) & 1u, limit);   // the epilogue has drained it
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t d = tmem_base + buf * (uint32_t)BN;
             for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % NS;
-                ok = mbar_wait(full(s), (it / NS) & 1u);
-                if constexpr (C::DECODE) ok = ok && mbar_wait(decoded(s), (it / NS) & 1u);
+                ok = mbar_wait(full(s), (it / NS) & 1u, limit);
+                if constexpr (C::DECODE) ok = ok && mbar_wait(decoded(s), (it / NS) & 1u, limit);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a = base + s * C::STAGE, b = a + TILE_A_BYTES;
@@ -285,7 +290,7 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         for (uint32_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++lt) {
             const int tm = t % tiles_m, tn = t / tiles_m;
             const uint32_t buf = lt & 1u;
-            ok = mbar_wait(acc_full(buf), (lt >> 1) & 1u);
+            ok = mbar_wait(acc_full(buf), (lt >> 1) & 1u, limit);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -330,7 +335,7 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
             for (uint32_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
                 for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % NS;
-                    ok = mbar_wait(full(s), (it / NS) & 1u);
+                    ok = mbar_wait(full(s), (it / NS) & 1u, limit);
                     if (!ok) break;
                     uint8_t *stage = base_ptr + s * C::STAGE;
                     const uint8_t *raw = stage + TILE_A_BYTES + TILE_B_BYTES + t * B;      // 8 codes = B bytes
@@ -404,7 +409,7 @@ bool make_raw_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t row_b
 
 template <int B, int E>
 int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const float *rowsum, float *y,
-           uint32_t M, uint32_t N, uint32_t K, uint32_t n_sm, uint32_t *status, cudaStream_t st)
+           uint32_t M, uint32_t N, uint32_t K, uint32_t n_sm, uint32_t *status, uint32_t inject_polls, cudaStream_t st)
 {
     using C = Cfg<B, E>;
     CUtensorMap map_w;
@@ -420,7 +425,7 @@ int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const f
     }
     const uint32_t ntiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
     const uint32_t grid = ntiles < n_sm ? ntiles : n_sm;
-    matmul_kernel<B, E><<<grid, C::THREADS, C::SMEM, st>>>(map_x, map_w, sb, rowsum, y, M, N, K, status);
+    matmul_kernel<B, E><<<grid, C::THREADS, C::SMEM, st>>>(map_x, map_w, sb, rowsum, y, M, N, K, status, inject_polls);
     return omc::note_cuda(cudaGetLastError());
 }
 
@@ -458,11 +463,13 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     const uint8_t *codes = packed + v.store_off;
     const float *sbv = sb + 2 * v.sb_slot;
     const uint32_t n_sm = plan->n_sm ? plan->n_sm : 1;
-    if (exp == 4) return launch<8, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
-    if (exp == 2) return launch<6, 2>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
+    const uint32_t inject = plan->inject_polls;      // diagnostics: applies to this launch only
+    plan->inject_polls = 0;
+    if (exp == 4) return launch<8, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    if (exp == 2) return launch<6, 2>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     switch (man) {
-    case 10: return launch<16, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
-    case 6: return launch<12, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
-    default: return launch<8, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, st);
+    case 10: return launch<16, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    case 6: return launch<12, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    default: return launch<8, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     }
 }

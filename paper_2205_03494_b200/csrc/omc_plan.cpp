@@ -50,6 +50,14 @@ static uint64_t splitmix64(uint64_t &state)
     return z ^ (z >> 31);
 }
 
+// The k-th output (k = round * 2^32 + client) of the stream seeded with base_seed: SplitMix64
+// keeps a counter as its state, so the stream can be entered anywhere.
+extern "C" uint64_t omc_plan_seed(uint64_t base_seed, uint32_t round, uint32_t client)
+{
+    uint64_t state = base_seed + ((((uint64_t)round << 32) | client) * 0x9E3779B97F4A7C15ull);
+    return splitmix64(state);
+}
+
 static uint64_t round_up(uint64_t x, uint64_t m) { return (x + m - 1) / m * m; }
 
 static uint32_t query_sm_count()
@@ -156,6 +164,7 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         pl->ops = ops;
         pl->d_vars = nullptr;
         pl->d_status = nullptr;
+        pl->inject_polls = 0;
         pl->d_run_start = nullptr;
         pl->d_run_var = nullptr;
         pl->d_dec_run_var = nullptr;

@@ -160,3 +160,20 @@ def test_division_of_the_tiles_into_runs():
             entered = int(np.searchsorted(qstarts, rs[r + 1]) - np.searchsorted(qstarts, rs[r]))
             assert run <= cost_share + 2, (r, run, cost_share)
             assert run + 3 * entered >= cost_share - 5, (r, run, entered, cost_share)
+
+
+def test_plan_seed_matches_oracle_and_published_values():
+    want = [int(l, 16) for l in open(os.path.join(os.path.dirname(__file__), "golden", "splitmix64_seed0.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert [omc.plan_seed(0, 0, c) for c in range(len(want))] == want
+    rng = np.random.default_rng(8)
+    for _ in range(200):
+        base = int(rng.integers(0, 2 ** 63)) * 2 + int(rng.integers(0, 2))
+        r, c = int(rng.integers(0, 2 ** 32)), int(rng.integers(0, 2 ** 32))
+        assert omc.plan_seed(base, r, c) == orc.plan_seed(base, r, c)
+    # N client plans from one seed: the library's plans equal the oracle's selections
+    wl = workloads.conformer_like(blocks=2)
+    for client in range(4):
+        seed = omc.plan_seed(77, 3, client)
+        plan = omc.Plan(wl.numel, wl.kinds, (3, 7), fraction=0.9, seed=seed)
+        assert plan.quantised == list(orc.select(wl.kinds, 0.9, orc.plan_seed(77, 3, client)))

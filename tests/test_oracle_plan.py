@@ -118,3 +118,26 @@ def test_whole_model_state_round():
     assert np.array_equal(ws[1], orc.sgd_var(variables[1], grads[1], 0.01))
     p, s, b = orc.compress_var(ws[0], 5, 2)
     assert np.array_equal(st["packed"][0], p) and st["s"][0] == s and st["b"][0] == b
+
+
+def test_plan_seed_is_the_kth_output_of_the_published_generator():
+    """Seeds per (round, client), Sec. 3.1: output number round * 2^32 + client of the stream seeded
+    with the job's seed.  For seed 0, round 0 these are the generator's published check values; for
+    other arguments the oracle's direct jump must land where stepping through the stream arrives."""
+    want = [int(l, 16) for l in open(os.path.join(GOLDEN, "splitmix64_seed0.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert [orc.plan_seed(0, 0, c) for c in range(len(want))] == want
+    for base in (0, 1, 0xDEADBEEF, 2 ** 64 - 1):
+        for c in (0, 1, 7, 500, 1999):
+            assert orc.plan_seed(base, 0, c) == orc.splitmix64(base, c)
+    # a round is 2^32 outputs further on: the same as entering the stream of another seed
+    gamma = 0x9E3779B97F4A7C15
+    for base, rnd, c in [(5, 1, 0), (5, 3, 9), (123456789, 1000, 77)]:
+        shifted = (base + ((rnd << 32) * gamma)) % 2 ** 64
+        assert orc.plan_seed(base, rnd, c) == orc.splitmix64(shifted, c)
+    # all different over a grid of rounds and clients, and the selections they give vary
+    seeds = {orc.plan_seed(42, r, c) for r in range(50) for c in range(128)}
+    assert len(seeds) == 50 * 128
+    kinds = np.zeros(40, int)
+    masks = {tuple(orc.select(kinds, 0.9, orc.plan_seed(42, r, c))) for r in range(4) for c in range(16)}
+    assert len(masks) > 55
