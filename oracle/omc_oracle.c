@@ -116,6 +116,62 @@ void orc_encode_array(const float *x, uint64_t n, int E, int M, uint32_t *codes)
 }
 
 /* ------------------------------------------------------------------------------------------ */
+/*
+ * Fixed-point variant.  Sec. 2.2 remarks that fixed-point (or other) formats can be used in place
+ * of the floating-point one and says nothing more, so everything here is a reading ("parity
+ * unpinned" by the paper): S1IxFy = one sign bit, x integer bits, y fraction bits, B = 1 + x + y;
+ * a code is the B-bit two's complement of an integer k in [-2^(x+y), 2^(x+y) - 1] and stands for
+ * k * 2^-y.  The scale is fixed by the format, not by the data: a scale taken from the data (a
+ * maximum) would need a pass over the updated values before the first code could be written,
+ * which the one-pass update of Sec. 2.1 has no room for; adapting to the variable is what the
+ * per-variable transformation of Sec. 2.3 does afterwards, as for the floating-point codes.
+ * Encoding: k = x * 2^y rounded to the nearest integer, ties to even, then clamped to the range
+ * (saturation: there is no infinity); NaN has no code either and becomes 0.
+ * x + y <= 23, so that every value is an FP32 value.
+ */
+int orc_fixed_format_ok(int I, int F) { return I >= 0 && I <= 8 && F >= 0 && I + F >= 1 && I + F <= 23; }
+
+float orc_decode_fixed(uint32_t code, int I, int F)
+{
+    const int B = 1 + I + F;
+    int64_t k = (int64_t)(code & ((1u << B) - 1u));
+    if (k >= ((int64_t)1 << (B - 1))) k -= ((int64_t)1 << B);      /* two's complement */
+    return (float)ldexp((double)k, -F);
+}
+
+uint32_t orc_encode_fixed(float x, int I, int F)
+{
+    const int B = 1 + I + F;
+    const uint32_t mask = (1u << B) - 1u;
+    if (isnan(x)) return 0u;
+    const double lo = -ldexp(1.0, I + F), hi = ldexp(1.0, I + F) - 1.0;
+    double k = nearbyint(ldexp((double)x, F));   /* exact scaling; default rounding mode = ties to even */
+    if (k < lo) k = lo;
+    if (k > hi) k = hi;
+    return (uint32_t)(int64_t)k & mask;
+}
+
+/* The two codecs behind one switch: fixed != 0 reads (E, M) as (integer bits, fraction bits). */
+static uint32_t enc_any(float x, int fixed, int E, int M)
+{
+    return fixed ? orc_encode_fixed(x, E, M) : orc_encode(x, E, M);
+}
+static float dec_any(uint32_t c, int fixed, int E, int M)
+{
+    return fixed ? orc_decode_fixed(c, E, M) : orc_decode(c, E, M);
+}
+
+void orc_decode_fixed_array(const uint32_t *codes, uint64_t n, int I, int F, float *out)
+{
+    for (uint64_t k = 0; k < n; ++k) out[k] = orc_decode_fixed(codes[k], I, F);
+}
+
+void orc_encode_fixed_array(const float *x, uint64_t n, int I, int F, uint32_t *codes)
+{
+    for (uint64_t k = 0; k < n; ++k) codes[k] = orc_encode_fixed(x[k], I, F);
+}
+
+/* ------------------------------------------------------------------------------------------ */
 /* Bit packing.  The paper stores "B-bit codes"; the layout is this library's (paper silent):    */
 /* little-endian bit stream, code k in bits [k*B, (k+1)*B), bit j of the stream = bit (j mod 8)  */
 /* of byte (j div 8); the stream is zero-padded to a multiple of 16 bytes.                       */
@@ -286,16 +342,17 @@ void orc_fit(const float *V, const float *Vt, uint64_t n, int pvt, float *s_out,
 /* ------------------------------------------------------------------------------------------ */
 /* Whole-variable operations (Sec. 2.1, Fig. 1).                                                */
 
-/* Initial compression of one variable: quantise V itself, fit (s, b) against it, pack. */
-void orc_compress_var(const float *V, uint64_t n, int E, int M, int pvt, uint8_t *packed,
-                      float *s_out, float *b_out)
+/* Initial compression of one variable: quantise V itself, fit (s, b) against it, pack.
+ * fixed != 0: the fixed-point codec with (E, M) = (integer bits, fraction bits). */
+void orc_compress_var_fx(const float *V, uint64_t n, int fixed, int E, int M, int pvt, uint8_t *packed,
+                         float *s_out, float *b_out)
 {
     const int B = 1 + E + M;
     uint32_t *codes = (uint32_t *)malloc(n * sizeof(uint32_t));
     float *Vt = (float *)malloc(n * sizeof(float));
     for (uint64_t k = 0; k < n; ++k) {
-        codes[k] = orc_encode(V[k], E, M);
-        Vt[k] = orc_decode(codes[k], E, M);
+        codes[k] = enc_any(V[k], fixed, E, M);
+        Vt[k] = dec_any(codes[k], fixed, E, M);
     }
     orc_fit(V, Vt, n, pvt, s_out, b_out, NULL);
     orc_pack(codes, n, B, packed);
@@ -303,14 +360,26 @@ void orc_compress_var(const float *V, uint64_t n, int E, int M, int pvt, uint8_t
     free(Vt);
 }
 
+void orc_compress_var(const float *V, uint64_t n, int E, int M, int pvt, uint8_t *packed,
+                      float *s_out, float *b_out)
+{
+    orc_compress_var_fx(V, n, 0, E, M, pvt, packed, s_out, b_out);
+}
+
 /* Forward path: Vbar_k = s*Vt_k + b, one correctly rounded fp32 fused multiply-add per element
  * (the rounding of this fp32 operation is a reading: the paper gives only the formula). */
-void orc_decompress_var(const uint8_t *packed, uint64_t n, int E, int M, float s, float b,
-                        float *out)
+void orc_decompress_var_fx(const uint8_t *packed, uint64_t n, int fixed, int E, int M, float s, float b,
+                           float *out)
 {
     const int B = 1 + E + M;
     for (uint64_t k = 0; k < n; ++k)
-        out[k] = fmaf(s, orc_decode(orc_unpack_one(packed, k, B), E, M), b);
+        out[k] = fmaf(s, dec_any(orc_unpack_one(packed, k, B), fixed, E, M), b);
+}
+
+void orc_decompress_var(const uint8_t *packed, uint64_t n, int E, int M, float s, float b,
+                        float *out)
+{
+    orc_decompress_var_fx(packed, n, 0, E, M, s, b, out);
 }
 
 /*
@@ -318,19 +387,25 @@ void orc_decompress_var(const uint8_t *packed, uint64_t n, int E, int M, float s
  * A NaN produced by the arithmetic has no payload fixed by IEEE-754; it is replaced by the
  * positive all-ones NaN so that the code written back is defined.  w_out (optional) receives W.
  */
-void orc_update_recompress_var(uint8_t *packed, uint64_t n, int E, int M, int pvt, float *s_io,
-                               float *b_io, const float *g, float lr, float *w_out)
+void orc_update_recompress_var_fx(uint8_t *packed, uint64_t n, int fixed, int E, int M, int pvt, float *s_io,
+                                  float *b_io, const float *g, float lr, float *w_out)
 {
     float *W = (float *)malloc(n * sizeof(float));
-    orc_decompress_var(packed, n, E, M, *s_io, *b_io, W);
+    orc_decompress_var_fx(packed, n, fixed, E, M, *s_io, *b_io, W);
     for (uint64_t k = 0; k < n; ++k) {
         float w = fmaf(-lr, g[k], W[k]);
         if (isnan(w)) w = bits_f32(0x7FFFFFFFu);
         W[k] = w;
     }
-    orc_compress_var(W, n, E, M, pvt, packed, s_io, b_io);
+    orc_compress_var_fx(W, n, fixed, E, M, pvt, packed, s_io, b_io);
     if (w_out) memcpy(w_out, W, n * sizeof(float));
     free(W);
+}
+
+void orc_update_recompress_var(uint8_t *packed, uint64_t n, int E, int M, int pvt, float *s_io,
+                               float *b_io, const float *g, float lr, float *w_out)
+{
+    orc_update_recompress_var_fx(packed, n, 0, E, M, pvt, s_io, b_io, g, lr, w_out);
 }
 
 /* Variables that stay in FP32 (Sec. 2.4): plain SGD step in place. */

@@ -47,6 +47,18 @@ def lib():
         L.orc_decode.restype = C.c_float
         L.orc_encode.argtypes = [C.c_float, C.c_int, C.c_int]
         L.orc_encode.restype = C.c_uint32
+        L.orc_fixed_format_ok.argtypes = [C.c_int, C.c_int]
+        L.orc_decode_fixed.argtypes = [C.c_uint32, C.c_int, C.c_int]
+        L.orc_decode_fixed.restype = C.c_float
+        L.orc_encode_fixed.argtypes = [C.c_float, C.c_int, C.c_int]
+        L.orc_encode_fixed.restype = C.c_uint32
+        L.orc_decode_fixed_array.argtypes = [u32p, C.c_uint64, C.c_int, C.c_int, f32p]
+        L.orc_encode_fixed_array.argtypes = [f32p, C.c_uint64, C.c_int, C.c_int, u32p]
+        L.orc_compress_var_fx.argtypes = [f32p, C.c_uint64, C.c_int, C.c_int, C.c_int, C.c_int, u8p, f32p, f32p]
+        L.orc_decompress_var_fx.argtypes = [u8p, C.c_uint64, C.c_int, C.c_int, C.c_int, C.c_float, C.c_float,
+                                            f32p]
+        L.orc_update_recompress_var_fx.argtypes = [u8p, C.c_uint64, C.c_int, C.c_int, C.c_int, C.c_int, f32p,
+                                                   f32p, f32p, C.c_float, f32p]
         L.orc_decode_array.argtypes = [u32p, C.c_uint64, C.c_int, C.c_int, f32p]
         L.orc_encode_array.argtypes = [f32p, C.c_uint64, C.c_int, C.c_int, u32p]
         L.orc_packed_bytes.argtypes = [C.c_uint64, C.c_int]
@@ -87,17 +99,20 @@ def _f32(a) -> np.ndarray:
 # --------------------------------------------------------------------------------------------
 # scalar / array codec
 
-def decode(codes, E: int, M: int) -> np.ndarray:
+def decode(codes, E: int, M: int, fixed: bool = False) -> np.ndarray:
+    """fixed=True: the fixed-point variant, (E, M) = (integer bits, fraction bits)."""
     codes = np.ascontiguousarray(codes, dtype=np.uint32).ravel()
     out = np.empty(codes.size, np.float32)
-    lib().orc_decode_array(_p(codes, C.c_uint32), codes.size, E, M, _p(out, C.c_float))
+    fn = lib().orc_decode_fixed_array if fixed else lib().orc_decode_array
+    fn(_p(codes, C.c_uint32), codes.size, E, M, _p(out, C.c_float))
     return out
 
 
-def encode(x, E: int, M: int) -> np.ndarray:
+def encode(x, E: int, M: int, fixed: bool = False) -> np.ndarray:
     x = _f32(x).ravel()
     out = np.empty(x.size, np.uint32)
-    lib().orc_encode_array(_p(x, C.c_float), x.size, E, M, _p(out, C.c_uint32))
+    fn = lib().orc_encode_fixed_array if fixed else lib().orc_encode_array
+    fn(_p(x, C.c_float), x.size, E, M, _p(out, C.c_uint32))
     return out
 
 
@@ -138,33 +153,33 @@ def fit(V, Vt, pvt: bool = True, want_sums: bool = False):
 # --------------------------------------------------------------------------------------------
 # per-variable operations
 
-def compress_var(V, E: int, M: int, pvt: bool = True):
+def compress_var(V, E: int, M: int, pvt: bool = True, fixed: bool = False):
     V = _f32(V).ravel()
     out = np.empty(packed_bytes(V.size, 1 + E + M), np.uint8)
     s, b = C.c_float(), C.c_float()
-    lib().orc_compress_var(_p(V, C.c_float), V.size, E, M, int(pvt), _p(out, C.c_uint8),
-                           C.byref(s), C.byref(b))
+    lib().orc_compress_var_fx(_p(V, C.c_float), V.size, int(fixed), E, M, int(pvt), _p(out, C.c_uint8),
+                              C.byref(s), C.byref(b))
     return out, np.float32(s.value), np.float32(b.value)
 
 
-def decompress_var(packed, n: int, E: int, M: int, s, b) -> np.ndarray:
+def decompress_var(packed, n: int, E: int, M: int, s, b, fixed: bool = False) -> np.ndarray:
     packed = np.ascontiguousarray(packed, dtype=np.uint8)
     out = np.empty(n, np.float32)
-    lib().orc_decompress_var(_p(packed, C.c_uint8), n, E, M, C.c_float(float(s)),
-                             C.c_float(float(b)), _p(out, C.c_float))
+    lib().orc_decompress_var_fx(_p(packed, C.c_uint8), n, int(fixed), E, M, C.c_float(float(s)),
+                                C.c_float(float(b)), _p(out, C.c_float))
     return out
 
 
 def update_recompress_var(packed, n: int, E: int, M: int, s, b, g, lr: float, pvt: bool = True,
-                          want_w: bool = False):
+                          want_w: bool = False, fixed: bool = False):
     """Returns (new_packed, s', b'[, W]); the input array is not modified."""
     packed = np.array(packed, dtype=np.uint8, copy=True)
     g = _f32(g).ravel()
     sc, bc = C.c_float(float(s)), C.c_float(float(b))
     w = np.empty(n, np.float32) if want_w else None
-    lib().orc_update_recompress_var(_p(packed, C.c_uint8), n, E, M, int(pvt), C.byref(sc),
-                                    C.byref(bc), _p(g, C.c_float), C.c_float(lr),
-                                    _p(w, C.c_float) if want_w else None)
+    lib().orc_update_recompress_var_fx(_p(packed, C.c_uint8), n, int(fixed), E, M, int(pvt), C.byref(sc),
+                                       C.byref(bc), _p(g, C.c_float), C.c_float(lr),
+                                       _p(w, C.c_float) if want_w else None)
     if want_w:
         return packed, np.float32(sc.value), np.float32(bc.value), w
     return packed, np.float32(sc.value), np.float32(bc.value)
@@ -230,15 +245,16 @@ def _map(fn, items, threads: int):
         return list(ex.map(fn, items))
 
 
-def compress(variables, selected, E: int, M: int, pvt: bool = True, threads: int = 1) -> dict:
-    """Model state: {'E','M','pvt','n': [...], 'sel': [...], 'packed': {i: u8}, 's': {i: f32},
+def compress(variables, selected, E: int, M: int, pvt: bool = True, threads: int = 1,
+             fixed: bool = False) -> dict:
+    """Model state: {'E','M','fixed','pvt','n': [...], 'sel': [...], 'packed': {i: u8}, 's': {i: f32},
     'b': {i: f32}, 'fp32': {i: f32 array}} -- variables not selected stay in FP32 (Sec. 2.4)."""
-    st = {"E": E, "M": M, "pvt": pvt, "n": [int(np.asarray(v).size) for v in variables],
+    st = {"E": E, "M": M, "fixed": bool(fixed), "pvt": pvt, "n": [int(np.asarray(v).size) for v in variables],
           "sel": [bool(x) for x in selected], "packed": {}, "s": {}, "b": {}, "fp32": {}}
 
     def one(i):
         if st["sel"][i]:
-            return compress_var(variables[i], E, M, pvt)
+            return compress_var(variables[i], E, M, pvt, fixed)
         return np.array(variables[i], dtype=np.float32, copy=True).ravel()
 
     for i, r in enumerate(_map(one, range(len(variables)), threads)):
@@ -253,7 +269,7 @@ def decompress(st: dict, threads: int = 1) -> list:
     def one(i):
         if st["sel"][i]:
             return decompress_var(st["packed"][i], st["n"][i], st["E"], st["M"], st["s"][i],
-                                  st["b"][i])
+                                  st["b"][i], st.get("fixed", False))
         return st["fp32"][i].copy()
 
     return _map(one, range(len(st["n"])), threads)
@@ -264,7 +280,8 @@ def update_recompress(st: dict, grads, lr: float, threads: int = 1, want_w: bool
     def one(i):
         if st["sel"][i]:
             return update_recompress_var(st["packed"][i], st["n"][i], st["E"], st["M"], st["s"][i],
-                                         st["b"][i], grads[i], lr, st["pvt"], want_w=want_w)
+                                         st["b"][i], grads[i], lr, st["pvt"], want_w=want_w,
+                                         fixed=st.get("fixed", False))
         return sgd_var(st["fp32"][i], grads[i], lr)
 
     ws = []
