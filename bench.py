@@ -298,8 +298,8 @@ class FusedRun:
         return out
 
 
-def config_label(wl):
-    return "%s S1E%dM%d p=%g" % (wl.name, wl.fmt[0], wl.fmt[1], wl.fraction)
+def config_label(wl, fixed=False):
+    return "%s S1%s%d%s%d p=%g" % (wl.name, "I" if fixed else "E", wl.fmt[0], "F" if fixed else "M", wl.fmt[1], wl.fraction)
 
 
 def bench_other_config(name, local, dev, stream, seconds):
@@ -349,7 +349,8 @@ def run_ours(args):
     if args.fraction:
         wl.fraction = args.fraction
     flags = (0 if args.no_pvt else omc.PLAN_PVT) | (0 if args.all_variables else omc.PLAN_WEIGHTS_ONLY)
-    plan = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=wl.fraction, seed=wl.sel_seed, flags=flags)
+    plan = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=wl.fraction, seed=wl.sel_seed, flags=flags,
+                    fixed=args.fixed)
     stream = torch.cuda.current_stream().cuda_stream
     run = FusedRun(wl, plan, dev, stream)
     packed, resid, sb, ws, grads = run.packed, run.resid, run.sb, run.ws, run.grads
@@ -465,8 +466,8 @@ def run_ours(args):
                                                     "gbs": extra["decompress"]["gbs"] * extra["decompress"]["ms"] / t_ms}
 
         # re-selection between two random 90% subsets (Sec. 3.1), state A -> state B
-        pa = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=1)
-        pb = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=2)
+        pa = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=1, fixed=args.fixed)
+        pb = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=2, fixed=args.fixed)
         if pa.n_quantised and pa.quantised != pb.quantised:
             bufs = {}
             for nm, pl in (("a", pa), ("b", pb)):
@@ -498,7 +499,7 @@ def run_ours(args):
         K = 8
         cl = []
         for k in range(K):
-            pl = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=100 + k)
+            pl = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=100 + k, fixed=args.fixed)
             b4 = (z(pl.packed_bytes, torch.uint8), z(pl.resid_elems, torch.float32),
                   z(2 * pl.n_quantised, torch.float32), z(pl.workspace_bytes, torch.uint8))
             pl.prepare(b4[3].data_ptr(), stream)
@@ -561,7 +562,7 @@ def run_ours(args):
     # ---- the other target configurations as sub-records (default workload, one GPU only)
     other_configs = []
     if rank == 0 and world == 1 and args.workload == "conformer" and not args.no_other_configs and \
-            not (args.format or args.fraction or args.no_pvt or args.all_variables):
+            not (args.format or args.fixed or args.fraction or args.no_pvt or args.all_variables):
         del packed, resid, sb, ws, grads
         run.packed = run.resid = run.sb = run.ws = run.grads = None
         torch.cuda.empty_cache()
@@ -595,7 +596,7 @@ def run_ours(args):
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "ms_per_step_spread": spread,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": config_label(wl),
+        "config": {"workload": config_label(wl, args.fixed),
                    "params": nparams, "variables": plan.nvars, "quantised_variables": plan.n_quantised,
                    "bytes_per_step": step_bytes, "lr": wl.lr, "pvt": not args.no_pvt, "weights_only": not args.all_variables, "gradients": "one seeded buffer reused every step",
                    "l2": "inputs per step (%.0f MB) exceed the 126 MB L2; no flush" % (step_bytes / 1e6),
@@ -606,7 +607,7 @@ def run_ours(args):
                 "h2d_bytes_per_step": 4 * plan.full_elems, "d2h_bytes_per_step": 8 * plan.n_quantised,
                 "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
         "gpu_launches": args.steps,
-        "roofline": run.roofline(ms_per_step, None if (args.format or args.fraction or args.no_pvt or args.all_variables)
+        "roofline": run.roofline(ms_per_step, None if (args.format or args.fixed or args.fraction or args.no_pvt or args.all_variables)
                                  else wl.name),
         "sustained": sustained,
         "other_configs": other_configs,
@@ -626,6 +627,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="conformer")
     ap.add_argument("--format", default="", help="override the workload's format: E,M (e.g. 3,7 = S1E3M7)")
+    ap.add_argument("--fixed", action="store_true",
+                    help="read --format as I,F of the fixed-point variant S1IxFy (e.g. 0,15 = Q15)")
     ap.add_argument("--fraction", type=float, default=0.0, help="override the quantised fraction of weight matrices")
     ap.add_argument("--no-pvt", action="store_true", help="ablation: without the per-variable transformation")
     ap.add_argument("--all-variables", action="store_true", help="ablation: biases and norms are eligible too")

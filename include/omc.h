@@ -41,10 +41,23 @@ extern "C" {
  * 2 <= exp_bits <= 8, 0 <= man_bits <= 23 (so 3 <= B <= 32).  S1E8M23 is FP32, S1E5M10 is FP16
  * (Sec. 2.2, Sec. 3.4); the family is the IEEE-754 interchange parametrisation (bias
  * 2^(E-1)-1, gradual underflow, top exponent field = Inf/NaN), rounding to nearest, ties to even.
- * `flags` must be 0. */
+ * `flags` is 0 for these.
+ *
+ * flags == OMC_FORMAT_FIXED_POINT selects the fixed-point variant that Sec. 2.2 mentions as an
+ * alternative without defining it; the definition here is this library's.  S1IxFy: exp_bits = x
+ * integer bits (0 .. 8), man_bits = y fraction bits, 1 <= x + y <= 23, B = 1 + x + y.  A code is
+ * the B-bit two's complement of an integer k in [-2^(x+y), 2^(x+y) - 1] and stands for k * 2^-y.
+ * Encoding rounds value * 2^y to the nearest integer, ties to even, and saturates at both ends
+ * (there is no infinity; +-Inf saturate too); NaN has no code and becomes 0.  The scale is fixed
+ * by the format and not taken from the data (that would cost the one-pass update a second pass);
+ * the per-variable transformation of Sec. 2.3 adapts to the variable as it does for the
+ * floating-point codes.  Layouts, packing and every call are the same; omc_matmul accepts only
+ * floating-point codes.  Q7, Q11 and Q15 (x = 0) have compiled kernels; the other formats run on
+ * the slower kernels that take the format at run time. */
 typedef struct {
     uint8_t sign_bits, exp_bits, man_bits, flags;
 } omc_format_t;
+#define OMC_FORMAT_FIXED_POINT 1u
 
 /* What a variable is (Sec. 2.4): only weight matrices are ever quantised. */
 enum { OMC_KIND_WEIGHT_MATRIX = 0, OMC_KIND_BIAS = 1, OMC_KIND_NORM = 2, OMC_KIND_OTHER = 3 };

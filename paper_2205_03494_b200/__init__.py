@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libomc.so")
 KIND_WEIGHT_MATRIX, KIND_BIAS, KIND_NORM, KIND_OTHER = 0, 1, 2, 3
 PLAN_PVT, PLAN_WEIGHTS_ONLY = 1, 2
 PLAN_DEFAULT = PLAN_PVT | PLAN_WEIGHTS_ONLY
+FORMAT_FIXED_POINT = 1
 
 EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_seed", "omc_plan_sizes",
            "omc_plan_var", "omc_plan_division", "omc_plan_prepare", "omc_plan_status", "omc_plan_inject_wait_timeout", "omc_compress", "omc_decompress",
@@ -90,14 +91,17 @@ def _check(status: int, where: str):
 class Plan:
     """Handle of an ``omc_plan_t``; attributes mirror omc_plan_sizes / omc_plan_var."""
 
-    def __init__(self, numel, kinds, fmt, fraction=1.0, seed=0, mask=None, flags=PLAN_DEFAULT):
+    def __init__(self, numel, kinds, fmt, fraction=1.0, seed=0, mask=None, flags=PLAN_DEFAULT, fixed=False):
+        """fmt = (E, M) of S1EyMz, or with fixed=True (integer bits, fraction bits) of the fixed-point
+        variant S1IxFy."""
         n = len(numel)
         descs = (VarDesc * max(n, 1))()
         for i in range(n):
             descs[i].numel, descs[i].kind, descs[i].reserved = int(numel[i]), int(kinds[i]), 0
         S, E, M = (1, fmt[0], fmt[1]) if len(fmt) == 2 else fmt
         self.E, self.M, self.B = int(E), int(M), 1 + int(E) + int(M)
-        f = Format(S, E, M, 0)
+        f = Format(S, E, M, FORMAT_FIXED_POINT if fixed else 0)
+        self.fixed = bool(fixed)
         mk = None
         if mask is not None:
             mk = (C.c_uint8 * n)(*[1 if m else 0 for m in mask])
@@ -205,11 +209,12 @@ def aggregate(plans, packed, resid, sb, out, stream=0):
     _check(lib().omc_aggregate(arr(plans), k, arr(packed), arr(resid), arr(sb), out, stream), "omc_aggregate")
 
 
-def compress_var_static(values, numel, fmt, packed, sb, flags=PLAN_PVT, stream=0):
+def compress_var_static(values, numel, fmt, packed, sb, flags=PLAN_PVT, stream=0, fixed=False):
     """omc_compress_var_static: one variable, no plan, no workspace, no allocation (addresses are
     ints).  Raises OmcError like the other calls (status -8 = numel beyond STATIC_MAX_NUMEL)."""
     S, E, M = (1, fmt[0], fmt[1]) if len(fmt) == 2 else fmt
-    _check(lib().omc_compress_var_static(values, int(numel), Format(S, E, M, 0), int(flags), packed, sb,
+    _check(lib().omc_compress_var_static(values, int(numel), Format(S, E, M, FORMAT_FIXED_POINT if fixed else 0),
+                                         int(flags), packed, sb,
                                          stream), "omc_compress_var_static")
 
 

@@ -17,6 +17,7 @@ namespace omc {
 template <int E_, int M_>
 struct Fmt {
     static_assert(E_ >= 2 && E_ <= 8 && M_ >= 0 && M_ <= 23, "format outside the accepted family");
+    static constexpr bool FIXED = false;
     static constexpr int E = E_, M = M_, B = 1 + E_ + M_;
     static constexpr int BIAS = (1 << (E_ - 1)) - 1;
     static constexpr int EMIN = 1 - BIAS, EMAX = BIAS;
@@ -38,11 +39,33 @@ struct Fmt {
     static constexpr uint32_t OVF_BITS = ovf_bits();
 };
 
+// The fixed-point variant (Sec. 2.2 names fixed-point formats as an alternative without defining
+// one): S1IxFy, a B = 1 + x + y bit two's-complement integer k standing for k * 2^-y, rounded to
+// nearest even, saturating at both ends (there is no infinity), NaN -> 0.  E and M carry x and y
+// so that the layout code (B bits per code, LU elements per lane) needs no second set of names.
+// The fast forms below need every |k| <= 2^22 (x + y <= 22): the FP32 adder does the rounding to
+// an integer (adding 1.5 * 2^23 leaves k in the low mantissa bits, as a two's complement), and a
+// code with its sign bit flipped is an unsigned offset that drops straight into a mantissa.
+template <int I_, int F_>
+struct FixFmt {
+    static_assert(I_ >= 0 && I_ <= 8 && F_ >= 0 && I_ + F_ >= 1 && I_ + F_ <= 22, "fixed-point format outside the compiled family");
+    static constexpr bool FIXED = true;
+    static constexpr int E = I_, M = F_, B = 1 + I_ + F_;
+    static constexpr int SH = 0;
+    static constexpr uint32_t CODE_MASK = (1u << B) - 1u;
+    static constexpr uint32_t SIGN_BIT = 1u << (I_ + F_);
+    static constexpr uint32_t MAG_MASK = SIGN_BIT - 1u, INF_MAG = 0xFFFFFFFFu, OVF_BITS = 0x7F800000u;
+    static constexpr float SCALE = (float)(1u << F_), INV_SCALE = 1.f / (float)(1u << F_);
+    static constexpr float LO = -(float)(1u << (I_ + F_)), HI = (float)((1u << (I_ + F_)) - 1u);
+    static constexpr float MAGIC = 12582912.f;                    // 1.5 * 2^23
+    static constexpr float OFFSET = 8388608.f + (float)(1u << (I_ + F_));   // 2^23 + 2^(B-1)
+};
+
 // Formats with E = 5 and M <= 10 are FP16 with the low mantissa bits dropped: code << (10-M) is
 // an IEEE half, so the hardware half conversions do the exponent work (specials included).
 template <class F>
 struct HalfPath {
-    static constexpr bool value = (F::E == 5 && F::M <= 10);
+    static constexpr bool value = (!F::FIXED && F::E == 5 && F::M <= 10);
 };
 
 // Formats whose codes, below the top of the range, are those of a hardware narrow-float type
@@ -50,7 +73,7 @@ struct HalfPath {
 template <class F>
 struct Fp8Path {
     static constexpr bool value =
-        (F::E == 5 && F::M == 2) || (F::E == 4 && F::M == 3) || (F::E == 2 && F::M == 3);
+        !F::FIXED && ((F::E == 5 && F::M == 2) || (F::E == 4 && F::M == 3) || (F::E == 2 && F::M == 3));
 };
 
 __device__ __forceinline__ uint32_t f2u(float x) { return __float_as_uint(x); }
@@ -63,7 +86,11 @@ __device__ __forceinline__ float u2f(uint32_t u) { return __uint_as_float(u); }
 template <class F>
 __device__ __forceinline__ float decode_fast(uint32_t c)
 {
-    if constexpr (F::E == 8) {
+    if constexpr (F::FIXED) {
+        // 2^23 + (k + 2^(B-1)) as a float, then (that - 2^23 - 2^(B-1)) * 2^-y in one exact operation
+        const float f = u2f(c ^ (F::SIGN_BIT | 0x4B000000u));
+        return __fmaf_rn(f, F::INV_SCALE, -F::OFFSET * F::INV_SCALE);
+    } else if constexpr (F::E == 8) {
         return u2f(c << F::SH);      // S1E8Mz is FP32 with the low mantissa bits dropped
     } else if constexpr (HalfPath<F>::value) {
         return __half2float(__ushort_as_half((unsigned short)(c << (10 - F::M))));   // exact, all codes
@@ -80,7 +107,7 @@ __device__ __forceinline__ float decode_fast(uint32_t c)
 template <class F>
 __device__ __forceinline__ bool code_is_special(uint32_t c)
 {
-    if constexpr (F::E == 8 || HalfPath<F>::value) return false;   // decode_fast is already exact
+    if constexpr (F::FIXED || F::E == 8 || HalfPath<F>::value) return false;   // decode_fast is already exact
     return (c & F::MAG_MASK) >= F::INF_MAG;
 }
 
@@ -88,7 +115,7 @@ __device__ __forceinline__ bool code_is_special(uint32_t c)
 template <class F>
 __device__ __forceinline__ float decode_exact(uint32_t c)
 {
-    if constexpr (F::E < 8 && !HalfPath<F>::value) {
+    if constexpr (!F::FIXED && F::E < 8 && !HalfPath<F>::value) {
         if ((c & F::MAG_MASK) >= F::INF_MAG) {
             const uint32_t m = c & ((1u << F::M) - 1u);
             return u2f(((c >> (F::E + F::M)) << 31) | 0x7F800000u | (m << F::SH));
@@ -105,7 +132,14 @@ template <class F>
 __device__ __forceinline__ uint32_t encode_fast(float w, float &vt)
 {
     const uint32_t u = f2u(w);
-    if constexpr (F::M == 23 && F::E == 8) {
+    if constexpr (F::FIXED) {
+        // clamp (the bounds are integers, so clamping before the rounding is clamping after it),
+        // round to an integer with the adder, read k off the mantissa
+        const float t = fminf(fmaxf(__fmul_rn(w, F::SCALE), F::LO), F::HI);
+        const float r = __fadd_rn(t, F::MAGIC);
+        vt = __fmaf_rn(r, F::INV_SCALE, -F::MAGIC * F::INV_SCALE);     // (r - MAGIC) * 2^-y, exact
+        return f2u(r) & F::CODE_MASK;
+    } else if constexpr (F::M == 23 && F::E == 8) {
         vt = w;
         return u;
     } else if constexpr (HalfPath<F>::value && F::M == 10) {
@@ -190,6 +224,7 @@ template <class F, bool KEEP_PAYLOAD>
 __device__ __forceinline__ bool needs_exact_encode(float w)
 {
     const uint32_t a = f2u(w) & 0x7FFFFFFFu;
+    if constexpr (F::FIXED) return a > 0x7F800000u;          // NaN only: everything else saturates
     if constexpr (HalfPath<F>::value && F::M == 10) return KEEP_PAYLOAD ? (a > 0x7F800000u) : false;
     if constexpr (F::E == 8) return a > 0x7F800000u;
     return a >= F::OVF_BITS;
@@ -213,7 +248,7 @@ __device__ __forceinline__ float absmax4(float a, float b, float c, float d)
 template <class F>
 __device__ __forceinline__ bool any_code_special4(const float (&dec)[4])
 {
-    if constexpr (F::E == 8 || HalfPath<F>::value) return false;
+    if constexpr (F::FIXED || F::E == 8 || HalfPath<F>::value) return false;
     else return absmax4(dec[0], dec[1], dec[2], dec[3]) >= u2f(F::pow2_bits(F::EMAX + 1));
 }
 
@@ -223,7 +258,7 @@ __device__ __forceinline__ bool any_needs_exact_encode4(const float (&w)[4])
     if constexpr (HalfPath<F>::value && F::M == 10 && !KEEP_PAYLOAD) return false;
     else {
         const float m = absmax4(w[0], w[1], w[2], w[3]);
-        if constexpr ((HalfPath<F>::value && F::M == 10) || F::E == 8) return m != m;      // NaN only
+        if constexpr (F::FIXED || (HalfPath<F>::value && F::M == 10) || F::E == 8) return m != m;      // NaN only
         else return !(m < u2f(F::OVF_BITS));                                               // overflow, Inf, NaN
     }
 }
@@ -235,6 +270,13 @@ __device__ __forceinline__ uint32_t encode_exact(float w, float &vt)
 {
     const uint32_t u = f2u(w);
     const uint32_t a = u & 0x7FFFFFFFu;
+    if constexpr (F::FIXED) {
+        if (a > 0x7F800000u) {      // NaN has no code: it becomes 0
+            vt = 0.f;
+            return 0u;
+        }
+        return encode_fast<F>(w, vt);
+    }
     const uint32_t sign = (u >> 31) << (F::E + F::M);
     if (a > 0x7F800000u) {
         uint32_t c;
@@ -281,7 +323,7 @@ __device__ __forceinline__ uint32_t get_code_at(const uint32_t (&w)[NW], int pos
 template <class F, int NW>
 __device__ __forceinline__ float decode_fast_at(const uint32_t (&w)[NW], int pos)
 {
-    static_assert(F::E < 8 && !HalfPath<F>::value, "generic path");
+    static_assert(!F::FIXED && F::E < 8 && !HalfPath<F>::value, "generic path");
     const int wi = pos >> 5, sh = pos & 31;
     uint32_t t;      // the code in the top B bits
     if (sh + F::B <= 32)

@@ -3,20 +3,32 @@
 // through 32 consecutive elements with a streaming bit reader / writer straight on global memory.
 // Same results, layouts, tile partition and fit as the specialised kernels; an order of magnitude
 // slower, which is the price of covering all of 2 <= E <= 8, 0 <= M <= 23 without 168 builds.
+#include <cmath>
+
 #include "kernels.cuh"
 
 namespace omc {
 
 struct DynFmt {
+    int fixed;               // the fixed-point variant S1IxFy: E = x, M = y
+    float scale, inv_scale, lo, hi;      // 2^y, 2^-y, -2^(x+y), 2^(x+y) - 1
     int E, M, B, SH;
     uint32_t mag_mask, inf_mag, ovf_bits, min_normal_bits, clamp_bits;
     float up, down, xs;      // 2^(127-BIAS), 2^(BIAS-127), 2^SH
 };
 
-static DynFmt make_dyn(int E, int M)
+static DynFmt make_dyn(int E, int M, int fixed)
 {
     DynFmt f{};
     f.E = E; f.M = M; f.B = 1 + E + M; f.SH = 23 - M;
+    f.fixed = fixed;
+    if (fixed) {
+        f.scale = std::ldexp(1.f, M);
+        f.inv_scale = std::ldexp(1.f, -M);
+        f.lo = -std::ldexp(1.f, E + M);
+        f.hi = std::ldexp(1.f, E + M) - 1.f;
+        return f;
+    }
     const int bias = (1 << (E - 1)) - 1, emin = 1 - bias, emax = bias;
     auto p2 = [](int k) { return (uint32_t)(k + 127) << 23; };
     auto asf = [](uint32_t u) { float x; memcpy(&x, &u, 4); return x; };
@@ -35,6 +47,10 @@ static DynFmt make_dyn(int E, int M)
 
 __device__ __forceinline__ float dyn_decode(const DynFmt &f, uint32_t c)
 {
+    if (f.fixed) {      // two's complement, k * 2^-y
+        const int k = (int)(c << (32 - f.B)) >> (32 - f.B);
+        return __fmul_rn((float)k, f.inv_scale);
+    }
     if (f.E == 8) return u2f(c << f.SH);
     const uint32_t mag = c & f.mag_mask;
     const uint32_t sign = (c >> (f.E + f.M)) << 31;
@@ -46,6 +62,12 @@ __device__ __forceinline__ float dyn_decode(const DynFmt &f, uint32_t c)
 __device__ __forceinline__ uint32_t dyn_encode(const DynFmt &f, float w, float &vt)
 {
     const uint32_t u = f2u(w), a = u & 0x7FFFFFFFu;
+    if (f.fixed) {      // nearest integer multiple of 2^-y, ties to even, saturating; NaN -> 0
+        if (a > 0x7F800000u) { vt = 0.f; return 0u; }
+        const int k = __float2int_rn(fminf(fmaxf(__fmul_rn(w, f.scale), f.lo), f.hi));
+        vt = __fmul_rn((float)k, f.inv_scale);
+        return (uint32_t)k & ((1u << f.B) - 1u);
+    }
     const uint32_t sign = (u >> 31) << (f.E + f.M);
     if (a > 0x7F800000u) {
         uint32_t c = sign | f.inf_mag;
@@ -169,10 +191,10 @@ __global__ void __launch_bounds__(THREADS) omc_dyn_kernel(const KParams p, const
 template <int MODE, bool WOUT>
 static void launch_dyn(const KParams &p, int grid, void *stream)
 {
-    omc_dyn_kernel<MODE, WOUT><<<grid, THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p, make_dyn((int)p.dyn_e, (int)p.dyn_m));
+    omc_dyn_kernel<MODE, WOUT><<<grid, THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p, make_dyn((int)p.dyn_e, (int)p.dyn_m, (int)p.dyn_fixed));
 }
 
-extern const FmtOps ops_dynamic = {-1, -1, launch_dyn<COMPRESS, false>, launch_dyn<DECOMPRESS, false>,
+extern const FmtOps ops_dynamic = {-1, -1, -1, launch_dyn<COMPRESS, false>, launch_dyn<DECOMPRESS, false>,
                                    launch_dyn<UPDATE, false>, launch_dyn<UPDATE, true>, nullptr, nullptr, nullptr};
 
 }  // namespace omc

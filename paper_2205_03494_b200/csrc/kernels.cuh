@@ -344,7 +344,7 @@ __device__ __forceinline__ void compute_group(const uint32_t (&win)[NWI], int g,
 {
     constexpr bool HAS_CIN = (MODE != COMPRESS);
     constexpr bool KEEP_PAYLOAD = (MODE == COMPRESS);    // UPDATE gives arithmetic NaNs one pattern
-    constexpr bool GENERIC = F::E < 8 && !HalfPath<F>::value;   // codes are isolated only on the careful path
+    constexpr bool GENERIC = !F::FIXED && F::E < 8 && !HalfPath<F>::value;   // codes are isolated only on the careful path
     uint32_t cin[4], cout[4];
     float vt[4];
     bool bad = false;
@@ -1578,7 +1578,7 @@ __global__ void __launch_bounds__(THREADS, Unit<F>::LU == 32 ? CTAS_PER_SM : 4) 
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) x[4 * g + j] = __fmaf_rn(c.s, dec[j], c.b);
                             }
-                        } else if constexpr (F::E < 8 && !HalfPath<F>::value) {
+                        } else if constexpr (!F::FIXED && F::E < 8 && !HalfPath<F>::value) {
                             // generic path: decode from the word, test four values at once for Inf/NaN codes
 #pragma unroll
                             for (int g = 0; g < AL / 4; ++g) {
@@ -1623,8 +1623,17 @@ void launch_aggregate(const AggParams &p, int grid, void *stream)
     omc_aggregate_kernel<F><<<grid, THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p);
 }
 
+#define OMC_DEFINE_FIXED_FORMAT(I_, F_)                                                         \
+    extern const FmtOps ops_I##I_##F##F_ = {I_, F_, 1, launch<FixFmt<I_, F_>, COMPRESS, false>, \
+                                            launch<FixFmt<I_, F_>, DECOMPRESS, false>,          \
+                                            launch<FixFmt<I_, F_>, UPDATE, false>,              \
+                                            launch<FixFmt<I_, F_>, UPDATE, true>,               \
+                                            launch<FixFmt<I_, F_>, UPDATE, false, true>,        \
+                                            launch_transition<FixFmt<I_, F_>>,                  \
+                                            launch_aggregate<FixFmt<I_, F_>>};
+
 #define OMC_DEFINE_FORMAT(E_, M_)                                                               \
-    extern const FmtOps ops_E##E_##M##M_ = {E_, M_, launch<Fmt<E_, M_>, COMPRESS, false>,       \
+    extern const FmtOps ops_E##E_##M##M_ = {E_, M_, 0, launch<Fmt<E_, M_>, COMPRESS, false>,    \
                                             launch<Fmt<E_, M_>, DECOMPRESS, false>,             \
                                             launch<Fmt<E_, M_>, UPDATE, false>,                 \
                                             launch<Fmt<E_, M_>, UPDATE, true>,                  \

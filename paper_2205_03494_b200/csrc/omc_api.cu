@@ -15,14 +15,20 @@ int note_cuda(cudaError_t e);
     X(3, 9) X(4, 8) X(5, 7)          /* the 13-bit formats of Sec. 3.5.3                      */ \
     X(8, 7) X(8, 23)                 /* bfloat16 and FP32 itself                              */
 OMC_FORMAT_LIST(OMC_DECLARE_FORMAT)
-extern const FmtOps ops_dynamic;   // any other format of the family, at run time
+// the fixed-point variant (Sec. 2.2): Q7, Q11 and Q15, the widths of the benchmark configurations
+#define OMC_DECLARE_FIXED_FORMAT(I_, F_) extern const FmtOps ops_I##I_##F##F_;
+#define OMC_FIXED_FORMAT_LIST(X) X(0, 7) X(0, 11) X(0, 15)
+OMC_FIXED_FORMAT_LIST(OMC_DECLARE_FIXED_FORMAT)
+extern const FmtOps ops_dynamic;   // any other format of either family, at run time
 
-const FmtOps *find_ops(int E, int M)
+const FmtOps *find_ops(int E, int M, int fixed)
 {
 #define OMC_ADDR(E_, M_) &ops_E##E_##M##M_,
-    static const FmtOps *const table[] = {OMC_FORMAT_LIST(OMC_ADDR)};
+#define OMC_FIXED_ADDR(I_, F_) &ops_I##I_##F##F_,
+    static const FmtOps *const table[] = {OMC_FORMAT_LIST(OMC_ADDR) OMC_FIXED_FORMAT_LIST(OMC_FIXED_ADDR)};
     for (const FmtOps *o : table)
-        if (o->E == E && o->M == M) return o;
+        if (o->E == E && o->M == M && o->fixed == (fixed ? 1 : 0)) return o;
+    if (fixed) return fixed_format_ok(E, M) ? &ops_dynamic : nullptr;
     if (E >= 2 && E <= 8 && M >= 0 && M <= 23) return &ops_dynamic;
     return nullptr;
 }
@@ -125,6 +131,7 @@ static KParams whole_model(const omc_plan_t *plan, void *workspace)
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
     p.dyn_e = plan->fmt.exp_bits;
     p.dyn_m = plan->fmt.man_bits;
+    p.dyn_fixed = plan->fmt.flags & OMC_FORMAT_FIXED_POINT;
     p.status = plan->d_status;
     p.queue = static_cast<uint32_t *>(workspace);       // the workspace header
     p.tickets = reinterpret_cast<uint32_t *>(static_cast<char *>(workspace) + plan->ws_tickets_off);
@@ -202,6 +209,7 @@ extern "C" int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, con
     p.pvt = (plan->flags & OMC_PLAN_PVT) ? 1u : 0u;
     p.dyn_e = plan->fmt.exp_bits;
     p.dyn_m = plan->fmt.man_bits;
+    p.dyn_fixed = plan->fmt.flags & OMC_FORMAT_FIXED_POINT;
     p.status = plan->d_status;
     p.packed = const_cast<uint8_t *>(packed);
     p.resid = const_cast<float *>(resid);
@@ -284,7 +292,8 @@ extern "C" int omc_transition(const omc_plan_t *from, const omc_plan_t *to, cons
     if (rc) return rc;
     rc = check_ready(to);
     if (rc) return rc;
-    if (from->nvars != to->nvars || from->fmt.exp_bits != to->fmt.exp_bits || from->fmt.man_bits != to->fmt.man_bits)
+    if (from->nvars != to->nvars || from->fmt.exp_bits != to->fmt.exp_bits || from->fmt.man_bits != to->fmt.man_bits ||
+        from->fmt.flags != to->fmt.flags)
         return OMC_ERR_PLAN_MISMATCH;
     for (uint32_t i = 0; i < to->nvars; ++i)
         if (from->vars[i].n != to->vars[i].n) return OMC_ERR_PLAN_MISMATCH;
@@ -335,7 +344,7 @@ extern "C" int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients,
         int rc = check_ready(pl);
         if (rc) return rc;
         if (pl->nvars != first->nvars || pl->fmt.exp_bits != first->fmt.exp_bits ||
-            pl->fmt.man_bits != first->fmt.man_bits)
+            pl->fmt.man_bits != first->fmt.man_bits || pl->fmt.flags != first->fmt.flags)
             return OMC_ERR_PLAN_MISMATCH;
         for (uint32_t i = 0; i < pl->nvars; ++i)
             if (pl->vars[i].n != first->vars[i].n) return OMC_ERR_PLAN_MISMATCH;

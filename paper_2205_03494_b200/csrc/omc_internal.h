@@ -68,6 +68,7 @@ struct KParams {
     const uint32_t *run_var;
     uint32_t pvt;
     uint32_t dyn_e, dyn_m;         // the format, for the kernels that take it at run time
+    uint32_t dyn_fixed;            // ... and whether it is the fixed-point variant (then integer / fraction bits)
     uint8_t *packed;
     float *resid;
     float *sb;
@@ -133,7 +134,8 @@ struct AggParams {
 };
 
 struct FmtOps {
-    int E, M;
+    int E, M;          // fixed != 0: integer bits and fraction bits of S1IxFy
+    int fixed;
     void (*compress)(const KParams &, int grid, void *stream);
     void (*decompress)(const KParams &, int grid, void *stream);
     void (*update)(const KParams &, int grid, void *stream);     // W not stored
@@ -142,7 +144,9 @@ struct FmtOps {
     void (*transition)(const KParams &, int grid, void *stream); // plan-to-plan; NULL if unsupported
     void (*aggregate)(const AggParams &, int grid, void *stream); // mean of replicas; NULL if unsupported
 };
-const FmtOps *find_ops(int E, int M);
+const FmtOps *find_ops(int E, int M, int fixed);
+// Limits of the fixed-point variant S1IxFy (every value k * 2^-y must be an FP32 value).
+inline bool fixed_format_ok(int I, int F) { return I >= 0 && I <= 8 && F >= 0 && I + F >= 1 && I + F <= 23; }
 
 // Divides the tiles of vars[0 .. nvars) (n, quantised, tile_start and ntiles filled in) into nruns
 // contiguous runs of about equal estimated cost: writes run_start[0 .. nruns], run_var[0 .. nruns)

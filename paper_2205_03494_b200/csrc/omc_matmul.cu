@@ -446,6 +446,7 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     if (!packed || !sb || !x_half || !y || !rowsum_scratch) return OMC_ERR_NULL_PTR;
     if (var >= plan->nvars || !plan->vars[var].quantised) return OMC_ERR_INVALID_ARG;
     const int exp = plan->fmt.exp_bits, man = plan->fmt.man_bits;
+    if (plan->fmt.flags) return OMC_ERR_BAD_FORMAT;          // floating-point codes only
     const bool half_family = exp == 5 && (man == 10 || man == 6 || man == 2);
     const bool narrow = (exp == 4 && man == 3) || (exp == 2 && man == 3);
     if (!half_family && !narrow) return OMC_ERR_BAD_FORMAT;

@@ -145,9 +145,12 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
     *out = nullptr;
     if (nvars == 0) return OMC_ERR_INVALID_ARG;
     if (flags & ~(uint32_t)OMC_PLAN_DEFAULT) return OMC_ERR_INVALID_ARG;
-    if (fmt.sign_bits != 1 || fmt.exp_bits < 2 || fmt.exp_bits > 8 || fmt.man_bits > 23 || fmt.flags != 0)
+    if (fmt.sign_bits != 1 || (fmt.flags & ~OMC_FORMAT_FIXED_POINT)) return OMC_ERR_BAD_FORMAT;
+    const int fixed = (fmt.flags & OMC_FORMAT_FIXED_POINT) ? 1 : 0;
+    if (fixed ? !omc::fixed_format_ok(fmt.exp_bits, fmt.man_bits)
+              : (fmt.exp_bits < 2 || fmt.exp_bits > 8 || fmt.man_bits > 23))
         return OMC_ERR_BAD_FORMAT;
-    const omc::FmtOps *ops = omc::find_ops(fmt.exp_bits, fmt.man_bits);
+    const omc::FmtOps *ops = omc::find_ops(fmt.exp_bits, fmt.man_bits, fixed);
     if (!ops) return OMC_ERR_BAD_FORMAT;
     if (!mask && !(fraction > 0.0 && fraction <= 1.0)) return OMC_ERR_INVALID_ARG;
     for (uint32_t i = 0; i < nvars; ++i)

@@ -120,9 +120,12 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     if (flags & ~(uint32_t)OMC_PLAN_PVT) return OMC_ERR_INVALID_ARG;
     if (numel == 0) return OMC_ERR_INVALID_ARG;
     if (numel > OMC_STATIC_MAX_NUMEL) return OMC_ERR_TOO_LARGE;
-    if (fmt.sign_bits != 1 || fmt.exp_bits < 2 || fmt.exp_bits > 8 || fmt.man_bits > 23 || fmt.flags != 0)
+    if (fmt.sign_bits != 1 || (fmt.flags & ~OMC_FORMAT_FIXED_POINT)) return OMC_ERR_BAD_FORMAT;
+    const int fixed = (fmt.flags & OMC_FORMAT_FIXED_POINT) ? 1 : 0;
+    if (fixed ? !omc::fixed_format_ok(fmt.exp_bits, fmt.man_bits)
+              : (fmt.exp_bits < 2 || fmt.exp_bits > 8 || fmt.man_bits > 23))
         return OMC_ERR_BAD_FORMAT;
-    const omc::FmtOps *ops = omc::find_ops(fmt.exp_bits, fmt.man_bits);
+    const omc::FmtOps *ops = omc::find_ops(fmt.exp_bits, fmt.man_bits, fixed);
     if (!ops) return OMC_ERR_BAD_FORMAT;
 
     unsigned char *scratch = nullptr;
@@ -161,6 +164,7 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     p.pvt = (flags & OMC_PLAN_PVT) ? 1u : 0u;
     p.dyn_e = fmt.exp_bits;
     p.dyn_m = fmt.man_bits;
+    p.dyn_fixed = (uint32_t)fixed;
     p.packed = packed;
     p.resid = nullptr;
     p.sb = sb;

@@ -28,10 +28,11 @@ class Lockstep:
     """Runs the oracle and the GPU side by side on a (sub)set of variables and compares."""
 
     def __init__(self, numel, kinds, fmt, params, *, fraction=1.0, seed=0, mask=None,
-                 flags=omc.PLAN_DEFAULT, sample=None, threads=4):
+                 flags=omc.PLAN_DEFAULT, sample=None, threads=4, fixed=False):
         self.E, self.M = fmt
+        self.fixed = fixed
         self.B = 1 + self.E + self.M
-        self.plan = omc.Plan(numel, kinds, fmt, fraction=fraction, seed=seed, mask=mask, flags=flags)
+        self.plan = omc.Plan(numel, kinds, fmt, fraction=fraction, seed=seed, mask=mask, flags=flags, fixed=fixed)
         self.pvt = bool(flags & omc.PLAN_PVT)
         self.dm = DeviceModel(self.plan)
         self.idx = list(range(len(numel))) if sample is None else list(sample)
@@ -44,7 +45,7 @@ class Lockstep:
         self.dm.compress(full)
         del full
         sel = [self.plan.quantised[i] for i in self.idx]
-        self.st = orc.compress([params[i] for i in self.idx], sel, self.E, self.M, self.pvt, threads)
+        self.st = orc.compress([params[i] for i in self.idx], sel, self.E, self.M, self.pvt, threads, fixed=fixed)
         self.check_state("compress")
 
     def check_state(self, what, resync=True):
@@ -66,7 +67,7 @@ class Lockstep:
                         # an ulp of the tiny b: 4 n 2^-53 mean|V| bounds it (worst-case summation).
                         n = self.plan.numel[i]
                         scale = float(np.mean(np.abs(orc.decompress_var(
-                            self.st["packed"][k], n, self.E, self.M, self.st["s"][k], self.st["b"][k]))))
+                            self.st["packed"][k], n, self.E, self.M, self.st["s"][k], self.st["b"][k], self.fixed))))
                         assert abs(float(g) - float(w)) <= 4 * n * 2.0 ** -53 * scale, (what, i, g, w, scale)
                         self.b_cancellation_cases += 1
                         fix.append((i, k))
@@ -381,7 +382,8 @@ def oracle_transition(st, sel_to):
     """The oracle's state under another selection, composed from its own operations: released
     variables are decompressed, newly selected ones compressed, the others kept."""
     E, M, pvt = st["E"], st["M"], st["pvt"]
-    new = {"E": E, "M": M, "pvt": pvt, "n": list(st["n"]), "sel": [bool(x) for x in sel_to],
+    fixed = st.get("fixed", False)
+    new = {"E": E, "M": M, "fixed": fixed, "pvt": pvt, "n": list(st["n"]), "sel": [bool(x) for x in sel_to],
            "packed": {}, "s": {}, "b": {}, "fp32": {}}
     for i, n in enumerate(st["n"]):
         was, now = st["sel"][i], bool(sel_to[i])
@@ -390,9 +392,9 @@ def oracle_transition(st, sel_to):
         elif not was and not now:
             new["fp32"][i] = st["fp32"][i]
         elif was:
-            new["fp32"][i] = orc.decompress_var(st["packed"][i], n, E, M, st["s"][i], st["b"][i])
+            new["fp32"][i] = orc.decompress_var(st["packed"][i], n, E, M, st["s"][i], st["b"][i], fixed)
         else:
-            new["packed"][i], new["s"][i], new["b"][i] = orc.compress_var(st["fp32"][i], E, M, pvt)
+            new["packed"][i], new["s"][i], new["b"][i] = orc.compress_var(st["fp32"][i], E, M, pvt, fixed)
     return new
 
 

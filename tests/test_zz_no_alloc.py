@@ -17,10 +17,10 @@ from harness import ulp_diff
 pytestmark = pytest.mark.gpu
 
 
-def reference(values: torch.Tensor, fmt, flags):
+def reference(values: torch.Tensor, fmt, flags, fixed=False):
     """omc_compress on a plan holding just this variable."""
     n = values.numel()
-    plan = omc.Plan([n], [omc.KIND_WEIGHT_MATRIX], fmt, flags=flags | omc.PLAN_WEIGHTS_ONLY)
+    plan = omc.Plan([n], [omc.KIND_WEIGHT_MATRIX], fmt, flags=flags | omc.PLAN_WEIGHTS_ONLY, fixed=fixed)
     dev = values.device
     packed = torch.zeros(plan.packed_bytes, dtype=torch.uint8, device=dev)
     resid = torch.zeros(16, dtype=torch.float32, device=dev)
@@ -34,14 +34,14 @@ def reference(values: torch.Tensor, fmt, flags):
     return packed.cpu().numpy(), sb.cpu().numpy()
 
 
-def static_call(values: torch.Tensor, fmt, flags):
+def static_call(values: torch.Tensor, fmt, flags, fixed=False):
     n = values.numel()
     B = 1 + fmt[0] + fmt[1]
     nbytes = ((n * B + 7) // 8 + 15) // 16 * 16
     packed = torch.full((nbytes,), 0xAB, dtype=torch.uint8, device=values.device)   # must be overwritten
     sb = torch.full((2,), 7.0, dtype=torch.float32, device=values.device)
     omc.compress_var_static(values.data_ptr(), n, fmt, packed.data_ptr(), sb.data_ptr(), flags=flags,
-                            stream=torch.cuda.current_stream().cuda_stream)
+                            stream=torch.cuda.current_stream().cuda_stream, fixed=fixed)
     torch.cuda.synchronize()
     assert omc.static_status(torch.cuda.current_stream().cuda_stream) == 0
     return packed.cpu().numpy(), sb.cpu().numpy()
@@ -57,18 +57,19 @@ def padded(n, gen, scale):
 def test_two_calls_in_a_row_match_omc_compress():
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234)
-    calls = [(3_000_001, (5, 10), omc.PLAN_PVT, 0.05),      # many warps, ragged end
-             (70_001, (5, 2), omc.PLAN_PVT, 0.3),           # fewer warps than the first call used
-             (513, (5, 6), 0, 0.02),                        # no transformation: s = 1, b = 0
-             (1, (4, 3), omc.PLAN_PVT, 1.0)]                # a single element
-    for n, fmt, flags, scale in calls:
+    calls = [(3_000_001, (5, 10), omc.PLAN_PVT, 0.05, False),      # many warps, ragged end
+             (70_001, (5, 2), omc.PLAN_PVT, 0.3, False),           # fewer warps than the first call used
+             (513, (5, 6), 0, 0.02, False),                        # no transformation: s = 1, b = 0
+             (200_003, (0, 11), omc.PLAN_PVT, 0.3, True),          # the fixed-point variant
+             (1, (4, 3), omc.PLAN_PVT, 1.0, False)]                # a single element
+    for n, fmt, flags, scale, fixed in calls:
         v = padded(n, gen, scale)
-        got_p, got_sb = static_call(v, fmt, flags)
-        want_p, want_sb = reference(v, fmt, flags)
+        got_p, got_sb = static_call(v, fmt, flags, fixed)
+        want_p, want_sb = reference(v, fmt, flags, fixed)
         assert np.array_equal(got_p, want_p), (n, fmt)
         assert np.array_equal(got_sb.view(np.uint32), want_sb.view(np.uint32)), (n, fmt, got_sb, want_sb)
         # and against the CPU oracle itself, so that a defect shared by both entry points shows
-        orc_p, orc_s, orc_b = orc.compress_var(v.cpu().numpy(), fmt[0], fmt[1], bool(flags & omc.PLAN_PVT))
+        orc_p, orc_s, orc_b = orc.compress_var(v.cpu().numpy(), fmt[0], fmt[1], bool(flags & omc.PLAN_PVT), fixed)
         assert np.array_equal(got_p, orc_p), (n, fmt)
         assert ulp_diff(got_sb[0], orc_s) <= 1 and ulp_diff(got_sb[1], orc_b) <= 1, (n, fmt, got_sb, orc_s, orc_b)
     # same input twice through the shared array: identical bytes
