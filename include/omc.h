@@ -261,6 +261,22 @@ int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint
                   const float *const *resid, const float *const *sb, float *out, void *stream);
 
 /*
+ * omc_aggregate_sum / omc_divide -- the same aggregation (Sec. 1, Sec. 2.5) when the clients'
+ * models sit on several GPUs.  Each GPU adds up its own clients with omc_aggregate_sum
+ * (out[e] = x_0[e] + ... + x_{K-1}[e], FP32, its clients in index order, no division; arguments
+ * as for omc_aggregate), the per-GPU sums are added across GPUs by the caller's collective (one
+ * all-reduce over `out`, which every GPU owns a full copy of: this library hands no memory of
+ * another GPU to any kernel), and omc_divide turns the total into the mean: values[e] /= divisor,
+ * one correctly rounded FP32 division, over a buffer in the plan's full layout (1 <= divisor <=
+ * 2^24: the total number of clients).  The order in which a collective adds the per-GPU sums is
+ * not defined, so with three or more GPUs the result can differ from omc_aggregate over all
+ * clients in the last bits: by at most (K - 1) * 2^-24 * sum_k |x_k[e]| / K for K clients.
+ */
+int omc_aggregate_sum(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
+                      const float *const *resid, const float *const *sb, float *out, void *stream);
+int omc_divide(const omc_plan_t *plan, float *values, uint32_t divisor, void *stream);
+
+/*
  * omc_matmul -- forward path of Fig. 1 with the decompression fused into the consumer (Sec. 2.1:
  * a layer's parameters are decompressed only when the layer needs them; here they never exist in
  * FP32 at all).  For variable `var` of the plan, read as an N x K matrix W (K contiguous):

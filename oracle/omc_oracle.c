@@ -431,6 +431,27 @@ void orc_aggregate_var(const float *const *x, uint32_t K, uint64_t n, float *out
     }
 }
 
+/*
+ * The same mean taken in two stages, for clients spread over several servers or GPUs: each holder
+ * adds up its own clients (client order, FP32, no division), the holders' sums are added in holder
+ * order, and the total is divided once by the number of all clients.  With one holder this is
+ * orc_aggregate_var.  (A reading like the mean itself; across holders the order of the additions
+ * is whatever the transport does, so a real run is only bounded by, not equal to, this order.)
+ */
+void orc_sum_var(const float *const *x, uint32_t K, uint64_t n, float *out)
+{
+    for (uint64_t e = 0; e < n; ++e) {
+        float acc = x[0][e];
+        for (uint32_t k = 1; k < K; ++k) acc = acc + x[k][e];
+        out[e] = acc;
+    }
+}
+
+void orc_divide_var(const float *x, uint64_t n, uint32_t K, float *out)
+{
+    for (uint64_t e = 0; e < n; ++e) out[e] = x[e] / (float)K;
+}
+
 /* ------------------------------------------------------------------------------------------ */
 /* Selection (Sec. 2.4, 2.5, 3.1) and size accounting (Tables 1 and 2).                         */
 

@@ -77,6 +77,8 @@ def lib():
                                                 f32p, f32p, C.c_float, f32p]
         L.orc_sgd_var.argtypes = [f32p, f32p, C.c_uint64, C.c_float]
         L.orc_aggregate_var.argtypes = [C.POINTER(f32p), C.c_uint32, C.c_uint64, f32p]
+        L.orc_sum_var.argtypes = [C.POINTER(f32p), C.c_uint32, C.c_uint64, f32p]
+        L.orc_divide_var.argtypes = [f32p, C.c_uint64, C.c_uint32, f32p]
         L.orc_splitmix64.argtypes = [C.c_uint64, C.c_uint32]
         L.orc_splitmix64.restype = C.c_uint64
         L.orc_plan_seed.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32]
@@ -201,6 +203,35 @@ def aggregate_var(client_values) -> np.ndarray:
     out = np.empty(n, np.float32)
     lib().orc_aggregate_var(ptrs, len(xs), n, _p(out, C.c_float))
     return out
+
+
+def sum_var(client_values) -> np.ndarray:
+    """Un-divided FP32 sum of one variable over clients, in index order."""
+    xs = [_f32(x).ravel() for x in client_values]
+    n = xs[0].size
+    ptrs = (C.POINTER(C.c_float) * len(xs))(*[_p(x, C.c_float) for x in xs])
+    out = np.empty(n, np.float32)
+    lib().orc_sum_var(ptrs, len(xs), n, _p(out, C.c_float))
+    return out
+
+
+def divide_var(x, K: int) -> np.ndarray:
+    x = _f32(x).ravel()
+    out = np.empty(x.size, np.float32)
+    lib().orc_divide_var(_p(x, C.c_float), x.size, K, _p(out, C.c_float))
+    return out
+
+
+def aggregate_two_stage(states_by_holder, threads: int = 1) -> list:
+    """Mean over the clients of several holders (servers, GPUs): per-holder sums in client order,
+    the holders' sums added in holder order, one division by the number of all clients."""
+    holders = [h for h in states_by_holder if h]
+    k_total = sum(len(h) for h in holders)
+    sums = []
+    for h in holders:
+        dec = [decompress(st, threads) for st in h]
+        sums.append([sum_var([d[i] for d in dec]) for i in range(len(dec[0]))])
+    return [divide_var(sum_var([s[i] for s in sums]), k_total) for i in range(len(sums[0]))]
 
 
 def aggregate(states, threads: int = 1) -> list:

@@ -1485,7 +1485,7 @@ __global__ void __launch_bounds__(THREADS, Unit<F>::LU == 32 ? CTAS_PER_SM : 4) 
     // rounded value of the same real number.
     const bool pow2 = (p.nclients & (p.nclients - 1)) == 0;
     const float kinv = 1.f / kf;
-    auto mean_of = [&](float a) { return pow2 ? __fmul_rn(a, kinv) : __fdiv_rn(a, kf); };
+    auto mean_of = [&](float a) { return !p.divide ? a : pow2 ? __fmul_rn(a, kinv) : __fdiv_rn(a, kf); };
     // per warp: what the unit loop needs to know about each client's copy of the current variable
     struct ClientVar { uint64_t base; uint32_t nwords; uint32_t quantised; float s, b; uint32_t pad[2]; };
     __shared__ ClientVar cv_all[WARPS_PER_CTA][MAX_CLIENTS];

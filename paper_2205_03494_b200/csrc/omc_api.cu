@@ -331,8 +331,8 @@ extern "C" int omc_transition(const omc_plan_t *from, const omc_plan_t *to, cons
     return omc::note_cuda(cudaGetLastError());
 }
 
-extern "C" int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
-                             const float *const *resid, const float *const *sb, float *out, void *stream)
+static int aggregate_impl(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
+                          const float *const *resid, const float *const *sb, float *out, uint32_t divide, void *stream)
 {
     if (!plans || !packed || !resid || !sb || !out) return OMC_ERR_NULL_PTR;
     if (n_clients == 0 || n_clients > (uint32_t)omc::MAX_CLIENTS) return OMC_ERR_INVALID_ARG;
@@ -358,11 +358,59 @@ extern "C" int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients,
     }
     if (!first->ops->aggregate) return OMC_ERR_BAD_FORMAT;
     p.nclients = n_clients;
+    p.divide = divide;
     p.nvars = first->nvars;
     p.tile_count = first->ntiles;
     const uint64_t max_warps = (uint64_t)first->n_cta * omc::WARPS_PER_CTA * 2;    // light kernel: 4 CTAs per SM fit
     p.nwarps = (uint32_t)(p.tile_count < max_warps ? p.tile_count : max_warps);
     p.out = out;
     first->ops->aggregate(p, grid_for(p.nwarps), stream);
+    return omc::note_cuda(cudaGetLastError());
+}
+
+extern "C" int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
+                             const float *const *resid, const float *const *sb, float *out, void *stream)
+{
+    return aggregate_impl(plans, n_clients, packed, resid, sb, out, 1u, stream);
+}
+
+extern "C" int omc_aggregate_sum(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
+                                 const float *const *resid, const float *const *sb, float *out, void *stream)
+{
+    return aggregate_impl(plans, n_clients, packed, resid, sb, out, 0u, stream);
+}
+
+namespace {
+// out[e] = out[e] / divisor, one correctly rounded FP32 division per element (a multiplication by
+// the exact reciprocal when the divisor is a power of two: the same real number, rounded once).
+__global__ void divide_kernel(float4 *__restrict__ x, uint64_t n4, float divisor, int pow2)
+{
+    const float inv = 1.f / divisor;
+    for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n4; i += (uint64_t)gridDim.x * blockDim.x) {
+        float4 v = x[i];
+        if (pow2) {
+            v.x = __fmul_rn(v.x, inv); v.y = __fmul_rn(v.y, inv); v.z = __fmul_rn(v.z, inv); v.w = __fmul_rn(v.w, inv);
+        } else {
+            v.x = __fdiv_rn(v.x, divisor); v.y = __fdiv_rn(v.y, divisor);
+            v.z = __fdiv_rn(v.z, divisor); v.w = __fdiv_rn(v.w, divisor);
+        }
+        x[i] = v;
+    }
+}
+}  // namespace
+
+extern "C" int omc_divide(const omc_plan_t *plan, float *values, uint32_t divisor, void *stream)
+{
+    int rc = check_ready(plan);
+    if (rc) return rc;
+    if (!values) return OMC_ERR_NULL_PTR;
+    if (misaligned(values)) return OMC_ERR_MISALIGNED;
+    if (divisor == 0 || divisor > (1u << 24)) return OMC_ERR_INVALID_ARG;       // exact as an FP32 value
+    const uint64_t n4 = (plan->full_elems + 3) / 4;
+    const uint64_t want = (n4 + 255) / 256;
+    const uint64_t cap = (uint64_t)plan->n_sm * 8;
+    const unsigned grid = (unsigned)(want < cap ? (want ? want : 1) : cap);
+    divide_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(reinterpret_cast<float4 *>(values), n4,
+                                                                        (float)divisor, (divisor & (divisor - 1)) == 0);
     return omc::note_cuda(cudaGetLastError());
 }

@@ -127,6 +127,7 @@ struct AggParams {
     const float *resid[MAX_CLIENTS];
     const float *sb[MAX_CLIENTS];
     uint32_t nclients;
+    uint32_t divide;                     // 1: out = sum / nclients; 0: out = the sum itself (first stage of a mean across GPUs)
     uint32_t nvars;
     uint64_t tile_count;
     uint32_t nwarps;

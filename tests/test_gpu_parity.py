@@ -502,3 +502,51 @@ def test_aggregate_client_replicas(fmt, K):
         assert same_f32(from_full(clients[1].plan, got, i), dec[1][i]), i
     L = omc.lib()
     assert L.omc_aggregate(None, 1, None, None, None, out.data_ptr(), None) == -3
+
+
+@pytest.mark.parametrize("fmt", [(5, 10), (5, 2), (3, 7)], ids=lambda f: "E%dM%d" % f)
+def test_aggregate_in_two_stages(fmt):
+    """The mean over clients held by several GPUs (omc_aggregate_sum per holder, the holders' sums
+    added, omc_divide), with the collective's addition stood in for by one FP32 addition in holder
+    order: bit-exact against the oracle's two-stage mean; one holder alone equals omc_aggregate."""
+    from paper_2205_03494_b200 import replicas
+    rng = np.random.default_rng(31)
+    numel = [3000, 1, 1024, 5121, 333, 40000, 77]
+    kinds = [0, 0, 0, 0, 1, 0, 2]
+    base = [(rng.standard_normal(n) * 0.1).astype(np.float32) for n in numel]
+    clients = []
+    for k in range(7):
+        params = [(p + rng.standard_normal(p.size).astype(np.float32) * np.float32(0.01)) for p in base]
+        clients.append(Lockstep(numel, kinds, fmt, params, fraction=0.6, seed=50 + k))
+    holders = [clients[:3], clients[3:5], clients[5:]]
+    st = torch.cuda.current_stream().cuda_stream
+    plan0 = clients[0].plan
+    sums = []
+    for h in holders:
+        buf = clients[0].dm.full_buffer("partial sum %d" % len(sums))
+        omc.aggregate_sum([c.plan for c in h], [c.dm.packed.data_ptr() for c in h], [c.dm.resid.data_ptr() for c in h],
+                          [c.dm.sb.data_ptr() for c in h], buf.data_ptr(), st)
+        sums.append(buf)
+    total = sums[0].clone()
+    for s in sums[1:]:
+        total += s                                  # what the all-reduce does, here in holder order
+    omc.divide(plan0, total.data_ptr(), 7, st)
+    torch.cuda.synchronize()
+    clients[0].dm.check_guards()
+    got = total.cpu().numpy()
+    want = orc.aggregate_two_stage([[c.st for c in h] for h in holders])
+    for i in range(len(numel)):
+        assert same_f32(from_full(plan0, got, i), want[i]), i
+    # one process, no process group: the two library steps in a row are omc_aggregate
+    out = torch.zeros(plan0.full_elems, dtype=torch.float32, device="cuda")
+    k = replicas.mean_of_local_and_remote_clients([c.plan for c in clients], [c.dm.packed.data_ptr() for c in clients],
+                                                  [c.dm.resid.data_ptr() for c in clients],
+                                                  [c.dm.sb.data_ptr() for c in clients], out, st)
+    ref = torch.zeros_like(out)
+    omc.aggregate([c.plan for c in clients], [c.dm.packed.data_ptr() for c in clients],
+                  [c.dm.resid.data_ptr() for c in clients], [c.dm.sb.data_ptr() for c in clients], ref.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert k == 7 and torch.equal(out.view(torch.int32), ref.view(torch.int32))
+    L = omc.lib()
+    assert L.omc_divide(plan0._h, out.data_ptr(), 0, None) == -1
+    assert L.omc_divide(plan0._h, None, 3, None) == -3

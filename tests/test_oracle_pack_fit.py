@@ -340,3 +340,27 @@ def test_aggregate_models_decompresses_each_client_first():
             want = want + x
         assert np.array_equal(got[i], want / np.float32(3))
     assert np.array_equal(states[1]["fp32"][0], base[0] + np.float32(0.01))
+
+
+def test_two_stage_mean_is_sum_then_one_division():
+    """Per-holder sums in client order, holders in order, one rounded division: exact rationals;
+    one holder alone is the plain mean; the result stays within the stated bound of it."""
+    rng = np.random.default_rng(21)
+    n = 50
+    xs = [(rng.standard_normal(n) * 10.0 ** rng.integers(-2, 2)).astype(np.float32) for _ in range(7)]
+    groups = [xs[:3], xs[3:5], xs[5:]]
+    got = orc.divide_var(orc.sum_var([orc.sum_var(g) for g in groups]), 7)
+    for e in range(n):
+        parts = []
+        for g in groups:
+            acc = np.float32(g[0][e])
+            for x in g[1:]:
+                acc = f32_round(Fraction(float(acc)) + Fraction(float(x[e])))
+            parts.append(acc)
+        tot = parts[0]
+        for p in parts[1:]:
+            tot = f32_round(Fraction(float(tot)) + Fraction(float(p)))
+        assert got[e] == f32_round(Fraction(float(tot)) / 7)
+    assert np.array_equal(orc.divide_var(orc.sum_var(xs), 7), orc.aggregate_var(xs))
+    bound = 6 * 2.0 ** -24 * np.sum(np.abs(xs), axis=0) / 7 + 2.0 ** -24 * np.abs(orc.aggregate_var(xs))
+    assert np.all(np.abs(got.astype(np.float64) - orc.aggregate_var(xs)) <= 2 * bound)
