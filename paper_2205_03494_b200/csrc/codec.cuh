@@ -160,6 +160,19 @@ __device__ __forceinline__ uint32_t encode_fast(float w, float &vt)
     } else {
         // Let the FP32 adder do the rounding: adding 2^(e_q+23-M), e_q = max(exponent, EMIN),
         // leaves exactly the bits above the target spacing 2^(e_q-M), rounded to nearest even.
+        if constexpr (F::M <= 22 && !HalfPath<F>::value) {
+            // The constant as 2^e_q (with w's sign) times 2^(23-M): the product is exact, so the two
+            // fused multiply-adds round exactly what the addition and the subtraction would, on
+            // the signed value.  A negative w that rounds to zero gives +0 here; the sums and
+            // the equality test do not tell the zeros apart, and the code takes its sign from w.
+            const uint32_t m = max(u & 0x7F800000u, F::pow2_bits(F::EMIN));
+            const float ms = u2f(m | (u & 0x80000000u));
+            constexpr float K = (float)(1u << F::SH);
+            vt = __fmaf_rn(ms, -K, __fmaf_rn(ms, K, w));
+            // vt is a value of the format: rebias its magnitude exactly, read the fields off the pattern
+            const float t = __fmul_rn(fabsf(vt), u2f(F::pow2_bits(F::BIAS - 127)));
+            return (f2u(t) >> F::SH) | ((u >> (31 - F::E - F::M)) & F::SIGN_BIT);
+        }
         const float a = fabsf(w);
         float r;
         if constexpr (F::M <= 22) {
@@ -330,17 +343,18 @@ __device__ __forceinline__ float decode_fast_at(const uint32_t (&w)[NW], int pos
         t = w[wi] << (32 - sh - F::B);
     else
         t = __funnelshift_r(w[wi], w[(wi + 1 < NW) ? wi + 1 : wi], sh + F::B - 32);
-    const uint32_t mag = (t >> (8 - F::E)) & (F::MAG_MASK << F::SH);
-    const float v = __fmul_rn(u2f(mag), u2f(F::pow2_bits(127 - F::BIAS)));
-    return u2f(f2u(v) | (t & 0x80000000u));
+    // an arithmetic shift keeps the sign at bit 31; the copies of it that follow are masked away
+    const uint32_t sm = (uint32_t)((int32_t)t >> (8 - F::E)) & (0x80000000u | (F::MAG_MASK << F::SH));
+    return __fmul_rn(u2f(sm), u2f(F::pow2_bits(127 - F::BIAS)));
 }
 
 template <class F, int NW>
 __device__ __forceinline__ void put_code_at(uint32_t (&w)[NW], int pos, uint32_t c)
 {
+    // the fields are disjoint, so adding is OR-ing, and a shift-and-add is one instruction
     const int wi = pos >> 5, sh = pos & 31;
-    w[wi] |= c << sh;
-    if (sh + F::B > 32) w[(wi + 1 < NW) ? wi + 1 : wi] |= c >> (32 - sh);
+    w[wi] += c << sh;
+    if (sh + F::B > 32) w[(wi + 1 < NW) ? wi + 1 : wi] += c >> (32 - sh);
 }
 
 }  // namespace omc
