@@ -286,9 +286,9 @@ int omc_divide(const omc_plan_t *plan, float *values, uint32_t divisor, void *st
  *   S1E5M10 (the codes are IEEE halves and feed the tensor cores as they are); S1E5M6, S1E5M2,
  *   S1E4M3 and S1E2M3 (every value of these formats is an FP16 value: the codes are expanded to
  *   halves inside the kernel, on the way into the operand tile; Inf and NaN codes included); other
- *   formats return OMC_ERR_BAD_FORMAT: the odd code widths (S1E5M7, S1E3M7, S1E3M9, S1E4M8 of
- *   Table 2 and Sec. 3.5.3) because 64 codes of a row are then not a multiple of the 16 bytes a
- *   bulk tensor copy is made of, S1E4M14 (Table 1) because its 15 significant bits are not an FP16
+ *   S1E3M7 (Table 2), S1E3M9, S1E4M8 and S1E5M7 (Sec. 3.5.3) the same way, with K % 128 == 0 (a row
+ *   of 11- or 13-bit codes must be whole 16-byte units for the bulk tensor copies); other formats
+ *   return OMC_ERR_BAD_FORMAT: S1E4M14 (Table 1) because its 15 significant bits are not an FP16
  *   value, the fixed-point variant because its codes are not floating-point patterns.  For those,
  *   omc_decompress the variable and multiply.
  *   var must be quantised and N*K == its numel; N % 128 == 0, K % 64 == 0 (else OMC_ERR_INVALID_ARG).

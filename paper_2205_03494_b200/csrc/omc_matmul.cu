@@ -41,14 +41,26 @@ constexpr uint32_t WAIT_LIMIT = 1u << 20;        // polls of one mbarrier before
 // three stages of 72 / 64 / 60 KB (X tile, operand tile, packed bytes of the tile) and sixteen
 // decoder warps.  E = 5 codes are FP16 patterns with the low mantissa bits dropped; S1E4M3 and
 // S1E2M3 codes go through the narrow-float conversion instructions.
+// Odd code widths (11 and 13 bits: S1E3M7 of Table 2, S1E3M9 / S1E4M8 / S1E5M7 of Sec. 3.5.3): the
+// 64 codes of a tile row are 8 B bytes, so every other K block starts 8 bytes off the 16-byte
+// grid that a bulk tensor copy has to start on.  The copy then starts at the boundary below and
+// is 8 bytes wider (BOX_BYTES), and the decoders index from the remainder; a row of the matrix
+// must itself be a multiple of 16 bytes (K % 128 == 0).  Every value of these formats is an FP16
+// value: E = 5 codes are FP16 patterns (code << 3), the others become FP16 patterns whose exponent
+// field is too small by 15 - bias, which one exact packed multiplication by 2^(15 - bias) repairs
+// for normal and subnormal codes alike; Inf / NaN codes are patched in afterwards.
 template <int B, int E>
 struct Cfg {
-    static_assert((E == 5 && (B == 16 || B == 12 || B == 8)) || (E == 4 && B == 8) || (E == 2 && B == 6), "");
+    static_assert((E == 5 && (B == 16 || B == 12 || B == 8)) || (E == 4 && B == 8) || (E == 2 && B == 6) ||
+                  (B == 13 && (E == 5 || E == 3 || E == 4)) || (B == 11 && E == 3), "");
     static constexpr bool DECODE = B != 16;
+    static constexpr bool ODD = (B % 2) != 0;
+    static constexpr int MAN = B - 1 - E;
     static constexpr int ROW_BYTES = BK * B / 8;                 // one tile row of codes
-    static constexpr int RAW_BYTES = DECODE ? BN * ROW_BYTES : 0;
+    static constexpr int BOX_BYTES = ODD ? (ROW_BYTES + 8 + 15) / 16 * 16 : ROW_BYTES;   // what one copy brings per row
+    static constexpr int RAW_BYTES = DECODE ? BN * BOX_BYTES : 0;
     static constexpr int STAGE = TILE_A_BYTES + TILE_B_BYTES + RAW_BYTES;
-    static constexpr int NSTAGES = DECODE ? 3 : 4;
+    static constexpr int NSTAGES = !DECODE ? 4 : (3 * STAGE + 1280 <= 227 * 1024 ? 3 : 2);
     static constexpr int SMEM = NSTAGES * STAGE + 1024 /* alignment slack */ + 256 /* barriers, tmem slot */;
     static constexpr int DEC_THREADS = DECODE ? MATMUL_DECODER_THREADS : 0;
     static constexpr int THREADS = 192 + DEC_THREADS;
@@ -195,6 +207,56 @@ __device__ __forceinline__ uint4 expand_chunk(const uint8_t *raw)
     }
 }
 
+// Odd widths: the chunk's B bytes start at any byte; four aligned words hold them.
+template <int B, int E>
+__device__ __forceinline__ uint4 expand_chunk_odd(const uint8_t *raw)
+{
+    constexpr int M = B - 1 - E, SHIFT = 10 - M;
+    constexpr uint32_t MAG = (1u << (E + M)) - 1u, CODE = (1u << B) - 1u, INF_MAG = ((1u << E) - 1u) << M;
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(raw);
+    const uint32_t sh = (a & 3u) * 8u;
+    uint32_t w0, w1, w2, w3;
+    asm volatile("ld.shared.u32 %0, [%4];\n\tld.shared.u32 %1, [%4+4];\n\tld.shared.u32 %2, [%4+8];\n\tld.shared.u32 %3, [%4+12];"
+                 : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(a & ~3u));
+    uint32_t v[4] = {__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh), __funnelshift_r(w2, w3, sh), w3 >> sh};
+    uint32_t h[4];
+    bool special = false;
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        uint32_t hp = 0u;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int pos = (2 * p + q) * B, wi = pos >> 5, bs = pos & 31;
+            uint32_t c = (bs + B <= 32) ? (v[wi] >> bs) : __funnelshift_r(v[wi], v[wi + 1 < 4 ? wi + 1 : wi], bs);
+            c &= CODE;
+            const uint32_t mag = c & MAG;
+            uint32_t hb = (mag << SHIFT) | ((c >> (E + M)) << 15);
+            if (E != 5 && mag >= INF_MAG) special = true;
+            hp |= hb << (16 * q);
+        }
+        if constexpr (E != 5) {      // exponent field + (15 - bias): one exact multiplication, subnormal codes included
+            const __half2 scale = __float2half2_rn((float)(1u << (15 - ((1 << (E - 1)) - 1))));
+            const __half2 r = __hmul2(*reinterpret_cast<const __half2 *>(&hp), scale);
+            hp = *reinterpret_cast<const uint32_t *>(&r);
+        }
+        h[p] = hp;
+    }
+    if (E != 5 && special) {         // rare: a weight is Inf or NaN
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int pos = j * B, wi = pos >> 5, bs = pos & 31;
+            uint32_t c = (bs + B <= 32) ? (v[wi] >> bs) : __funnelshift_r(v[wi], v[wi + 1 < 4 ? wi + 1 : wi], bs);
+            c &= CODE;
+            const uint32_t mag = c & MAG;
+            if (mag >= INF_MAG) {
+                const uint32_t hb = ((c >> (E + M)) << 15) | (mag == INF_MAG ? 0x7C00u : 0x7E00u);
+                h[j >> 1] = (j & 1) ? ((h[j >> 1] & 0x0000FFFFu) | (hb << 16)) : ((h[j >> 1] & 0xFFFF0000u) | hb);
+            }
+        }
+    }
+    return make_uint4(h[0], h[1], h[2], h[3]);
+}
+
 template <int B, int E>
 __global__ void __launch_bounds__(Cfg<B, E>::THREADS, 1)
 matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
@@ -253,8 +315,8 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 if (skip_loads) continue;
                 const uint32_t a = base + s * C::STAGE;
                 tma_load_2d(a, &map_x, (int)(kb * BK), tm * BM, full(s));
-                if constexpr (C::DECODE)
-                    tma_load_2d(a + TILE_A_BYTES + TILE_B_BYTES, &map_w, (int)(kb * C::ROW_BYTES), tn * BN, full(s));
+                if constexpr (C::DECODE)      // odd widths: from the 16-byte boundary at or below the K block's first byte
+                    tma_load_2d(a + TILE_A_BYTES + TILE_B_BYTES, &map_w, (int)((kb * C::ROW_BYTES) & ~15u), tn * BN, full(s));
                 else
                     tma_load_2d(a + TILE_A_BYTES, &map_w, (int)(kb * BK), tn * BN, full(s));
             }
@@ -340,10 +402,15 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                     uint8_t *stage = base_ptr + s * C::STAGE;
                     const uint8_t *raw = stage + TILE_A_BYTES + TILE_B_BYTES + t * B;      // 8 codes = B bytes
                     uint8_t *dst = stage + TILE_A_BYTES;
+                    const uint32_t off = C::ODD ? ((kb * C::ROW_BYTES) & 15u) : 0u;      // where the K block starts in its copy
 #pragma unroll
                     for (int i = 0; i < BN * 8 / C::DEC_THREADS; ++i) {
                         const int r = i * (C::DEC_THREADS / 8) + (t >> 3);
-                        const uint4 o = expand_chunk<B, E>(raw + i * C::DEC_THREADS * B);
+                        uint4 o;
+                        if constexpr (C::ODD)
+                            o = expand_chunk_odd<B, E>(stage + TILE_A_BYTES + TILE_B_BYTES + r * C::BOX_BYTES + off + c * B);
+                        else
+                            o = expand_chunk<B, E>(raw + i * C::DEC_THREADS * B);
                         // 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r mod 8)
                         *reinterpret_cast<uint4 *>(dst + r * 128 + ((c ^ (r & 7)) << 4)) = o;
                     }
@@ -413,7 +480,7 @@ int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const f
 {
     using C = Cfg<B, E>;
     CUtensorMap map_w;
-    if (C::DECODE ? !make_raw_map(&map_w, codes, N, (uint64_t)K * B / 8, C::ROW_BYTES) : !make_map(&map_w, codes, N, K, BN))
+    if (C::DECODE ? !make_raw_map(&map_w, codes, N, (uint64_t)K * B / 8, C::BOX_BYTES) : !make_map(&map_w, codes, N, K, BN))
         return OMC_ERR_CUDA;
     static bool configured[64] = {};
     int dev = 0;
@@ -449,7 +516,9 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     if (plan->fmt.flags) return OMC_ERR_BAD_FORMAT;          // floating-point codes only
     const bool half_family = exp == 5 && (man == 10 || man == 6 || man == 2);
     const bool narrow = (exp == 4 && man == 3) || (exp == 2 && man == 3);
-    if (!half_family && !narrow) return OMC_ERR_BAD_FORMAT;
+    const bool odd = (exp == 5 && man == 7) || (exp == 3 && man == 7) || (exp == 3 && man == 9) || (exp == 4 && man == 8);
+    if (!half_family && !narrow && !odd) return OMC_ERR_BAD_FORMAT;
+    if (odd && K % 128 != 0) return OMC_ERR_INVALID_ARG;      // a row of 11- or 13-bit codes must be whole 16-byte units
     if (M == 0 || N == 0 || K == 0 || N % 128 != 0 || K % BK != 0 || (uint64_t)N * K != plan->vars[var].n)
         return OMC_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(packed) | reinterpret_cast<uintptr_t>(x_half) | reinterpret_cast<uintptr_t>(y) |
@@ -466,6 +535,12 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     const uint32_t n_sm = plan->n_sm ? plan->n_sm : 1;
     const uint32_t inject = plan->inject_polls;      // diagnostics: applies to this launch only
     plan->inject_polls = 0;
+    if (odd) {
+        if (exp == 5) return launch<13, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        if (exp == 4) return launch<13, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        if (man == 9) return launch<13, 3>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        return launch<11, 3>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    }
     if (exp == 4) return launch<8, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     if (exp == 2) return launch<6, 2>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     switch (man) {

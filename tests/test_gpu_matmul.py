@@ -57,10 +57,54 @@ def test_matmul_from_codes_matches_definition(M, N, K, fmt):
     assert np.all(np.abs(got - want) <= bound), float(np.max(np.abs(got - want) / bound))
 
 
+@pytest.mark.parametrize("fmt", [(5, 7), (3, 7), (3, 9), (4, 8)], ids=lambda f: "E%dM%d" % f)
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (200, 256, 384), (1000, 384, 512), (4000, 4224, 256)])
+def test_matmul_from_odd_width_codes(M, N, K, fmt):
+    """The 11- and 13-bit formats of Table 2 and Sec. 3.5.3: a K block of their codes starts 8
+    bytes off the 16-byte grid every other time, the E = 3 and E = 4 formats are FP16 values only
+    after a change of the exponent bias, and their subnormal codes are normal FP16 numbers.  Weights
+    are scaled so that they reach from the format's subnormal range to near its largest value."""
+    E_, M_ = fmt
+    rng = np.random.default_rng(M + N + K + E_)
+    top = 2.0 ** ((1 << (E_ - 1)) - 1) * (2 - 2.0 ** -M_)
+    scale = min(0.2 * top, 2.0)
+    w = (rng.standard_normal(N * K) * scale * 10.0 ** rng.uniform(-4, 0, N * K)).astype(np.float32)
+    w = np.clip(w, -0.9 * top, 0.9 * top)
+    numel, kinds = [333, N * K, 64], [0, 0, 1]
+    params = [rng.standard_normal(333).astype(np.float32) * np.float32(0.1), w, np.zeros(64, np.float32)]
+    plan = omc.Plan(numel, kinds, fmt)
+    dm = DeviceModel(plan)
+    dm.compress(dm.upload_full(params))
+    st = orc.compress(params, plan.quantised, *fmt)
+    x = (rng.standard_normal((M, K)) * 0.5).astype(np.float16)
+    xd = torch.from_numpy(x).cuda()
+    yg = Guarded(M * N, torch.float32, "cuda", fill=float("nan"))
+    y = yg.t[:M * N].view(M, N)
+    scratch = torch.zeros(M, dtype=torch.float32, device="cuda")
+    omc.matmul(plan, 1, dm.packed.data_ptr(), dm.sb.data_ptr(), xd.data_ptr(), M, N, K, y.data_ptr(),
+               scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert plan.status() == 0 and yg.intact()
+    s_, b_ = float(st["s"][1]), float(st["b"][1])
+    wbar = orc.decompress_var(st["packed"][1], N * K, E_, M_, st["s"][1], st["b"][1]).reshape(N, K).astype(np.float64)
+    wt = orc.decode(orc.unpack(st["packed"][1], N * K, 1 + E_ + M_), E_, M_).reshape(N, K).astype(np.float64)
+    x64 = x.astype(np.float64)
+    want = x64 @ wbar.T
+    bound = (4 * K + 8) * 2.0 ** -24 * (abs(s_) * (np.abs(x64) @ np.abs(wt).T)
+                                        + abs(b_) * np.abs(x64).sum(1, keepdims=True)) + 1e-30
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.all(np.abs(got - want) <= bound), float(np.max(np.abs(got - want) / bound))
+    # a row of 11- or 13-bit codes must be whole 16-byte units: K = 64 is refused before any launch
+    if (N * K) % 64 == 0:
+        assert omc.lib().omc_matmul(plan._h, 1, dm.packed.data_ptr(), dm.sb.data_ptr(), xd.data_ptr(), M, N * K // 64, 64,
+                                    y.data_ptr(), scratch.data_ptr(), None) == -1
+
+
 def test_matmul_argument_checks():
     plan = omc.Plan([128 * 64, 100], [0, 1], (5, 10))
     dm = DeviceModel(plan)
-    p8 = omc.Plan([128 * 64], [0], (3, 7))
+    p8 = omc.Plan([128 * 64], [0], (4, 14))
     d8 = DeviceModel(p8)
     x = torch.zeros(128 * 64, dtype=torch.float16, device="cuda")
     y = torch.zeros(128 * 128, dtype=torch.float32, device="cuda")
@@ -76,14 +120,14 @@ def test_matmul_argument_checks():
     torch.cuda.synchronize()
 
 
-@pytest.mark.parametrize("fmt", [(4, 3), (2, 3)], ids=lambda f: "E%dM%d" % f)
+@pytest.mark.parametrize("fmt", [(4, 3), (2, 3), (3, 7), (4, 8), (3, 9)], ids=lambda f: "E%dM%d" % f)
 def test_matmul_weights_at_the_top_of_the_range(fmt):
     """Weights that are infinite, NaN or the largest finite value of S1E4M3 / S1E2M3: the hardware
     narrow-float types have other values at those codes, so the decoder patches them.  A row of W
     with an infinity gives an infinite or NaN output column, a row with the largest finite value
     the exact product."""
     E, M = fmt
-    N, K, Mr = 128, 64, 128
+    N, K, Mr = 128, 128, 128
     top = 2.0 ** ((1 << (E - 1)) - 1) * (2 - 2.0 ** -M)
     w = np.full((N, K), 0.5 * top, np.float32)           # a value of the format in both cases
     w[3, 5] = np.inf
