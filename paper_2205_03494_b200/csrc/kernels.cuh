@@ -75,8 +75,9 @@ struct Smem {
     static constexpr int OUT = OUT_C + OUT_F;
     static constexpr int PER_WARP = NSTAGES * STAGE + OUTBUFS * OUT;
     static_assert(!ROWS || (STAGE % 128 == 0 && OUT % 128 == 0 && CB % 128 == 0), "row layout: FP32 granules stay 128-byte aligned");
-    static constexpr int BAR_PAD = (8 * MAX_STAGES * WARPS_PER_CTA + 127) / 128 * 128;   // the mbarriers
-    static constexpr int TOTAL = BAR_PAD + WARPS_PER_CTA * PER_WARP;
+    static constexpr int WARPS = (MODE == DECOMPRESS) ? WARPS_PER_CTA : fit_warps_per_cta(F::B, F::FIXED);
+    static constexpr int BAR_PAD = (8 * MAX_STAGES * WARPS + 127) / 128 * 128;   // the mbarriers
+    static constexpr int TOTAL = BAR_PAD + WARPS * PER_WARP;
     static_assert(STAGE % 16 == 0 && CB % 16 == 0, "bulk copies move multiples of 16 bytes");
 };
 
@@ -811,7 +812,7 @@ __device__ __forceinline__ bool compute_unit_b12(const uint32_t (&win)[3], const
             vt[2 * k + 1] = u2f(f2u(r1) | (u1 & 0x80000000u));
             const __half2 h = __floats2half2_rn(vt[2 * k], vt[2 * k + 1]);   // exact: both are FP16 values
             const uint32_t x = *reinterpret_cast<const uint32_t *>(&h);      // code 2k << 4 | code 2k+1 << 20
-            // the pair's 24 bits; what is left above them is never selected by the byte permutes below
+            // the pair as 24 bits: code 2k in bits 0..11, code 2k+1 in bits 12..23
             const uint32_t lo = x >> 4, hi = x >> 8;
             pr[k] = (lo & 0xFFFu) | (hi & ~0xFFFu);
         }
@@ -1223,7 +1224,7 @@ __device__ __noinline__ void fp32_queue(const KParams &p, int lane)
 // instead of the runs; a separate instantiation, because the call costs the kernels of
 // all-quantised models 3 to 8 %.
 template <class F, int MODE, bool WOUT, bool QUEUE = false>
-__global__ void __launch_bounds__(THREADS, MODE == DECOMPRESS ? DECOMPRESS_CTAS_PER_SM : CTAS_PER_SM)
+__global__ void __launch_bounds__(32 * Smem<F, MODE, WOUT>::WARPS, MODE == DECOMPRESS ? DECOMPRESS_CTAS_PER_SM : CTAS_PER_SM)
 omc_kernel(const KParams p)
 {
     using SM = Smem<F, MODE, WOUT>;
@@ -1233,7 +1234,7 @@ omc_kernel(const KParams p)
     int lane;
     asm volatile("mov.u32 %0, %%laneid;" : "=r"(lane));
     const int wid = threadIdx.x >> 5;
-    const uint32_t warp = blockIdx.x * WARPS_PER_CTA + wid;
+    const uint32_t warp = blockIdx.x * SM::WARPS + wid;
     if (warp >= p.nwarps) return;
 
     // this warp's slice of shared memory: the input stages, then the output buffers
@@ -1312,7 +1313,7 @@ void launch(const KParams &p, int grid, void *stream)
         cudaFuncSetAttribute(omc_kernel<F, MODE, WOUT, QUEUE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL);
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    omc_kernel<F, MODE, WOUT, QUEUE><<<grid, THREADS, SM::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
+    omc_kernel<F, MODE, WOUT, QUEUE><<<grid, 32 * SM::WARPS, SM::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1329,7 +1330,8 @@ struct TransitionSmem {
     using C = Smem<F, COMPRESS, false>;
     using D = Smem<F, DECOMPRESS, false>;
     static constexpr int PER_WARP = C::PER_WARP > D::PER_WARP ? C::PER_WARP : D::PER_WARP;
-    static constexpr int TOTAL = C::BAR_PAD + WARPS_PER_CTA * PER_WARP;
+    static constexpr int WARPS = C::WARPS;
+    static constexpr int TOTAL = C::BAR_PAD + WARPS * PER_WARP;
 };
 
 // 16-byte copy of `count` units by one warp, eight loads in flight per lane.
@@ -1348,13 +1350,13 @@ __device__ __forceinline__ void warp_copy16(uint4 *__restrict__ to, const uint4 
 }
 
 template <class F>
-__global__ void __launch_bounds__(THREADS, CTAS_PER_SM) omc_transition_kernel(const KParams p)
+__global__ void __launch_bounds__(32 * TransitionSmem<F>::WARPS, CTAS_PER_SM) omc_transition_kernel(const KParams p)
 {
     using TS = TransitionSmem<F>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const int lane = threadIdx.x & 31;
     const int wid = threadIdx.x >> 5;
-    const uint32_t warp = blockIdx.x * WARPS_PER_CTA + wid;
+    const uint32_t warp = blockIdx.x * TS::WARPS + wid;
     if (warp >= p.nwarps) return;
     WarpPipe pipe;
     pipe.wbase = smem_raw + TS::C::BAR_PAD + wid * TS::PER_WARP;
@@ -1445,7 +1447,7 @@ void launch_transition(const KParams &p, int grid, void *stream)
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(THREADS);
+    cfg.blockDim = dim3(32 * TransitionSmem<F>::WARPS);
     cfg.dynamicSmemBytes = TransitionSmem<F>::TOTAL;
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
@@ -1624,7 +1626,8 @@ void launch_aggregate(const AggParams &p, int grid, void *stream)
 }
 
 #define OMC_DEFINE_FIXED_FORMAT(I_, F_)                                                         \
-    extern const FmtOps ops_I##I_##F##F_ = {I_, F_, 1, launch<FixFmt<I_, F_>, COMPRESS, false>, \
+    extern const FmtOps ops_I##I_##F##F_ = {I_, F_, 1, fit_warps_per_cta(1 + I_ + F_, true),    \
+                                            launch<FixFmt<I_, F_>, COMPRESS, false>,            \
                                             launch<FixFmt<I_, F_>, DECOMPRESS, false>,          \
                                             launch<FixFmt<I_, F_>, UPDATE, false>,              \
                                             launch<FixFmt<I_, F_>, UPDATE, true>,               \
@@ -1633,7 +1636,8 @@ void launch_aggregate(const AggParams &p, int grid, void *stream)
                                             launch_aggregate<FixFmt<I_, F_>>};
 
 #define OMC_DEFINE_FORMAT(E_, M_)                                                               \
-    extern const FmtOps ops_E##E_##M##M_ = {E_, M_, 0, launch<Fmt<E_, M_>, COMPRESS, false>,    \
+    extern const FmtOps ops_E##E_##M##M_ = {E_, M_, 0, fit_warps_per_cta(1 + E_ + M_, false),   \
+                                            launch<Fmt<E_, M_>, COMPRESS, false>,               \
                                             launch<Fmt<E_, M_>, DECOMPRESS, false>,             \
                                             launch<Fmt<E_, M_>, UPDATE, false>,                 \
                                             launch<Fmt<E_, M_>, UPDATE, true>,                  \

@@ -157,7 +157,10 @@ static bool use_fp32_queue(const omc_plan_t *plan, KParams &p)
     return true;
 }
 
-static int grid_for(uint32_t nwarps) { return (int)((nwarps + omc::WARPS_PER_CTA - 1) / omc::WARPS_PER_CTA); }
+static int grid_for(uint32_t nwarps, int warps_per_cta = omc::WARPS_PER_CTA)
+{
+    return (int)((nwarps + warps_per_cta - 1) / warps_per_cta);
+}
 
 extern "C" int omc_compress(const omc_plan_t *plan, const float *params, uint8_t *packed, float *resid,
                             float *sb, void *workspace, void *stream)
@@ -171,7 +174,7 @@ extern "C" int omc_compress(const omc_plan_t *plan, const float *params, uint8_t
         return OMC_ERR_MISALIGNED;
     KParams p = whole_model(plan, workspace);
     p.packed = packed; p.resid = resid; p.sb = sb; p.fin = params;
-    plan->ops->compress(p, grid_for(p.nwarps), stream);
+    plan->ops->compress(p, grid_for(p.nwarps, plan->ops->fit_warps), stream);
     return omc::note_cuda(cudaGetLastError());
 }
 
@@ -235,11 +238,11 @@ extern "C" int omc_update_recompress(const omc_plan_t *plan, uint8_t *packed, fl
     p.packed = packed; p.resid = resid; p.sb = sb; p.fin = grads; p.fout = debug_w_out;
     p.neg_lr = -lr;
     if (debug_w_out)
-        plan->ops->update_w(p, grid_for(p.nwarps), stream);
+        plan->ops->update_w(p, grid_for(p.nwarps, plan->ops->fit_warps), stream);
     else if (use_fp32_queue(plan, p))
-        plan->ops->update_q(p, grid_for(p.nwarps), stream);
+        plan->ops->update_q(p, grid_for(p.nwarps, plan->ops->fit_warps), stream);
     else
-        plan->ops->update(p, grid_for(p.nwarps), stream);
+        plan->ops->update(p, grid_for(p.nwarps, plan->ops->fit_warps), stream);
     return omc::note_cuda(cudaGetLastError());
 }
 
@@ -327,7 +330,7 @@ extern "C" int omc_transition(const omc_plan_t *from, const omc_plan_t *to, cons
     p.run_var = to->d_trans.run_var;
     p.trans_vars = to->d_trans.vars;
     p.nruns_dev = to->d_trans.nruns;
-    to->ops->transition(p, grid_for(p.nwarps), stream);
+    to->ops->transition(p, grid_for(p.nwarps, to->ops->fit_warps), stream);
     return omc::note_cuda(cudaGetLastError());
 }
 

@@ -239,7 +239,7 @@ extern "C" int omc_plan(const omc_var_desc_t *vars, uint32_t nvars, omc_format_t
         // ---- division of the tiles among warps
         pl->n_sm = query_sm_count();
         pl->n_cta = pl->n_sm * omc::CTAS_PER_SM;
-        const uint64_t max_warps = (uint64_t)pl->n_cta * omc::WARPS_PER_CTA;
+        const uint64_t max_warps = (uint64_t)pl->n_cta * ops->fit_warps;      // the fitting kernels' launch
         pl->nwarps = (uint32_t)(tiles < max_warps ? tiles : max_warps);
         // Kernels that fit (s, b) take one run per warp: a run ends with a hand-over of the sums,
         // which costs more than working side by side with the other warps gains.

@@ -136,7 +136,7 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     // one variable, one tile list, divided among the warps exactly as omc_plan divides a model
     const uint32_t B = 1u + fmt.exp_bits + fmt.man_bits;
     const uint64_t tiles = (numel + omc::TILE - 1) / omc::TILE;
-    const uint64_t max_warps = (uint64_t)sms * omc::CTAS_PER_SM * omc::WARPS_PER_CTA;
+    const uint64_t max_warps = (uint64_t)sms * omc::CTAS_PER_SM * ops->fit_warps;
     const uint32_t nwarps = (uint32_t)(tiles < max_warps ? tiles : max_warps);
     if (nwarps > MAX_SLOTS) return OMC_ERR_TOO_LARGE;
     const uint32_t nruns = nwarps;          // one run per warp, as in omc_compress
@@ -172,7 +172,7 @@ extern "C" int omc_compress_var_static(const float *values, uint64_t numel, omc_
     p.tickets = reinterpret_cast<uint32_t *>(scratch + OFF_TICKET);
     p.status = reinterpret_cast<uint32_t *>(scratch + OFF_STATUS);
     p.slots = reinterpret_cast<omc::Partial *>(scratch + OFF_SLOTS);
-    ops->compress(p, (int)((nwarps + omc::WARPS_PER_CTA - 1) / omc::WARPS_PER_CTA), stream);
+    ops->compress(p, (int)((nwarps + ops->fit_warps - 1) / ops->fit_warps), stream);
     return omc::note_cuda(cudaGetLastError());
 }
 
