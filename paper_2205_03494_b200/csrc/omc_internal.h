@@ -15,10 +15,11 @@ constexpr int THREADS = 32 * WARPS_PER_CTA;
 // Warps per CTA of the kernels that fit (s, b) (compress, fused round, transition).  Eight warps
 // leave a thread 128 registers; the 12- and 19-bit kernels, which need more to keep several
 // elements' arithmetic in flight, run faster with six warps and up to 168 registers (measured:
-// S1E5M6 on the 1.6-billion set 3-5 % per clock, S1E4M14 5 %; the 16- and 8-bit kernels lose 2-3 %).
-constexpr int fit_warps_per_cta(int code_bits, bool fixed_point)
+// S1E5M6 on the 1.6-billion set 3-5 % per clock, S1E4M14 5 %, Q11 4 %; the 16- and 8-bit kernels lose 2-3 %,
+// the 11- and 13-bit ones gain a per cent and a half, which their compress kernel would lose again).
+constexpr int fit_warps_per_cta(int code_bits, bool /*fixed_point*/)
 {
-    return (!fixed_point && (code_bits == 12 || code_bits == 19)) ? 6 : WARPS_PER_CTA;
+    return (code_bits == 12 || code_bits == 19) ? 6 : WARPS_PER_CTA;
 }
 constexpr int CTAS_PER_SM = 2;
 // The decompress kernel divides its tiles at launch, so its grid is independent of the plan's division.
