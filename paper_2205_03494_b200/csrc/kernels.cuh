@@ -148,6 +148,15 @@ struct Acc {
         sxy = fma(dw, dv, sxy);
         syy = fma(dv, dv, syy);
     }
+    // the same with Vt already in fp64 (converted straight from its FP16 pattern)
+    __device__ __forceinline__ void add_d(float w, double dv)
+    {
+        const double dw = (double)w;
+        sx += dw;
+        sy += dv;
+        sxy = fma(dw, dv, sxy);
+        syy = fma(dv, dv, syy);
+    }
     __device__ __forceinline__ void merge(const Acc &o)
     {
         sx += o.sx; sy += o.sy; sxy += o.sxy; syy += o.syy;
@@ -520,11 +529,10 @@ __device__ __forceinline__ void compute_unit_rows(const uint32_t *cin, const flo
 // of infinity; e4m3 and e2m3 have finite values where the family has Inf/NaN), and every code that
 // high, read or produced, sends the unit to compute_unit.
 
-// Four codes, one per byte -> four FP32 values (exact).
+// Four codes, one per byte -> two pairs of FP16 patterns (exact).
 template <class F>
-__device__ __forceinline__ void fp8x4_decode(uint32_t cw, float (&v)[4])
+__device__ __forceinline__ void fp8x4_halves(uint32_t cw, uint32_t &h01, uint32_t &h23)
 {
-    uint32_t h01, h23;       // two FP16 pairs
     if constexpr (F::E == 5) {                   // a code is the top byte of its FP16 pattern
         h01 = __byte_perm(cw, 0u, 0x1404);
         h23 = __byte_perm(cw, 0u, 0x3424);
@@ -541,9 +549,26 @@ __device__ __forceinline__ void fp8x4_decode(uint32_t cw, float (&v)[4])
             "cvt.rn.f16x2.e2m3x2 %1, hi;\n\t}"
             : "=r"(h01), "=r"(h23) : "r"(cw));
     }
+}
+
+template <class F>
+__device__ __forceinline__ void fp8x4_decode(uint32_t cw, float (&v)[4])
+{
+    uint32_t h01, h23;
+    fp8x4_halves<F>(cw, h01, h23);
     const __half2 a = *reinterpret_cast<const __half2 *>(&h01), c = *reinterpret_cast<const __half2 *>(&h23);
     v[0] = __low2float(a); v[1] = __high2float(a);
     v[2] = __low2float(c); v[3] = __high2float(c);
+}
+
+// A pair of FP16 patterns -> two fp64 values, without the detour through FP32.
+__device__ __forceinline__ void half2_to_doubles(uint32_t h2, double &lo, double &hi)
+{
+    asm("{\n\t.reg .b16 l, h;\n\t"
+        "mov.b32 {l, h}, %2;\n\t"
+        "cvt.f64.f16 %0, l;\n\t"
+        "cvt.f64.f16 %1, h;\n\t}"
+        : "=d"(lo), "=d"(hi) : "r"(h2));
 }
 
 // Four FP32 values -> four codes, one per byte (element 0 in the low byte).  Saturating: a
@@ -652,8 +677,8 @@ __device__ __forceinline__ void compute_unit_fp8(const uint32_t (&win)[Unit<F>::
     for (int j = 0; j < NW; ++j) wout_sp[j] = 0u;
 #pragma unroll
     for (int g = 0; g < NG; ++g) {
-        float w[4], vt[4];
-        uint32_t special = 0u;
+        float w[4];
+        uint32_t special = 0u, vh01 = 0u, vh23 = 0u;
         if constexpr (MODE != COMPRESS) {
             float dec[4];
             fp8x4_decode<F>(cin[g], dec);
@@ -670,7 +695,7 @@ __device__ __forceinline__ void compute_unit_fp8(const uint32_t (&win)[Unit<F>::
         if constexpr (MODE != DECOMPRESS) {
             cout[g] = fp8x4_encode<F>(w);
             special |= fp8x4_any_at_least<F, TOP_OUT>(cout[g]);
-            fp8x4_decode<F>(cout[g], vt);
+            fp8x4_halves<F>(cout[g], vh01, vh23);        // Q^-1 of the new codes, as FP16 patterns
         }
         if (special) {
             // on copies, so that only they (and not the registers of the main path) have addresses
@@ -688,8 +713,11 @@ __device__ __forceinline__ void compute_unit_fp8(const uint32_t (&win)[Unit<F>::
             for (int j = 0; j < 4; ++j) w[j] = w_c[j];
             if constexpr (MODE != DECOMPRESS) cout[g] = 0u;
         } else if constexpr (MODE != DECOMPRESS) {
+            double dv[4];
+            half2_to_doubles(vh01, dv[0], dv[1]);
+            half2_to_doubles(vh23, dv[2], dv[3]);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc.add(w[j], vt[j]);
+            for (int j = 0; j < 4; ++j) acc.add_d(w[j], dv[j]);
             if (g == 0) ref = __byte_perm(cout[0], 0u, 0x0000);     // element 0's code in all four bytes
             diff |= cout[g] ^ ref;
         }
