@@ -532,7 +532,7 @@ def run_ours(args):
         xh = (torch.randn(Mm, Km, device=dev) * 0.5).half()
         yo = torch.empty(Mm, Nm, dtype=torch.float32, device=dev)
         rs = torch.empty(Mm, dtype=torch.float32, device=dev)
-        for mfmt in ((5, 10), (5, 6), (5, 2), (4, 3), (2, 3), (5, 7), (3, 7), (3, 9), (4, 8)):
+        for mfmt in ((5, 10), (5, 6), (5, 2), (4, 3), (2, 3), (5, 7), (3, 7), (3, 9), (4, 8), (4, 14)):
             key = "matmul_from_codes_8192x8192x2048_S1E%dM%d" % mfmt
             try:
                 pm = omc.Plan([Nm * Km], [0], mfmt)

@@ -287,10 +287,11 @@ int omc_divide(const omc_plan_t *plan, float *values, uint32_t divisor, void *st
  *   S1E4M3 and S1E2M3 (every value of these formats is an FP16 value: the codes are expanded to
  *   halves inside the kernel, on the way into the operand tile; Inf and NaN codes included); other
  *   S1E3M7 (Table 2), S1E3M9, S1E4M8 and S1E5M7 (Sec. 3.5.3) the same way, with K % 128 == 0 (a row
- *   of 11- or 13-bit codes must be whole 16-byte units for the bulk tensor copies); other formats
- *   return OMC_ERR_BAD_FORMAT: S1E4M14 (Table 1) because its 15 significant bits are not an FP16
- *   value, the fixed-point variant because its codes are not floating-point patterns.  For those,
- *   omc_decompress the variable and multiply.
+ *   of 11-, 13- or 19-bit codes must be whole 16-byte units for the bulk tensor copies); S1E4M14
+ *   (Table 1) has 15 significant bits, more than FP16 holds, so each weight enters as two FP16
+ *   terms whose sum is the weight exactly and every K step makes two products into the same FP32
+ *   accumulator.  Other formats return OMC_ERR_BAD_FORMAT (the fixed-point variant among them: its
+ *   codes are not floating-point patterns); for those, omc_decompress the variable and multiply.
  *   var must be quantised and N*K == its numel; N % 128 == 0, K % 64 == 0 (else OMC_ERR_INVALID_ARG).
  *   packed, sb      device, the model state (read only).
  *   x_half          device, M x K IEEE halves, K contiguous, 16-byte aligned.

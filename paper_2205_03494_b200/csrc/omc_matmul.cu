@@ -31,10 +31,11 @@ constexpr int MATMUL_DECODER_THREADS = 512;      // sixteen decoder warps (measu
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64;       // CTA tile; BK halves = one 128-byte swizzle row
+constexpr int BM = 128, BK = 64;                 // CTA tile rows; BK halves = one 128-byte swizzle row
+constexpr int BN_WIDE = 256, BN_SPLIT = 128;     // CTA tile columns: 256, or 128 for the two-term format
 constexpr int UMMA_K = 16;                       // K of one tcgen05.mma with 16-bit inputs
-constexpr int TILE_A_BYTES = BM * BK * 2, TILE_B_BYTES = BN * BK * 2;
-constexpr int TMEM_COLS = 512;                   // two accumulators of 128 lanes x 256 FP32 columns
+constexpr int TILE_A_BYTES = BM * BK * 2;
+constexpr int TMEM_COLS = 512;                   // two accumulators of 128 lanes x (up to) 256 FP32 columns
 constexpr uint32_t WAIT_LIMIT = 1u << 20;        // polls of one mbarrier before giving up
 
 // B = bits per code, E = exponent bits.  16: no decode stage, four stages of 48 KB.  12 / 8 / 6:
@@ -52,14 +53,23 @@ constexpr uint32_t WAIT_LIMIT = 1u << 20;        // polls of one mbarrier before
 template <int B, int E>
 struct Cfg {
     static_assert((E == 5 && (B == 16 || B == 12 || B == 8)) || (E == 4 && B == 8) || (E == 2 && B == 6) ||
-                  (B == 13 && (E == 5 || E == 3 || E == 4)) || (B == 11 && E == 3), "");
+                  (B == 13 && (E == 5 || E == 3 || E == 4)) || (B == 11 && E == 3) || (B == 19 && E == 4), "");
     static constexpr bool DECODE = B != 16;
     static constexpr bool ODD = (B % 2) != 0;
+    // S1E4M14 (Table 1) has 15 significant bits, four more than an FP16 value: a weight is split
+    // exactly into hi + lo, both FP16 values (hi = the weight rounded to FP16, lo = the rest, at
+    // most 5 significant bits and never below 2^-20), the tile has two operand tiles and every K
+    // step two products into the same accumulator.  The tile is 128 columns wide then.
+    static constexpr bool SPLIT = (B == 19);
+    static constexpr int BN = SPLIT ? BN_SPLIT : BN_WIDE;
+    static constexpr int TILE_B_BYTES = BN * BK * 2;              // one operand tile
+    static constexpr int OPERAND_BYTES = (SPLIT ? 2 : 1) * TILE_B_BYTES;
+    static constexpr uint32_t IDESC = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
     static constexpr int MAN = B - 1 - E;
     static constexpr int ROW_BYTES = BK * B / 8;                 // one tile row of codes
     static constexpr int BOX_BYTES = ODD ? (ROW_BYTES + 8 + 15) / 16 * 16 : ROW_BYTES;   // what one copy brings per row
     static constexpr int RAW_BYTES = DECODE ? BN * BOX_BYTES : 0;
-    static constexpr int STAGE = TILE_A_BYTES + TILE_B_BYTES + RAW_BYTES;
+    static constexpr int STAGE = TILE_A_BYTES + OPERAND_BYTES + RAW_BYTES;
     static constexpr int NSTAGES = !DECODE ? 4 : (3 * STAGE + 1280 <= 227 * 1024 ? 3 : 2);
     static constexpr int SMEM = NSTAGES * STAGE + 1024 /* alignment slack */ + 256 /* barriers, tmem slot */;
     static constexpr int DEC_THREADS = DECODE ? MATMUL_DECODER_THREADS : 0;
@@ -110,16 +120,15 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_byte_addr)
 {
     return (uint64_t)((smem_byte_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: D = FP32 (bits 4-5 = 1), A = B = FP16 (0), both K-major, N/8 at bit 17, M/16 at bit 24.
-constexpr uint32_t IDESC = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate)
+// Instruction descriptor (Cfg::IDESC): D = FP32 (bits 4-5 = 1), A = B = FP16 (0), both K-major, N/8 at bit 17,
+// M/16 at bit 24.
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate, uint32_t idesc)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "r"(accumulate), "r"(0u) : "memory");
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
@@ -257,6 +266,50 @@ __device__ __forceinline__ uint4 expand_chunk_odd(const uint8_t *raw)
     return make_uint4(h[0], h[1], h[2], h[3]);
 }
 
+// S1E4M14: eight 19-bit codes (19 bytes from any byte) -> eight FP16 pairs (hi, lo) with
+// hi + lo = the weight exactly.  The weight is built as an FP32 value first (fields in place, one
+// exact multiplication by 2^(127 - 7) that also normalises subnormal codes), hi is its FP16
+// rounding, lo the FP16 value of the exact FP32 remainder.  Inf / NaN codes: hi = Inf / NaN, lo = 0.
+__device__ __forceinline__ void expand_chunk_split(const uint8_t *raw, uint4 &hi4, uint4 &lo4)
+{
+    constexpr int B = 19, E = 4, M = 14;
+    constexpr uint32_t MAG = (1u << (E + M)) - 1u, CODE = (1u << B) - 1u, INF_MAG = ((1u << E) - 1u) << M;
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(raw);
+    const uint32_t sh = (a & 3u) * 8u;
+    uint32_t w[6];
+    asm volatile("ld.shared.u32 %0, [%6];\n\tld.shared.u32 %1, [%6+4];\n\tld.shared.u32 %2, [%6+8];\n\t"
+                 "ld.shared.u32 %3, [%6+12];\n\tld.shared.u32 %4, [%6+16];\n\tld.shared.u32 %5, [%6+20];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]) : "r"(a & ~3u));
+    uint32_t v[5];
+#pragma unroll
+    for (int i = 0; i < 5; ++i) v[i] = __funnelshift_r(w[i], w[i + 1], sh);
+    uint32_t h[4], l[4];
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        h[p] = 0u;
+        l[p] = 0u;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int pos = (2 * p + q) * B, wi = pos >> 5, bs = pos & 31;
+            uint32_t c = (bs + B <= 32) ? (v[wi] >> bs) : __funnelshift_r(v[wi], v[wi + 1 < 5 ? wi + 1 : wi], bs);
+            c &= CODE;
+            const uint32_t mag = c & MAG, sign = (c >> (E + M)) << 31;
+            const float val = __fmul_rn(__uint_as_float(sign | (mag << (23 - M))), __uint_as_float((uint32_t)(127 - 7 + 127) << 23));
+            __half hh = __float2half_rn(val);
+            __half ll = __float2half_rn(__fsub_rn(val, __half2float(hh)));
+            uint32_t hb = __half_as_ushort(hh), lb = __half_as_ushort(ll);
+            if (mag >= INF_MAG) {
+                hb = (sign >> 16) | (mag == INF_MAG ? 0x7C00u : 0x7E00u);
+                lb = 0u;
+            }
+            h[p] |= hb << (16 * q);
+            l[p] |= lb << (16 * q);
+        }
+    }
+    hi4 = make_uint4(h[0], h[1], h[2], h[3]);
+    lo4 = make_uint4(l[0], l[1], l[2], l[3]);
+}
+
 template <int B, int E>
 __global__ void __launch_bounds__(Cfg<B, E>::THREADS, 1)
 matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
@@ -280,6 +333,7 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     const uint32_t tmem_slot = bars + 8u * (3 * NS + 4);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t nkb = K / BK;
+    constexpr int BN = C::BN, TILE_B_BYTES = C::TILE_B_BYTES;
     const uint32_t tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN, ntiles = tiles_m * tiles_n;
 
     if (tid == 0) {
@@ -316,7 +370,7 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 const uint32_t a = base + s * C::STAGE;
                 tma_load_2d(a, &map_x, (int)(kb * BK), tm * BM, full(s));
                 if constexpr (C::DECODE)      // odd widths: from the 16-byte boundary at or below the K block's first byte
-                    tma_load_2d(a + TILE_A_BYTES + TILE_B_BYTES, &map_w, (int)((kb * C::ROW_BYTES) & ~15u), tn * BN, full(s));
+                    tma_load_2d(a + TILE_A_BYTES + C::OPERAND_BYTES, &map_w, (int)((kb * C::ROW_BYTES) & ~15u), tn * BN, full(s));
                 else
                     tma_load_2d(a + TILE_A_BYTES, &map_w, (int)(kb * BK), tn * BN, full(s));
             }
@@ -338,8 +392,11 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a = base + s * C::STAGE, b = a + TILE_A_BYTES;
 #pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k)
-                    umma_f16(d, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), (kb | k) != 0);
+                for (int k = 0; k < BK / UMMA_K; ++k) {
+                    umma_f16(d, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), (kb | k) != 0, C::IDESC);
+                    if constexpr (C::SPLIT)      // the low parts of the weights, into the same accumulator
+                        umma_f16(d, umma_desc(a + k * UMMA_K * 2), umma_desc(b + TILE_B_BYTES + k * UMMA_K * 2), 1u, C::IDESC);
+                }
                 umma_commit(empty(s));
             }
             if (ok) umma_commit(acc_full(buf));     // complete once all MMAs issued so far have finished
@@ -400,15 +457,19 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                     ok = mbar_wait(full(s), (it / NS) & 1u, limit);
                     if (!ok) break;
                     uint8_t *stage = base_ptr + s * C::STAGE;
-                    const uint8_t *raw = stage + TILE_A_BYTES + TILE_B_BYTES + t * B;      // 8 codes = B bytes
+                    const uint8_t *raw = stage + TILE_A_BYTES + C::OPERAND_BYTES + t * B;      // 8 codes = B bytes
                     uint8_t *dst = stage + TILE_A_BYTES;
                     const uint32_t off = C::ODD ? ((kb * C::ROW_BYTES) & 15u) : 0u;      // where the K block starts in its copy
 #pragma unroll
                     for (int i = 0; i < BN * 8 / C::DEC_THREADS; ++i) {
                         const int r = i * (C::DEC_THREADS / 8) + (t >> 3);
                         uint4 o;
-                        if constexpr (C::ODD)
-                            o = expand_chunk_odd<B, E>(stage + TILE_A_BYTES + TILE_B_BYTES + r * C::BOX_BYTES + off + c * B);
+                        if constexpr (C::SPLIT) {
+                            uint4 lo;
+                            expand_chunk_split(stage + TILE_A_BYTES + C::OPERAND_BYTES + r * C::BOX_BYTES + off + c * B, o, lo);
+                            *reinterpret_cast<uint4 *>(dst + TILE_B_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) = lo;
+                        } else if constexpr (C::ODD)
+                            o = expand_chunk_odd<B, E>(stage + TILE_A_BYTES + C::OPERAND_BYTES + r * C::BOX_BYTES + off + c * B);
                         else
                             o = expand_chunk<B, E>(raw + i * C::DEC_THREADS * B);
                         // 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r mod 8)
@@ -461,13 +522,13 @@ bool make_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t cols, uin
 }
 
 // The packed codes of an N x K matrix as bytes: [rows x row_bytes], boxes of 256 rows x box_bytes, no swizzle.
-bool make_raw_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t row_bytes, uint32_t box_bytes)
+bool make_raw_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t row_bytes, uint32_t box_bytes, uint32_t box_rows)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {row_bytes, rows};
     const cuuint64_t strides[1] = {row_bytes};
-    const cuuint32_t box[2] = {box_bytes, BN};
+    const cuuint32_t box[2] = {box_bytes, box_rows};
     const cuuint32_t elem[2] = {1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(ptr), dims, strides, box, elem,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -480,7 +541,8 @@ int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const f
 {
     using C = Cfg<B, E>;
     CUtensorMap map_w;
-    if (C::DECODE ? !make_raw_map(&map_w, codes, N, (uint64_t)K * B / 8, C::BOX_BYTES) : !make_map(&map_w, codes, N, K, BN))
+    constexpr int BN = C::BN;
+    if (C::DECODE ? !make_raw_map(&map_w, codes, N, (uint64_t)K * B / 8, C::BOX_BYTES, BN) : !make_map(&map_w, codes, N, K, BN))
         return OMC_ERR_CUDA;
     static bool configured[64] = {};
     int dev = 0;
@@ -516,7 +578,8 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     if (plan->fmt.flags) return OMC_ERR_BAD_FORMAT;          // floating-point codes only
     const bool half_family = exp == 5 && (man == 10 || man == 6 || man == 2);
     const bool narrow = (exp == 4 && man == 3) || (exp == 2 && man == 3);
-    const bool odd = (exp == 5 && man == 7) || (exp == 3 && man == 7) || (exp == 3 && man == 9) || (exp == 4 && man == 8);
+    const bool split = exp == 4 && man == 14;
+    const bool odd = (exp == 5 && man == 7) || (exp == 3 && man == 7) || (exp == 3 && man == 9) || (exp == 4 && man == 8) || split;
     if (!half_family && !narrow && !odd) return OMC_ERR_BAD_FORMAT;
     if (odd && K % 128 != 0) return OMC_ERR_INVALID_ARG;      // a row of 11- or 13-bit codes must be whole 16-byte units
     if (M == 0 || N == 0 || K == 0 || N % 128 != 0 || K % BK != 0 || (uint64_t)N * K != plan->vars[var].n)
@@ -535,6 +598,7 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     const uint32_t n_sm = plan->n_sm ? plan->n_sm : 1;
     const uint32_t inject = plan->inject_polls;      // diagnostics: applies to this launch only
     plan->inject_polls = 0;
+    if (split) return launch<19, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     if (odd) {
         if (exp == 5) return launch<13, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
         if (exp == 4) return launch<13, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);

@@ -57,13 +57,15 @@ def test_matmul_from_codes_matches_definition(M, N, K, fmt):
     assert np.all(np.abs(got - want) <= bound), float(np.max(np.abs(got - want) / bound))
 
 
-@pytest.mark.parametrize("fmt", [(5, 7), (3, 7), (3, 9), (4, 8)], ids=lambda f: "E%dM%d" % f)
+@pytest.mark.parametrize("fmt", [(5, 7), (3, 7), (3, 9), (4, 8), (4, 14)], ids=lambda f: "E%dM%d" % f)
 @pytest.mark.parametrize("M,N,K", [(128, 128, 128), (200, 256, 384), (1000, 384, 512), (4000, 4224, 256)])
 def test_matmul_from_odd_width_codes(M, N, K, fmt):
     """The 11- and 13-bit formats of Table 2 and Sec. 3.5.3: a K block of their codes starts 8
     bytes off the 16-byte grid every other time, the E = 3 and E = 4 formats are FP16 values only
-    after a change of the exponent bias, and their subnormal codes are normal FP16 numbers.  Weights
-    are scaled so that they reach from the format's subnormal range to near its largest value."""
+    after a change of the exponent bias, and their subnormal codes are normal FP16 numbers.  S1E4M14
+    (Table 1, 19 bits) has more significant bits than FP16: its weights go in as two FP16 terms and
+    every K step makes two products.  Weights are scaled so that they reach from the format's
+    subnormal range to near its largest value."""
     E_, M_ = fmt
     rng = np.random.default_rng(M + N + K + E_)
     top = 2.0 ** ((1 << (E_ - 1)) - 1) * (2 - 2.0 ** -M_)
@@ -104,7 +106,7 @@ def test_matmul_from_odd_width_codes(M, N, K, fmt):
 def test_matmul_argument_checks():
     plan = omc.Plan([128 * 64, 100], [0, 1], (5, 10))
     dm = DeviceModel(plan)
-    p8 = omc.Plan([128 * 64], [0], (4, 14))
+    p8 = omc.Plan([128 * 64], [0], (6, 5))
     d8 = DeviceModel(p8)
     x = torch.zeros(128 * 64, dtype=torch.float16, device="cuda")
     y = torch.zeros(128 * 128, dtype=torch.float32, device="cuda")
@@ -120,7 +122,7 @@ def test_matmul_argument_checks():
     torch.cuda.synchronize()
 
 
-@pytest.mark.parametrize("fmt", [(4, 3), (2, 3), (3, 7), (4, 8), (3, 9)], ids=lambda f: "E%dM%d" % f)
+@pytest.mark.parametrize("fmt", [(4, 3), (2, 3), (3, 7), (4, 8), (3, 9), (4, 14)], ids=lambda f: "E%dM%d" % f)
 def test_matmul_weights_at_the_top_of_the_range(fmt):
     """Weights that are infinite, NaN or the largest finite value of S1E4M3 / S1E2M3: the hardware
     narrow-float types have other values at those codes, so the decoder patches them.  A row of W
