@@ -176,7 +176,8 @@ int omc_plan_status(const omc_plan_t *plan, void *stream, uint32_t *host_status)
 /*
  * omc_plan_inject_wait_timeout -- diagnostics for the bounded waits (the paper has no counterpart).
  * The next kernel launched with this plan (omc_compress, omc_decompress, omc_update_recompress,
- * omc_transition with the plan as destination, omc_matmul) announces its asynchronous loads to
+ * omc_transition with the plan as destination, omc_aggregate and omc_aggregate_sum with the plan
+ * first in the list, omc_matmul) announces its asynchronous loads to
  * their barriers without issuing them and gives up each wait after `polls` polls (1 .. 2^24):
  * every wait runs out with no copy in flight, the kernel sets the status word and returns, its
  * outputs are garbage.  Afterwards omc_plan_status reports non-zero; call omc_plan_prepare again
@@ -254,7 +255,10 @@ int omc_transition(const omc_plan_t *from, const omc_plan_t *to, const uint8_t *
  * fma(s_k, Vt_k, b_k) if k quantised the variable and its FP32 value otherwise.
  *   plans[K]   host array: each client's prepared plan (same variables and format, own selection).
  *   packed[K], resid[K], sb[K]   host arrays of device pointers: each client's state, read only.
- *   out        device, full layout, written.       1 <= K <= 16 (else OMC_ERR_INVALID_ARG).
+ *   out        device, full layout, written (the padding after each variable with zeros).
+ *   1 <= K <= 16 (else OMC_ERR_INVALID_ARG).
+ * The kernel streams the codes through shared memory with bounded waits like the other calls; one
+ * that runs out sets the status word of plans[0] (omc_plan_status).
  * Formats without a compiled specialisation return OMC_ERR_BAD_FORMAT.
  */
 int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,

@@ -329,12 +329,11 @@ __device__ __forceinline__ uint32_t get_code_at(const uint32_t (&w)[NW], int pos
     return c & F::CODE_MASK;
 }
 
-// decode_fast of the code at bit position `pos`, without isolating the code first: one shift
-// puts the code's sign at bit 31 (whatever follows the code stays in the low bits), a second one
-// and a mask put exponent and mantissa where FP32 keeps them, and the sign is merged after the
-// rebias multiplication.  Formats on the generic path only (E < 8, not the FP16 family).
+// The code at bit position `pos` with its fields where FP32 keeps them, before the rebias
+// multiplication: decode_fast(code) = placed * 2^(127-BIAS) exactly.  A code with an all-ones
+// exponent field gives a magnitude of at least u2f(INF_MAG << SH), every other code less.
 template <class F, int NW>
-__device__ __forceinline__ float decode_fast_at(const uint32_t (&w)[NW], int pos)
+__device__ __forceinline__ float placed_at(const uint32_t (&w)[NW], int pos)
 {
     static_assert(!F::FIXED && F::E < 8 && !HalfPath<F>::value, "generic path");
     const int wi = pos >> 5, sh = pos & 31;
@@ -344,8 +343,17 @@ __device__ __forceinline__ float decode_fast_at(const uint32_t (&w)[NW], int pos
     else
         t = __funnelshift_r(w[wi], w[(wi + 1 < NW) ? wi + 1 : wi], sh + F::B - 32);
     // an arithmetic shift keeps the sign at bit 31; the copies of it that follow are masked away
-    const uint32_t sm = (uint32_t)((int32_t)t >> (8 - F::E)) & (0x80000000u | (F::MAG_MASK << F::SH));
-    return __fmul_rn(u2f(sm), u2f(F::pow2_bits(127 - F::BIAS)));
+    return u2f((uint32_t)((int32_t)t >> (8 - F::E)) & (0x80000000u | (F::MAG_MASK << F::SH)));
+}
+
+// decode_fast of the code at bit position `pos`, without isolating the code first: one shift
+// puts the code's sign at bit 31 (whatever follows the code stays in the low bits), a second one
+// and a mask put exponent and mantissa where FP32 keeps them, and the sign is merged after the
+// rebias multiplication.  Formats on the generic path only (E < 8, not the FP16 family).
+template <class F, int NW>
+__device__ __forceinline__ float decode_fast_at(const uint32_t (&w)[NW], int pos)
+{
+    return __fmul_rn(placed_at<F, NW>(w, pos), u2f(F::pow2_bits(127 - F::BIAS)));
 }
 
 template <class F, int NW>

@@ -194,7 +194,7 @@ static void launch_dyn(const KParams &p, int grid, void *stream)
     omc_dyn_kernel<MODE, WOUT><<<grid, THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p, make_dyn((int)p.dyn_e, (int)p.dyn_m, (int)p.dyn_fixed));
 }
 
-extern const FmtOps ops_dynamic = {-1, -1, -1, WARPS_PER_CTA, launch_dyn<COMPRESS, false>, launch_dyn<DECOMPRESS, false>,
+extern const FmtOps ops_dynamic = {-1, -1, -1, WARPS_PER_CTA, CTAS_PER_SM, launch_dyn<COMPRESS, false>, launch_dyn<DECOMPRESS, false>,
                                    launch_dyn<UPDATE, false>, launch_dyn<UPDATE, true>, nullptr, nullptr, nullptr};
 
 }  // namespace omc

@@ -1491,170 +1491,349 @@ void launch_transition(const KParams &p, int grid, void *stream)
 // Sec. 2.5: each client quantises its own subset, so the server receives precise values of a
 // parameter from the clients that kept it in FP32).  out = (x_0 + x_1 + ... + x_{K-1}) / K per
 // element, FP32, clients added in index order, one rounded division at the end, where x_k is
-// client k's decompressed value fma(s_k, Vt_k, b_k) or its FP32 value.  Plain predicated
-// 128-bit global accesses; every element is read once per client and written once.
+// client k's decompressed value fma(s_k, Vt_k, b_k) or its FP32 value.
+//
+// The tiles are cut into short runs of equal length, dealt out to the warps in turn.  Tile by tile a
+// warp walks the clients in index order with the tile's 32 sums per lane in registers; the codes of
+// the (tile, client) pairs ahead are already on their way into a ring of shared-memory slots, one
+// bulk copy each, so that the bytes in flight do not depend on how many registers a lane has left.
+// FP32 copies of a tile are read with plain vector loads when their turn comes, their lines asked
+// for (an L2 prefetch) when the producer passes them.  Every element is read once per client and
+// written once.  The waits are on the warp's own copies and bounded, as in the other kernels.
 
+// What the tile loop needs to know about one client's copy of the current variable.
+struct AggClientVar {
+    uint64_t base;        // the variable's codes, or its FP32 values
+    uint32_t last_bytes;  // how many bytes of codes its last tile has (padding included)
+    uint32_t quantised;
+    float s, b;
+    float sk;             // s * 2^(127-BIAS) where agg_add can use it (folded != 0)
+    uint32_t folded;
+};
+
+// Shared memory of one warp: a ring of slots, each one client's codes of one tile.
 template <class F>
-__global__ void __launch_bounds__(THREADS, Unit<F>::LU == 32 ? CTAS_PER_SM : 4) omc_aggregate_kernel(const AggParams p)
+struct AggSmem {
+    static constexpr int CB = TILE * F::B / 8;
+    static constexpr int RING_BYTES = 8192;
+    static constexpr int MAX_SLOTS = 8;         // mbarriers reserved per warp
+    static constexpr int NSLOT = RING_BYTES / CB < 2 ? 2 : RING_BYTES / CB > MAX_SLOTS ? MAX_SLOTS : RING_BYTES / CB;
+    static constexpr int PER_WARP = NSLOT * CB;
+    static constexpr int BAR_PAD = (8 * MAX_SLOTS * WARPS_PER_CTA + 127) / 128 * 128;
+    static constexpr int TOTAL = BAR_PAD + WARPS_PER_CTA * PER_WARP;
+    static_assert(CB % 16 == 0, "bulk copies move multiples of 16 bytes");
+};
+
+// Formats whose codes the aggregation decodes by placing the fields (codec.cuh, placed_at).
+template <class F>
+struct PlacedPath {
+    static constexpr bool value = !F::FIXED && F::E < 8 && !HalfPath<F>::value && !Fp8Path<F>::value;
+};
+
+// acc[j] (+)= fma(s, Vt_j, b) for the AL consecutive elements whose codes are the ANW words of
+// `win`; FIRST: the sum starts with this client.
+// FOLDED (PlacedPath only): `sk` is s * 2^(127-BIAS), computed without overflow, hence exactly:
+// Vt = placed * 2^(127-BIAS) exactly, so fma(sk, placed, b) rounds the same real number as
+// fma(s, Vt, b), and the rebias multiplication is never made.
+template <class F, int AL, int ANW, bool FIRST, bool FOLDED>
+__device__ __forceinline__ void agg_add(const uint32_t (&win)[ANW], float s, float sk, float b, float *acc)
+{
+    float x[AL];
+    if constexpr (Fp8Path<F>::value) {
+        // four codes at a time through the narrow-float conversions; Inf/NaN codes redone
+#pragma unroll
+        for (int g = 0; g < AL / 4; ++g) {
+            float dec[4];
+            uint32_t c4;            // the group's codes, one per byte
+            if constexpr (F::B == 8) c4 = win[g];
+            else c4 = spread6(g == 0 ? win[0] : g == 1 ? __funnelshift_r(win[0], win[1], 24)
+                              : g == 2 ? __funnelshift_r(win[1], win[2], 16) : win[2] >> 8);
+            fp8x4_decode<F>(c4, dec);
+            if (F::E != 5 && fp8x4_any_at_least<F, F::INF_MAG>(c4)) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) dec[j] = decode_exact<F>((c4 >> (8 * j)) & 0xFFu);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) x[4 * g + j] = __fmaf_rn(s, dec[j], b);
+        }
+    } else if constexpr (PlacedPath<F>::value) {
+        // eight values at a time, tested together for Inf/NaN codes
+        constexpr int G = AL >= 8 ? 8 : 4;
+#pragma unroll
+        for (int g = 0; g < AL / G; ++g) {
+            float v[G];
+#pragma unroll
+            for (int j = 0; j < G; ++j) v[j] = placed_at<F, ANW>(win, (G * g + j) * F::B);
+            float m = absmax4(v[0], v[1], v[2], v[3]);
+            if constexpr (G == 8) m = fmaxf(m, absmax4(v[4], v[5], v[6], v[7]));
+            if (m >= u2f(F::INF_MAG << F::SH)) {
+#pragma unroll
+                for (int j = 0; j < G; ++j)
+                    x[G * g + j] = __fmaf_rn(s, decode_exact<F>(get_code_at<F, ANW>(win, (G * g + j) * F::B)), b);
+            } else {
+#pragma unroll
+                for (int j = 0; j < G; ++j)
+                    x[G * g + j] = FOLDED ? __fmaf_rn(sk, v[j], b)
+                                          : __fmaf_rn(s, __fmul_rn(v[j], u2f(F::pow2_bits(127 - F::BIAS))), b);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < AL; ++j) x[j] = __fmaf_rn(s, decode_exact<F>(get_code_at<F, ANW>(win, j * F::B)), b);
+    }
+#pragma unroll
+    for (int j = 0; j < AL; ++j) acc[j] = FIRST ? x[j] : __fadd_rn(acc[j], x[j]);
+}
+
+// One client's codes of one tile, in a slot of the ring: each lane adds its 32 values to its sums.
+template <class F, bool FIRST, bool FOLDED>
+__device__ __forceinline__ void agg_tile_codes(const uint32_t *sw, float s, float sk, float b, float (&acc)[32], int lane)
 {
     using U = Unit<F>;
-    constexpr int LU = U::LU, NW = U::NWORDS;
-    const int lane = threadIdx.x & 31;
-    const uint32_t warp = blockIdx.x * WARPS_PER_CTA + (threadIdx.x >> 5);
+    // A lane takes AL consecutive elements at a time, at least four (one 16-byte store), NQ times per tile.
+    constexpr int UF = U::LU < 4 ? 4 / U::LU : 1, AL = U::LU * UF, ANW = U::NWORDS * UF, NQ = 32 / AL;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        uint32_t win[ANW];
+        const uint32_t *uw = sw + (q * 32 + lane) * ANW;
+        if constexpr (ANW % 4 == 0) {
+#pragma unroll
+            for (int j = 0; j < ANW / 4; ++j) {
+                const uint4 w4 = reinterpret_cast<const uint4 *>(uw)[j];
+                win[4 * j] = w4.x; win[4 * j + 1] = w4.y; win[4 * j + 2] = w4.z; win[4 * j + 3] = w4.w;
+            }
+        } else if constexpr (ANW % 2 == 0) {
+#pragma unroll
+            for (int j = 0; j < ANW / 2; ++j) {
+                const uint2 w2 = reinterpret_cast<const uint2 *>(uw)[j];
+                win[2 * j] = w2.x; win[2 * j + 1] = w2.y;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < ANW; ++j) win[j] = uw[j];
+        }
+        agg_add<F, AL, ANW, FIRST, FOLDED>(win, s, sk, b, acc + q * AL);
+    }
+}
+
+// One client's FP32 values of one tile, element e of the tile at r[e]: the same elements per lane.
+// WHOLE: the tile lies inside the variable; otherwise only the first `n_pad` floats exist.
+template <class F, bool FIRST, bool WHOLE>
+__device__ __forceinline__ void agg_tile_fp32(const float *r, uint32_t n_pad, float (&acc)[32], int lane)
+{
+    using U = Unit<F>;
+    constexpr int UF = U::LU < 4 ? 4 / U::LU : 1, AL = U::LU * UF, NQ = 32 / AL;
+    float4 f[8];
+#pragma unroll
+    for (int q = 0; q < NQ; ++q)
+#pragma unroll
+        for (int j = 0; j < AL / 4; ++j) {
+            const uint32_t e = (uint32_t)(q * 32 + lane) * AL + 4 * j;
+            f[q * (AL / 4) + j] = (WHOLE || e < n_pad) ? __ldcs(reinterpret_cast<const float4 *>(r + e))
+                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        acc[4 * i] = FIRST ? f[i].x : __fadd_rn(acc[4 * i], f[i].x);
+        acc[4 * i + 1] = FIRST ? f[i].y : __fadd_rn(acc[4 * i + 1], f[i].y);
+        acc[4 * i + 2] = FIRST ? f[i].z : __fadd_rn(acc[4 * i + 2], f[i].z);
+        acc[4 * i + 3] = FIRST ? f[i].w : __fadd_rn(acc[4 * i + 3], f[i].w);
+    }
+}
+
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+template <class F>
+__global__ void __launch_bounds__(THREADS, aggregate_ctas_per_sm(F::B)) omc_aggregate_kernel(const AggParams p)
+{
+    using U = Unit<F>;
+    using AS = AggSmem<F>;
+    constexpr int UF = U::LU < 4 ? 4 / U::LU : 1, AL = U::LU * UF, NQ = 32 / AL;
+    constexpr uint32_t CB = AS::CB, NSLOT = AS::NSLOT;
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    __shared__ AggClientVar cv_all[WARPS_PER_CTA][MAX_CLIENTS];
+    int lane;
+    asm volatile("mov.u32 %0, %%laneid;" : "=r"(lane));
+    const int wid = threadIdx.x >> 5;
+    const uint32_t warp = blockIdx.x * WARPS_PER_CTA + wid;
     if (warp >= p.nwarps) return;
-    uint64_t t = (uint64_t)warp * p.tile_count / p.nwarps;
-    const uint64_t tend = (uint64_t)(warp + 1) * p.tile_count / p.nwarps;
+    uint8_t *const ring = smem_raw + AS::BAR_PAD + wid * AS::PER_WARP;
+    const uint32_t bar0 = smem_addr(smem_raw) + (uint32_t)wid * AS::MAX_SLOTS * 8u;
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < (int)NSLOT; ++i) mbar_init(bar0 + 8u * i, 1u);
+        fence_mbar_init();
+        fence_proxy_async();
+    }
+    __syncwarp();
+    AggClientVar *cv = cv_all[wid];
+    const uint32_t K = p.nclients;
+    const uint32_t wait_limit = p.wait_limit ? p.wait_limit : WAIT_LIMIT;
+    const bool skip_loads = p.skip_loads != 0u;
+    uint32_t phases = 0u;            // bit i: the parity the next wait on slot i looks for
+    uint32_t pslot = 0u, cslot = 0u; // the slot filled next, the slot read next
+    uint32_t in_ring = 0u;           // copies issued and not yet consumed
+    bool failed = false;
+    // FP32 copies the producer has passed and the consumer has not yet read: at most FP32_AHEAD, so
+    // that what is prefetched for all warps together stays a fraction of the L2
+    constexpr uint32_t FP32_AHEAD = 3;
+    uint32_t fp32_ahead = 0u;
+    const float kf = (float)K;
+    // Dividing by a power of two is a multiplication by its exact reciprocal: both are the correctly
+    // rounded value of the same real number.
+    const bool pow2 = (K & (K - 1)) == 0;
+    const float kinv = 1.f / kf;
+    const bool divide = p.divide != 0u;
+    auto mean_of = [&](float a) { return !divide ? a : pow2 ? __fmul_rn(a, kinv) : __fdiv_rn(a, kf); };
+
+    // Short runs of equal length, dealt out to the warps in turn: what a tile costs depends on how many
+    // clients hold it in FP32, and a long stretch of costly tiles is shared by all warps this way.
+    for (uint32_t run = warp; run < p.nruns && !failed; run += p.nwarps) {
+    uint64_t t = (uint64_t)run * p.tile_count / p.nruns;
+    const uint64_t tend = (uint64_t)(run + 1) * p.tile_count / p.nruns;
     uint32_t lo = 0, hi = p.nvars;
     while (hi - lo > 1) {
         const uint32_t mid = (lo + hi) >> 1;
         if (__ldg(&p.vars[0][mid].tile_start) <= t) lo = mid; else hi = mid;
     }
     uint32_t v = lo;
-    const float kf = (float)p.nclients;
-    // Dividing by a power of two is a multiplication by its exact reciprocal: both are the correctly
-    // rounded value of the same real number.
-    const bool pow2 = (p.nclients & (p.nclients - 1)) == 0;
-    const float kinv = 1.f / kf;
-    auto mean_of = [&](float a) { return !p.divide ? a : pow2 ? __fmul_rn(a, kinv) : __fdiv_rn(a, kf); };
-    // per warp: what the unit loop needs to know about each client's copy of the current variable
-    struct ClientVar { uint64_t base; uint32_t nwords; uint32_t quantised; float s, b; uint32_t pad[2]; };
-    __shared__ ClientVar cv_all[WARPS_PER_CTA][MAX_CLIENTS];
-    ClientVar *cv = cv_all[threadIdx.x >> 5];
-    while (t < tend) {
+
+    while (t < tend && !failed) {
         const VarDev var = load_var(p.vars[0] + v);
         __syncwarp();
-        if ((uint32_t)lane < p.nclients) {
+        if ((uint32_t)lane < K) {
             const VarDev vk = load_var(p.vars[lane] + v);
-            ClientVar c;
+            AggClientVar c;
             c.quantised = vk.quantised;
-            c.nwords = (uint32_t)(vk.packed_bytes / 4);
+            c.last_bytes = vk.ntiles ? (uint32_t)(vk.packed_bytes - (uint64_t)(vk.ntiles - 1) * CB) : 0u;
             c.base = vk.quantised ? reinterpret_cast<uint64_t>(p.packed[lane] + vk.store_off)
                                   : reinterpret_cast<uint64_t>(p.resid[lane] + vk.store_off);
             c.s = vk.quantised ? __ldg(p.sb[lane] + 2 * vk.sb_slot) : 1.f;
             c.b = vk.quantised ? __ldg(p.sb[lane] + 2 * vk.sb_slot + 1) : 0.f;
-            c.pad[0] = c.pad[1] = 0u;
+            c.sk = c.s;
+            c.folded = 0u;
+            if constexpr (PlacedPath<F>::value) {
+                c.sk = __fmul_rn(c.s, u2f(F::pow2_bits(127 - F::BIAS)));
+                c.folded = fabsf(c.sk) < u2f(0x7F800000u) ? 1u : 0u;       // no overflow: the product is exact
+            }
             cv[lane] = c;
         }
         __syncwarp();
         const uint32_t local = (uint32_t)(t - var.tile_start);
         const uint64_t left = tend - t;
         const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
-        const uint64_t e_begin = (uint64_t)local * TILE;
-        const uint64_t e_end = (uint64_t)(local + cnt) * TILE < var.n ? (uint64_t)(local + cnt) * TILE : var.n;
-        const uint64_t n_pad = (var.n + 3) & ~3ull;
-        // A lane takes AL consecutive elements per step: at least 8, so that its codes are 8 to 16
-        // contiguous bytes per client (one vector load where the width allows it).
-        constexpr int UF = LU < 8 ? 8 / LU : 1, AL = LU * UF, ANW = NW * UF;
-        for (uint64_t e0 = e_begin + (uint64_t)lane * AL; e0 < e_end; e0 += 32 * AL) {
-            float acc[AL];
-#pragma unroll
-            for (int j = 0; j < AL; ++j) acc[j] = 0.f;
-            const uint64_t w0 = e0 / AL * ANW;
-            // clients in batches: first every load of the batch, then the arithmetic, in index order
-            constexpr int KB = AL >= 32 ? 1 : 4, WMAX = ANW > AL ? ANW : AL;
-            for (uint32_t k0 = 0; k0 < p.nclients; k0 += KB) {
-                uint32_t w[KB][WMAX];
-#pragma unroll
-                for (int kk = 0; kk < KB; ++kk) {
-                    if (k0 + kk >= p.nclients) break;
-                    const ClientVar c = cv[k0 + kk];
-                    if (c.quantised) {
-                        // packed sizes are multiples of 16 bytes: an aligned 8- or 16-byte group is inside or outside as a whole
-                        const uint32_t *cw = reinterpret_cast<const uint32_t *>(c.base) + w0;
-                        if constexpr (ANW == 4) {
-                            const uint4 q = (w0 < c.nwords) ? __ldcs(reinterpret_cast<const uint4 *>(cw)) : make_uint4(0u, 0u, 0u, 0u);
-                            w[kk][0] = q.x; w[kk][1] = q.y; w[kk][2] = q.z; w[kk][3] = q.w;
-                        } else if constexpr (ANW == 2) {
-                            const uint2 q = (w0 < c.nwords) ? __ldcs(reinterpret_cast<const uint2 *>(cw)) : make_uint2(0u, 0u);
-                            w[kk][0] = q.x; w[kk][1] = q.y;
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < ANW; ++j) w[kk][j] = (w0 + j < c.nwords) ? __ldcs(cw + j) : 0u;
-                        }
-                    } else {
-                        const float *r = reinterpret_cast<const float *>(c.base) + e0;
-#pragma unroll
-                        for (int j = 0; j < AL / 4; ++j) {
-                            const float4 q = (e0 + 4 * j < n_pad) ? __ldcs(reinterpret_cast<const float4 *>(r) + j)
-                                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
-                            w[kk][4 * j] = __float_as_uint(q.x); w[kk][4 * j + 1] = __float_as_uint(q.y);
-                            w[kk][4 * j + 2] = __float_as_uint(q.z); w[kk][4 * j + 3] = __float_as_uint(q.w);
-                        }
+
+        // the producer's place in this variable's (tile, client) pairs
+        uint32_t ptile = 0u, pk = 0u;
+        auto fill = [&]() {                     // called by the whole warp
+            while (ptile < cnt && in_ring < NSLOT && fp32_ahead < FP32_AHEAD) {
+                const AggClientVar c = cv[pk];
+                if (c.quantised) {
+                    // packed sizes are multiples of 16 bytes, and so is what is left of one in its last tile
+                    const uint64_t off = (uint64_t)(local + ptile) * CB;
+                    const uint32_t bytes = local + ptile + 1 == var.ntiles ? c.last_bytes : CB;
+                    if (lane == 0) {
+                        const uint32_t bar = bar0 + 8u * pslot;
+                        mbar_expect_tx(bar, bytes);
+                        if (!skip_loads)
+                            bulk_load(smem_addr(ring + pslot * CB), reinterpret_cast<const uint8_t *>(c.base) + off, bytes, bar);
                     }
+                    pslot = pslot + 1 == NSLOT ? 0u : pslot + 1;
+                    ++in_ring;
+                } else {
+                    // an FP32 copy is read with plain loads when its turn comes: ask for its lines now
+                    const uint64_t e = (uint64_t)(local + ptile) * TILE + (uint32_t)lane * 32u;
+                    if (e < var.n) prefetch_l2(reinterpret_cast<const float *>(c.base) + e);
+                    ++fp32_ahead;
                 }
-#pragma unroll
-                for (int kk = 0; kk < KB; ++kk) {
-                    if (k0 + kk >= p.nclients) break;
-                    const ClientVar c = cv[k0 + kk];
-                    float x[AL];
-                    if (c.quantised) {
-                        uint32_t win[ANW];
-#pragma unroll
-                        for (int j = 0; j < ANW; ++j) win[j] = w[kk][j];
-                        if constexpr (Fp8Path<F>::value) {
-                            // four codes at a time through the narrow-float conversions; Inf/NaN codes redone
-#pragma unroll
-                            for (int g = 0; g < AL / 4; ++g) {
-                                float dec[4];
-                                uint32_t c4;            // the group's codes, one per byte
-                                if constexpr (F::B == 8) c4 = win[g];
-                                else c4 = spread6(g == 0 ? win[0] : g == 1 ? __funnelshift_r(win[0], win[1], 24)
-                                                  : g == 2 ? __funnelshift_r(win[1], win[2], 16) : win[2] >> 8);
-                                fp8x4_decode<F>(c4, dec);
-                                if (F::E != 5 && fp8x4_any_at_least<F, F::INF_MAG>(c4)) {
-#pragma unroll
-                                    for (int j = 0; j < 4; ++j) dec[j] = decode_exact<F>((c4 >> (8 * j)) & 0xFFu);
-                                }
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) x[4 * g + j] = __fmaf_rn(c.s, dec[j], c.b);
-                            }
-                        } else if constexpr (!F::FIXED && F::E < 8 && !HalfPath<F>::value) {
-                            // generic path: decode from the word, test four values at once for Inf/NaN codes
-#pragma unroll
-                            for (int g = 0; g < AL / 4; ++g) {
-                                float dec[4];
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) dec[j] = decode_fast_at<F, ANW>(win, (4 * g + j) * F::B);
-                                if (any_code_special4<F>(dec)) {
-#pragma unroll
-                                    for (int j = 0; j < 4; ++j) dec[j] = decode_exact<F>(get_code_at<F, ANW>(win, (4 * g + j) * F::B));
-                                }
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) x[4 * g + j] = __fmaf_rn(c.s, dec[j], c.b);
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < AL; ++j)
-                                x[j] = __fmaf_rn(c.s, decode_exact<F>(get_code_at<F, ANW>(win, j * F::B)), c.b);
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < AL; ++j) x[j] = __uint_as_float(w[kk][j]);
-                    }
-#pragma unroll
-                    for (int j = 0; j < AL; ++j) acc[j] = (k0 + kk == 0) ? x[j] : __fadd_rn(acc[j], x[j]);
-                }
+                if (++pk == K) { pk = 0u; ++ptile; }
             }
-            float *o = p.out + var.full_off + e0;
+        };
+
+        for (uint32_t ti = 0; ti < cnt && !failed; ++ti) {
+            fill();
+            const uint64_t e_tile = (uint64_t)(local + ti) * TILE;
+            const bool whole = e_tile + TILE <= var.n;
+            const uint32_t n_here = whole ? (uint32_t)TILE : (uint32_t)(var.n - e_tile);     // the tile's elements
+            const uint32_t n_pad = (n_here + 3u) & ~3u;
+            float acc[32];
+            // client k's turn; false: the wait for its codes ran out
+            auto client = [&](auto first, uint32_t k) -> bool {
+                constexpr bool FIRST = decltype(first)::value;
+                const AggClientVar c = cv[k];
+                if (c.quantised) {
+                    const uint32_t bar = bar0 + 8u * cslot, parity = (phases >> cslot) & 1u;
+                    phases ^= 1u << cslot;
+                    uint32_t polls = 0;
+                    while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) {
+                        if (++polls > wait_limit) return false;
+                    }
+                    const uint32_t *sw = reinterpret_cast<const uint32_t *>(ring + cslot * CB);
+                    if constexpr (PlacedPath<F>::value) {
+                        if (c.folded) agg_tile_codes<F, FIRST, true>(sw, c.s, c.sk, c.b, acc, lane);
+                        else agg_tile_codes<F, FIRST, false>(sw, c.s, c.sk, c.b, acc, lane);
+                    } else {
+                        agg_tile_codes<F, FIRST, false>(sw, c.s, c.s, c.b, acc, lane);
+                    }
+                    __syncwarp();               // every lane has read the slot: it may be filled again
+                    cslot = cslot + 1 == NSLOT ? 0u : cslot + 1;
+                    --in_ring;
+                    fill();
+                } else {
+                    const float *r = reinterpret_cast<const float *>(c.base) + e_tile;
+                    if (whole) agg_tile_fp32<F, FIRST, true>(r, n_pad, acc, lane);
+                    else agg_tile_fp32<F, FIRST, false>(r, n_pad, acc, lane);
+                    --fp32_ahead;
+                    fill();
+                }
+                return true;
+            };
+            failed = !client(std::true_type{}, 0u);
+            for (uint32_t k = 1; k < K && !failed; ++k) failed = !client(std::false_type{}, k);
+            if (failed) break;
+            float *o = p.out + var.full_off + e_tile;
 #pragma unroll
-            for (int j = 0; j < AL / 4; ++j)
-                if (e0 + 4 * j < n_pad)
-                    reinterpret_cast<float4 *>(o)[j] = make_float4(mean_of(acc[4 * j]), mean_of(acc[4 * j + 1]),
-                                                                   mean_of(acc[4 * j + 2]), mean_of(acc[4 * j + 3]));
+            for (int q = 0; q < NQ; ++q)
+#pragma unroll
+                for (int j = 0; j < AL / 4; ++j) {
+                    const uint32_t e = (uint32_t)(q * 32 + lane) * AL + 4 * j;
+                    const int i = q * AL + 4 * j;
+                    float4 m = make_float4(mean_of(acc[i]), mean_of(acc[i + 1]), mean_of(acc[i + 2]), mean_of(acc[i + 3]));
+                    if (whole) {
+                        *reinterpret_cast<float4 *>(o + e) = m;
+                    } else if (e < n_pad) {
+                        if (e + 3 >= n_here) {          // the padding after the variable's last element: zeros
+                            if (e + 1 >= n_here) m.y = 0.f;
+                            if (e + 2 >= n_here) m.z = 0.f;
+                            m.w = 0.f;
+                        }
+                        *reinterpret_cast<float4 *>(o + e) = m;
+                    }
+                }
         }
         t += cnt;
         ++v;
     }
+    }
+    if (failed && lane == 0) atomicExch(p.status, 1u);       // a bulk load never arrived
 }
 
 template <class F>
 void launch_aggregate(const AggParams &p, int grid, void *stream)
 {
-    omc_aggregate_kernel<F><<<grid, THREADS, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    static bool configured[64] = {};    // once per device and instantiation
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        cudaFuncSetAttribute(omc_aggregate_kernel<F>, cudaFuncAttributeMaxDynamicSharedMemorySize, AggSmem<F>::TOTAL);
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    omc_aggregate_kernel<F><<<grid, THREADS, AggSmem<F>::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
 }
 
 #define OMC_DEFINE_FIXED_FORMAT(I_, F_)                                                         \
     extern const FmtOps ops_I##I_##F##F_ = {I_, F_, 1, fit_warps_per_cta(1 + I_ + F_, true),    \
+                                            aggregate_ctas_per_sm(1 + I_ + F_),                 \
                                             launch<FixFmt<I_, F_>, COMPRESS, false>,            \
                                             launch<FixFmt<I_, F_>, DECOMPRESS, false>,          \
                                             launch<FixFmt<I_, F_>, UPDATE, false>,              \
@@ -1665,6 +1844,7 @@ void launch_aggregate(const AggParams &p, int grid, void *stream)
 
 #define OMC_DEFINE_FORMAT(E_, M_)                                                               \
     extern const FmtOps ops_E##E_##M##M_ = {E_, M_, 0, fit_warps_per_cta(1 + E_ + M_, false),   \
+                                            aggregate_ctas_per_sm(1 + E_ + M_),                 \
                                             launch<Fmt<E_, M_>, COMPRESS, false>,               \
                                             launch<Fmt<E_, M_>, DECOMPRESS, false>,             \
                                             launch<Fmt<E_, M_>, UPDATE, false>,                 \

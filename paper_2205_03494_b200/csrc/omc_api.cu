@@ -364,9 +364,14 @@ static int aggregate_impl(const omc_plan_t *const *plans, uint32_t n_clients, co
     p.divide = divide;
     p.nvars = first->nvars;
     p.tile_count = first->ntiles;
-    const uint64_t max_warps = (uint64_t)first->n_cta * omc::WARPS_PER_CTA * 2;    // light kernel: 4 CTAs per SM fit
+    const uint64_t max_warps = (uint64_t)first->n_sm * first->ops->agg_ctas * omc::WARPS_PER_CTA;
     p.nwarps = (uint32_t)(p.tile_count < max_warps ? p.tile_count : max_warps);
+    p.nruns = omc::runs_for(p.tile_count, p.nwarps, omc::aggregate_tiles_per_run(n_clients), omc::DECODE_MAX_RUNS);
     p.out = out;
+    p.status = first->d_status;
+    p.wait_limit = first->inject_polls;       // the diagnostic of omc_plan_inject_wait_timeout, for one launch
+    p.skip_loads = first->inject_polls ? 1u : 0u;
+    first->inject_polls = 0;
     first->ops->aggregate(p, grid_for(p.nwarps), stream);
     return omc::note_cuda(cudaGetLastError());
 }

@@ -22,6 +22,9 @@ constexpr int fit_warps_per_cta(int code_bits, bool /*fixed_point*/)
     return (code_bits == 12 || code_bits == 19) ? 6 : WARPS_PER_CTA;
 }
 constexpr int CTAS_PER_SM = 2;
+// CTAs per SM of the aggregation: with 8-bit codes it fits the 80 registers that three leave it
+// (measured 11-14 % faster than two); with any other width it spills there (up to 29 % slower).
+constexpr int aggregate_ctas_per_sm(int code_bits) { return code_bits == 8 ? 3 : CTAS_PER_SM; }
 // The decompress kernel divides its tiles at launch, so its grid is independent of the plan's division.
 constexpr int DECOMPRESS_CTAS_PER_SM = 2;
 constexpr int DEFAULT_SMS = 148;   // B200; used when no device can be queried at plan time
@@ -140,13 +143,18 @@ struct AggParams {
     uint32_t nvars;
     uint64_t tile_count;
     uint32_t nwarps;
+    uint32_t nruns;                      // equal runs of tiles, run r to warp r mod nwarps
     float *out;                          // full layout
+    uint32_t *status;                    // set to 1 by a warp whose wait for a bulk copy ran out
+    uint32_t wait_limit;                 // polls of one mbarrier before giving up; 0: the default
+    uint32_t skip_loads;                 // diagnostics: announce the bulk loads, do not issue them
 };
 
 struct FmtOps {
     int E, M;          // fixed != 0: integer bits and fraction bits of S1IxFy
     int fixed;
     int fit_warps;     // warps per CTA of compress / update / transition (the decoder and the aggregation use WARPS_PER_CTA)
+    int agg_ctas;      // CTAs per SM of the aggregation
     void (*compress)(const KParams &, int grid, void *stream);
     void (*decompress)(const KParams &, int grid, void *stream);
     void (*update)(const KParams &, int grid, void *stream);     // W not stored
@@ -170,6 +178,11 @@ uint32_t runs_for(uint64_t tiles, uint32_t nwarps, uint32_t tiles_per_run, uint3
 // pipeline granules per run; one-tile runs are slower than none at all).
 constexpr uint32_t decode_tiles_per_run(uint32_t code_bits) { return code_bits >= 16 ? 4u : 2u; }
 constexpr uint32_t DECODE_MAX_RUNS = 1u << 22;
+// The aggregation's runs, in tiles: about 64 (tile, client) pairs each.
+constexpr uint32_t aggregate_tiles_per_run(uint32_t nclients)
+{
+    return nclients >= 16 ? 4u : nclients <= 2 ? 32u : 64u / nclients;
+}
 
 #ifdef __CUDACC__
 // The tiles [t, tend) of run `run`.

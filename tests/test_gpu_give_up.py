@@ -56,6 +56,40 @@ def test_wait_runs_out_then_plan_works_again(call, fmt):
     ls.check_decompress()
 
 
+@pytest.mark.parametrize("fmt", [(5, 10), (5, 2), (3, 7)], ids=lambda f: "E%dM%d" % f)
+def test_aggregate_wait_runs_out_then_works_again(fmt):
+    """omc_aggregate streams the clients' codes through bounded waits of its own; the give-up is
+    reported through the first plan's status word."""
+    rng = np.random.default_rng(23)
+    clients = []
+    for k in range(3):
+        params = [(rng.standard_normal(n) * 0.1).astype(np.float32) for n in NUMEL]
+        clients.append(Lockstep(NUMEL, KINDS, fmt, params, fraction=0.7, seed=5 + k))
+    plan0, dm0 = clients[0].plan, clients[0].dm
+    st = torch.cuda.current_stream().cuda_stream
+    out = dm0.full_buffer("mean")
+    run = lambda: omc.aggregate([c.plan for c in clients], [c.dm.packed.data_ptr() for c in clients],
+                                [c.dm.resid.data_ptr() for c in clients], [c.dm.sb.data_ptr() for c in clients],
+                                out.data_ptr(), st)
+    plan0.inject_wait_timeout(1 << 10)
+    run()
+    torch.cuda.synchronize()
+    assert plan0.status(st) != 0
+    for c in clients:
+        c.dm.check_guards()
+    plan0.prepare(dm0.ws.data_ptr(), st)
+    assert plan0.status(st) == 0
+    run()
+    torch.cuda.synchronize()
+    assert plan0.status(st) == 0
+    dm0.check_guards()
+    got = out.cpu().numpy()
+    want = orc.aggregate([c.st for c in clients])
+    for i in range(len(NUMEL)):
+        o = plan0.full_off[i]
+        assert np.array_equal(got[o:o + NUMEL[i]].view(np.uint32), want[i].view(np.uint32)), i
+
+
 def test_matmul_wait_runs_out_then_works_again():
     rng = np.random.default_rng(3)
     N, K, M = 256, 128, 200

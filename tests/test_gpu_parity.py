@@ -466,8 +466,9 @@ def test_transition_refuses_mismatched_plans():
     torch.cuda.synchronize()
 
 
-@pytest.mark.parametrize("K", [5, 8], ids=lambda k: "K%d" % k)
-@pytest.mark.parametrize("fmt", [(5, 2), (5, 6), (5, 10), (3, 7), (4, 14)], ids=lambda f: "E%dM%d" % f)
+@pytest.mark.parametrize("K", [5, 8, 16], ids=lambda k: "K%d" % k)
+@pytest.mark.parametrize("fmt", [(5, 2), (4, 3), (2, 3), (5, 6), (5, 10), (3, 7), (5, 7), (4, 14), (8, 7), (8, 23)],
+                         ids=lambda f: "E%dM%d" % f)
 def test_aggregate_client_replicas(fmt, K):
     """Server-side mean of K clients that each quantised their own random subset (Sec. 2.5) against
     the oracle's aggregate (every client decompressed, FP32 mean in client order, one division)."""
@@ -488,6 +489,8 @@ def test_aggregate_client_replicas(fmt, K):
                   [c.dm.resid.data_ptr() for c in clients], [c.dm.sb.data_ptr() for c in clients],
                   out.data_ptr(), torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
+    for c in clients:
+        c.dm.check_guards()
     got = out.cpu().numpy()
     dec = [orc.decompress(c.st) for c in clients]
     want = orc.aggregate([c.st for c in clients])
@@ -502,6 +505,38 @@ def test_aggregate_client_replicas(fmt, K):
         assert same_f32(from_full(clients[1].plan, got, i), dec[1][i]), i
     L = omc.lib()
     assert L.omc_aggregate(None, 1, None, None, None, out.data_ptr(), None) == -3
+
+
+@pytest.mark.parametrize("fmt", [(3, 7), (4, 14), (5, 7), (4, 3), (5, 6)], ids=lambda f: "E%dM%d" % f)
+def test_aggregate_with_extreme_transformations(fmt):
+    """(s, b) are data to the aggregation: whatever a client delivers, each value is
+    fma(s, Vt, b).  Huge, tiny, negative and non-finite scales, written into the clients' (s, b)
+    arrays on both sides, take the kernel off any path that pre-scales s."""
+    rng = np.random.default_rng(41)
+    numel = [2048, 700, 1024, 3333, 5000, 64, 1500]
+    kinds = [0] * len(numel)
+    odd = [(1e30, 0.5), (np.inf, 0.0), (np.nan, 1.0), (1e-42, -2.0), (-3.0e37, 1e38), (16.0, 0.0), (-0.0, -0.0)]
+    clients = []
+    for k in range(4):
+        params = [(rng.standard_normal(n) * 0.1).astype(np.float32) for n in numel]
+        c = Lockstep(numel, kinds, fmt, params, seed=70 + k)
+        for i in range(len(numel)):
+            if (i + k) % 2 == 0:
+                sv, bv = odd[(i + 2 * k) % len(odd)]
+                slot = c.plan.sb_slot[i]
+                c.dm.sb[2 * slot], c.dm.sb[2 * slot + 1] = float(sv), float(bv)
+                c.st["s"][i], c.st["b"][i] = np.float32(sv), np.float32(bv)
+        clients.append(c)
+    out = clients[0].dm.full_buffer("mean")
+    omc.aggregate([c.plan for c in clients], [c.dm.packed.data_ptr() for c in clients],
+                  [c.dm.resid.data_ptr() for c in clients], [c.dm.sb.data_ptr() for c in clients],
+                  out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    clients[0].dm.check_guards()
+    got = out.cpu().numpy()
+    want = orc.aggregate([c.st for c in clients])
+    for i in range(len(numel)):
+        assert same_f32(from_full(clients[0].plan, got, i), want[i]), i
 
 
 @pytest.mark.parametrize("fmt", [(5, 10), (5, 2), (3, 7)], ids=lambda f: "E%dM%d" % f)
