@@ -1278,6 +1278,12 @@ omc_kernel(const KParams p)
         fence_proxy_async();
     }
     __syncwarp();
+    // Where the launch is the programmatic dependent of the kernel before it on the stream
+    // (KParams::dependent), the launch and the set-up above overlap that kernel's last warps; nothing
+    // of global memory is touched before it has completed.  The kernel after this one may be set up
+    // the same way.  In an ordinary launch both instructions do nothing.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     for (uint32_t run = warp; run < p.nruns && !pipe.failed; run += p.nwarps) {
         uint64_t t, tend;
@@ -1341,7 +1347,21 @@ void launch(const KParams &p, int grid, void *stream)
         cudaFuncSetAttribute(omc_kernel<F, MODE, WOUT, QUEUE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL);
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    omc_kernel<F, MODE, WOUT, QUEUE><<<grid, 32 * SM::WARPS, SM::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
+    if (p.dependent) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(32 * SM::WARPS);
+        cfg.dynamicSmemBytes = SM::TOTAL;
+        cfg.stream = static_cast<cudaStream_t>(stream);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaLaunchKernelEx(&cfg, omc_kernel<F, MODE, WOUT, QUEUE>, p);
+    } else {
+        omc_kernel<F, MODE, WOUT, QUEUE><<<grid, 32 * SM::WARPS, SM::TOTAL, static_cast<cudaStream_t>(stream)>>>(p);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------

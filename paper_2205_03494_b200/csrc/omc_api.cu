@@ -119,6 +119,7 @@ static KParams whole_model(const omc_plan_t *plan, void *workspace)
 {
     KParams p{};
     take_injection(plan, p);
+    p.dependent = 1u;
     p.vars = plan->d_vars;
     p.var_begin = 0;
     p.var_end = plan->nvars;
@@ -193,6 +194,7 @@ extern "C" int omc_decompress(const omc_plan_t *plan, const uint8_t *packed, con
     if (misaligned(packed) || misaligned(resid) || misaligned(sb) || misaligned(out)) return OMC_ERR_MISALIGNED;
     KParams p{};
     take_injection(plan, p);
+    p.dependent = n_vars != plan->nvars ? 1u : 0u;
     p.vars = plan->d_vars;
     p.var_begin = first_var;
     p.var_end = first_var + n_vars;

@@ -110,6 +110,13 @@ struct KParams {
     // so that the waits run out with nothing in flight.
     uint32_t wait_limit;
     uint32_t skip_loads;
+    // Host side: launch as the programmatic dependent of the kernel before it on the stream.  On for
+    // the fused round and compress (measured on the 100M set: 1.5-2.6 % per round in a row of rounds,
+    // nothing lost on the larger sets) and for omc_decompress of a part of the model (17 block-wise
+    // calls 12.3 -> 10.7 us each); off for whole-model decompress calls in a row, which lose with
+    // 8-bit codes (0.0845 -> 0.0926 ms: the CTAs of a dependent launch take their SMs in the order
+    // in which the kernel before it leaves them).
+    uint32_t dependent;
 };
 
 // omc_transition's own division of the work, made on the device before each launch.
