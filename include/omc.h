@@ -13,6 +13,11 @@
  *     the caller, 16-byte aligned, valid until the work queued on `stream` has finished.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device calls only
  *     enqueue work; they do not synchronise.  Apart from omc_plan_prepare they allocate nothing.
+ *     Work queued on one stream runs in stream order.  The library's kernels allow the launch of
+ *     a programmatic dependent early (griddepcontrol.launch_dependents) and wait for the kernel
+ *     before them themselves; a kernel of the caller's that is launched with programmatic stream
+ *     serialization right after a library call must, like any such kernel, call
+ *     cudaGridDependencySynchronize() before it reads what that call wrote.
  *   - Non-finite values are data, never errors: they propagate as IEEE-754 prescribes.
  *   - A plan is not thread-safe; distinct plans are independent.
  *
