@@ -532,14 +532,17 @@ def run_ours(args):
         xh = (torch.randn(Mm, Km, device=dev) * 0.5).half()
         yo = torch.empty(Mm, Nm, dtype=torch.float32, device=dev)
         rs = torch.empty(Mm, dtype=torch.float32, device=dev)
-        for mfmt in ((5, 10), (5, 6), (5, 2), (4, 3), (2, 3), (5, 7), (3, 7), (3, 9), (4, 8), (4, 14)):
-            key = "matmul_from_codes_8192x8192x2048_S1E%dM%d" % mfmt
+        for mfmt in ((5, 10), (5, 6), (5, 2), (4, 3), (2, 3), (5, 7), (3, 7), (3, 9), (4, 8), (4, 14),
+                     (0, 7, "fixed"), (0, 11, "fixed"), (0, 15, "fixed")):
+            mfixed = len(mfmt) == 3
+            mfmt = mfmt[:2]
+            key = "matmul_from_codes_8192x8192x2048_" + ("S1I%dF%d" if mfixed else "S1E%dM%d") % mfmt
             try:
-                pm = omc.Plan([Nm * Km], [0], mfmt)
+                pm = omc.Plan([Nm * Km], [0], mfmt, fixed=mfixed)
                 bm = (z(pm.packed_bytes, torch.uint8), z(16, torch.float32), z(2, torch.float32),
                       z(pm.workspace_bytes, torch.uint8))
                 pm.prepare(bm[3].data_ptr(), stream)
-                wfmt = wsrc * 25.0 if mfmt == (2, 3) else wsrc       # S1E2M3 resolves nothing below 1/8
+                wfmt = wsrc * 25.0 if mfmt == (2, 3) and not mfixed else wsrc       # S1E2M3 resolves nothing below 1/8
                 pm.compress(wfmt.data_ptr(), bm[0].data_ptr(), bm[1].data_ptr(), bm[2].data_ptr(), bm[3].data_ptr(), stream)
                 torch.cuda.synchronize()
                 del wfmt

@@ -56,9 +56,9 @@ extern "C" {
  * (there is no infinity; +-Inf saturate too); NaN has no code and becomes 0.  The scale is fixed
  * by the format and not taken from the data (that would cost the one-pass update a second pass);
  * the per-variable transformation of Sec. 2.3 adapts to the variable as it does for the
- * floating-point codes.  Layouts, packing and every call are the same; omc_matmul accepts only
- * floating-point codes.  Q7, Q11 and Q15 (x = 0) have compiled kernels; the other formats run on
- * the slower kernels that take the format at run time. */
+ * floating-point codes.  Layouts, packing and every call are the same.  Q7, Q11 and Q15 (x = 0)
+ * have compiled kernels (omc_matmul accepts these three); the other formats run on the slower
+ * kernels that take the format at run time. */
 typedef struct {
     uint8_t sign_bits, exp_bits, man_bits, flags;
 } omc_format_t;
@@ -299,8 +299,9 @@ int omc_divide(const omc_plan_t *plan, float *values, uint32_t divisor, void *st
  *   of 11-, 13- or 19-bit codes must be whole 16-byte units for the bulk tensor copies); S1E4M14
  *   (Table 1) has 15 significant bits, more than FP16 holds, so each weight enters as two FP16
  *   terms whose sum is the weight exactly and every K step makes two products into the same FP32
- *   accumulator.  Other formats return OMC_ERR_BAD_FORMAT (the fixed-point variant among them: its
- *   codes are not floating-point patterns); for those, omc_decompress the variable and multiply.
+ *   accumulator.  Of the fixed-point variant S1I0F7 and S1I0F11 (every value is an FP16 value)
+ *   and S1I0F15 (two FP16 terms per weight, like S1E4M14).  Other formats return
+ *   OMC_ERR_BAD_FORMAT; for those, omc_decompress the variable and multiply.
  *   var must be quantised and N*K == its numel; N % 128 == 0, K % 64 == 0 (else OMC_ERR_INVALID_ARG).
  *   packed, sb      device, the model state (read only).
  *   x_half          device, M x K IEEE halves, K contiguous, 16-byte aligned.

@@ -50,17 +50,22 @@ constexpr uint32_t WAIT_LIMIT = 1u << 20;        // polls of one mbarrier before
 // value: E = 5 codes are FP16 patterns (code << 3), the others become FP16 patterns whose exponent
 // field is too small by 15 - bias, which one exact packed multiplication by 2^(15 - bias) repairs
 // for normal and subnormal codes alike; Inf / NaN codes are patched in afterwards.
+// E = 0 stands for the fixed-point variant S1I0Fy with y = B - 1 (B = 8, 12, 16).
 template <int B, int E>
 struct Cfg {
     static_assert((E == 5 && (B == 16 || B == 12 || B == 8)) || (E == 4 && B == 8) || (E == 2 && B == 6) ||
-                  (B == 13 && (E == 5 || E == 3 || E == 4)) || (B == 11 && E == 3) || (B == 19 && E == 4), "");
-    static constexpr bool DECODE = B != 16;
+                  (B == 13 && (E == 5 || E == 3 || E == 4)) || (B == 11 && E == 3) || (B == 19 && E == 4) ||
+                  (E == 0 && (B == 8 || B == 12 || B == 16)), "");
+    static constexpr bool FIXED = E == 0;        // S1I0Fy, y = B - 1: two's complement k, value k * 2^-y
+    static constexpr bool DECODE = B != 16 || FIXED;
     static constexpr bool ODD = (B % 2) != 0;
     // S1E4M14 (Table 1) has 15 significant bits, four more than an FP16 value: a weight is split
     // exactly into hi + lo, both FP16 values (hi = the weight rounded to FP16, lo = the rest, at
     // most 5 significant bits and never below 2^-20), the tile has two operand tiles and every K
     // step two products into the same accumulator.  The tile is 128 columns wide then.
-    static constexpr bool SPLIT = (B == 19);
+    // S1I0F15 has 15 significant bits as well: k = 64 hi + lo with -512 <= hi < 512 and 0 <= lo < 64,
+    // the weight is hi * 2^-9 + lo * 2^-15, two FP16 values again.
+    static constexpr bool SPLIT = (B == 19) || (FIXED && B == 16);
     static constexpr int BN = SPLIT ? BN_SPLIT : BN_WIDE;
     static constexpr int TILE_B_BYTES = BN * BK * 2;              // one operand tile
     static constexpr int OPERAND_BYTES = (SPLIT ? 2 : 1) * TILE_B_BYTES;
@@ -181,11 +186,70 @@ __device__ __forceinline__ void narrow_to_halves(uint32_t c4, uint32_t &h01, uin
     }
 }
 
+// Fixed-point codes (two's complement k in B bits, value k * 2^-(B-1)) as FP16 values, without an
+// integer-to-float conversion: flipping the sign bit gives k + 2^(B-1) >= 0; up to ten bits of a
+// non-negative integer j dropped into the mantissa of 1024 make the FP16 value 1024 + j, and one
+// fused multiply-add, exact because its result is an FP16 value, scales it and takes the offset off.
+__device__ __forceinline__ uint32_t hfma2_bits(uint32_t a, float mul, float add)
+{
+    const __half2 r = __hfma2(*reinterpret_cast<const __half2 *>(&a), __float2half2_rn(mul), __float2half2_rn(add));
+    return *reinterpret_cast<const uint32_t *>(&r);
+}
+// S1I0F7, four codes of one word: 1024 + (k + 128) = 1152 + k, times 2^-7, minus 9.
+__device__ __forceinline__ void fixed8_to_halves(uint32_t c4, uint32_t &h01, uint32_t &h23)
+{
+    const uint32_t x = c4 ^ 0x80808080u;
+    h01 = hfma2_bits(__byte_perm(x, 0x64646464u, 0x5140), 0.0078125f, -9.f);
+    h23 = hfma2_bits(__byte_perm(x, 0x64646464u, 0x5342), 0.0078125f, -9.f);
+}
+// S1I0F11, two codes in the low 12 bits of each half of `pr`: j = k + 2048 has twelve bits, the low
+// ten go into one FP16 value (1024 + lo), the top two into another (1024 + 256 hi); then
+// (1024 + 256 hi) 2^-9 - 3.5 = hi/2 - 1.5 and (1024 + lo) 2^-11 + that = (lo + 1024 hi) / 2048 - 1 = k / 2048.
+__device__ __forceinline__ uint32_t fixed12_to_halves(uint32_t pr)
+{
+    const uint32_t x = pr ^ 0x08000800u;
+    const uint32_t lo = (x & 0x03FF03FFu) | 0x64006400u, hi = ((x >> 2) & 0x03000300u) | 0x64006400u;
+    const __half2 c = __hfma2(*reinterpret_cast<const __half2 *>(&hi), __float2half2_rn(0.001953125f), __float2half2_rn(-3.5f));
+    const __half2 r = __hfma2(*reinterpret_cast<const __half2 *>(&lo), __float2half2_rn(0.00048828125f), c);
+    return *reinterpret_cast<const uint32_t *>(&r);
+}
+// S1I0F15, two codes of one word: j = k + 32768; the top ten bits give hi + 512, the low six lo.
+// (1024 + hi + 512) 2^-9 - 3 = hi 2^-9;  (1024 + lo) 2^-15 - 2^-5 = lo 2^-15 (an FP16 subnormal below 2^-14).
+__device__ __forceinline__ void fixed16_to_halves(uint32_t c2, uint32_t &hi, uint32_t &lo)
+{
+    const uint32_t x = c2 ^ 0x80008000u;
+    hi = hfma2_bits(((x >> 6) & 0x03FF03FFu) | 0x64006400u, 0.001953125f, -3.f);
+    lo = hfma2_bits((x & 0x003F003Fu) | 0x64006400u, 0.000030517578125f, -0.03125f);
+}
+// Eight S1I0F15 codes (16 bytes) -> eight FP16 pairs (hi, lo) with hi + lo = the weight exactly.
+__device__ __forceinline__ void expand_chunk_split_fixed16(const uint8_t *raw, uint4 &hi4, uint4 &lo4)
+{
+    const uint4 w = *reinterpret_cast<const uint4 *>(raw);
+    fixed16_to_halves(w.x, hi4.x, lo4.x);
+    fixed16_to_halves(w.y, hi4.y, lo4.y);
+    fixed16_to_halves(w.z, hi4.z, lo4.z);
+    fixed16_to_halves(w.w, hi4.w, lo4.w);
+}
+
 // Eight codes (one 16-byte chunk of halves) from their B packed bytes.
 template <int B, int E>
 __device__ __forceinline__ uint4 expand_chunk(const uint8_t *raw)
 {
-    if constexpr (B == 8 && E == 5) {        // a code is the top byte of its half
+    if constexpr (B == 8 && E == 0) {        // S1I0F7
+        const uint2 w = *reinterpret_cast<const uint2 *>(raw);
+        uint4 o;
+        fixed8_to_halves(w.x, o.x, o.y);
+        fixed8_to_halves(w.y, o.z, o.w);
+        return o;
+    } else if constexpr (B == 12 && E == 0) {    // S1I0F11: pair p is bytes 3p .. 3p+2
+        const uint32_t *rw = reinterpret_cast<const uint32_t *>(raw);
+        const uint32_t w0 = rw[0], w1 = rw[1], w2 = rw[2];
+        const uint32_t t0 = __byte_perm(w0, 0u, 0x2110), t1 = __byte_perm(w0, w1, 0x5443);
+        const uint32_t t2 = __byte_perm(w1, w2, 0x4332), t3 = __byte_perm(w2, 0u, 0x3221);
+        auto pair = [](uint32_t t) { return (t & 0x00000FFFu) | ((t >> 4) & 0x0FFF0000u); };
+        return make_uint4(fixed12_to_halves(pair(t0)), fixed12_to_halves(pair(t1)), fixed12_to_halves(pair(t2)),
+                          fixed12_to_halves(pair(t3)));
+    } else if constexpr (B == 8 && E == 5) {        // a code is the top byte of its half
         const uint2 w = *reinterpret_cast<const uint2 *>(raw);
         return make_uint4(__byte_perm(w.x, 0u, 0x1404), __byte_perm(w.x, 0u, 0x3424),
                           __byte_perm(w.y, 0u, 0x1404), __byte_perm(w.y, 0u, 0x3424));
@@ -466,7 +530,10 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                         uint4 o;
                         if constexpr (C::SPLIT) {
                             uint4 lo;
-                            expand_chunk_split(stage + TILE_A_BYTES + C::OPERAND_BYTES + r * C::BOX_BYTES + off + c * B, o, lo);
+                            if constexpr (C::FIXED)
+                                expand_chunk_split_fixed16(stage + TILE_A_BYTES + C::OPERAND_BYTES + r * C::BOX_BYTES + c * B, o, lo);
+                            else
+                                expand_chunk_split(stage + TILE_A_BYTES + C::OPERAND_BYTES + r * C::BOX_BYTES + off + c * B, o, lo);
                             *reinterpret_cast<uint4 *>(dst + TILE_B_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) = lo;
                         } else if constexpr (C::ODD)
                             o = expand_chunk_odd<B, E>(stage + TILE_A_BYTES + C::OPERAND_BYTES + r * C::BOX_BYTES + off + c * B);
@@ -575,12 +642,14 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     if (!packed || !sb || !x_half || !y || !rowsum_scratch) return OMC_ERR_NULL_PTR;
     if (var >= plan->nvars || !plan->vars[var].quantised) return OMC_ERR_INVALID_ARG;
     const int exp = plan->fmt.exp_bits, man = plan->fmt.man_bits;
-    if (plan->fmt.flags) return OMC_ERR_BAD_FORMAT;          // floating-point codes only
-    const bool half_family = exp == 5 && (man == 10 || man == 6 || man == 2);
-    const bool narrow = (exp == 4 && man == 3) || (exp == 2 && man == 3);
-    const bool split = exp == 4 && man == 14;
-    const bool odd = (exp == 5 && man == 7) || (exp == 3 && man == 7) || (exp == 3 && man == 9) || (exp == 4 && man == 8) || split;
-    if (!half_family && !narrow && !odd) return OMC_ERR_BAD_FORMAT;
+    const bool fixed = (plan->fmt.flags & OMC_FORMAT_FIXED_POINT) != 0;
+    if (fixed && !(exp == 0 && (man == 7 || man == 11 || man == 15))) return OMC_ERR_BAD_FORMAT;   // S1I0F7 / F11 / F15
+    const bool half_family = !fixed && exp == 5 && (man == 10 || man == 6 || man == 2);
+    const bool narrow = !fixed && ((exp == 4 && man == 3) || (exp == 2 && man == 3));
+    const bool split = !fixed && exp == 4 && man == 14;
+    const bool odd = !fixed && ((exp == 5 && man == 7) || (exp == 3 && man == 7) || (exp == 3 && man == 9) ||
+                               (exp == 4 && man == 8) || split);
+    if (!fixed && !half_family && !narrow && !odd) return OMC_ERR_BAD_FORMAT;
     if (odd && K % 128 != 0) return OMC_ERR_INVALID_ARG;      // a row of 11- or 13-bit codes must be whole 16-byte units
     if (M == 0 || N == 0 || K == 0 || N % 128 != 0 || K % BK != 0 || (uint64_t)N * K != plan->vars[var].n)
         return OMC_ERR_INVALID_ARG;
@@ -598,6 +667,11 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     const uint32_t n_sm = plan->n_sm ? plan->n_sm : 1;
     const uint32_t inject = plan->inject_polls;      // diagnostics: applies to this launch only
     plan->inject_polls = 0;
+    if (fixed) {
+        if (man == 7) return launch<8, 0>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        if (man == 11) return launch<12, 0>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        return launch<16, 0>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    }
     if (split) return launch<19, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     if (odd) {
         if (exp == 5) return launch<13, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);

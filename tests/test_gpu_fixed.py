@@ -170,7 +170,7 @@ def test_fixed_point_format_limits_and_matmul_refusal():
         if rc == 0:
             L.omc_plan_destroy(h)
     assert L.omc_plan(d, 1, omc.Format(1, 5, 2, 2), 1.0, 0, None, omc.PLAN_DEFAULT, omc.C.byref(h)) == -2   # unknown flag
-    plan = omc.Plan([128 * 64], [0], (0, 7), fixed=True)
+    plan = omc.Plan([128 * 64], [0], (2, 9), fixed=True)        # omc_matmul decodes S1I0F7 / F11 / F15 only
     dm = DeviceModel(plan)
     x = torch.zeros(128 * 64, dtype=torch.float16, device="cuda")
     y = torch.zeros(128 * 128, dtype=torch.float32, device="cuda")

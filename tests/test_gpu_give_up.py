@@ -95,8 +95,8 @@ def test_matmul_wait_runs_out_then_works_again():
     N, K, M = 256, 128, 200
     w = (rng.standard_normal(N * K) * 0.05).astype(np.float32)
     x = (rng.standard_normal((M, K)) * 0.5).astype(np.float16)
-    for fmt in [(5, 10), (5, 2)]:
-        plan = omc.Plan([N * K], [0], fmt)
+    for fmt, fixed in [((5, 10), False), ((5, 2), False), ((0, 15), True)]:
+        plan = omc.Plan([N * K], [0], fmt, fixed=fixed)
         dm = DeviceModel(plan)
         dm.compress(dm.upload_full([w]))
         xd = torch.from_numpy(x).cuda()
@@ -114,8 +114,8 @@ def test_matmul_wait_runs_out_then_works_again():
         run()
         torch.cuda.synchronize()
         assert plan.status(st) == 0
-        state = orc.compress([w], [True], *fmt)
-        wbar = orc.decompress_var(state["packed"][0], N * K, fmt[0], fmt[1], state["s"][0], state["b"][0])
+        state = orc.compress([w], [True], *fmt, fixed=fixed)
+        wbar = orc.decompress_var(state["packed"][0], N * K, fmt[0], fmt[1], state["s"][0], state["b"][0], fixed)
         want = x.astype(np.float64) @ wbar.reshape(N, K).astype(np.float64).T
         assert np.allclose(y.cpu().numpy(), want, rtol=1e-4, atol=1e-4)
 

@@ -103,6 +103,72 @@ def test_matmul_from_odd_width_codes(M, N, K, fmt):
                                     y.data_ptr(), scratch.data_ptr(), None) == -1
 
 
+@pytest.mark.parametrize("fmt", [(0, 7), (0, 11), (0, 15)], ids=lambda f: "I%dF%d" % f)
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 256, 192), (1000, 384, 512), (4000, 4224, 192)])
+def test_matmul_from_fixed_point_codes(M, N, K, fmt):
+    """The fixed-point variant (Sec. 2.2): two's-complement codes become FP16 values in the decoder
+    warps without an integer conversion; S1I0F15 has more significant bits than FP16 and goes in as
+    two terms.  The weights cover the whole range, both ends (the most negative code -1 and the
+    largest value 1 - 2^-y, reached by saturation) and the smallest steps included."""
+    I_, F_ = fmt
+    rng = np.random.default_rng(M + N + K + F_)
+    w = (rng.standard_normal(N * K) * 0.4 * 10.0 ** rng.uniform(-4, 0, N * K)).astype(np.float32)
+    w[:64] = np.linspace(-1.5, 1.5, 64, dtype=np.float32)        # saturates at both ends
+    w[64:72] = [-1.0, 1.0, 2.0 ** -F_, -(2.0 ** -F_), 0.0, -0.0, 1 - 2.0 ** -F_, 2.0 ** -(F_ + 2)]
+    numel, kinds = [333, N * K, 64], [0, 0, 1]
+    params = [rng.standard_normal(333).astype(np.float32) * np.float32(0.1), w, np.zeros(64, np.float32)]
+    plan = omc.Plan(numel, kinds, fmt, fixed=True)
+    dm = DeviceModel(plan)
+    dm.compress(dm.upload_full(params))
+    st = orc.compress(params, plan.quantised, I_, F_, fixed=True)
+    x = (rng.standard_normal((M, K)) * 0.5).astype(np.float16)
+    xd = torch.from_numpy(x).cuda()
+    yg = Guarded(M * N, torch.float32, "cuda", fill=float("nan"))
+    y = yg.t[:M * N].view(M, N)
+    scratch = torch.zeros(M, dtype=torch.float32, device="cuda")
+    omc.matmul(plan, 1, dm.packed.data_ptr(), dm.sb.data_ptr(), xd.data_ptr(), M, N, K, y.data_ptr(),
+               scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert plan.status() == 0 and yg.intact()
+    s_, b_ = float(st["s"][1]), float(st["b"][1])
+    wbar = orc.decompress_var(st["packed"][1], N * K, I_, F_, st["s"][1], st["b"][1], fixed=True).reshape(N, K).astype(np.float64)
+    codes = orc.unpack(st["packed"][1], N * K, 1 + I_ + F_)
+    wt = orc.decode(codes, I_, F_, fixed=True).reshape(N, K).astype(np.float64)
+    assert wt.min() == -1.0 and wt.max() == 1 - 2.0 ** -F_          # both ends of the range are in the matrix
+    x64 = x.astype(np.float64)
+    want = x64 @ wbar.T
+    bound = (4 * K + 8) * 2.0 ** -24 * (abs(s_) * (np.abs(x64) @ np.abs(wt).T)
+                                        + abs(b_) * np.abs(x64).sum(1, keepdims=True)) + 1e-30
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.all(np.abs(got - want) <= bound), float(np.max(np.abs(got - want) / bound))
+
+
+def test_matmul_fixed_point_exact_small_case():
+    """With s = 1, b = 0, one-hot rows of X and weights that are whole codes, every output is one
+    weight exactly: the decoders' FP16 values are the codes' values bit for bit, for every code of
+    the three formats."""
+    for F_ in (7, 11, 15):
+        N, K, M = 128, 512, 512
+        B = 1 + F_
+        ks = (np.arange(N * K, dtype=np.int64) % (1 << B)) - (1 << (B - 1))     # every code (all 65536 of S1I0F15 once)
+        w = (ks.astype(np.float64) * 2.0 ** -F_).astype(np.float32)
+        plan = omc.Plan([N * K], [0], (0, F_), fixed=True, flags=omc.PLAN_WEIGHTS_ONLY)    # no transformation
+        dm = DeviceModel(plan)
+        dm.compress(dm.upload_full([w]))
+        x = np.zeros((M, K), np.float16)
+        x[np.arange(M), np.arange(M) % K] = 1.0                                   # row m picks column m of W^T
+        xd = torch.from_numpy(x).cuda()
+        y = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+        scratch = torch.zeros(M, dtype=torch.float32, device="cuda")
+        omc.matmul(plan, 0, dm.packed.data_ptr(), dm.sb.data_ptr(), xd.data_ptr(), M, N, K, y.data_ptr(),
+                   scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert plan.status() == 0
+        want = w.reshape(N, K)[:, np.arange(M) % K].T                              # y[m, n] = W[n, m]
+        assert np.array_equal(y.cpu().numpy(), want), F_
+
+
 def test_matmul_argument_checks():
     plan = omc.Plan([128 * 64, 100], [0, 1], (5, 10))
     dm = DeviceModel(plan)
@@ -119,6 +185,10 @@ def test_matmul_argument_checks():
     assert L.omc_matmul(p8._h, 0, d8.packed.data_ptr(), d8.sb.data_ptr(), x.data_ptr(), 128, 128, 64, y.data_ptr(),
                         y.data_ptr(), None) == -2
     assert L.omc_matmul(plan._h, 0, *a, 128, 128, 64, None, y.data_ptr(), None) == -3
+    pf = omc.Plan([128 * 64], [0], (1, 6), fixed=True)          # a fixed-point format the product has no decoder for
+    df = DeviceModel(pf)
+    assert L.omc_matmul(pf._h, 0, df.packed.data_ptr(), df.sb.data_ptr(), x.data_ptr(), 128, 128, 64, y.data_ptr(),
+                        y.data_ptr(), None) == -2
     torch.cuda.synchronize()
 
 
