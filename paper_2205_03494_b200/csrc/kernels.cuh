@@ -1552,11 +1552,12 @@ struct PlacedPath {
 
 // acc[j] (+)= fma(s, Vt_j, b) for the AL consecutive elements whose codes are the ANW words of
 // `win`; FIRST: the sum starts with this client.
-// FOLDED (PlacedPath only): `sk` is s * 2^(127-BIAS), computed without overflow, hence exactly:
-// Vt = placed * 2^(127-BIAS) exactly, so fma(sk, placed, b) rounds the same real number as
-// fma(s, Vt, b), and the rebias multiplication is never made.
-template <class F, int AL, int ANW, bool FIRST, bool FOLDED>
-__device__ __forceinline__ void agg_add(const uint32_t (&win)[ANW], float s, float sk, float b, float *acc)
+// PlacedPath formats: `sk` is s * 2^(127-BIAS).  Where that did not overflow (`folded`) it is exact,
+// and as Vt = placed * 2^(127-BIAS) exactly, fma(sk, placed, b) rounds the same real number as
+// fma(s, Vt, b): the rebias multiplication is never made.  A variable whose s is that large takes
+// the path of the Inf/NaN codes, element by element, for all of its values.
+template <class F, int AL, int ANW, bool FIRST>
+__device__ __forceinline__ void agg_add(const uint32_t (&win)[ANW], float s, float sk, float b, bool folded, float *acc)
 {
     float x[AL];
     if constexpr (Fp8Path<F>::value) {
@@ -1586,15 +1587,13 @@ __device__ __forceinline__ void agg_add(const uint32_t (&win)[ANW], float s, flo
             for (int j = 0; j < G; ++j) v[j] = placed_at<F, ANW>(win, (G * g + j) * F::B);
             float m = absmax4(v[0], v[1], v[2], v[3]);
             if constexpr (G == 8) m = fmaxf(m, absmax4(v[4], v[5], v[6], v[7]));
-            if (m >= u2f(F::INF_MAG << F::SH)) {
+            if (m >= u2f(F::INF_MAG << F::SH) || !folded) {
 #pragma unroll
                 for (int j = 0; j < G; ++j)
                     x[G * g + j] = __fmaf_rn(s, decode_exact<F>(get_code_at<F, ANW>(win, (G * g + j) * F::B)), b);
             } else {
 #pragma unroll
-                for (int j = 0; j < G; ++j)
-                    x[G * g + j] = FOLDED ? __fmaf_rn(sk, v[j], b)
-                                          : __fmaf_rn(s, __fmul_rn(v[j], u2f(F::pow2_bits(127 - F::BIAS))), b);
+                for (int j = 0; j < G; ++j) x[G * g + j] = __fmaf_rn(sk, v[j], b);
             }
         }
     } else {
@@ -1606,8 +1605,9 @@ __device__ __forceinline__ void agg_add(const uint32_t (&win)[ANW], float s, flo
 }
 
 // One client's codes of one tile, in a slot of the ring: each lane adds its 32 values to its sums.
-template <class F, bool FIRST, bool FOLDED>
-__device__ __forceinline__ void agg_tile_codes(const uint32_t *sw, float s, float sk, float b, float (&acc)[32], int lane)
+template <class F, bool FIRST>
+__device__ __forceinline__ void agg_tile_codes(const uint32_t *sw, float s, float sk, float b, bool folded,
+                                               float (&acc)[32], int lane)
 {
     using U = Unit<F>;
     // A lane takes AL consecutive elements at a time, at least four (one 16-byte store), NQ times per tile.
@@ -1632,7 +1632,7 @@ __device__ __forceinline__ void agg_tile_codes(const uint32_t *sw, float s, floa
 #pragma unroll
             for (int j = 0; j < ANW; ++j) win[j] = uw[j];
         }
-        agg_add<F, AL, ANW, FIRST, FOLDED>(win, s, sk, b, acc + q * AL);
+        agg_add<F, AL, ANW, FIRST>(win, s, sk, b, folded, acc + q * AL);
     }
 }
 
@@ -1789,12 +1789,8 @@ __global__ void __launch_bounds__(THREADS, aggregate_ctas_per_sm(F::B)) omc_aggr
                         if (++polls > wait_limit) return false;
                     }
                     const uint32_t *sw = reinterpret_cast<const uint32_t *>(ring + cslot * CB);
-                    if constexpr (PlacedPath<F>::value) {
-                        if (c.folded) agg_tile_codes<F, FIRST, true>(sw, c.s, c.sk, c.b, acc, lane);
-                        else agg_tile_codes<F, FIRST, false>(sw, c.s, c.sk, c.b, acc, lane);
-                    } else {
-                        agg_tile_codes<F, FIRST, false>(sw, c.s, c.s, c.b, acc, lane);
-                    }
+                    if constexpr (PlacedPath<F>::value) agg_tile_codes<F, FIRST>(sw, c.s, c.sk, c.b, c.folded != 0u, acc, lane);
+                    else agg_tile_codes<F, FIRST>(sw, c.s, c.s, c.b, true, acc, lane);
                     __syncwarp();               // every lane has read the slot: it may be filled again
                     cslot = cslot + 1 == NSLOT ? 0u : cslot + 1;
                     --in_ring;

@@ -22,8 +22,9 @@ constexpr int fit_warps_per_cta(int code_bits, bool /*fixed_point*/)
     return (code_bits == 12 || code_bits == 19) ? 6 : WARPS_PER_CTA;
 }
 constexpr int CTAS_PER_SM = 2;
-// CTAs per SM of the aggregation: with 8-bit codes it fits the 80 registers that three leave it
-// (measured 11-14 % faster than two); with any other width it spills there (up to 29 % slower).
+// CTAs per SM of the aggregation: with 8-bit codes it gets by on the 80 registers that three leave it
+// (nine words spilled, outside the tile loop; measured 11-14 % faster than two); with any other
+// width it spills inside the loop (up to 29 % slower).
 constexpr int aggregate_ctas_per_sm(int code_bits) { return code_bits == 8 ? 3 : CTAS_PER_SM; }
 // The decompress kernel divides its tiles at launch, so its grid is independent of the plan's division.
 constexpr int DECOMPRESS_CTAS_PER_SM = 2;
