@@ -497,14 +497,15 @@ def run_ours(args):
 
         # server-side mean of 8 client replicas, each with its own random 90% subset (Sec. 2.5)
         K = 8
-        cl = []
-        for k in range(K):
+        cl16 = []
+        for k in range(16):
             pl = omc.Plan(wl.numel, wl.kinds, wl.fmt, fraction=0.9, seed=100 + k, fixed=args.fixed)
             b4 = (z(pl.packed_bytes, torch.uint8), z(pl.resid_elems, torch.float32),
                   z(2 * pl.n_quantised, torch.float32), z(pl.workspace_bytes, torch.uint8))
             pl.prepare(b4[3].data_ptr(), stream)
             pl.compress(out.data_ptr(), b4[0].data_ptr(), b4[1].data_ptr(), b4[2].data_ptr(), b4[3].data_ptr(), stream)
-            cl.append((pl, b4))
+            cl16.append((pl, b4))
+        cl = cl16[:K]
         mean = torch.empty(plan.full_elems, dtype=torch.float32, device=dev)
         try:
             fn = lambda: omc.aggregate([c[0] for c in cl], [c[1][0].data_ptr() for c in cl],
@@ -523,6 +524,34 @@ def run_ours(args):
                                        for pl, _ in cl for n, q in zip(pl.numel, pl.quantised))
             extra["aggregate_8_clients"] = {"ms": t_ms, "params_per_s": nparams / (t_ms * 1e-3),
                                             "gbs": nbytes / (t_ms * 1e6)}
+            # the paper's round (Sec. 3.1: 128 clients), more than one call takes: eight batches of 16
+            # (omc_aggregate_sum, seven times omc_aggregate_add, omc_divide); sixteen different
+            # states, the same sixteen in every batch (3.6 GB a batch: nothing of it is left in the
+            # L2 when the next batch reads it)
+            lists = lambda cs: ([c[0] for c in cs], [c[1][0].data_ptr() for c in cs], [c[1][1].data_ptr() for c in cs],
+                                [c[1][2].data_ptr() for c in cs])
+            batches = [lists(cl16) for _ in range(8)]
+
+            def fn128():
+                omc.aggregate_sum(*batches[0], mean.data_ptr(), stream)
+                for bt in batches[1:]:
+                    omc.aggregate_add(*bt, mean.data_ptr(), stream)
+                omc.divide(cl[0][0], mean.data_ptr(), 128, stream)
+            for _ in range(2):
+                fn128()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(5):
+                fn128()
+            e1.record()
+            torch.cuda.synchronize()
+            t_ms = e0.elapsed_time(e1) / 5
+            # the clients' bytes; `out` written once, then read and written by each further batch and by the division
+            per_client = sum(((n * pl.B + 7) // 8) if q else 4 * n
+                             for pl, _ in cl16 for n, q in zip(pl.numel, pl.quantised))
+            nbytes128 = 8 * per_client + (4 + 8 * 8) * nparams
+            extra["aggregate_128_clients_in_8_calls"] = {"ms": t_ms, "params_per_s": nparams / (t_ms * 1e-3),
+                                                         "gbs": nbytes128 / (t_ms * 1e6)}
         except omc.OmcError as err:
             extra["aggregate_8_clients"] = {"unavailable": str(err)}
 

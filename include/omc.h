@@ -181,8 +181,8 @@ int omc_plan_status(const omc_plan_t *plan, void *stream, uint32_t *host_status)
 /*
  * omc_plan_inject_wait_timeout -- diagnostics for the bounded waits (the paper has no counterpart).
  * The next kernel launched with this plan (omc_compress, omc_decompress, omc_update_recompress,
- * omc_transition with the plan as destination, omc_aggregate and omc_aggregate_sum with the plan
- * first in the list, omc_matmul) announces its asynchronous loads to
+ * omc_transition with the plan as destination, omc_aggregate, omc_aggregate_sum and
+ * omc_aggregate_add with the plan first in the list, omc_matmul) announces its asynchronous loads to
  * their barriers without issuing them and gives up each wait after `polls` polls (1 .. 2^24):
  * every wait runs out with no copy in flight, the kernel sets the status word and returns, its
  * outputs are garbage.  Afterwards omc_plan_status reports non-zero; call omc_plan_prepare again
@@ -284,6 +284,18 @@ int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint
 int omc_aggregate_sum(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
                       const float *const *resid, const float *const *sb, float *out, void *stream);
 int omc_divide(const omc_plan_t *plan, float *values, uint32_t divisor, void *stream);
+
+/*
+ * omc_aggregate_add -- more clients than one call takes (a round of the paper's experiments has
+ * more than 16, Sec. 3.1): out[e] = out[e] + x_0[e] + ... + x_{K-1}[e], FP32, starting from what
+ * `out` holds and adding this call's clients in index order (arguments as for omc_aggregate_sum;
+ * `out` is read and written; the padding after each variable is written with zeros).
+ * omc_aggregate_sum over the first batch of clients, omc_aggregate_add over each further batch
+ * and omc_divide by the number of all clients make exactly the additions, in exactly the order,
+ * of one omc_aggregate over all of them: the result is the same bit for bit.
+ */
+int omc_aggregate_add(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
+                      const float *const *resid, const float *const *sb, float *out, void *stream);
 
 /*
  * omc_matmul -- forward path of Fig. 1 with the decompression fused into the consumer (Sec. 2.1:

@@ -21,7 +21,7 @@ FORMAT_FIXED_POINT = 1
 
 EXPORTS = ["omc_strerror", "omc_last_cuda_error", "omc_plan", "omc_plan_destroy", "omc_plan_seed", "omc_plan_sizes",
            "omc_plan_var", "omc_plan_division", "omc_plan_prepare", "omc_plan_status", "omc_plan_inject_wait_timeout", "omc_compress", "omc_decompress",
-           "omc_update_recompress", "omc_update_recompress_host", "omc_transition", "omc_aggregate", "omc_aggregate_sum", "omc_divide", "omc_matmul",
+           "omc_update_recompress", "omc_update_recompress_host", "omc_transition", "omc_aggregate", "omc_aggregate_sum", "omc_aggregate_add", "omc_divide", "omc_matmul",
            "omc_compress_var_static", "omc_static_status"]
 STATIC_MAX_NUMEL = 1 << 28
 
@@ -78,6 +78,7 @@ def lib():
         L.omc_matmul.argtypes = [vp, C.c_uint32, vp, vp, vp, C.c_uint32, C.c_uint32, C.c_uint32, vp, vp, vp]
         L.omc_aggregate.argtypes = [C.POINTER(vp), C.c_uint32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp, vp]
         L.omc_aggregate_sum.argtypes = L.omc_aggregate.argtypes
+        L.omc_aggregate_add.argtypes = L.omc_aggregate.argtypes
         L.omc_divide.argtypes = [vp, vp, C.c_uint32, vp]
         L.omc_compress_var_static.argtypes = [vp, C.c_uint64, Format, C.c_uint32, vp, vp, vp]
         L.omc_static_status.argtypes = [vp, u32p]
@@ -216,6 +217,16 @@ def aggregate_sum(plans, packed, resid, sb, out, stream=0):
     k = len(plans)
     arr = lambda xs: (C.c_void_p * k)(*[x if not hasattr(x, "_h") else x._h.value for x in xs])
     _check(lib().omc_aggregate_sum(arr(plans), k, arr(packed), arr(resid), arr(sb), out, stream), "omc_aggregate_sum")
+
+
+MAX_CLIENTS_PER_CALL = 16      # of omc_aggregate, omc_aggregate_sum and omc_aggregate_add
+
+
+def aggregate_add(plans, packed, resid, sb, out, stream=0):
+    """omc_aggregate_add: this batch of clients added, in index order, to the sum `out` already holds."""
+    k = len(plans)
+    arr = lambda xs: (C.c_void_p * k)(*[x if not hasattr(x, "_h") else x._h.value for x in xs])
+    _check(lib().omc_aggregate_add(arr(plans), k, arr(packed), arr(resid), arr(sb), out, stream), "omc_aggregate_add")
 
 
 def divide(plan: Plan, values, divisor: int, stream=0):

@@ -1511,7 +1511,9 @@ void launch_transition(const KParams &p, int grid, void *stream)
 // Sec. 2.5: each client quantises its own subset, so the server receives precise values of a
 // parameter from the clients that kept it in FP32).  out = (x_0 + x_1 + ... + x_{K-1}) / K per
 // element, FP32, clients added in index order, one rounded division at the end, where x_k is
-// client k's decompressed value fma(s_k, Vt_k, b_k) or its FP32 value.
+// client k's decompressed value fma(s_k, Vt_k, b_k) or its FP32 value.  Without the division it is
+// the sum, and the sum may start from what `out` holds: more clients than one launch takes are
+// added batch after batch, in the same order of additions as in one pass.
 //
 // The tiles are cut into short runs of equal length, dealt out to the warps in turn.  Tile by tile a
 // warp walks the clients in index order with the tile's 32 sums per lane in registers; the codes of
@@ -1703,7 +1705,7 @@ __global__ void __launch_bounds__(THREADS, aggregate_ctas_per_sm(F::B)) omc_aggr
     // rounded value of the same real number.
     const bool pow2 = (K & (K - 1)) == 0;
     const float kinv = 1.f / kf;
-    const bool divide = p.divide != 0u;
+    const bool divide = p.divide != 0u, accumulate = p.accumulate != 0u;
     auto mean_of = [&](float a) { return !divide ? a : pow2 ? __fmul_rn(a, kinv) : __fdiv_rn(a, kf); };
 
     // Short runs of equal length, dealt out to the warps in turn: what a tile costs depends on how many
@@ -1804,10 +1806,17 @@ __global__ void __launch_bounds__(THREADS, aggregate_ctas_per_sm(F::B)) omc_aggr
                 }
                 return true;
             };
-            failed = !client(std::true_type{}, 0u);
-            for (uint32_t k = 1; k < K && !failed; ++k) failed = !client(std::false_type{}, k);
-            if (failed) break;
             float *o = p.out + var.full_off + e_tile;
+            uint32_t k = 0;
+            if (accumulate) {       // the sum so far, left in `out` by the call before
+                if (whole) agg_tile_fp32<F, true, true>(o, n_pad, acc, lane);
+                else agg_tile_fp32<F, true, false>(o, n_pad, acc, lane);
+            } else {
+                failed = !client(std::true_type{}, 0u);
+                k = 1;
+            }
+            for (; k < K && !failed; ++k) failed = !client(std::false_type{}, k);
+            if (failed) break;
 #pragma unroll
             for (int q = 0; q < NQ; ++q)
 #pragma unroll

@@ -337,7 +337,8 @@ extern "C" int omc_transition(const omc_plan_t *from, const omc_plan_t *to, cons
 }
 
 static int aggregate_impl(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
-                          const float *const *resid, const float *const *sb, float *out, uint32_t divide, void *stream)
+                          const float *const *resid, const float *const *sb, float *out, uint32_t divide,
+                          uint32_t accumulate, void *stream)
 {
     if (!plans || !packed || !resid || !sb || !out) return OMC_ERR_NULL_PTR;
     if (n_clients == 0 || n_clients > (uint32_t)omc::MAX_CLIENTS) return OMC_ERR_INVALID_ARG;
@@ -364,6 +365,7 @@ static int aggregate_impl(const omc_plan_t *const *plans, uint32_t n_clients, co
     if (!first->ops->aggregate) return OMC_ERR_BAD_FORMAT;
     p.nclients = n_clients;
     p.divide = divide;
+    p.accumulate = accumulate;
     p.nvars = first->nvars;
     p.tile_count = first->ntiles;
     const uint64_t max_warps = (uint64_t)first->n_sm * first->ops->agg_ctas * omc::WARPS_PER_CTA;
@@ -381,13 +383,19 @@ static int aggregate_impl(const omc_plan_t *const *plans, uint32_t n_clients, co
 extern "C" int omc_aggregate(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
                              const float *const *resid, const float *const *sb, float *out, void *stream)
 {
-    return aggregate_impl(plans, n_clients, packed, resid, sb, out, 1u, stream);
+    return aggregate_impl(plans, n_clients, packed, resid, sb, out, 1u, 0u, stream);
 }
 
 extern "C" int omc_aggregate_sum(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
                                  const float *const *resid, const float *const *sb, float *out, void *stream)
 {
-    return aggregate_impl(plans, n_clients, packed, resid, sb, out, 0u, stream);
+    return aggregate_impl(plans, n_clients, packed, resid, sb, out, 0u, 0u, stream);
+}
+
+extern "C" int omc_aggregate_add(const omc_plan_t *const *plans, uint32_t n_clients, const uint8_t *const *packed,
+                                 const float *const *resid, const float *const *sb, float *out, void *stream)
+{
+    return aggregate_impl(plans, n_clients, packed, resid, sb, out, 0u, 1u, stream);
 }
 
 namespace {

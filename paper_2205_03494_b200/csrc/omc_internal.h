@@ -148,6 +148,7 @@ struct AggParams {
     const float *sb[MAX_CLIENTS];
     uint32_t nclients;
     uint32_t divide;                     // 1: out = sum / nclients; 0: out = the sum itself (first stage of a mean across GPUs)
+    uint32_t accumulate;                 // 1: the sum starts from what `out` holds (clients beyond the first MAX_CLIENTS)
     uint32_t nvars;
     uint64_t tile_count;
     uint32_t nwarps;

@@ -1,8 +1,9 @@
 """Aggregation of client replicas that live on several GPUs (Sec. 1: the clients' models are sent
 back and aggregated; Sec. 2.5: every client compresses its own subset).
 
-Plumbing only: the two library calls do the arithmetic on each GPU (omc_aggregate_sum adds up the
-GPU's own clients, omc_divide turns the total into the mean); in between, one all-reduce of
+Plumbing only: the library calls do the arithmetic on each GPU (omc_aggregate_sum adds up the
+GPU's own clients, omc_aggregate_add those beyond the first sixteen, omc_divide turns the total
+into the mean); in between, one all-reduce of
 ``torch.distributed`` adds the per-GPU sums and another the client counts.  Every buffer handed to
 the collective is owned by the calling rank; no kernel of the library ever sees another GPU's
 memory.  The two steps are passed in as callables so that the bookkeeping can be run on CPU ranks
@@ -46,10 +47,14 @@ def mean_of_local_and_remote_clients(plans, packed, resid, sb, out, stream=0, gr
     layout_plan = plans[0] if plans else layout_plan
 
     def local_sum(t):
-        if plans:
-            omc.aggregate_sum(plans, packed, resid, sb, t.data_ptr(), stream)
-        else:
+        # any number of clients: the first batch starts the sum, each further batch is added to it,
+        # in client order throughout
+        if not plans:
             t.zero_()
+        step = omc.MAX_CLIENTS_PER_CALL
+        for a in range(0, len(plans), step):
+            call = omc.aggregate_sum if a == 0 else omc.aggregate_add
+            call(plans[a:a + step], packed[a:a + step], resid[a:a + step], sb[a:a + step], t.data_ptr(), stream)
 
     return mean_across_ranks(out, len(plans), local_sum,
                              lambda t, k: omc.divide(layout_plan, t.data_ptr(), k, stream), group)

@@ -539,6 +539,47 @@ def test_aggregate_with_extreme_transformations(fmt):
         assert same_f32(from_full(clients[0].plan, got, i), want[i]), i
 
 
+@pytest.mark.parametrize("fmt", [(5, 10), (5, 2), (3, 7), (4, 14)], ids=lambda f: "E%dM%d" % f)
+def test_aggregate_more_clients_than_one_call_takes(fmt):
+    """Forty clients in batches of 16, 16 and 8 (omc_aggregate_sum, then omc_aggregate_add twice,
+    then omc_divide): the same FP32 additions in the same order as one pass over all forty, so the
+    result equals the oracle's mean over the forty bit for bit."""
+    from paper_2205_03494_b200 import replicas
+    rng = np.random.default_rng(57)
+    numel = [3000, 1, 1024, 5121, 333, 20000, 77]
+    kinds = [0, 0, 0, 0, 1, 0, 2]
+    base = [(rng.standard_normal(n) * 0.1).astype(np.float32) for n in numel]
+    clients = []
+    for k in range(40):
+        params = [(p + rng.standard_normal(p.size).astype(np.float32) * np.float32(0.01)) for p in base]
+        if k == 21:
+            params[0][:4] = [np.inf, np.nan, -0.0, 1e-45]
+        clients.append(Lockstep(numel, kinds, fmt, params, fraction=0.6, seed=300 + k))
+    st = torch.cuda.current_stream().cuda_stream
+    plan0 = clients[0].plan
+    args = lambda cs: ([c.plan for c in cs], [c.dm.packed.data_ptr() for c in cs], [c.dm.resid.data_ptr() for c in cs],
+                       [c.dm.sb.data_ptr() for c in cs])
+    out = clients[0].dm.full_buffer("running sum")
+    out.fill_(123.0)                                  # the first batch must not read it
+    omc.aggregate_sum(*args(clients[:16]), out.data_ptr(), st)
+    omc.aggregate_add(*args(clients[16:32]), out.data_ptr(), st)
+    omc.aggregate_add(*args(clients[32:]), out.data_ptr(), st)
+    omc.divide(plan0, out.data_ptr(), 40, st)
+    torch.cuda.synchronize()
+    clients[0].dm.check_guards()
+    got = out.cpu().numpy()
+    want = orc.aggregate([c.st for c in clients])
+    for i in range(len(numel)):
+        assert same_f32(from_full(plan0, got, i), want[i]), i
+    # the helper cuts any number of local clients into such batches
+    out2 = torch.zeros(plan0.full_elems, dtype=torch.float32, device="cuda")
+    k = replicas.mean_of_local_and_remote_clients(*args(clients), out2, st)
+    torch.cuda.synchronize()
+    assert k == 40 and torch.equal(out2.view(torch.int32), out.view(torch.int32))
+    L = omc.lib()
+    assert L.omc_aggregate_add(None, 1, None, None, None, out.data_ptr(), None) == -3
+
+
 @pytest.mark.parametrize("fmt", [(5, 10), (5, 2), (3, 7)], ids=lambda f: "E%dM%d" % f)
 def test_aggregate_in_two_stages(fmt):
     """The mean over clients held by several GPUs (omc_aggregate_sum per holder, the holders' sums

@@ -364,3 +364,21 @@ def test_two_stage_mean_is_sum_then_one_division():
     assert np.array_equal(orc.divide_var(orc.sum_var(xs), 7), orc.aggregate_var(xs))
     bound = 6 * 2.0 ** -24 * np.sum(np.abs(xs), axis=0) / 7 + 2.0 ** -24 * np.abs(orc.aggregate_var(xs))
     assert np.all(np.abs(got.astype(np.float64) - orc.aggregate_var(xs)) <= 2 * bound)
+
+
+def test_sum_continued_batch_after_batch_is_the_one_pass_sum():
+    """A sum that starts from the sum so far and adds the next batch of clients in order makes the
+    additions of one pass over all clients, in the same order: forty clients in batches of 16, 16
+    and 8 give the one-pass sum and mean bit for bit (the first element checked in exact rationals)."""
+    rng = np.random.default_rng(33)
+    n = 64
+    xs = [(rng.standard_normal(n) * 10.0 ** rng.integers(-3, 3)).astype(np.float32) for _ in range(40)]
+    run = orc.sum_var(xs[:16])
+    run = orc.sum_var([run] + xs[16:32])
+    run = orc.sum_var([run] + xs[32:])
+    assert np.array_equal(run.view(np.uint32), orc.sum_var(xs).view(np.uint32))
+    assert np.array_equal(orc.divide_var(run, 40).view(np.uint32), orc.aggregate_var(xs).view(np.uint32))
+    acc = np.float32(xs[0][0])
+    for x in xs[1:]:
+        acc = f32_round(Fraction(float(acc)) + Fraction(float(x[0])))
+    assert run[0] == acc
