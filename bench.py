@@ -631,7 +631,10 @@ def run_ours(args):
         "config": {"workload": config_label(wl, args.fixed),
                    "params": nparams, "variables": plan.nvars, "quantised_variables": plan.n_quantised,
                    "bytes_per_step": step_bytes, "lr": wl.lr, "pvt": not args.no_pvt, "weights_only": not args.all_variables, "gradients": "one seeded buffer reused every step",
-                   "l2": "inputs per step (%.0f MB) exceed the 126 MB L2; no flush" % (step_bytes / 1e6),
+                   "l2": ("inputs per step (%.0f MB) exceed the 126 MB L2; no flush" % (step_bytes / 1e6)
+                          if step_bytes > 126e6 else
+                          "inputs per step (%.1f MB) fit the 126 MB L2 and are not flushed: a latency figure, "
+                          "not a bandwidth one" % (step_bytes / 1e6)),
                    "multi_gpu": "replicas only"},
         "hbm_gbs": achieved, "pct_of_8tbs": 100 * achieved / NOMINAL_HBM_GBS,
         "clocks": clocks,
