@@ -202,13 +202,16 @@ __device__ __forceinline__ void fixed8_to_halves(uint32_t c4, uint32_t &h01, uin
     h01 = hfma2_bits(__byte_perm(x, 0x64646464u, 0x5140), 0.0078125f, -9.f);
     h23 = hfma2_bits(__byte_perm(x, 0x64646464u, 0x5342), 0.0078125f, -9.f);
 }
-// S1I0F11, two codes in the low 12 bits of each half of `pr`: j = k + 2048 has twelve bits, the low
-// ten go into one FP16 value (1024 + lo), the top two into another (1024 + 256 hi); then
-// (1024 + 256 hi) 2^-9 - 3.5 = hi/2 - 1.5 and (1024 + lo) 2^-11 + that = (lo + 1024 hi) / 2048 - 1 = k / 2048.
-__device__ __forceinline__ uint32_t fixed12_to_halves(uint32_t pr)
+// S1I0F11, two codes: `t` holds three bytes of the stream as (b0 b1 | b1 b2), so code 0 is the low
+// 12 bits of the low half and code 1 the high 12 bits of the high half; one shift and a byte permute
+// put both in the low 12 bits of their halves (what lies above is masked away below).
+// j = k + 2048 = code xor 0x800 has twelve bits: the low ten go into one FP16 value (1024 + lo), the
+// top two into another (1024 + 256 hi; the xor only touches bit 11 and is folded into the constant);
+// then (1024 + 256 hi) 2^-9 - 3.5 = hi/2 - 1.5 and (1024 + lo) 2^-11 + that = (lo + 1024 hi) / 2048 - 1 = k / 2048.
+__device__ __forceinline__ uint32_t fixed12_to_halves(uint32_t t)
 {
-    const uint32_t x = pr ^ 0x08000800u;
-    const uint32_t lo = (x & 0x03FF03FFu) | 0x64006400u, hi = ((x >> 2) & 0x03000300u) | 0x64006400u;
+    const uint32_t v = __byte_perm(t, t >> 4, 0x7610);
+    const uint32_t lo = (v & 0x03FF03FFu) | 0x64006400u, hi = ((v >> 2) & 0x03000300u) ^ 0x66006600u;
     const __half2 c = __hfma2(*reinterpret_cast<const __half2 *>(&hi), __float2half2_rn(0.001953125f), __float2half2_rn(-3.5f));
     const __half2 r = __hfma2(*reinterpret_cast<const __half2 *>(&lo), __float2half2_rn(0.00048828125f), c);
     return *reinterpret_cast<const uint32_t *>(&r);
@@ -246,9 +249,7 @@ __device__ __forceinline__ uint4 expand_chunk(const uint8_t *raw)
         const uint32_t w0 = rw[0], w1 = rw[1], w2 = rw[2];
         const uint32_t t0 = __byte_perm(w0, 0u, 0x2110), t1 = __byte_perm(w0, w1, 0x5443);
         const uint32_t t2 = __byte_perm(w1, w2, 0x4332), t3 = __byte_perm(w2, 0u, 0x3221);
-        auto pair = [](uint32_t t) { return (t & 0x00000FFFu) | ((t >> 4) & 0x0FFF0000u); };
-        return make_uint4(fixed12_to_halves(pair(t0)), fixed12_to_halves(pair(t1)), fixed12_to_halves(pair(t2)),
-                          fixed12_to_halves(pair(t3)));
+        return make_uint4(fixed12_to_halves(t0), fixed12_to_halves(t1), fixed12_to_halves(t2), fixed12_to_halves(t3));
     } else if constexpr (B == 8 && E == 5) {        // a code is the top byte of its half
         const uint2 w = *reinterpret_cast<const uint2 *>(raw);
         return make_uint4(__byte_perm(w.x, 0u, 0x1404), __byte_perm(w.x, 0u, 0x3424),
