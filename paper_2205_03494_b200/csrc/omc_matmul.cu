@@ -281,36 +281,39 @@ __device__ __forceinline__ uint4 expand_chunk(const uint8_t *raw)
     }
 }
 
-// Odd widths: the chunk's B bytes start at any byte; four aligned words hold them.
+// Odd widths: the chunk's B bytes start at any byte; four aligned words hold them.  A code is taken
+// with its sign at bit 31 (one shift, or a funnel shift where it straddles two words); one arithmetic
+// shift then puts exponent and mantissa where FP16 keeps them, with copies of the sign above, and a
+// mask keeps bit 15 of those and drops what follows the code: the low half of the pair from a shift
+// by 21 - E, the high half from a shift by 5 - E, so the pair needs no further assembly.
 template <int B, int E>
 __device__ __forceinline__ uint4 expand_chunk_odd(const uint8_t *raw)
 {
-    constexpr int M = B - 1 - E, SHIFT = 10 - M;
-    constexpr uint32_t MAG = (1u << (E + M)) - 1u, CODE = (1u << B) - 1u, INF_MAG = ((1u << E) - 1u) << M;
+    constexpr int M = B - 1 - E;
+    constexpr uint32_t MAG = (1u << (E + M)) - 1u, INF_MAG = ((1u << E) - 1u) << M;
+    constexpr uint32_t HMASK = 0x8000u | (MAG << (10 - M));
     const uint32_t a = (uint32_t)__cvta_generic_to_shared(raw);
     const uint32_t sh = (a & 3u) * 8u;
     uint32_t w0, w1, w2, w3;
     asm volatile("ld.shared.u32 %0, [%4];\n\tld.shared.u32 %1, [%4+4];\n\tld.shared.u32 %2, [%4+8];\n\tld.shared.u32 %3, [%4+12];"
                  : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(a & ~3u));
     uint32_t v[4] = {__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh), __funnelshift_r(w2, w3, sh), w3 >> sh};
+    auto top = [&](int j) -> uint32_t {          // code j in the top B bits of the result
+        const int pos = j * B, wi = pos >> 5, bs = pos & 31;
+        return (bs + B <= 32) ? (v[wi] << (32 - bs - B)) : __funnelshift_r(v[wi], v[wi + 1 < 4 ? wi + 1 : wi], bs + B - 32);
+    };
     uint32_t h[4];
     bool special = false;
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
-        uint32_t hp = 0u;
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const int pos = (2 * p + q) * B, wi = pos >> 5, bs = pos & 31;
-            uint32_t c = (bs + B <= 32) ? (v[wi] >> bs) : __funnelshift_r(v[wi], v[wi + 1 < 4 ? wi + 1 : wi], bs);
-            c &= CODE;
-            const uint32_t mag = c & MAG;
-            uint32_t hb = (mag << SHIFT) | ((c >> (E + M)) << 15);
-            if (E != 5 && mag >= INF_MAG) special = true;
-            hp |= hb << (16 * q);
-        }
-        if constexpr (E != 5) {      // exponent field + (15 - bias): one exact multiplication, subnormal codes included
-            const __half2 scale = __float2half2_rn((float)(1u << (15 - ((1 << (E - 1)) - 1))));
-            const __half2 r = __hmul2(*reinterpret_cast<const __half2 *>(&hp), scale);
+        const uint32_t lo = (uint32_t)((int32_t)top(2 * p) >> (21 - E)) & HMASK;
+        uint32_t hp = ((uint32_t)((int32_t)top(2 * p + 1) >> (5 - E)) & (HMASK << 16)) | lo;
+        if constexpr (E != 5) {
+            // exponent field + (15 - bias): one exact multiplication, subnormal codes included; a code with
+            // an all-ones exponent field then has a magnitude of at least 2^(2^E - 1 - bias), every other less
+            constexpr int BIAS = (1 << (E - 1)) - 1;
+            const __half2 r = __hmul2(*reinterpret_cast<const __half2 *>(&hp), __float2half2_rn((float)(1u << (15 - BIAS))));
+            special |= !__hblt2(__habs2(r), __float2half2_rn((float)(1u << ((1 << E) - 1 - BIAS))));
             hp = *reinterpret_cast<const uint32_t *>(&r);
         }
         h[p] = hp;
@@ -318,9 +321,7 @@ __device__ __forceinline__ uint4 expand_chunk_odd(const uint8_t *raw)
     if (E != 5 && special) {         // rare: a weight is Inf or NaN
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const int pos = j * B, wi = pos >> 5, bs = pos & 31;
-            uint32_t c = (bs + B <= 32) ? (v[wi] >> bs) : __funnelshift_r(v[wi], v[wi + 1 < 4 ? wi + 1 : wi], bs);
-            c &= CODE;
+            const uint32_t c = top(j) >> (32 - B);
             const uint32_t mag = c & MAG;
             if (mag >= INF_MAG) {
                 const uint32_t hb = ((c >> (E + M)) << 15) | (mag == INF_MAG ? 0x7C00u : 0x7E00u);
@@ -332,13 +333,14 @@ __device__ __forceinline__ uint4 expand_chunk_odd(const uint8_t *raw)
 }
 
 // S1E4M14: eight 19-bit codes (19 bytes from any byte) -> eight FP16 pairs (hi, lo) with
-// hi + lo = the weight exactly.  The weight is built as an FP32 value first (fields in place, one
-// exact multiplication by 2^(127 - 7) that also normalises subnormal codes), hi is its FP16
-// rounding, lo the FP16 value of the exact FP32 remainder.  Inf / NaN codes: hi = Inf / NaN, lo = 0.
+// hi + lo = the weight exactly.  The weight is built as an FP32 value first (fields in place by one
+// arithmetic shift and a mask, as above, then one exact multiplication by 2^(127 - 7) that also
+// normalises subnormal codes), hi is its FP16 rounding, lo the FP16 value of the exact FP32
+// remainder.  Inf / NaN codes: hi = Inf / NaN, lo = 0.
 __device__ __forceinline__ void expand_chunk_split(const uint8_t *raw, uint4 &hi4, uint4 &lo4)
 {
     constexpr int B = 19, E = 4, M = 14;
-    constexpr uint32_t MAG = (1u << (E + M)) - 1u, CODE = (1u << B) - 1u, INF_MAG = ((1u << E) - 1u) << M;
+    constexpr uint32_t MAG = (1u << (E + M)) - 1u, INF_MAG = ((1u << E) - 1u) << M;
     const uint32_t a = (uint32_t)__cvta_generic_to_shared(raw);
     const uint32_t sh = (a & 3u) * 8u;
     uint32_t w[6];
@@ -348,27 +350,38 @@ __device__ __forceinline__ void expand_chunk_split(const uint8_t *raw, uint4 &hi
     uint32_t v[5];
 #pragma unroll
     for (int i = 0; i < 5; ++i) v[i] = __funnelshift_r(w[i], w[i + 1], sh);
+    auto top = [&](int j) -> uint32_t {          // code j in the top 19 bits of the result
+        const int pos = j * B, wi = pos >> 5, bs = pos & 31;
+        return (bs + B <= 32) ? (v[wi] << (32 - bs - B)) : __funnelshift_r(v[wi], v[wi + 1 < 5 ? wi + 1 : wi], bs + B - 32);
+    };
     uint32_t h[4], l[4];
+    bool special = false;
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
-        h[p] = 0u;
-        l[p] = 0u;
+        float val[2];
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
-            const int pos = (2 * p + q) * B, wi = pos >> 5, bs = pos & 31;
-            uint32_t c = (bs + B <= 32) ? (v[wi] >> bs) : __funnelshift_r(v[wi], v[wi + 1 < 5 ? wi + 1 : wi], bs);
-            c &= CODE;
-            const uint32_t mag = c & MAG, sign = (c >> (E + M)) << 31;
-            const float val = __fmul_rn(__uint_as_float(sign | (mag << (23 - M))), __uint_as_float((uint32_t)(127 - 7 + 127) << 23));
-            __half hh = __float2half_rn(val);
-            __half ll = __float2half_rn(__fsub_rn(val, __half2float(hh)));
-            uint32_t hb = __half_as_ushort(hh), lb = __half_as_ushort(ll);
+            const uint32_t placed = (uint32_t)((int32_t)top(2 * p + q) >> (8 - E)) & (0x80000000u | (MAG << (23 - M)));
+            val[q] = __fmul_rn(__uint_as_float(placed), __uint_as_float((uint32_t)(127 - 7 + 127) << 23));
+        }
+        special |= !(fmaxf(fabsf(val[0]), fabsf(val[1])) < 256.f);      // an all-ones exponent field: 2^8 or more
+        // both roundings as packed conversions of the pair (the one-value conversion runs at a quarter of the rate)
+        const __half2 hh = __floats2half2_rn(val[0], val[1]);
+        const float2 hf = __half22float2(hh);
+        const __half2 ll = __floats2half2_rn(__fsub_rn(val[0], hf.x), __fsub_rn(val[1], hf.y));
+        h[p] = *reinterpret_cast<const uint32_t *>(&hh);
+        l[p] = *reinterpret_cast<const uint32_t *>(&ll);
+    }
+    if (special) {          // rare: a weight is Inf or NaN
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t c = top(j) >> (32 - B);
+            const uint32_t mag = c & MAG;
             if (mag >= INF_MAG) {
-                hb = (sign >> 16) | (mag == INF_MAG ? 0x7C00u : 0x7E00u);
-                lb = 0u;
+                const uint32_t hb = ((c >> (E + M)) << 15) | (mag == INF_MAG ? 0x7C00u : 0x7E00u);
+                h[j >> 1] = (j & 1) ? ((h[j >> 1] & 0x0000FFFFu) | (hb << 16)) : ((h[j >> 1] & 0xFFFF0000u) | hb);
+                l[j >> 1] &= (j & 1) ? 0x0000FFFFu : 0xFFFF0000u;
             }
-            h[p] |= hb << (16 * q);
-            l[p] |= lb << (16 * q);
         }
     }
     hi4 = make_uint4(h[0], h[1], h[2], h[3]);
