@@ -1711,134 +1711,135 @@ __global__ void __launch_bounds__(THREADS, aggregate_ctas_per_sm(F::B)) omc_aggr
     // Short runs of equal length, dealt out to the warps in turn: what a tile costs depends on how many
     // clients hold it in FP32, and a long stretch of costly tiles is shared by all warps this way.
     for (uint32_t run = warp; run < p.nruns && !failed; run += p.nwarps) {
-    uint64_t t = (uint64_t)run * p.tile_count / p.nruns;
-    const uint64_t tend = (uint64_t)(run + 1) * p.tile_count / p.nruns;
-    uint32_t lo = 0, hi = p.nvars;
-    while (hi - lo > 1) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (__ldg(&p.vars[0][mid].tile_start) <= t) lo = mid; else hi = mid;
-    }
-    uint32_t v = lo;
-
-    while (t < tend && !failed) {
-        const VarDev var = load_var(p.vars[0] + v);
-        __syncwarp();
-        if ((uint32_t)lane < K) {
-            const VarDev vk = load_var(p.vars[lane] + v);
-            AggClientVar c;
-            c.quantised = vk.quantised;
-            c.last_bytes = vk.ntiles ? (uint32_t)(vk.packed_bytes - (uint64_t)(vk.ntiles - 1) * CB) : 0u;
-            c.base = vk.quantised ? reinterpret_cast<uint64_t>(p.packed[lane] + vk.store_off)
-                                  : reinterpret_cast<uint64_t>(p.resid[lane] + vk.store_off);
-            c.s = vk.quantised ? __ldg(p.sb[lane] + 2 * vk.sb_slot) : 1.f;
-            c.b = vk.quantised ? __ldg(p.sb[lane] + 2 * vk.sb_slot + 1) : 0.f;
-            c.sk = c.s;
-            c.folded = 0u;
-            if constexpr (PlacedPath<F>::value) {
-                c.sk = __fmul_rn(c.s, u2f(F::pow2_bits(127 - F::BIAS)));
-                c.folded = fabsf(c.sk) < u2f(0x7F800000u) ? 1u : 0u;       // no overflow: the product is exact
-            }
-            cv[lane] = c;
+        uint64_t t = (uint64_t)run * p.tile_count / p.nruns;
+        const uint64_t tend = (uint64_t)(run + 1) * p.tile_count / p.nruns;
+        uint32_t lo = 0, hi = p.nvars;
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (__ldg(&p.vars[0][mid].tile_start) <= t) lo = mid; else hi = mid;
         }
-        __syncwarp();
-        const uint32_t local = (uint32_t)(t - var.tile_start);
-        const uint64_t left = tend - t;
-        const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
+        uint32_t v = lo;
 
-        // the producer's place in this variable's (tile, client) pairs
-        uint32_t ptile = 0u, pk = 0u;
-        auto fill = [&]() {                     // called by the whole warp
-            while (ptile < cnt && in_ring < NSLOT && fp32_ahead < FP32_AHEAD) {
-                const AggClientVar c = cv[pk];
-                if (c.quantised) {
-                    // packed sizes are multiples of 16 bytes, and so is what is left of one in its last tile
-                    const uint64_t off = (uint64_t)(local + ptile) * CB;
-                    const uint32_t bytes = local + ptile + 1 == var.ntiles ? c.last_bytes : CB;
-                    if (lane == 0) {
-                        const uint32_t bar = bar0 + 8u * pslot;
-                        mbar_expect_tx(bar, bytes);
-                        if (!skip_loads)
-                            bulk_load(smem_addr(ring + pslot * CB), reinterpret_cast<const uint8_t *>(c.base) + off, bytes, bar);
-                    }
-                    pslot = pslot + 1 == NSLOT ? 0u : pslot + 1;
-                    ++in_ring;
-                } else {
-                    // an FP32 copy is read with plain loads when its turn comes: ask for its lines now
-                    const uint64_t e = (uint64_t)(local + ptile) * TILE + (uint32_t)lane * 32u;
-                    if (e < var.n) prefetch_l2(reinterpret_cast<const float *>(c.base) + e);
-                    ++fp32_ahead;
+        while (t < tend && !failed) {
+            const VarDev var = load_var(p.vars[0] + v);
+            __syncwarp();
+            if ((uint32_t)lane < K) {
+                const VarDev vk = load_var(p.vars[lane] + v);
+                AggClientVar c;
+                c.quantised = vk.quantised;
+                c.last_bytes = vk.ntiles ? (uint32_t)(vk.packed_bytes - (uint64_t)(vk.ntiles - 1) * CB) : 0u;
+                c.base = vk.quantised ? reinterpret_cast<uint64_t>(p.packed[lane] + vk.store_off)
+                                      : reinterpret_cast<uint64_t>(p.resid[lane] + vk.store_off);
+                c.s = vk.quantised ? __ldg(p.sb[lane] + 2 * vk.sb_slot) : 1.f;
+                c.b = vk.quantised ? __ldg(p.sb[lane] + 2 * vk.sb_slot + 1) : 0.f;
+                c.sk = c.s;
+                c.folded = 0u;
+                if constexpr (PlacedPath<F>::value) {
+                    c.sk = __fmul_rn(c.s, u2f(F::pow2_bits(127 - F::BIAS)));
+                    c.folded = fabsf(c.sk) < u2f(0x7F800000u) ? 1u : 0u;       // no overflow: the product is exact
                 }
-                if (++pk == K) { pk = 0u; ++ptile; }
+                cv[lane] = c;
             }
-        };
+            __syncwarp();
+            const uint32_t local = (uint32_t)(t - var.tile_start);
+            const uint64_t left = tend - t;
+            const uint32_t cnt = (uint32_t)((uint64_t)(var.ntiles - local) < left ? (var.ntiles - local) : left);
 
-        for (uint32_t ti = 0; ti < cnt && !failed; ++ti) {
-            fill();
-            const uint64_t e_tile = (uint64_t)(local + ti) * TILE;
-            const bool whole = e_tile + TILE <= var.n;
-            const uint32_t n_here = whole ? (uint32_t)TILE : (uint32_t)(var.n - e_tile);     // the tile's elements
-            const uint32_t n_pad = (n_here + 3u) & ~3u;
-            float acc[32];
-            // client k's turn; false: the wait for its codes ran out
-            auto client = [&](auto first, uint32_t k) -> bool {
-                constexpr bool FIRST = decltype(first)::value;
-                const AggClientVar c = cv[k];
-                if (c.quantised) {
-                    const uint32_t bar = bar0 + 8u * cslot, parity = (phases >> cslot) & 1u;
-                    phases ^= 1u << cslot;
-                    uint32_t polls = 0;
-                    while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) {
-                        if (++polls > wait_limit) return false;
-                    }
-                    const uint32_t *sw = reinterpret_cast<const uint32_t *>(ring + cslot * CB);
-                    if constexpr (PlacedPath<F>::value) agg_tile_codes<F, FIRST>(sw, c.s, c.sk, c.b, c.folded != 0u, acc, lane);
-                    else agg_tile_codes<F, FIRST>(sw, c.s, c.s, c.b, true, acc, lane);
-                    __syncwarp();               // every lane has read the slot: it may be filled again
-                    cslot = cslot + 1 == NSLOT ? 0u : cslot + 1;
-                    --in_ring;
-                    fill();
-                } else {
-                    const float *r = reinterpret_cast<const float *>(c.base) + e_tile;
-                    if (whole) agg_tile_fp32<F, FIRST, true>(r, n_pad, acc, lane);
-                    else agg_tile_fp32<F, FIRST, false>(r, n_pad, acc, lane);
-                    --fp32_ahead;
-                    fill();
-                }
-                return true;
-            };
-            float *o = p.out + var.full_off + e_tile;
-            uint32_t k = 0;
-            if (accumulate) {       // the sum so far, left in `out` by the call before
-                if (whole) agg_tile_fp32<F, true, true>(o, n_pad, acc, lane);
-                else agg_tile_fp32<F, true, false>(o, n_pad, acc, lane);
-            } else {
-                failed = !client(std::true_type{}, 0u);
-                k = 1;
-            }
-            for (; k < K && !failed; ++k) failed = !client(std::false_type{}, k);
-            if (failed) break;
-#pragma unroll
-            for (int q = 0; q < NQ; ++q)
-#pragma unroll
-                for (int j = 0; j < AL / 4; ++j) {
-                    const uint32_t e = (uint32_t)(q * 32 + lane) * AL + 4 * j;
-                    const int i = q * AL + 4 * j;
-                    float4 m = make_float4(mean_of(acc[i]), mean_of(acc[i + 1]), mean_of(acc[i + 2]), mean_of(acc[i + 3]));
-                    if (whole) {
-                        *reinterpret_cast<float4 *>(o + e) = m;
-                    } else if (e < n_pad) {
-                        if (e + 3 >= n_here) {          // the padding after the variable's last element: zeros
-                            if (e + 1 >= n_here) m.y = 0.f;
-                            if (e + 2 >= n_here) m.z = 0.f;
-                            m.w = 0.f;
+            // the producer's place in this variable's (tile, client) pairs
+            uint32_t ptile = 0u, pk = 0u;
+            auto fill = [&]() {                     // called by the whole warp
+                while (ptile < cnt && in_ring < NSLOT && fp32_ahead < FP32_AHEAD) {
+                    const AggClientVar c = cv[pk];
+                    if (c.quantised) {
+                        // packed sizes are multiples of 16 bytes, and so is what is left of one in its last tile
+                        const uint64_t off = (uint64_t)(local + ptile) * CB;
+                        const uint32_t bytes = local + ptile + 1 == var.ntiles ? c.last_bytes : CB;
+                        if (lane == 0) {
+                            const uint32_t bar = bar0 + 8u * pslot;
+                            mbar_expect_tx(bar, bytes);
+                            if (!skip_loads)
+                                bulk_load(smem_addr(ring + pslot * CB), reinterpret_cast<const uint8_t *>(c.base) + off, bytes,
+                                          bar);
                         }
-                        *reinterpret_cast<float4 *>(o + e) = m;
+                        pslot = pslot + 1 == NSLOT ? 0u : pslot + 1;
+                        ++in_ring;
+                    } else {
+                        // an FP32 copy is read with plain loads when its turn comes: ask for its lines now
+                        const uint64_t e = (uint64_t)(local + ptile) * TILE + (uint32_t)lane * 32u;
+                        if (e < var.n) prefetch_l2(reinterpret_cast<const float *>(c.base) + e);
+                        ++fp32_ahead;
                     }
+                    if (++pk == K) { pk = 0u; ++ptile; }
                 }
+            };
+
+            for (uint32_t ti = 0; ti < cnt && !failed; ++ti) {
+                fill();
+                const uint64_t e_tile = (uint64_t)(local + ti) * TILE;
+                const bool whole = e_tile + TILE <= var.n;
+                const uint32_t n_here = whole ? (uint32_t)TILE : (uint32_t)(var.n - e_tile);     // the tile's elements
+                const uint32_t n_pad = (n_here + 3u) & ~3u;
+                float acc[32];
+                // client k's turn; false: the wait for its codes ran out
+                auto client = [&](auto first, uint32_t k) -> bool {
+                    constexpr bool FIRST = decltype(first)::value;
+                    const AggClientVar c = cv[k];
+                    if (c.quantised) {
+                        const uint32_t bar = bar0 + 8u * cslot, parity = (phases >> cslot) & 1u;
+                        phases ^= 1u << cslot;
+                        uint32_t polls = 0;
+                        while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(bar, parity))) {
+                            if (++polls > wait_limit) return false;
+                        }
+                        const uint32_t *sw = reinterpret_cast<const uint32_t *>(ring + cslot * CB);
+                        if constexpr (PlacedPath<F>::value) agg_tile_codes<F, FIRST>(sw, c.s, c.sk, c.b, c.folded != 0u, acc, lane);
+                        else agg_tile_codes<F, FIRST>(sw, c.s, c.s, c.b, true, acc, lane);
+                        __syncwarp();               // every lane has read the slot: it may be filled again
+                        cslot = cslot + 1 == NSLOT ? 0u : cslot + 1;
+                        --in_ring;
+                        fill();
+                    } else {
+                        const float *r = reinterpret_cast<const float *>(c.base) + e_tile;
+                        if (whole) agg_tile_fp32<F, FIRST, true>(r, n_pad, acc, lane);
+                        else agg_tile_fp32<F, FIRST, false>(r, n_pad, acc, lane);
+                        --fp32_ahead;
+                        fill();
+                    }
+                    return true;
+                };
+                float *o = p.out + var.full_off + e_tile;
+                uint32_t k = 0;
+                if (accumulate) {       // the sum so far, left in `out` by the call before
+                    if (whole) agg_tile_fp32<F, true, true>(o, n_pad, acc, lane);
+                    else agg_tile_fp32<F, true, false>(o, n_pad, acc, lane);
+                } else {
+                    failed = !client(std::true_type{}, 0u);
+                    k = 1;
+                }
+                for (; k < K && !failed; ++k) failed = !client(std::false_type{}, k);
+                if (failed) break;
+#pragma unroll
+                for (int q = 0; q < NQ; ++q)
+#pragma unroll
+                    for (int j = 0; j < AL / 4; ++j) {
+                        const uint32_t e = (uint32_t)(q * 32 + lane) * AL + 4 * j;
+                        const int i = q * AL + 4 * j;
+                        float4 m = make_float4(mean_of(acc[i]), mean_of(acc[i + 1]), mean_of(acc[i + 2]), mean_of(acc[i + 3]));
+                        if (whole) {
+                            *reinterpret_cast<float4 *>(o + e) = m;
+                        } else if (e < n_pad) {
+                            if (e + 3 >= n_here) {          // the padding after the variable's last element: zeros
+                                if (e + 1 >= n_here) m.y = 0.f;
+                                if (e + 2 >= n_here) m.z = 0.f;
+                                m.w = 0.f;
+                            }
+                            *reinterpret_cast<float4 *>(o + e) = m;
+                        }
+                    }
+            }
+            t += cnt;
+            ++v;
         }
-        t += cnt;
-        ++v;
-    }
     }
     if (failed && lane == 0) atomicExch(p.status, 1u);       // a bulk load never arrived
 }
