@@ -616,6 +616,201 @@ bool make_raw_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t row_b
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// ---------------------------------------------------------------------------------------------
+// S1E5M10 on pairs of SMs.  Two CTAs of a cluster share one 256 x 256 tile of Y: each holds its own
+// 128 rows of X and its own 128 rows of the codes per K block (32 KB instead of the 48 KB of the
+// one-SM kernel for the same number of products, and six stages instead of four), the leader's
+// MMA thread issues tcgen05.mma.cta_group::2 (M = 256: the upper 128 rows accumulate in the
+// leader's tensor memory, the lower in its peer's; the 256 columns of the B operand are read from
+// both CTAs' shared memory), and each CTA's epilogue warps store their own 128 rows.
+//   full(s)      lives in the leader: its producer announces the bytes of both CTAs; both producers'
+//                copies complete on it (bulk tensor copies in their cta_group::2 form, which may
+//                signal the barrier of the pair's other CTA; no multicast).
+//   empty(s)     one in each CTA, for its producer: the MMA thread's commit reaches both.
+//   acc_full(b)  one in each CTA, for its epilogue: the commit after a tile's last MMA reaches both.
+//   acc_empty(b) lives in the leader, 256 arrivals: the epilogue threads of both CTAs.
+// The barriers are initialised before a cluster-wide barrier and nothing of the peer is touched
+// before it; a second one before the tensor memory is released keeps either CTA alive while the
+// other may still signal it.  Every mbarrier wait is bounded; a wait that runs out ends that role's
+// loop, so that both CTAs always reach the closing barrier.
+constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_BN_HALF = 128;                                   // rows of the codes per CTA
+constexpr int PAIR_STAGE = TILE_A_BYTES + PAIR_BN_HALF * BK * 2;     // 32 KB
+constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE + 1024 + 256;
+constexpr int PAIR_THREADS = 192;
+constexpr uint32_t PAIR_IDESC = (1u << 4) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+
+__device__ __forceinline__ uint32_t cluster_cta_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// The shared::cluster address of the same location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_barrier()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Tile into this CTA's shared memory; the bytes complete on `bar`, a shared::cluster address in either CTA of the pair.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_f16_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+// Arrives, once the MMAs issued so far have finished, on the barrier at this address in both CTAs.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(both) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+__global__ void __launch_bounds__(PAIR_THREADS, 1)
+matmul_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                   const float *__restrict__ sb, const float *__restrict__ rowsum, float *__restrict__ y,
+                   uint32_t M, uint32_t N, uint32_t K, uint32_t *status, uint32_t inject_polls)
+{
+    constexpr int NS = PAIR_STAGES;
+    const uint32_t limit = inject_polls ? inject_polls : WAIT_LIMIT;
+    const bool skip_loads = inject_polls != 0u;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (saddr(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bars = base + NS * PAIR_STAGE;   // full[NS], empty[NS], acc_full[2], acc_empty[2], tmem slot
+    auto full = [&](int s) { return bars + 8u * s; };
+    auto empty = [&](int s) { return bars + 8u * (NS + s); };
+    auto acc_full = [&](int b) { return bars + 8u * (2 * NS + b); };
+    auto acc_empty = [&](int b) { return bars + 8u * (2 * NS + 2 + b); };
+    const uint32_t tmem_slot = bars + 8u * (2 * NS + 4);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_cta_rank();          // 0: the leader
+    const uint32_t nkb = K / BK;
+    const uint32_t tiles_m = (M + 255) / 256, tiles_n = (N + 255) / 256, ntiles = tiles_m * tiles_n;
+    const uint32_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 256); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // the same warp of both CTAs allocates the pair's tensor memory
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"((uint32_t)TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_barrier();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+
+    bool ok = true;
+    if (tid == 0) {
+        // ---- producer of this CTA: its 128 rows of X and its 128 rows of the codes per K block
+        uint32_t it = 0;
+        for (uint32_t t = pair; t < ntiles && ok; t += npairs) {
+            const int tm = t % tiles_m, tn = t / tiles_m;
+            for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
+                const int s = it % NS;
+                if (it >= (uint32_t)NS) ok = mbar_wait(empty(s), ((it / NS) - 1) & 1u, limit);
+                if (!ok) break;
+                if (rank == 0) mbar_expect_tx(full(s), 2u * PAIR_STAGE);        // the bytes of both CTAs
+                if (skip_loads) continue;
+                const uint32_t a = base + s * PAIR_STAGE, lead_full = map_to_cta(full(s), 0u);
+                tma_load_2d_pair(a, &map_x, (int)(kb * BK), tm * 256 + (int)rank * 128, lead_full);
+                tma_load_2d_pair(a + TILE_A_BYTES, &map_w, (int)(kb * BK), tn * 256 + (int)rank * PAIR_BN_HALF, lead_full);
+            }
+        }
+    } else if (tid == 32 && rank == 0) {
+        // ---- MMA issuer (leader only): accumulator lt mod 2 in both CTAs' tensor memory
+        uint32_t it = 0, lt = 0;
+        for (uint32_t t = pair; t < ntiles && ok; t += npairs, ++lt) {
+            const uint32_t buf = lt & 1u;
+            if (lt >= 2) ok = mbar_wait(acc_empty(buf), ((lt >> 1) - 1) & 1u, limit);   // both epilogues have drained it
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t d = tmem_base + buf * 256u;
+            for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
+                const int s = it % NS;
+                ok = mbar_wait(full(s), (it / NS) & 1u, limit);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a = base + s * PAIR_STAGE, b = a + TILE_A_BYTES;
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k)
+                    umma_f16_pair(d, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), (kb | k) != 0, PAIR_IDESC);
+                umma_commit_pair(empty(s));          // the stage goes back to both producers
+            }
+            if (ok) umma_commit_pair(acc_full(buf));
+        }
+    } else if (warp >= 2 && warp < 6) {
+        // ---- epilogue of this CTA: its 128 rows of the tile; tensor-memory lane quarter = warp mod 4
+        const int q = warp & 3;
+        const float s = __ldg(sb), b = __ldg(sb + 1);
+        uint32_t lt = 0;
+        for (uint32_t t = pair; t < ntiles; t += npairs, ++lt) {
+            const int tm = t % tiles_m, tn = t / tiles_m;
+            const uint32_t buf = lt & 1u;
+            ok = mbar_wait(acc_full(buf), (lt >> 1) & 1u, limit);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t row = tm * 256 + rank * 128 + q * 32 + lane;
+            const float bias = (row < M) ? b * __ldg(rowsum + row) : 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 256; c0 += 32) {
+                uint32_t v[32];
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * 256u + (uint32_t)c0;
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                      "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                      "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                      "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                    : "r"(taddr));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const uint32_t col = tn * 256 + c0;
+                if (row < M && col < N) {
+                    float4 *dst = reinterpret_cast<float4 *>(y + (size_t)row * N + col);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        dst[j] = make_float4(__fmaf_rn(s, __uint_as_float(v[4 * j]), bias), __fmaf_rn(s, __uint_as_float(v[4 * j + 1]), bias),
+                                             __fmaf_rn(s, __uint_as_float(v[4 * j + 2]), bias), __fmaf_rn(s, __uint_as_float(v[4 * j + 3]), bias));
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive_cluster(map_to_cta(acc_empty(buf), 0u));
+        }
+    }
+    if (!ok) atomicExch(status, 2u);
+
+    // ---- both CTAs are through with each other's barriers and tensor memory before either lets go
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_barrier();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+}
+
 template <int B, int E>
 int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const float *rowsum, float *y,
            uint32_t M, uint32_t N, uint32_t K, uint32_t n_sm, uint32_t *status, uint32_t inject_polls, cudaStream_t st)
@@ -637,6 +832,38 @@ int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const f
     const uint32_t grid = ntiles < n_sm ? ntiles : n_sm;
     matmul_kernel<B, E><<<grid, C::THREADS, C::SMEM, st>>>(map_x, map_w, sb, rowsum, y, M, N, K, status, inject_polls);
     return omc::note_cuda(cudaGetLastError());
+}
+
+// S1E5M10 on pairs of SMs (matmul_pair_kernel): clusters of two CTAs, one cluster per pair of SMs.
+int launch_pair(const CUtensorMap &map_x, const void *codes, const float *sb, const float *rowsum, float *y,
+                uint32_t M, uint32_t N, uint32_t K, uint32_t n_sm, uint32_t *status, uint32_t inject_polls, cudaStream_t st)
+{
+    CUtensorMap map_w;
+    if (!make_map(&map_w, codes, N, K, PAIR_BN_HALF)) return OMC_ERR_CUDA;
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        int rc = omc::note_cuda(cudaFuncSetAttribute(matmul_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM));
+        if (rc) return rc;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    const uint32_t ntiles = ((M + 255) / 256) * ((N + 255) / 256);
+    const uint32_t max_pairs = n_sm / 2 ? n_sm / 2 : 1;
+    const uint32_t npairs = ntiles < max_pairs ? ntiles : max_pairs;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * npairs);
+    cfg.blockDim = dim3(PAIR_THREADS);
+    cfg.dynamicSmemBytes = PAIR_SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return omc::note_cuda(cudaLaunchKernelEx(&cfg, matmul_pair_kernel, map_x, map_w, sb, rowsum, y, M, N, K, status, inject_polls));
 }
 
 }  // namespace
@@ -696,7 +923,11 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     if (exp == 4) return launch<8, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     if (exp == 2) return launch<6, 2>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     switch (man) {
-    case 10: return launch<16, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    case 10:
+        // a tile of the two-SM kernel is 256 x 256: smaller products stay on the one-SM kernel
+        if (M >= 256 && N >= 256 && n_sm >= 2)
+            return launch_pair(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        return launch<16, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     case 6: return launch<12, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     default: return launch<8, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     }

@@ -95,7 +95,9 @@ def test_matmul_wait_runs_out_then_works_again():
     N, K, M = 256, 128, 200
     w = (rng.standard_normal(N * K) * 0.05).astype(np.float32)
     x = (rng.standard_normal((M, K)) * 0.5).astype(np.float16)
-    for fmt, fixed in [((5, 10), False), ((5, 2), False), ((0, 15), True)]:
+    for fmt, fixed, M in [((5, 10), False, 200), ((5, 10), False, 300), ((5, 2), False, 200), ((0, 15), True, 200)]:
+        # 300 rows of S1E5M10 take the kernel that pairs two SMs on a tile
+        x = (rng.standard_normal((M, K)) * 0.5).astype(np.float16)
         plan = omc.Plan([N * K], [0], fmt, fixed=fixed)
         dm = DeviceModel(plan)
         dm.compress(dm.upload_full([w]))
