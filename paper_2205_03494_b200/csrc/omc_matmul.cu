@@ -15,6 +15,7 @@
 //   S1E5M10: the codes are halves already; TMA puts them into the 128-byte-swizzled operand tile.
 //   S1E5M6 / S1E5M2: the tile's packed bytes arrive through a byte-typed tensor map, and eight more
 //   warps expand them (byte permutes and shifts only) into the swizzled operand tile.
+//   S1E5M10 with at least 256 rows and columns runs on pairs of SMs instead (matmul_pair_kernel below).
 // Every wait is bounded; a wait that runs out sets the plan's status word, and the tensor memory is
 // released on every path.
 #include <cuda.h>
@@ -142,6 +143,9 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 
 __global__ void rowsum_kernel(const __half *__restrict__ x, uint32_t M, uint32_t K, float *__restrict__ out)
 {
+    // the product that follows is launched as this kernel's programmatic dependent and may start at once;
+    // its epilogue waits for this kernel before it reads the sums
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // one warp per row; fixed order (lane-strided partial sums, then a shuffle tree)
     const uint32_t row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= M) return;
@@ -483,6 +487,7 @@ matmul_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         // ---- epilogue: tensor-memory lane quarter = warp mod 4; one thread = one row of the tile
         const int q = warp & 3;
         const float s = __ldg(sb), b = __ldg(sb + 1);
+        asm volatile("griddepcontrol.wait;" ::: "memory");      // the row sums of X are complete and visible
         uint32_t lt = 0;
         for (uint32_t t = blockIdx.x; t < ntiles; t += gridDim.x, ++lt) {
             const int tm = t % tiles_m, tn = t / tiles_m;
@@ -764,6 +769,7 @@ matmul_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
         // ---- epilogue of this CTA: its 128 rows of the tile; tensor-memory lane quarter = warp mod 4
         const int q = warp & 3;
         const float s = __ldg(sb), b = __ldg(sb + 1);
+        asm volatile("griddepcontrol.wait;" ::: "memory");      // the row sums of X are complete and visible
         uint32_t lt = 0;
         for (uint32_t t = pair; t < ntiles; t += npairs, ++lt) {
             const int tm = t % tiles_m, tn = t / tiles_m;
@@ -830,8 +836,18 @@ int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const f
     }
     const uint32_t ntiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
     const uint32_t grid = ntiles < n_sm ? ntiles : n_sm;
-    matmul_kernel<B, E><<<grid, C::THREADS, C::SMEM, st>>>(map_x, map_w, sb, rowsum, y, M, N, K, status, inject_polls);
-    return omc::note_cuda(cudaGetLastError());
+    // the programmatic dependent of rowsum_kernel: set-up, copies and products overlap it
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(C::THREADS);
+    cfg.dynamicSmemBytes = C::SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return omc::note_cuda(cudaLaunchKernelEx(&cfg, matmul_kernel<B, E>, map_x, map_w, sb, rowsum, y, M, N, K, status, inject_polls));
 }
 
 // S1E5M10 on pairs of SMs (matmul_pair_kernel): clusters of two CTAs, one cluster per pair of SMs.
@@ -856,13 +872,15 @@ int launch_pair(const CUtensorMap &map_x, const void *codes, const float *sb, co
     cfg.blockDim = dim3(PAIR_THREADS);
     cfg.dynamicSmemBytes = PAIR_SMEM;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // the programmatic dependent of rowsum_kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return omc::note_cuda(cudaLaunchKernelEx(&cfg, matmul_pair_kernel, map_x, map_w, sb, rowsum, y, M, N, K, status, inject_polls));
 }
 
