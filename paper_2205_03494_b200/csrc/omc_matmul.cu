@@ -622,9 +622,9 @@ bool make_raw_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t row_b
 }
 
 // ---------------------------------------------------------------------------------------------
-// S1E5M10 on pairs of SMs.  Two CTAs of a cluster share one 256 x 256 tile of Y: each holds its own
-// 128 rows of X and its own 128 rows of the codes per K block (32 KB instead of the 48 KB of the
-// one-SM kernel for the same number of products, and six stages instead of four), the leader's
+// The same product on pairs of SMs.  Two CTAs of a cluster share one 256 x 256 tile of Y: each holds its own
+// 128 rows of X and its own 128 rows of the codes per K block (with S1E5M10 32 KB instead of the 48 KB
+// of the one-SM kernel for the same number of products, and six stages instead of four), the leader's
 // MMA thread issues tcgen05.mma.cta_group::2 (M = 256: the upper 128 rows accumulate in the
 // leader's tensor memory, the lower in its peer's; the 256 columns of the B operand are read from
 // both CTAs' shared memory), and each CTA's epilogue warps store their own 128 rows.
@@ -638,12 +638,33 @@ bool make_raw_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t row_b
 // before it; a second one before the tensor memory is released keeps either CTA alive while the
 // other may still signal it.  Every mbarrier wait is bounded; a wait that runs out ends that role's
 // loop, so that both CTAs always reach the closing barrier.
-constexpr int PAIR_STAGES = 6;
-constexpr int PAIR_BN_HALF = 128;                                   // rows of the codes per CTA
-constexpr int PAIR_STAGE = TILE_A_BYTES + PAIR_BN_HALF * BK * 2;     // 32 KB
-constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE + 1024 + 256;
-constexpr int PAIR_THREADS = 192;
-constexpr uint32_t PAIR_IDESC = (1u << 4) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+// Formats that are decoded on the way in: each CTA's decoder warps expand its own 128 rows (half the
+// decoding per SM of the one-SM kernel), from packed bytes that arrive on a barrier of its own
+// (rawfull(s): an ordinary bulk tensor copy); the leader's decoders arrive on decoded(s) in the
+// leader, and the peer's idle MMA thread waits for its own decoders and forwards one arrival across
+// the pair, so that the leader's MMA thread sees both halves ready with two waits.
+template <int B, int E>
+struct PairCfg {
+    using C1 = Cfg<B, E>;
+    static constexpr bool DECODE = C1::DECODE, ODD = C1::ODD, SPLIT = C1::SPLIT, FIXED = C1::FIXED;
+    static constexpr int HALF = 128;                                  // rows of the codes per CTA
+    static constexpr int TILE_B_BYTES = HALF * BK * 2;                // one operand tile of this CTA
+    static constexpr int OPERAND_BYTES = (SPLIT ? 2 : 1) * TILE_B_BYTES;
+    static constexpr int ROW_BYTES = C1::ROW_BYTES, BOX_BYTES = C1::BOX_BYTES;
+    static constexpr int RAW_BYTES = DECODE ? HALF * BOX_BYTES : 0;
+    static constexpr int STAGE = TILE_A_BYTES + OPERAND_BYTES + RAW_BYTES;
+    static constexpr int MAX_STAGES = 6;
+    static constexpr int FIT = (227 * 1024 - 1280) / STAGE;
+    static constexpr int NSTAGES = FIT < MAX_STAGES ? FIT : MAX_STAGES;
+    static constexpr int SMEM = NSTAGES * STAGE + 1024 /* alignment slack */ + 256 /* barriers, tmem slot */;
+    static constexpr int DEC_THREADS = DECODE ? MATMUL_DECODER_THREADS : 0;
+    static constexpr int THREADS = 192 + DEC_THREADS;
+    // what completes on the leader's full(s): the X tiles of both CTAs, and without decoding their operand tiles too
+    static constexpr uint32_t FULL_TX = 2u * (TILE_A_BYTES + (DECODE ? 0 : TILE_B_BYTES));
+    static constexpr uint32_t IDESC = (1u << 4) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+    static_assert(STAGE % 1024 == 0, "operand tiles stay 1024-byte aligned");
+    static_assert(NSTAGES >= 2 && 8 * (4 * NSTAGES + 5) <= 256, "stages and their barriers fit");
+};
 
 __device__ __forceinline__ uint32_t cluster_cta_rank()
 {
@@ -683,27 +704,37 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                  ::"r"(bar), "h"(both) : "memory");
 }
+// Arrival on a barrier of the pair's other CTA (or this one), in the plain form: a release of cluster
+// scope on every arrival makes the forwarder of the decoders' completion the slowest link of the
+// pipeline (measured: S1E5M2 0.51 ms against 0.27 ms), and what it would order is already ordered,
+// since the operand bytes stay in the shared memory of the SM that wrote them, were handed to the
+// asynchronous proxy there (fence.proxy.async by their writers, before their own arrival), and are
+// read by that SM's half of the pair's MMA, which is issued only after this arrival was seen.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
-__global__ void __launch_bounds__(PAIR_THREADS, 1)
+template <int B, int E>
+__global__ void __launch_bounds__(PairCfg<B, E>::THREADS, 1)
 matmul_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                    const float *__restrict__ sb, const float *__restrict__ rowsum, float *__restrict__ y,
                    uint32_t M, uint32_t N, uint32_t K, uint32_t *status, uint32_t inject_polls)
 {
-    constexpr int NS = PAIR_STAGES;
+    using C = PairCfg<B, E>;
+    constexpr int NS = C::NSTAGES, TILE_B_BYTES = C::TILE_B_BYTES;
     const uint32_t limit = inject_polls ? inject_polls : WAIT_LIMIT;
     const bool skip_loads = inject_polls != 0u;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (saddr(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bars = base + NS * PAIR_STAGE;   // full[NS], empty[NS], acc_full[2], acc_empty[2], tmem slot
+    const uint32_t bars = base + NS * C::STAGE;   // full[NS], rawfull[NS], decoded[NS], empty[NS], acc_full[2], acc_empty[2], tmem slot
     auto full = [&](int s) { return bars + 8u * s; };
-    auto empty = [&](int s) { return bars + 8u * (NS + s); };
-    auto acc_full = [&](int b) { return bars + 8u * (2 * NS + b); };
-    auto acc_empty = [&](int b) { return bars + 8u * (2 * NS + 2 + b); };
-    const uint32_t tmem_slot = bars + 8u * (2 * NS + 4);
+    auto rawfull = [&](int s) { return bars + 8u * (NS + s); };
+    auto decoded = [&](int s) { return bars + 8u * (2 * NS + s); };
+    auto empty = [&](int s) { return bars + 8u * (3 * NS + s); };
+    auto acc_full = [&](int b) { return bars + 8u * (4 * NS + b); };
+    auto acc_empty = [&](int b) { return bars + 8u * (4 * NS + 2 + b); };
+    const uint32_t tmem_slot = bars + 8u * (4 * NS + 4);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_cta_rank();          // 0: the leader
     const uint32_t nkb = K / BK;
@@ -711,7 +742,13 @@ matmul_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     const uint32_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
 
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(full(s), 1);
+            mbar_init(rawfull(s), 1);
+            // the leader's: its own decoders and the arrival its peer forwards
+            mbar_init(decoded(s), C::DECODE ? C::DEC_THREADS + (rank == 0 ? 1 : 0) : 1);
+            mbar_init(empty(s), 1);
+        }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 256); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -728,7 +765,7 @@ matmul_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
 
     bool ok = true;
     if (tid == 0) {
-        // ---- producer of this CTA: its 128 rows of X and its 128 rows of the codes per K block
+        // ---- producer of this CTA: its 128 rows of X and its 128 rows of the codes (halves, or their packed bytes) per K block
         uint32_t it = 0;
         for (uint32_t t = pair; t < ntiles && ok; t += npairs) {
             const int tm = t % tiles_m, tn = t / tiles_m;
@@ -736,11 +773,16 @@ matmul_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
                 const int s = it % NS;
                 if (it >= (uint32_t)NS) ok = mbar_wait(empty(s), ((it / NS) - 1) & 1u, limit);
                 if (!ok) break;
-                if (rank == 0) mbar_expect_tx(full(s), 2u * PAIR_STAGE);        // the bytes of both CTAs
+                if (rank == 0) mbar_expect_tx(full(s), C::FULL_TX);              // the bytes of both CTAs
+                if constexpr (C::DECODE) mbar_expect_tx(rawfull(s), C::RAW_BYTES);
                 if (skip_loads) continue;
-                const uint32_t a = base + s * PAIR_STAGE, lead_full = map_to_cta(full(s), 0u);
+                const uint32_t a = base + s * C::STAGE, lead_full = map_to_cta(full(s), 0u);
                 tma_load_2d_pair(a, &map_x, (int)(kb * BK), tm * 256 + (int)rank * 128, lead_full);
-                tma_load_2d_pair(a + TILE_A_BYTES, &map_w, (int)(kb * BK), tn * 256 + (int)rank * PAIR_BN_HALF, lead_full);
+                if constexpr (C::DECODE)      // odd widths: from the 16-byte boundary at or below the K block's first byte
+                    tma_load_2d(a + TILE_A_BYTES + C::OPERAND_BYTES, &map_w, (int)((kb * C::ROW_BYTES) & ~15u),
+                                tn * 256 + (int)rank * C::HALF, rawfull(s));
+                else
+                    tma_load_2d_pair(a + TILE_A_BYTES, &map_w, (int)(kb * BK), tn * 256 + (int)rank * C::HALF, lead_full);
             }
         }
     } else if (tid == 32 && rank == 0) {
@@ -755,15 +797,32 @@ matmul_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % NS;
                 ok = mbar_wait(full(s), (it / NS) & 1u, limit);
+                if constexpr (C::DECODE) ok = ok && mbar_wait(decoded(s), (it / NS) & 1u, limit);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a = base + s * PAIR_STAGE, b = a + TILE_A_BYTES;
+                const uint32_t a = base + s * C::STAGE, b = a + TILE_A_BYTES;
 #pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k)
-                    umma_f16_pair(d, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), (kb | k) != 0, PAIR_IDESC);
+                for (int k = 0; k < BK / UMMA_K; ++k) {
+                    umma_f16_pair(d, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), (kb | k) != 0, C::IDESC);
+                    if constexpr (C::SPLIT)      // the low parts of the weights, into the same accumulator
+                        umma_f16_pair(d, umma_desc(a + k * UMMA_K * 2), umma_desc(b + TILE_B_BYTES + k * UMMA_K * 2), 1u, C::IDESC);
+                }
                 umma_commit_pair(empty(s));          // the stage goes back to both producers
             }
             if (ok) umma_commit_pair(acc_full(buf));
+        }
+    } else if (tid == 32) {
+        // ---- the peer's MMA thread has no products to issue: it tells the leader when its decoders are through
+        if constexpr (C::DECODE) {
+            uint32_t it = 0;
+            for (uint32_t t = pair; t < ntiles && ok; t += npairs) {
+                for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % NS;
+                    ok = mbar_wait(decoded(s), (it / NS) & 1u, limit);
+                    if (!ok) break;
+                    mbar_arrive_cluster(map_to_cta(decoded(s), 0u));
+                }
+            }
         }
     } else if (warp >= 2 && warp < 6) {
         // ---- epilogue of this CTA: its 128 rows of the tile; tensor-memory lane quarter = warp mod 4
@@ -805,6 +864,46 @@ matmul_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive_cluster(map_to_cta(acc_empty(buf), 0u));
+        }
+    } else if (warp >= 6) {
+        if constexpr (C::DECODE) {
+            // ---- decoders of this CTA: its 128 rows are 1024 chunks of 8 codes; thread t takes chunks t and t + 512.
+            // rawfull(s) of block it implies that the MMAs of block it - NS have released the operand tile.
+            uint8_t *const base_ptr = smem_raw + (base - saddr(smem_raw));
+            const int t = tid - 192;
+            const int c = t & 7;
+            uint32_t it = 0;
+            for (uint32_t tile = pair; tile < ntiles && ok; tile += npairs) {
+                for (uint32_t kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % NS;
+                    ok = mbar_wait(rawfull(s), (it / NS) & 1u, limit);
+                    if (!ok) break;
+                    uint8_t *stage = base_ptr + s * C::STAGE;
+                    const uint8_t *raw = stage + TILE_A_BYTES + C::OPERAND_BYTES + t * B;      // 8 codes = B bytes
+                    uint8_t *dst = stage + TILE_A_BYTES;
+                    const uint32_t off = C::ODD ? ((kb * C::ROW_BYTES) & 15u) : 0u;      // where the K block starts in its copy
+#pragma unroll
+                    for (int i = 0; i < C::HALF * 8 / C::DEC_THREADS; ++i) {
+                        const int r = i * (C::DEC_THREADS / 8) + (t >> 3);
+                        uint4 o;
+                        if constexpr (C::SPLIT) {
+                            uint4 lo;
+                            if constexpr (C::FIXED)
+                                expand_chunk_split_fixed16(stage + TILE_A_BYTES + C::OPERAND_BYTES + r * C::BOX_BYTES + c * B, o, lo);
+                            else
+                                expand_chunk_split(stage + TILE_A_BYTES + C::OPERAND_BYTES + r * C::BOX_BYTES + off + c * B, o, lo);
+                            *reinterpret_cast<uint4 *>(dst + TILE_B_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) = lo;
+                        } else if constexpr (C::ODD)
+                            o = expand_chunk_odd<B, E>(stage + TILE_A_BYTES + C::OPERAND_BYTES + r * C::BOX_BYTES + off + c * B);
+                        else
+                            o = expand_chunk<B, E>(raw + i * C::DEC_THREADS * B);
+                        // 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r mod 8)
+                        *reinterpret_cast<uint4 *>(dst + r * 128 + ((c ^ (r & 7)) << 4)) = o;
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // visible to the tensor cores
+                    mbar_arrive(decoded(s));
+                }
+            }
         }
     }
     if (!ok) atomicExch(status, 2u);
@@ -850,17 +949,20 @@ int launch(const CUtensorMap &map_x, const void *codes, const float *sb, const f
     return omc::note_cuda(cudaLaunchKernelEx(&cfg, matmul_kernel<B, E>, map_x, map_w, sb, rowsum, y, M, N, K, status, inject_polls));
 }
 
-// S1E5M10 on pairs of SMs (matmul_pair_kernel): clusters of two CTAs, one cluster per pair of SMs.
+// The kernel on pairs of SMs: clusters of two CTAs, one cluster per pair of SMs.
+template <int B, int E>
 int launch_pair(const CUtensorMap &map_x, const void *codes, const float *sb, const float *rowsum, float *y,
                 uint32_t M, uint32_t N, uint32_t K, uint32_t n_sm, uint32_t *status, uint32_t inject_polls, cudaStream_t st)
 {
+    using C = PairCfg<B, E>;
     CUtensorMap map_w;
-    if (!make_map(&map_w, codes, N, K, PAIR_BN_HALF)) return OMC_ERR_CUDA;
+    if (C::DECODE ? !make_raw_map(&map_w, codes, N, (uint64_t)K * B / 8, C::BOX_BYTES, C::HALF) : !make_map(&map_w, codes, N, K, C::HALF))
+        return OMC_ERR_CUDA;
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        int rc = omc::note_cuda(cudaFuncSetAttribute(matmul_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM));
+        int rc = omc::note_cuda(cudaFuncSetAttribute(matmul_pair_kernel<B, E>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
         if (rc) return rc;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
@@ -869,8 +971,8 @@ int launch_pair(const CUtensorMap &map_x, const void *codes, const float *sb, co
     const uint32_t npairs = ntiles < max_pairs ? ntiles : max_pairs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * npairs);
-    cfg.blockDim = dim3(PAIR_THREADS);
-    cfg.dynamicSmemBytes = PAIR_SMEM;
+    cfg.blockDim = dim3(C::THREADS);
+    cfg.dynamicSmemBytes = C::SMEM;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -881,7 +983,16 @@ int launch_pair(const CUtensorMap &map_x, const void *codes, const float *sb, co
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return omc::note_cuda(cudaLaunchKernelEx(&cfg, matmul_pair_kernel, map_x, map_w, sb, rowsum, y, M, N, K, status, inject_polls));
+    return omc::note_cuda(cudaLaunchKernelEx(&cfg, matmul_pair_kernel<B, E>, map_x, map_w, sb, rowsum, y, M, N, K, status, inject_polls));
+}
+
+// A tile of the kernel on pairs of SMs is 256 x 256: smaller products stay on the one-SM kernel.
+template <int B, int E>
+int launch_either(const CUtensorMap &map_x, const void *codes, const float *sb, const float *rowsum, float *y,
+                  uint32_t M, uint32_t N, uint32_t K, uint32_t n_sm, uint32_t *status, uint32_t inject_polls, cudaStream_t st)
+{
+    if (M >= 256 && N >= 256 && n_sm >= 2) return launch_pair<B, E>(map_x, codes, sb, rowsum, y, M, N, K, n_sm, status, inject_polls, st);
+    return launch<B, E>(map_x, codes, sb, rowsum, y, M, N, K, n_sm, status, inject_polls, st);
 }
 
 }  // namespace
@@ -927,26 +1038,22 @@ extern "C" int omc_matmul(const omc_plan_t *plan, uint32_t var, const uint8_t *p
     const uint32_t inject = plan->inject_polls;      // diagnostics: applies to this launch only
     plan->inject_polls = 0;
     if (fixed) {
-        if (man == 7) return launch<8, 0>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
-        if (man == 11) return launch<12, 0>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
-        return launch<16, 0>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        if (man == 7) return launch_either<8, 0>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        if (man == 11) return launch_either<12, 0>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        return launch_either<16, 0>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     }
-    if (split) return launch<19, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    if (split) return launch_either<19, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     if (odd) {
-        if (exp == 5) return launch<13, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
-        if (exp == 4) return launch<13, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
-        if (man == 9) return launch<13, 3>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
-        return launch<11, 3>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        if (exp == 5) return launch_either<13, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        if (exp == 4) return launch_either<13, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        if (man == 9) return launch_either<13, 3>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+        return launch_either<11, 3>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     }
-    if (exp == 4) return launch<8, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
-    if (exp == 2) return launch<6, 2>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    if (exp == 4) return launch_either<8, 4>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    if (exp == 2) return launch_either<6, 2>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     switch (man) {
-    case 10:
-        // a tile of the two-SM kernel is 256 x 256: smaller products stay on the one-SM kernel
-        if (M >= 256 && N >= 256 && n_sm >= 2)
-            return launch_pair(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
-        return launch<16, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
-    case 6: return launch<12, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
-    default: return launch<8, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    case 10: return launch_either<16, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    case 6: return launch_either<12, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
+    default: return launch_either<8, 5>(map_x, codes, sbv, rowsum_scratch, y, M, N, K, n_sm, plan->d_status, inject, st);
     }
 }

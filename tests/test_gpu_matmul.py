@@ -148,8 +148,8 @@ def test_matmul_fixed_point_exact_small_case():
     """With s = 1, b = 0, one-hot rows of X and weights that are whole codes, every output is one
     weight exactly: the decoders' FP16 values are the codes' values bit for bit, for every code of
     the three formats."""
-    for F_ in (7, 11, 15):
-        N, K, M = 128, 512, 512
+    for F_, (N, K, M) in [(f, shape) for f in (7, 11, 15) for shape in ((128, 512, 512), (256, 256, 256))]:
+        # 128 rows of W: one SM per tile; 256 x 256: the kernel on pairs of SMs
         B = 1 + F_
         ks = (np.arange(N * K, dtype=np.int64) % (1 << B)) - (1 << (B - 1))     # every code (all 65536 of S1I0F15 once)
         w = (ks.astype(np.float64) * 2.0 ** -F_).astype(np.float32)
@@ -157,7 +157,8 @@ def test_matmul_fixed_point_exact_small_case():
         dm = DeviceModel(plan)
         dm.compress(dm.upload_full([w]))
         x = np.zeros((M, K), np.float16)
-        x[np.arange(M), np.arange(M) % K] = 1.0                                   # row m picks column m of W^T
+        assert M == K
+        x[np.arange(M), np.arange(M)] = 1.0                                       # row m picks column m of W^T
         xd = torch.from_numpy(x).cuda()
         y = torch.zeros((M, N), dtype=torch.float32, device="cuda")
         scratch = torch.zeros(M, dtype=torch.float32, device="cuda")
@@ -165,8 +166,8 @@ def test_matmul_fixed_point_exact_small_case():
                    scratch.data_ptr(), torch.cuda.current_stream().cuda_stream)
         torch.cuda.synchronize()
         assert plan.status() == 0
-        want = w.reshape(N, K)[:, np.arange(M) % K].T                              # y[m, n] = W[n, m]
-        assert np.array_equal(y.cpu().numpy(), want), F_
+        want = w.reshape(N, K).T                                                   # y[m, n] = W[n, m]
+        assert np.array_equal(y.cpu().numpy(), want), (F_, N)
 
 
 def test_matmul_argument_checks():
@@ -192,14 +193,16 @@ def test_matmul_argument_checks():
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("size", [128, 384], ids=lambda n: "n%d" % n)
 @pytest.mark.parametrize("fmt", [(4, 3), (2, 3), (3, 7), (4, 8), (3, 9), (4, 14)], ids=lambda f: "E%dM%d" % f)
-def test_matmul_weights_at_the_top_of_the_range(fmt):
+def test_matmul_weights_at_the_top_of_the_range(fmt, size):
     """Weights that are infinite, NaN or the largest finite value of S1E4M3 / S1E2M3: the hardware
     narrow-float types have other values at those codes, so the decoder patches them.  A row of W
     with an infinity gives an infinite or NaN output column, a row with the largest finite value
-    the exact product."""
+    the exact product.  (128: the kernel with one SM per tile; 384: the one on pairs of SMs, the
+    second CTA's rows included.)"""
     E, M = fmt
-    N, K, Mr = 128, 128, 128
+    N, K, Mr = size, 128, size
     top = 2.0 ** ((1 << (E - 1)) - 1) * (2 - 2.0 ** -M)
     w = np.full((N, K), 0.5 * top, np.float32)           # a value of the format in both cases
     w[3, 5] = np.inf
@@ -207,6 +210,8 @@ def test_matmul_weights_at_the_top_of_the_range(fmt):
     w[11, 0] = np.nan
     w[20, :] = top
     w[21, :] = -top
+    w[N - 5, :] = top                                     # in the second CTA's half of a pair's tile
+    w[N - 9, 17] = -np.inf
     plan = omc.Plan([N * K], [0], fmt, flags=omc.PLAN_WEIGHTS_ONLY)       # no transformation: s = 1, b = 0
     dm = DeviceModel(plan)
     dm.compress(dm.upload_full([w.reshape(-1)]))
@@ -221,4 +226,5 @@ def test_matmul_weights_at_the_top_of_the_range(fmt):
     assert np.all(got[:, 3] == np.inf) and np.all(got[:, 7] == -np.inf) and np.all(np.isnan(got[:, 11]))
     assert np.all(got[:, 20] == np.float32(top * K)) and np.all(got[:, 21] == np.float32(-top * K))
     assert np.all(got[:, 0] == np.float32(0.5 * top * K))
+    assert np.all(got[:, N - 5] == np.float32(top * K)) and np.all(got[:, N - 9] == -np.inf)
 
