@@ -15,7 +15,7 @@
 //   S1E5M10: the codes are halves already; TMA puts them into the 128-byte-swizzled operand tile.
 //   S1E5M6 / S1E5M2: the tile's packed bytes arrive through a byte-typed tensor map, and eight more
 //   warps expand them (byte permutes and shifts only) into the swizzled operand tile.
-//   S1E5M10 with at least 256 rows and columns runs on pairs of SMs instead (matmul_pair_kernel below).
+//   Products of at least 256 rows and columns run on pairs of SMs instead (matmul_pair_kernel below).
 // Every wait is bounded; a wait that runs out sets the plan's status word, and the tensor memory is
 // released on every path.
 #include <cuda.h>
