@@ -170,6 +170,33 @@ def test_matmul_fixed_point_exact_small_case():
         assert np.array_equal(y.cpu().numpy(), want), (F_, N)
 
 
+@pytest.mark.parametrize("fmt,fixed", [((5, 10), False), ((5, 2), False), ((3, 7), False), ((4, 14), False),
+                                       ((0, 11), True), ((0, 15), True)], ids=lambda v: str(v))
+def test_matmul_repeated_launches_give_the_same_bits(fmt, fixed):
+    """Ten launches in a row on pairs of SMs (several tiles per pair, ragged M and N): the same bits
+    every time and a clean status word, i.e. no stage was read before it was ready."""
+    rng = np.random.default_rng(5)
+    M, N, K = 1000, 384, 512
+    w = (rng.standard_normal(N * K) * 0.05).astype(np.float32)
+    plan = omc.Plan([N * K], [0], fmt, fixed=fixed)
+    dm = DeviceModel(plan)
+    dm.compress(dm.upload_full([w]))
+    xd = torch.from_numpy((rng.standard_normal((M, K)) * 0.5).astype(np.float16)).cuda()
+    scratch = torch.zeros(M, dtype=torch.float32, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    first = None
+    for i in range(10):
+        y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        omc.matmul(plan, 0, dm.packed.data_ptr(), dm.sb.data_ptr(), xd.data_ptr(), M, N, K, y.data_ptr(),
+                   scratch.data_ptr(), st)
+        torch.cuda.synchronize()
+        assert plan.status(st) == 0 and not torch.isnan(y).any()
+        if first is None:
+            first = y
+        else:
+            assert torch.equal(first.view(torch.int32), y.view(torch.int32)), i
+
+
 def test_matmul_argument_checks():
     plan = omc.Plan([128 * 64, 100], [0, 1], (5, 10))
     dm = DeviceModel(plan)
