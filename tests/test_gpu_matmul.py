@@ -18,12 +18,13 @@ pytestmark = pytest.mark.gpu
 
 @pytest.mark.parametrize("fmt", [(5, 10), (5, 6), (5, 2), (4, 3), (2, 3)], ids=lambda f: "E%dM%d" % f)
 @pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 256, 192), (1000, 384, 512), (64, 128, 1024),
-                                   (4000, 4224, 192)])
+                                   (4000, 4224, 192), (256, 256, 64), (300, 256, 1024)])
 def test_matmul_from_codes_matches_definition(M, N, K, fmt):
     """The last shape has 32 x 17 = 544 tiles of 128 x 256 (M and N not multiples of the tile), so
     every persistent CTA walks over three or four tiles: both accumulators in tensor memory are
     reused, the producer runs ahead across tile boundaries, and the epilogue of one tile overlaps
-    the products of the next."""
+    the products of the next.  From 256 rows and columns on the product runs on pairs of SMs; the last
+    two shapes are its smallest (one tile, one K block) and one tile with more K blocks than stages."""
     rng = np.random.default_rng(M + N + K)
     numel = [777, N * K, 64, 128 * 64]
     kinds = [0, 0, 1, 0]
